@@ -1,0 +1,323 @@
+"""QAQ oracle bindings -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+
+Thin ctypes access to ``oracle/qaq_oracle.cpp`` (a plain CPU restatement of the QAQ
+hot path written from arXiv 2403.04643).  Only tests, the smoke check and the
+benchmark's CPU-baseline leg import this package; the CUDA library and its Python
+binding never do, and the two share no code.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "qaq_oracle.cpp")
+_LIB = os.path.join(_HERE, "libqaq_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no CUDA).  -ffp-contract=off keeps every
+    binary32 operation separately rounded, which the integer decisions rely on."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fPIC", "-shared", "-pthread",
+               "-o", _LIB, _SRC]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _p(a, ct):
+    return None if a is None else a.ctypes.data_as(C.POINTER(ct))
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        L = C.CDLL(_LIB)
+        L.qaq_oracle_half_to_float.restype = C.c_float
+        L.qaq_oracle_half_to_float.argtypes = [C.c_uint16]
+        L.qaq_oracle_token_bytes.restype = C.c_long
+        L.qaq_oracle_token_bytes.argtypes = [C.c_int, C.c_int]
+        L.qaq_oracle_bits_ladder.restype = C.c_int
+        L.qaq_oracle_bits_ladder.argtypes = [C.c_float, C.c_float, C.c_int, C.c_int]
+        L.qaq_oracle_key_bits.restype = C.c_int
+        L.qaq_oracle_key_bits.argtypes = [C.c_float, C.c_float, C.c_float, C.c_int, C.c_int]
+        L.qaq_oracle_value_bits.restype = C.c_int
+        L.qaq_oracle_value_bits.argtypes = [C.c_float, C.c_float, C.c_float, C.c_float, C.c_int, C.c_int]
+        L.qaq_oracle_dequant.restype = C.c_float
+        L.qaq_oracle_dequant.argtypes = [C.c_uint8, C.c_float, C.c_float]
+        L.qaq_oracle_quantize.restype = C.c_long
+        L.qaq_oracle_code_bits.restype = C.c_double
+        L.qaq_oracle_cr_paper.restype = C.c_double
+        L.qaq_oracle_cr_paper.argtypes = [C.c_double, C.c_double, C.c_long, C.c_long, C.c_long, C.c_int]
+        L.qaq_oracle_run_batch.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+# ---------------------------------------------------------------------------------
+# scalar / single-(b,h) wrappers
+# ---------------------------------------------------------------------------------
+def half_to_float(h: int) -> float:
+    return float(lib().qaq_oracle_half_to_float(int(h)))
+
+
+def token_bytes(D: int, B: int) -> int:
+    return int(lib().qaq_oracle_token_bytes(D, B))
+
+
+def thresholds(x_u16: np.ndarray, alpha: float):
+    x = np.ascontiguousarray(x_u16, dtype=np.uint16).ravel()
+    lo, hi = C.c_float(), C.c_float()
+    lib().qaq_oracle_thresholds(_p(x, C.c_uint16), C.c_long(x.size), C.c_double(alpha), C.byref(lo), C.byref(hi))
+    return np.float32(lo.value), np.float32(hi.value)
+
+
+def policy(sigmaS_max: float, sigmaX_max: float, qnorm2: float, T: int):
+    cK, cV = C.c_float(), C.c_float()
+    lib().qaq_oracle_policy(C.c_double(sigmaS_max), C.c_double(sigmaX_max), C.c_double(qnorm2), C.c_long(T),
+                            C.byref(cK), C.byref(cV))
+    return np.float32(cK.value), np.float32(cV.value)
+
+
+def window_max(ring: np.ndarray, nvalid: np.ndarray):
+    ring = np.ascontiguousarray(ring, dtype=np.float32)
+    W, T = ring.shape
+    nvalid = np.ascontiguousarray(nvalid, dtype=np.uint8)
+    out = np.empty(T, dtype=np.float32)
+    lib().qaq_oracle_window_max(_p(ring, C.c_float), _p(nvalid, C.c_uint8), C.c_int(W), C.c_long(T), _p(out, C.c_float))
+    return out
+
+
+def masked_range(x_u16: np.ndarray, lo, hi):
+    x = np.ascontiguousarray(x_u16, dtype=np.uint16)
+    mn, mx = C.c_float(), C.c_float()
+    lib().qaq_oracle_masked_range(_p(x, C.c_uint16), C.c_int(x.size), C.c_float(lo), C.c_float(hi),
+                                  C.byref(mn), C.byref(mx))
+    return np.float32(mn.value), np.float32(mx.value)
+
+
+def bits_ladder(r, c, bmin, bmax) -> int:
+    return int(lib().qaq_oracle_bits_ladder(C.c_float(r), C.c_float(c), bmin, bmax))
+
+
+def key_bits(mn, mx, cK, bmin, bmax) -> int:
+    return int(lib().qaq_oracle_key_bits(C.c_float(mn), C.c_float(mx), C.c_float(cK), bmin, bmax))
+
+
+def value_bits(mn, mx, shat, cV, bmin, bmax) -> int:
+    return int(lib().qaq_oracle_value_bits(C.c_float(mn), C.c_float(mx), C.c_float(shat), C.c_float(cV), bmin, bmax))
+
+
+def select_bits(K, V, thr, ring, nvalid, cK, cV, bmin, bmax):
+    """K, V: [T, D] uint16; thr: 4 floats; ring: [W, T]; nvalid: [T]."""
+    K = np.ascontiguousarray(K, dtype=np.uint16)
+    V = np.ascontiguousarray(V, dtype=np.uint16)
+    T, D = K.shape
+    thr = np.ascontiguousarray(thr, dtype=np.float32)
+    ring = np.ascontiguousarray(ring, dtype=np.float32)
+    nvalid = np.ascontiguousarray(nvalid, dtype=np.uint8)
+    W = ring.shape[0]
+    bK = np.empty(T, dtype=np.uint8)
+    bV = np.empty(T, dtype=np.uint8)
+    lib().qaq_oracle_select_bits(_p(K, C.c_uint16), _p(V, C.c_uint16), C.c_long(T), C.c_int(D), _p(thr, C.c_float),
+                                 _p(ring, C.c_float), _p(nvalid, C.c_uint8), C.c_int(W), C.c_float(cK), C.c_float(cV),
+                                 C.c_int(bmin), C.c_int(bmax), _p(bK, C.c_uint8), _p(bV, C.c_uint8))
+    return bK, bV
+
+
+def token_codes(x_u16, lo, hi, B):
+    x = np.ascontiguousarray(x_u16, dtype=np.uint16)
+    D = x.size
+    codes = np.empty(D, dtype=np.uint8)
+    flag = np.empty(D, dtype=np.uint8)
+    mn, step = C.c_float(), C.c_float()
+    lib().qaq_oracle_token_codes(_p(x, C.c_uint16), C.c_int(D), C.c_float(lo), C.c_float(hi), C.c_int(B),
+                                 C.byref(mn), C.byref(step), _p(codes, C.c_uint8), _p(flag, C.c_uint8))
+    return np.float32(mn.value), np.float32(step.value), codes, flag
+
+
+def dequant(code, mn, step) -> np.float32:
+    return np.float32(lib().qaq_oracle_dequant(int(code), C.c_float(mn), C.c_float(step)))
+
+
+def pack_token(codes, B):
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    D = codes.size
+    out = np.empty(token_bytes(D, B), dtype=np.uint8)
+    lib().qaq_oracle_pack_token(_p(codes, C.c_uint8), C.c_int(D), C.c_int(B), _p(out, C.c_uint8))
+    return out
+
+
+def unpack_token(data, D, B):
+    data = np.ascontiguousarray(data, dtype=np.uint8)
+    out = np.empty(D, dtype=np.uint8)
+    lib().qaq_oracle_unpack_token(_p(data, C.c_uint8), C.c_int(D), C.c_int(B), _p(out, C.c_uint8))
+    return out
+
+
+@dataclass
+class QuantTensor:
+    """Canonical quantized form of one (b,h) tensor."""
+    T: int
+    D: int
+    bits: np.ndarray      # [T] u8
+    mn: np.ndarray        # [T] f32
+    step: np.ndarray      # [T] f32
+    off: np.ndarray       # [T+1] u32 byte offsets
+    stream: np.ndarray    # [off[T]] u8
+    rowptr: np.ndarray    # [T+1] u32
+    ch: np.ndarray        # [n_out] u8
+    val: np.ndarray       # [n_out] u16 (binary16 bits)
+
+
+def quantize(x_u16, lo, hi, bits) -> QuantTensor:
+    x = np.ascontiguousarray(x_u16, dtype=np.uint16)
+    T, D = x.shape
+    bits = np.ascontiguousarray(bits, dtype=np.uint8)
+    mn = np.empty(T, np.float32)
+    step = np.empty(T, np.float32)
+    off = np.empty(T + 1, np.uint32)
+    cap = T * D + 16
+    stream = np.zeros(cap, np.uint8)
+    rowptr = np.empty(T + 1, np.uint32)
+    ocap = T * D + 1
+    ch = np.empty(ocap, np.uint8)
+    val = np.empty(ocap, np.uint16)
+    n = lib().qaq_oracle_quantize(_p(x, C.c_uint16), C.c_long(T), C.c_int(D), C.c_float(lo), C.c_float(hi),
+                                  _p(bits, C.c_uint8), _p(mn, C.c_float), _p(step, C.c_float), _p(off, C.c_uint32),
+                                  _p(stream, C.c_uint8), C.c_long(cap), _p(rowptr, C.c_uint32), _p(ch, C.c_uint8),
+                                  _p(val, C.c_uint16), C.c_long(ocap))
+    assert n >= 0
+    return QuantTensor(T, D, bits.copy(), mn, step, off, stream[: int(off[T])].copy(), rowptr, ch[:n].copy(), val[:n].copy())
+
+
+def reconstruct(qt: QuantTensor) -> np.ndarray:
+    out = np.empty((qt.T, qt.D), np.float32)
+    stream = np.ascontiguousarray(qt.stream) if qt.stream.size else np.zeros(1, np.uint8)
+    ch = np.ascontiguousarray(qt.ch) if qt.ch.size else np.zeros(1, np.uint8)
+    val = np.ascontiguousarray(qt.val) if qt.val.size else np.zeros(1, np.uint16)
+    bits = np.ascontiguousarray(qt.bits); mn = np.ascontiguousarray(qt.mn); step = np.ascontiguousarray(qt.step)
+    off = np.ascontiguousarray(qt.off); rowptr = np.ascontiguousarray(qt.rowptr)
+    lib().qaq_oracle_reconstruct(C.c_long(qt.T), C.c_int(qt.D), _p(bits, C.c_uint8), _p(mn, C.c_float),
+                                 _p(step, C.c_float), _p(off, C.c_uint32), _p(stream, C.c_uint8),
+                                 _p(rowptr, C.c_uint32), _p(ch, C.c_uint8), _p(val, C.c_uint16), _p(out, C.c_float))
+    return out
+
+
+def attention_dense(q_u16, Khat, Vhat, scale):
+    q = np.ascontiguousarray(q_u16, dtype=np.uint16)
+    Khat = np.ascontiguousarray(Khat, dtype=np.float32)
+    Vhat = np.ascontiguousarray(Vhat, dtype=np.float32)
+    T, D = Khat.shape
+    X = np.empty(D, np.float64)
+    S = np.empty(T, np.float64)
+    lib().qaq_oracle_attention_dense(_p(q, C.c_uint16), _p(Khat, C.c_float), _p(Vhat, C.c_float), C.c_long(T), C.c_int(D),
+                                     C.c_double(scale), _p(X, C.c_double), _p(S, C.c_double))
+    return X, S
+
+
+def attention_fp16(q_u16, K_u16, V_u16, scale):
+    q = np.ascontiguousarray(q_u16, dtype=np.uint16)
+    K = np.ascontiguousarray(K_u16, dtype=np.uint16)
+    V = np.ascontiguousarray(V_u16, dtype=np.uint16)
+    T, D = K.shape
+    X = np.empty(D, np.float64)
+    S = np.empty(T, np.float64)
+    lib().qaq_oracle_attention_fp16(_p(q, C.c_uint16), _p(K, C.c_uint16), _p(V, C.c_uint16), C.c_long(T), C.c_int(D),
+                                    C.c_double(scale), _p(X, C.c_double), _p(S, C.c_double))
+    return X, S
+
+
+def decode(q_u16, qk: QuantTensor, qv: QuantTensor, scale):
+    return attention_dense(q_u16, reconstruct(qk), reconstruct(qv), scale)
+
+
+def code_bits(bits, D) -> float:
+    bits = np.ascontiguousarray(bits, dtype=np.uint8)
+    return float(lib().qaq_oracle_code_bits(_p(bits, C.c_uint8), C.c_long(bits.size), C.c_int(D)))
+
+
+def cr_paper(cbk, cbv, nok, nov, T, D) -> float:
+    return float(lib().qaq_oracle_cr_paper(cbk, cbv, nok, nov, T, D))
+
+
+# ---------------------------------------------------------------------------------
+# batch runner (all (b,h) of one layer), optionally threaded
+# ---------------------------------------------------------------------------------
+class _Batch(C.Structure):
+    _fields_ = [
+        ("BH", C.c_long), ("T", C.c_long), ("D", C.c_int), ("W", C.c_int), ("bmin", C.c_int), ("bmax", C.c_int),
+        ("alpha", C.c_double), ("scale", C.c_double), ("cK", C.c_float), ("cV", C.c_float),
+        ("use_given_thr", C.c_int), ("use_given_bits", C.c_int), ("run_decode", C.c_int),
+        ("K", C.c_void_p), ("V", C.c_void_p), ("q", C.c_void_p), ("ring", C.c_void_p), ("nvalid", C.c_void_p),
+        ("thr", C.c_void_p), ("bitsK", C.c_void_p), ("bitsV", C.c_void_p),
+        ("mnK", C.c_void_p), ("stepK", C.c_void_p), ("mnV", C.c_void_p), ("stepV", C.c_void_p),
+        ("offK", C.c_void_p), ("offV", C.c_void_p), ("rowptrK", C.c_void_p), ("rowptrV", C.c_void_p),
+        ("streamK", C.c_void_p), ("streamV", C.c_void_p), ("stream_cap", C.c_long),
+        ("chK", C.c_void_p), ("chV", C.c_void_p), ("valK", C.c_void_p), ("valV", C.c_void_p), ("out_cap", C.c_long),
+        ("noutK", C.c_void_p), ("noutV", C.c_void_p), ("X", C.c_void_p), ("S", C.c_void_p),
+    ]
+
+
+@dataclass
+class BatchResult:
+    thr: np.ndarray
+    bitsK: np.ndarray
+    bitsV: np.ndarray
+    K: list   # QuantTensor per (b,h)
+    V: list
+    X: np.ndarray   # [BH, D] float64 (None when decode was skipped)
+    S: np.ndarray   # [BH, T] float64
+    threads: int
+
+
+def run_batch(K, V, q, ring, nvalid, *, alpha, cK, cV, bmin, bmax, scale, thr=None, bitsK=None, bitsV=None,
+              run_decode=True, n_threads=1, out_cap=None, want_scores=True, materialize=True) -> BatchResult:
+    """K, V: [BH, T, D] uint16; q: [BH, D] uint16; ring: [BH, W, T] f32; nvalid: [BH, T] u8."""
+    K = np.ascontiguousarray(K, dtype=np.uint16)
+    V = np.ascontiguousarray(V, dtype=np.uint16)
+    BH, T, D = K.shape
+    q = np.ascontiguousarray(q, dtype=np.uint16)
+    ring = np.ascontiguousarray(ring, dtype=np.float32)
+    nvalid = np.ascontiguousarray(nvalid, dtype=np.uint8)
+    W = ring.shape[1]
+    given_thr = thr is not None
+    thr_a = np.ascontiguousarray(thr, dtype=np.float32).reshape(BH, 4).copy() if given_thr else np.zeros((BH, 4), np.float32)
+    given_bits = bitsK is not None
+    bK = np.ascontiguousarray(bitsK, dtype=np.uint8).reshape(BH, T).copy() if given_bits else np.zeros((BH, T), np.uint8)
+    bV = np.ascontiguousarray(bitsV, dtype=np.uint8).reshape(BH, T).copy() if given_bits else np.zeros((BH, T), np.uint8)
+    scap = T * D + 16
+    ocap = out_cap if out_cap is not None else max(64, T * D // 4)
+    f32 = lambda: np.empty((BH, T), np.float32)
+    u32 = lambda: np.empty((BH, T + 1), np.uint32)
+    mnK, stepK, mnV, stepV = f32(), f32(), f32(), f32()
+    offK, offV, rpK, rpV = u32(), u32(), u32(), u32()
+    sK = np.zeros((BH, scap), np.uint8)
+    sV = np.zeros((BH, scap), np.uint8)
+    chK = np.empty((BH, ocap), np.uint8); chV = np.empty((BH, ocap), np.uint8)
+    vK = np.empty((BH, ocap), np.uint16); vV = np.empty((BH, ocap), np.uint16)
+    noK = np.zeros(BH, np.int64); noV = np.zeros(BH, np.int64)
+    X = np.zeros((BH, D), np.float64)
+    S = np.zeros((BH, T), np.float64) if want_scores else None
+    vp = lambda a: None if a is None else a.ctypes.data
+    b = _Batch(BH, T, D, W, bmin, bmax, float(alpha), float(scale), float(cK), float(cV),
+               int(given_thr), int(given_bits), int(run_decode),
+               vp(K), vp(V), vp(q), vp(ring), vp(nvalid), vp(thr_a), vp(bK), vp(bV),
+               vp(mnK), vp(stepK), vp(mnV), vp(stepV), vp(offK), vp(offV), vp(rpK), vp(rpV),
+               vp(sK), vp(sV), scap, vp(chK), vp(chV), vp(vK), vp(vV), ocap, vp(noK), vp(noV), vp(X), vp(S))
+    used = lib().qaq_oracle_run_batch(C.byref(b), C.c_int(n_threads))
+    assert (noK >= 0).all() and (noV >= 0).all(), "oracle outlier capacity too small"
+    Ks, Vs = [], []
+    if materialize:
+        for i in range(BH):
+            Ks.append(QuantTensor(T, D, bK[i], mnK[i], stepK[i], offK[i], sK[i, : int(offK[i, T])], rpK[i],
+                                  chK[i, : noK[i]], vK[i, : noK[i]]))
+            Vs.append(QuantTensor(T, D, bV[i], mnV[i], stepV[i], offV[i], sV[i, : int(offV[i, T])], rpV[i],
+                                  chV[i, : noV[i]], vV[i, : noV[i]]))
+    return BatchResult(thr_a, bK, bV, Ks, Vs, X if run_decode else None, S if run_decode else None, used)
