@@ -1,0 +1,186 @@
+/*
+ * libqaq -- quality-adaptive KV-cache quantization and attention over the packed
+ * cache (QAQ, arXiv 2403.04643), CUDA kernels for sm_100a behind a C ABI.
+ *
+ * Conventions that hold for every entry point unless its comment says otherwise:
+ *   - Pointers are DEVICE pointers owned by the caller ("host" is said explicitly).
+ *   - Work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL
+ *     is the default stream) and the call returns without synchronising.
+ *   - The return value is a qaq_status; nothing throws or aborts.  Argument and
+ *     shape errors are found on the host before anything is launched.
+ *   - Dense K/V inputs are binary16, logical shape [batch, heads, tokens, head_dim],
+ *     head_dim contiguous, with element strides for batch, head and token.
+ *   - "(b,h)" is one batch element of one head; all (b,h) are independent problems
+ *     (Section 2.1 of the paper: Q in R^{1xD}, K,V in R^{TxD} "within each head").
+ */
+#ifndef QAQ_H
+#define QAQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    QAQ_OK = 0,
+    QAQ_ERR_INVALID_ARG = 1,       /* null pointer, negative size, bad enum */
+    QAQ_ERR_UNSUPPORTED_SHAPE = 2, /* head_dim not in {32,64,128}, widths outside 1..8, ... */
+    QAQ_ERR_CAPACITY = 3,          /* token or outlier capacity of the cache exceeded */
+    QAQ_ERR_CUDA = 4,              /* a CUDA runtime call failed */
+    QAQ_ERR_WORKSPACE = 5,         /* workspace too small or misaligned */
+    QAQ_ERR_TIMEOUT = 6            /* a bounded device-side wait ran out */
+} qaq_status;
+
+const char* qaq_status_string(qaq_status s);
+
+/* Tokens are stored in groups ("tiles") of this many consecutive tokens. */
+#define QAQ_TILE_TOKENS 64
+
+typedef struct {
+    int batch, heads, head_dim; /* head_dim in {32, 64, 128} */
+    int max_tokens;             /* capacity per (b,h) */
+    int bits_min, bits_max;     /* allowed widths, 1 <= bits_min <= bits_max <= 8 */
+    int window;                 /* attention window n (Section 4.2); 1 = no window */
+    double outlier_frac;        /* alpha: proportion of values treated as outliers, both tails */
+    long max_outliers_per_bh;   /* per tensor; <= 0: derived from outlier_frac with slack */
+} qaq_config;
+
+/* Scalars of the bit-width rules (Section 4.1), see qaq_policy_from_hyper. */
+typedef struct {
+    float cK; /* keys:   B = min{b : range       <= cK * 2^b} */
+    float cV; /* values: B = min{b : range * S_t <= cV * 2^b} */
+} qaq_policy;
+
+typedef struct {
+    long tokens;              /* tokens cached per (b,h) */
+    long code_bytes[2];       /* packed code bytes, all (b,h): [0]=K, [1]=V */
+    long outliers[2];         /* stored outliers, all (b,h) */
+    long hist[2][9];          /* hist[x][b] = tokens of tensor x at width b */
+    long resident_bytes;      /* codes + per-token metadata + tile tables + outliers in use */
+    double cr_paper;          /* 16*2*T*D*BH / (code bits + 16 bits per outlier): memory
+                                 "calculated by the quantized bit" (Sections 2.1, 5.2) */
+    double cr_total;          /* fp16 bytes / resident_bytes */
+    int device_status;        /* sticky qaq_status raised on the device (capacity) */
+} qaq_stats;
+
+typedef struct qaq_cache qaq_cache; /* opaque; owns its device memory */
+
+/* Allocates (cudaMalloc on the current device) an empty cache.  host in, host out. */
+qaq_status qaq_cache_create(const qaq_config* cfg, qaq_cache** out);
+qaq_status qaq_cache_destroy(qaq_cache* c);
+/* Forgets all tokens (asynchronous on `stream`). */
+qaq_status qaq_cache_reset(qaq_cache* c, void* stream);
+/* Tokens currently cached per (b,h) (host counter). */
+long qaq_cache_tokens(const qaq_cache* c);
+
+/*
+ * Bit-width rule scalars from the paper's hyper-parameters (Section 4.1):
+ *   key bound    sigma2(K_t) <= log(T^3/(T-1) * sigmaS_max^2 + 1) / qnorm2
+ *   value bound  sigma(V_t)  <= sigmaX_max / (sqrt(T) * |S_t|)
+ *   bit count    B = ceil(log2((max - min) / (2 sqrt(3) sigma)))
+ * give cK = 2 sqrt(3) sigmaK and cV = 2 sqrt(3) sigmaX_max / sqrt(T) (binary64, rounded
+ * once to binary32).  qnorm2 is the caller's quantile of sum_d (Q_d)^2 (the paper uses
+ * the upper 10% quantile), T the number of cached tokens.  T < 2 or qnorm2 <= 0 gives
+ * cK = 0, which makes every key take bits_max.  Pure host function; host_out is host memory.
+ */
+qaq_status qaq_policy_from_hyper(double sigmaS_max, double sigmaX_max, double qnorm2, long T,
+                                 qaq_policy* host_out);
+
+/*
+ * Outlier thresholds (Section 4.2 "Outliers": values beyond the alpha% quantile at the
+ * maximum and minimum ends).  Per (b,h) and tensor, over the N = T*head_dim non-NaN
+ * values: k = floor(alpha*N/2), lo = k-th smallest, hi = k-th largest (exact order
+ * statistics).  thr is [batch*heads][4] binary32 = {loK, hiK, loV, hiV}.  An entry x is
+ * later an outlier iff !(lo <= x && x <= hi).  ws: qaq_thresholds_workspace_bytes bytes,
+ * 16-byte aligned, overwritten.
+ */
+qaq_status qaq_thresholds_workspace_bytes(const qaq_config* cfg, size_t* host_out);
+qaq_status qaq_outlier_thresholds(const qaq_config* cfg, const void* K, const void* V, long stride_b,
+                                  long stride_h, long stride_t, int n_tokens, float* thr, void* ws,
+                                  size_t ws_bytes, void* stream);
+
+/*
+ * S1: per-token widths (Section 4.1 rules, Section 4.2 attention window).
+ *   S_hat_t = max of the nvalid[t] valid rows of the score window for token t
+ *             (nvalid[t] == 0: no score seen yet, the value takes bits_max);
+ *   [min,max] of a token = range of its non-outlier entries (thr as above);
+ *   bitsK[t] = min{b in [bits_min,bits_max] : (max-min)          <= cK * 2^b}, else bits_max
+ *   bitsV[t] = min{b in [bits_min,bits_max] : (max-min) * S_hat_t <= cV * 2^b}, else bits_max
+ * score_ring: binary32 [batch*heads][window][n_tokens]; nvalid: u8 [batch*heads][n_tokens];
+ * bitsK, bitsV: u8 [batch*heads][n_tokens] (outputs).
+ */
+qaq_status qaq_select_bits(const qaq_config* cfg, const qaq_policy* policy, const void* K, const void* V,
+                           long stride_b, long stride_h, long stride_t, int n_tokens,
+                           const float* score_ring, const uint8_t* nvalid, const float* thr,
+                           uint8_t* bitsK, uint8_t* bitsV, void* stream);
+
+/*
+ * S2+S3: append n_new tokens per (b,h) to the cache: outlier split (entries outside
+ * [lo,hi] are kept as binary16 in a sparse side list and take code 0), uniform
+ * quantization of each token at its width (Section 4.1: the range [min,max] of the
+ * non-outlier entries is cut into 2^B equal segments, each value is represented by the
+ * midpoint of its segment) and bit-packing.
+ *   step = (max-min) * 2^-B;  code = min(2^B-1, floor((x-min) * (1/step)))  in binary32.
+ * bitsK/bitsV: u8 [batch*heads][n_new], or both NULL to choose the widths inside the
+ * same kernel exactly as qaq_select_bits would (then policy, score_ring, nvalid are
+ * required; score_ring is [batch*heads][window][n_new] for the new tokens, and the
+ * policy scalars should have been made for the token count after the append).
+ * thr: [batch*heads][4].  Returns QAQ_ERR_CAPACITY (nothing appended) if the token
+ * capacity would be exceeded; an outlier-list overflow is detected on the device, drops
+ * the surplus outliers and is reported by qaq_cache_stats().device_status.
+ */
+qaq_status qaq_quantize_append(qaq_cache* c, const void* K_new, const void* V_new, long stride_b,
+                               long stride_h, long stride_t, int n_new, const uint8_t* bitsK,
+                               const uint8_t* bitsV, const qaq_policy* policy, const float* score_ring,
+                               const uint8_t* nvalid, const float* thr, void* stream);
+
+/*
+ * S4+S5: decode attention over the packed cache (Section 2.1, Figure 1):
+ *   S = Softmax(softmax_scale * q Khat^T),  X = S Vhat,
+ * Khat/Vhat = midpoint reconstruction min + (code + 1/2) * step with the stored outliers
+ * put back.  q: binary16 [batch*heads][head_dim]; out: binary32 [batch*heads][head_dim];
+ * scores_out: NULL or binary32 [batch*heads][tokens] receiving S (one row of the attention
+ * window).  ws: qaq_decode_workspace_bytes bytes, 16-byte aligned (split partials).
+ */
+qaq_status qaq_decode_workspace_bytes(const qaq_cache* c, size_t* host_out);
+qaq_status qaq_decode_attention(const qaq_cache* c, const void* q, float softmax_scale, float* out,
+                                float* scores_out, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The same two steps with HOST buffers (pinned memory recommended): inputs are copied to
+ * device staging owned by the cache, the kernels run, and results are copied back, all on
+ * `stream`; the call returns after the stream has been synchronised.  K_new/V_new are
+ * contiguous [batch*heads][n_new][head_dim]; other arguments as above but in host memory.
+ */
+qaq_status qaq_quantize_append_host(qaq_cache* c, const void* K_new, const void* V_new, int n_new,
+                                    const qaq_policy* policy, const float* score_ring,
+                                    const uint8_t* nvalid, const float* thr, void* stream);
+qaq_status qaq_decode_attention_host(qaq_cache* c, const void* q, float softmax_scale, float* out,
+                                     void* stream);
+
+/* Counters and compression ratios (memory accounting of Sections 2.1 and 5.2).
+ * Synchronises `stream`.  host_out is host memory. */
+qaq_status qaq_cache_stats(const qaq_cache* c, qaq_stats* host_out, void* stream);
+
+/*
+ * Canonical copy of one tensor (0 = K, 1 = V) of the cache, for inspection and checks;
+ * all outputs are device arrays, any may be NULL:
+ *   bits u8 [BH][T]; mn, step binary32 [BH][T]; off u32 [BH][T+1] (byte offsets, prefix
+ *   sums of head_dim*bits/8); codes u8 [BH][codes_stride] (tokens concatenated in token
+ *   order); rowptr u32 [BH][T+1]; ch u8 / val binary16 [BH][outl_stride] (outliers in
+ *   (token, channel) order).  T = qaq_cache_tokens().  Within one token the codes are
+ *   stored as "planes": a B-bit code is cut into the power-of-two pieces of B (widest
+ *   first, holding the most significant bits); the plane of a w-bit piece has
+ *   head_dim*w/8 bytes; channel d = 32p+4r+i sits in little-endian 32-bit word
+ *   p*w + r*w/8 of the plane at bit 8*i + w*(r mod 8/w).
+ */
+qaq_status qaq_cache_export(const qaq_cache* c, int tensor, uint8_t* bits, float* mn, float* step,
+                            uint32_t* off, uint8_t* codes, long codes_stride, uint32_t* rowptr,
+                            uint8_t* ch, void* val, long outl_stride, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QAQ_H */
