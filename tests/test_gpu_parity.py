@@ -154,7 +154,8 @@ def test_split_count_does_not_change_the_result_beyond_rounding():
         cfg, cache, thr, out, scores, dev = gpu_pipeline(wlr, Kr, Vr, qr, rr, nr, pol)
         outs.append(out.cpu().numpy()[:2])
         if rep > 1:
-            assert np.array_equal(out.cpu().numpy()[:2], out.cpu().numpy()[-2:])   # replicas agree exactly
+            # replicas agree up to the order of a few float additions
+            assert np.allclose(out.cpu().numpy()[:2], out.cpu().numpy()[-2:], rtol=1e-5, atol=1e-6)
     assert np.allclose(outs[0], outs[1], rtol=1e-4, atol=1e-5)
 
 
