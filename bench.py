@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the QAQ hot path (arXiv 2403.04643) on B200.
+
+One step = one pass of the whole hot path over one synthetic LLaMA-7B-shaped KV cache
+(default workload C3: 32 layers x batch 8 x 32 heads x 4096 tokens x head_dim 128):
+per layer  outlier thresholds -> fused bit selection + outlier split + quantize + pack
+(`qaq_quantize_append`) -> decode attention over the packed cache (`qaq_decode_attention`).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload C3]
+
+Prints ONE JSON line (rank 0).  `value` = algorithmic GB/s of the whole step, summed over
+ranks (each rank holds its own batch: weak scaling, no data-path collective).
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2403_04643_b200 import synth  # noqa: E402
+
+METRIC = "QAQ quantize GB/s + packed decode-attn tokens/s, % of B200 HBM peak"
+QNORM2 = 1.16   # stand-in for the upper-10% quantile of sum_d (q_d / sqrt(D))^2 of N(0,1) queries
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    parts = [p.strip() for p in line.split(",")]
+                    if len(parts) < 6:
+                        continue
+                    try:
+                        sm.append(float(parts[0])); mx.append(float(parts[1]))
+                    except ValueError:
+                        continue
+                    for n, v in zip(names, parts[2:6]):
+                        if v.lower().startswith("active"):
+                            reasons.add(n)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+        return out
+
+
+# ----------------------------------------------------------------------------- byte accounting
+def algorithmic_bytes(wl, st, n_layers_stats=1):
+    """Per-layer algorithmic bytes of each stage from the cache statistics of one layer."""
+    BH, T, D, W = wl.bh, wl.tokens, wl.head_dim, wl.window
+    th = BH * T                                        # token-heads
+    ntile = BH * math.ceil(T / 64)
+    codes = st.code_bytes[0] + st.code_bytes[1]
+    outl = 4 * (st.outliers[0] + st.outliers[1])
+    meta = 2 * 5 * th + 2 * 16 * ntile                 # width + min/max per token and tensor; tile tables
+    fp16 = 2 * 2 * D * th
+    return {
+        "thresholds": fp16,                            # one read of K and V
+        "quantize": fp16 + (4 * W + 1) * th + codes + meta + outl,
+        "decode": codes + meta + outl + BH * D * (2 + 4),
+        "fp16": fp16,
+    }
+
+
+# ----------------------------------------------------------------------------- CPU baseline (oracle)
+def oracle_sample(wl, hyper, n_bh, threads, device):
+    """Times the oracle (thresholds + select + quantize + decode) on n_bh (b,h) of layer 0."""
+    import numpy as np
+    import oracle
+    small = synth.scaled(wl, batch=1, heads=n_bh, layers=1)
+    K, V = synth.make_kv(small, 0, device=device)
+    q = synth.make_query(small, 0, device=device)
+    ring, nv = synth.make_score_ring(small, 0, device=device)
+    u16 = lambda t: t.cpu().contiguous().numpy().view(np.uint16)
+    T, D = wl.tokens, wl.head_dim
+    cK, cV = oracle.policy(hyper[0], hyper[1], hyper[2], T)
+    args = (u16(K).reshape(n_bh, T, D), u16(V).reshape(n_bh, T, D), u16(q).reshape(n_bh, D),
+            ring.cpu().numpy().reshape(n_bh, wl.window, T), nv.cpu().numpy().reshape(n_bh, T))
+    kw = dict(alpha=wl.alpha, cK=cK, cV=cV, bmin=wl.bits_min, bmax=wl.bits_max, scale=1.0 / math.sqrt(D),
+              n_threads=threads, out_cap=max(1024, T * D // 2), want_scores=False, materialize=False)
+
+    def run():
+        t0 = time.perf_counter()
+        r = oracle.run_batch(*args, **kw)
+        return time.perf_counter() - t0, r
+    return run
+
+
+def per_th_bytes(wl, mean_bits=(4.0, 3.0)):
+    """Algorithmic bytes per token-head of the whole step at nominal widths (for the oracle's GB/s)."""
+    D, W = wl.head_dim, wl.window
+    codes = D * (mean_bits[0] + mean_bits[1]) / 8
+    outl = 2 * wl.alpha * D * 4
+    fp16 = 4 * D
+    return fp16 + (fp16 + 4 * W + 1 + codes + 10 + outl) + (codes + 10 + outl)
+
+
+# ----------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C3", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (0 = the workload's)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = synth.CONFIGS[args.workload]
+    if args.layers > 0:
+        wl = synth.scaled(wl, layers=args.layers)
+    hyper_qn = QNORM2
+    peak, peak_kind = measured_peaks()
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        return reference_arm(args, wl, hyper_qn)
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    from paper_2403_04643_b200 import qaq
+    from paper_2403_04643_b200.calibrate import calibrate
+    qaq.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    BH, T, D, W, L = wl.bh, wl.tokens, wl.head_dim, wl.window, wl.layers
+    scale = 1.0 / math.sqrt(D)
+    cfg = qaq.make_config(wl.batch, wl.heads, D, T, wl.bits_min, wl.bits_max, W, wl.alpha)
+    # ---- resident inputs (each rank its own batch: seed offset by rank)
+    wl_r = synth.scaled(wl, seed=wl.seed + 7777 * rank)
+    layers = []
+    for l in range(L):
+        K, V = synth.make_kv(wl_r, l, device=dev)
+        q = synth.make_query(wl_r, l, device=dev)
+        ring, nv = synth.make_score_ring(wl_r, l, device=dev)
+        layers.append(dict(K=K, V=V, q=q, ring=ring, nv=nv, cache=qaq.Cache(cfg),
+                           thr=torch.empty((BH, 4), dtype=torch.float32, device=dev),
+                           out=torch.empty((BH, D), dtype=torch.float32, device=dev)))
+    torch.cuda.synchronize()
+    # ---- hyper-parameters: calibrated once on layer 0 (mean widths ~4 / ~3)
+    L0 = layers[0]
+    qaq.qaq_outlier_thresholds(cfg, L0["K"], L0["V"], L0["thr"])
+    sS, sX, pol = calibrate(cfg, L0["K"], L0["V"], L0["ring"], L0["nv"], L0["thr"], T, hyper_qn)
+
+    def step(timers=None):
+        for Ly in layers:
+            c = Ly["cache"]
+            c.reset()
+            if timers: timers["thr"][0].append(ev())
+            qaq.qaq_outlier_thresholds(cfg, Ly["K"], Ly["V"], Ly["thr"])
+            if timers: timers["thr"][1].append(ev()); timers["quant"][0].append(timers["thr"][1][-1])
+            qaq.qaq_quantize_append(c, Ly["K"], Ly["V"], Ly["thr"], policy=pol, ring=Ly["ring"], nvalid=Ly["nv"])
+            if timers: timers["quant"][1].append(ev()); timers["dec"][0].append(timers["quant"][1][-1])
+            qaq.qaq_decode_attention(c, Ly["q"], scale, out=Ly["out"])
+            if timers: timers["dec"][1].append(ev())
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        return e
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    timers = {"thr": ([], []), "quant": ([], []), "dec": ([], [])}
+    e0 = ev()
+    for _ in range(args.steps):
+        step(timers)
+    e1 = ev()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    stage_ms = {k: sum(a.elapsed_time(b) for a, b in zip(*v)) / len(v[0]) for k, v in timers.items()}
+
+    st = qaq.qaq_cache_stats(layers[0]["cache"])
+    assert st.device_status == 0
+    ab = algorithmic_bytes(wl, st)
+    step_bytes = L * (ab["thresholds"] + ab["quantize"] + ab["decode"])
+    value = world * step_bytes / (ms_step * 1e-3) / 1e9
+    quant_gbs = ab["quantize"] / (stage_ms["quant"] * 1e-3) / 1e9
+    dec_gbs = ab["decode"] / (stage_ms["dec"] * 1e-3) / 1e9
+    thr_gbs = ab["thresholds"] / (stage_ms["thr"] * 1e-3) / 1e9
+
+    out = {
+        "metric": METRIC, "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "layers": L, "batch": wl.batch, "heads": wl.heads, "head_dim": D, "tokens": T,
+                   "window": W, "alpha": wl.alpha, "widths": [wl.bits_min, wl.bits_max],
+                   "sigmaS_max": sS, "sigmaX_max": sX, "mean_bits": [round(st.code_bytes[0] * 8 / (BH * T * D), 3),
+                                                                     round(st.code_bytes[1] * 8 / (BH * T * D), 3)],
+                   "cr_paper": round(st.cr_paper, 3), "cr_total": round(st.cr_total, 3),
+                   "l2": "each layer's inputs (>0.5 GB) and packed cache exceed L2; no flush needed",
+                   "per_rank": "own batch, no collective"},
+        "stages": {
+            "thresholds": {"ms_per_layer": round(stage_ms["thr"], 4), "gbs": round(thr_gbs, 1), "frac_of_hbm": round(thr_gbs / peak, 3)},
+            "quantize": {"ms_per_layer": round(stage_ms["quant"], 4), "gbs": round(quant_gbs, 1), "frac_of_hbm": round(quant_gbs / peak, 3),
+                         "fp16_input_gbs": round(ab["fp16"] / (stage_ms["quant"] * 1e-3) / 1e9, 1)},
+            "decode": {"ms_per_layer": round(stage_ms["dec"], 4), "gbs": round(dec_gbs, 1), "frac_of_hbm": round(dec_gbs / peak, 3),
+                       "cached_tokens_per_s": round(wl.batch * T / (stage_ms["dec"] * 1e-3), 1),
+                       "generated_tokens_per_s": round(wl.batch / (L * stage_ms["dec"] * 1e-3), 2)},
+        },
+        "roofline": {"kernel": "quant_kernel (fused select + outlier split + quantize + pack)", "bound": "hbm",
+                     "achieved": round(quant_gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(quant_gbs / peak, 3),
+                     "traffic": None, "peak_kind": peak_kind, "bytes_per_launch": ab["quantize"]},
+        "roofline_decode": {"kernel": "decode_kernel (+ merge)", "bound": "hbm", "achieved": round(dec_gbs, 1), "peak": peak,
+                            "unit": "GB/s", "frac": round(dec_gbs / peak, 3), "traffic": None, "peak_kind": peak_kind,
+                            "bytes_per_launch": ab["decode"]},
+        "gpu_launches": args.steps * L * 6,
+        "clocks": clocks,
+    }
+
+    # ---- end to end through the host-buffer C-ABI entry points (pinned host memory, copies in the timed region)
+    if not args.no_e2e:
+        Ly = layers[0]
+        pin = lambda t: t.cpu().contiguous().pin_memory()
+        hK, hV, hq, hr, hn, ht = pin(Ly["K"]), pin(Ly["V"]), pin(Ly["q"]), pin(Ly["ring"]), pin(Ly["nv"]), pin(Ly["thr"])
+        hout = torch.empty((BH, D), dtype=torch.float32).pin_memory()
+        n_e2e = max(1, min(args.steps, 2))
+
+        def e2e_step():
+            for Lz in layers:      # every layer gets the bytes of a full layer from the host
+                Lz["cache"].reset()
+                qaq.qaq_quantize_append_host(Lz["cache"], hK, hV, pol, hr, hn, ht)
+                qaq.qaq_decode_attention_host(Lz["cache"], hq, scale, hout)
+        e2e_step()
+        barrier()
+        a = ev()
+        for _ in range(n_e2e):
+            e2e_step()
+        b = ev()
+        barrier()
+        ms_e2e = a.elapsed_time(b) / n_e2e
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        h2d = L * (hK.numel() * 2 * 2 + hr.numel() * 4 + hn.numel() + ht.numel() * 4 + hq.numel() * 2)
+        e2e_bytes = L * (ab["quantize"] + ab["decode"])
+        out["e2e"] = {"value": round(world * e2e_bytes / (ms_e2e * 1e-3) / 1e9, 2), "unit": "GB/s",
+                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": L * hout.numel() * 4, "ms_per_step": round(ms_e2e, 3),
+                      "steps": n_e2e, "note": "quantize_append_host + decode_attention_host per layer; thresholds resident"}
+
+    # ---- CPU oracle beside it (rank 0, N = 1 only): a bounded sample of the same workload
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(wl, (sS, sX, hyper_qn))
+
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
+def cpu_baseline(wl, hyper, budget_s=20.0):
+    cores = os.cpu_count() or 1
+    n_bh = min(wl.bh, 16 * cores)
+    run = oracle_sample(wl, hyper, n_bh, cores, "cpu")
+    dt, r = run()
+    reps = 1
+    total = dt
+    while total + dt < budget_s and reps < 4:
+        d2, r = run()
+        total += d2
+        reps += 1
+    sec = total / reps
+    gbs = n_bh * wl.tokens * per_th_bytes(wl) / sec / 1e9
+    return {"value": round(gbs, 4), "unit": "GB/s", "cores": int(r.threads), "kind": "oracle",
+            "sample": f"{n_bh} of {wl.bh} (b,h) of layer 0 ({wl.tokens} tokens each): thresholds + select + quantize + decode, "
+                      f"{reps} repetition(s), {sec:.2f} s each; bytes at nominal widths (4,3)",
+            "cached_tokens_per_s": round(n_bh * wl.tokens / wl.heads / sec, 1)}
+
+
+def reference_arm(args, wl, hyper_qn):
+    """The oracle as the reference arm: every step is a bounded sample of the workload."""
+    cores = os.cpu_count() or 1
+    hyper = (0.002, 0.01, hyper_qn)
+    n_bh = min(wl.bh, 16 * cores)
+    run = oracle_sample(wl, hyper, n_bh, cores, "cpu")
+    for _ in range(min(args.warmup, 1)):
+        run()
+    ts = []
+    threads = cores
+    for _ in range(max(1, min(args.steps, 5))):
+        dt, r = run()
+        ts.append(dt)
+        threads = r.threads
+    sec = sum(ts) / len(ts)
+    gbs = n_bh * wl.tokens * per_th_bytes(wl) / sec / 1e9
+    sample = f"{n_bh} of {wl.bh} (b,h) of one layer per step ({wl.tokens} tokens each), {len(ts)} timed step(s)"
+    out = {"impl": "reference", "metric": METRIC, "value": round(gbs, 4), "unit": "GB/s", "n_gpus": args.gpus,
+           "steps": len(ts), "warmup": min(args.warmup, 1), "ms_per_step": round(sec * 1e3, 2), "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+           "config": {"workload": wl.name, "layers": wl.layers, "batch": wl.batch, "heads": wl.heads, "head_dim": wl.head_dim,
+                      "tokens": wl.tokens, "window": wl.window, "alpha": wl.alpha},
+           "cpu_baseline": {"value": round(gbs, 4), "unit": "GB/s", "cores": int(threads), "kind": "oracle", "sample": sample},
+           "e2e": {"value": round(gbs, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
