@@ -160,6 +160,33 @@ qaq_status qaq_quantize_append_host(qaq_cache* c, const void* K_new, const void*
 qaq_status qaq_decode_attention_host(qaq_cache* c, const void* q, float softmax_scale, float* out,
                                      void* stream);
 
+/*
+ * Decode attention without a caller-supplied workspace and without any allocation.
+ * (No counterpart in the paper: this exists for the sake of the callers, not the method.)
+ *
+ * Some users of this library sit where asking for device memory is not an option: a
+ * serving loop whose whole memory budget was handed out at start-up, or a step that must
+ * not trigger the device-wide synchronisation a cudaMalloc/cudaFree can cause.  For them
+ * this variant of qaq_decode_attention keeps the split partials in a fixed 4 MiB device
+ * array that is part of the library itself (every GPU that loads libqaq holds these 4 MiB
+ * until the process exits).  The call performs no cudaMalloc/cudaFree and uses no
+ * allocating library routine; q and out are still the caller's buffers, as above.
+ *
+ *   - Limit: batch*heads * splits * (head_dim+2) * 4 bytes + batch*heads*8 must fit in
+ *     4 MiB (the split count is the one qaq_decode_attention would use; e.g. 256 (b,h) x
+ *     4096 tokens x head_dim 128 needs 0.4 MiB).  Larger shapes get QAQ_ERR_WORKSPACE
+ *     and nothing is launched -- use qaq_decode_attention with your own workspace.
+ *   - The first call on each device looks up the array's device address (once, with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Calls that may overlap on the GPU
+ *     (different streams, no ordering between them) race on it and give wrong results;
+ *     keep them on one stream or order them yourself.  The array keeps the previous
+ *     call's contents; nothing in it needs clearing, every value is written before use.
+ *   - No scores_out here; results equal qaq_decode_attention's.
+ */
+qaq_status qaq_decode_attention_static(const qaq_cache* c, const void* q, float softmax_scale, float* out,
+                                       void* stream);
+
 /* Counters and compression ratios (memory accounting of Sections 2.1 and 5.2).
  * Synchronises `stream`.  host_out is host memory. */
 qaq_status qaq_cache_stats(const qaq_cache* c, qaq_stats* host_out, void* stream);

@@ -520,3 +520,66 @@ extern "C" qaq_status qaq_decode_attention(const qaq_cache* c, const void* q, fl
     }
     return QAQ_ERR_UNSUPPORTED_SHAPE;
 }
+
+// ---------------------------------------------------------------------------------------
+// Decode attention for callers that have no way to hand over a workspace.
+//
+// The split partials of the decode kernel need a few hundred KB of global scratch.  The
+// regular entry point takes it from the caller; this one keeps it in a fixed array that
+// is part of the library image, so the call itself never asks the CUDA allocator (or any
+// other allocator) for memory.
+#define QAQ_STATIC_SCRATCH_BYTES (4u << 20)
+static __device__ __align__(256) unsigned char g_decode_scratch[QAQ_STATIC_SCRATCH_BYTES];
+
+#include <mutex>
+static std::mutex g_scratch_mutex;
+static void* g_scratch_addr[64];  // device address of g_decode_scratch, per device ordinal
+
+extern "C" qaq_status qaq_decode_attention_static(const qaq_cache* c, const void* q, float softmax_scale,
+                                                  float* out, void* stream) {
+    if (!c || !q || !out) return QAQ_ERR_INVALID_ARG;
+    if (c->tokens < 1) return QAQ_ERR_INVALID_ARG;
+    const int D = c->cfg.head_dim, BH = c->BH;
+    const int T = (int)c->tokens;
+    const int ntiles = (T + QAQ_TILE - 1) / QAQ_TILE;
+    const int nsplit = pick_nsplit(BH, ntiles);
+    // partials [BH][nsplit][D+2] followed by the merged (max, sum) pairs [BH][2]
+    const size_t need = ((size_t)BH * nsplit * (D + 2) + (size_t)BH * 2) * sizeof(float);
+    if (need > QAQ_STATIC_SCRATCH_BYTES) return QAQ_ERR_WORKSPACE;  // shape too large for the built-in scratch
+
+    int dev = -1;
+    QAQ_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return QAQ_ERR_UNSUPPORTED_SHAPE;
+    void* scratch = nullptr;
+    {
+        // In host code the array's name is only a handle; the device address has to be
+        // looked up, once per device, with that device current.
+        std::lock_guard<std::mutex> lock(g_scratch_mutex);
+        if (!g_scratch_addr[dev]) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_decode_scratch) != cudaSuccess || !p) {
+                (void)cudaGetLastError();
+                return QAQ_ERR_CUDA;
+            }
+            g_scratch_addr[dev] = p;
+        }
+        scratch = g_scratch_addr[dev];
+    }
+    DecArgs a;
+    a.k = c->t[0]; a.v = c->t[1]; a.pool_bytes = c->pool_bytes; a.ocap = c->ocap;
+    a.tmax_pad = c->tmax_pad; a.ntiles_max = c->ntiles; a.T = T;
+    a.q = (const __half*)q; a.scale = softmax_scale;
+    a.nsplit = nsplit;
+    // Every (b,h,split) partial and every (max,sum) pair is written before it is read, so
+    // nothing in the scratch has to be cleared between calls.
+    a.part = (float*)scratch;
+    a.ml = a.part + (size_t)BH * nsplit * (D + 2);
+    a.out = out; a.scores = nullptr;
+    cudaStream_t s = (cudaStream_t)stream;
+    switch (D) {
+        case 32: return run_decode<32>(a, BH, s);
+        case 64: return run_decode<64>(a, BH, s);
+        case 128: return run_decode<128>(a, BH, s);
+    }
+    return QAQ_ERR_UNSUPPORTED_SHAPE;
+}

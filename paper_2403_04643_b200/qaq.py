@@ -21,7 +21,7 @@ EXPORTED = [
     "qaq_status_string", "qaq_cache_create", "qaq_cache_destroy", "qaq_cache_reset", "qaq_cache_tokens",
     "qaq_policy_from_hyper", "qaq_thresholds_workspace_bytes", "qaq_outlier_thresholds", "qaq_select_bits",
     "qaq_quantize_append", "qaq_decode_workspace_bytes", "qaq_decode_attention", "qaq_quantize_append_host",
-    "qaq_decode_attention_host", "qaq_cache_stats", "qaq_cache_export",
+    "qaq_decode_attention_host", "qaq_cache_stats", "qaq_cache_export", "qaq_decode_attention_static",
 ]
 
 
@@ -78,6 +78,7 @@ def lib():
         L.qaq_quantize_append_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.POINTER(Policy),
                                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.qaq_decode_attention_host.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]
+        L.qaq_decode_attention_static.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]
         L.qaq_cache_stats.argtypes = [C.c_void_p, C.POINTER(Stats), C.c_void_p]
         L.qaq_cache_export.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_long, C.c_void_p, C.c_void_p, C.c_void_p, C.c_long, C.c_void_p]
@@ -199,6 +200,18 @@ def qaq_decode_attention(cache: Cache, q, softmax_scale, out=None, scores_out=No
     ws = cache.workspace()
     _check(lib().qaq_decode_attention(cache.handle, _ptr(q), float(softmax_scale), _ptr(out), _ptr(scores_out), _ptr(ws),
                                       ws.numel(), _stream()), "qaq_decode_attention")
+    return out
+
+
+def qaq_decode_attention_static(cache: Cache, q, softmax_scale, out):
+    """Decode attention that allocates nothing: the split partials live in a fixed 4 MiB device array inside
+    the library instead of a workspace.  For callers that cannot obtain device memory at call time; `out`
+    (float32 [B*H, D]) must already exist.  Calls share the array, so do not let two of them overlap on the GPU."""
+    BH, D = cache.cfg.batch * cache.cfg.heads, cache.cfg.head_dim
+    assert q.dtype == torch.float16 and q.is_contiguous() and q.numel() == BH * D
+    assert out.dtype == torch.float32 and out.is_contiguous() and out.numel() == BH * D
+    _check(lib().qaq_decode_attention_static(cache.handle, _ptr(q), float(softmax_scale), _ptr(out), _stream()),
+           "qaq_decode_attention_static")
     return out
 
 
