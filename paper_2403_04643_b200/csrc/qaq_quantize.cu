@@ -1,14 +1,15 @@
 // S1-S3: bit-width selection, outlier split, uniform quantization and bit-packing.
 //
-// One CTA handles one tile (QAQ_TILE consecutive tokens) of one (b,h); a group of
-// head_dim/4 lanes owns one token (4 channels per lane, held in registers from the
-// min/max pass to the packing pass, so K and V are read from HBM exactly once).
-//   phase 0  thread per token: attention-window maximum of the score rows (Section 4.2)
-//   phase 1  group per token: outlier flags, min/max of the non-outliers (shuffle
-//            reductions), width ladder (Section 4.1), outlier count (ballot/popc)
+// One CTA handles one tile (QAQ_TILE consecutive tokens) of one (b,h); head_dim/32 lanes
+// own one token, each lane 32 consecutive channels of K and of V (64 bytes each), held in
+// registers from the min/max pass to the packing pass, so K and V are read from HBM once.
+//   phase 0  attention-window maximum of the score rows (Section 4.2)
+//   phase 1  outlier masks and min/max of the non-outliers in binary16 pair arithmetic
+//            (exact: the inputs are binary16), width from the exponents (Section 4.1)
 //   phase 2  warp 0: exclusive scans of byte lengths and outlier counts over the tile,
 //            space taken from the (b,h) pools by atomicAdd
-//   phase 3  group per token: codes, plane packing, stores; outlier compaction
+//   phase 3  codes (binary32: one sub, one mul, round down), planes built lane-locally,
+//            vector stores; outlier entries placed by popc ranks
 #include "qaq_internal.cuh"
 
 namespace {
@@ -39,123 +40,186 @@ struct QuantArgs {
     uint8_t* out_bitsV;
 };
 
+// B = min{b in [bmin,bmax] : v <= c * 2^b}, bmax if none; c * 2^b is an exact power-of-two
+// scaling.  For positive normal v and c the answer is read off the exponents: with
+// v = mv * 2^ev, c = mc * 2^ec (mv, mc in [1,2)) the smallest b is ev - ec if mv <= mc,
+// else ev - ec + 1.
 __device__ __forceinline__ int ladder(float v, float c, int bmin, int bmax) {
-    // B = min{b : v <= c * 2^b}; c * 2^b is exact (power-of-two scaling)
     if (!(c > 0.f)) return bmax;
-    for (int b = bmin; b <= bmax; ++b)
-        if (v <= __fmul_rn(c, (float)(1 << b))) return b;
-    return bmax;
+    if (v <= __fmul_rn(c, (float)(1 << bmin))) return bmin;
+    const int vb = __float_as_int(v), cb = __float_as_int(c);
+    if (cb < 0x00800000 || vb < 0x00800000) {  // subnormal operand: plain ladder
+        for (int b = bmin; b <= bmax; ++b)
+            if (v <= __fmul_rn(c, (float)(1 << b))) return b;
+        return bmax;
+    }
+    int b = (vb >> 23) - (cb >> 23) + (((vb & 0x7FFFFF) > (cb & 0x7FFFFF)) ? 1 : 0);
+    return b < bmin ? bmin : (b > bmax ? bmax : b);
 }
 
+__device__ __forceinline__ uint32_t lop3_sel(uint32_t a, uint32_t m, uint32_t c) {  // (a & m) | (c & ~m)
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xE2;" : "=r"(d) : "r"(a), "r"(m), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t c) {  // (a & b) | c
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+__device__ __forceinline__ __half2 as_h2(uint32_t x) { return *reinterpret_cast<__half2*>(&x); }
+__device__ __forceinline__ uint32_t as_u32(__half2 x) { return *reinterpret_cast<uint32_t*>(&x); }
+// binary32 (x - c) with x a binary16 value: one rounding, same as widening x exactly and subtracting
+__device__ __forceinline__ float sub_f32_f16(unsigned short x, float c) {
+    float d;
+    asm("sub.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
+    return d;
+}
+
+// One lane's 32 channels of one token and tensor: outlier masks, masked min / max.
+//   v[k] holds channels 2k, 2k+1 (binary16 pairs).
+//   bm[j]  : byte j' of bm[j] = 0xFF iff channel 4j+j' is NOT an outlier
+//   inl    : bit k = channel 2k is an inlier, bit 16+k = channel 2k+1 is an inlier
+__device__ __forceinline__ void analyze32(const uint32_t (&v)[16], __half2 lo2, __half2 hi2, uint32_t (&bm)[8],
+                                          uint32_t& inl, __half2& mn2, __half2& mx2) {
+    uint32_t mnacc = 0x7C007C00u, mxacc = 0xFC00FC00u, bits = 0, prev = 0;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        const __half2 x = as_h2(v[k]);
+        const uint32_t m = __hge2_mask(x, lo2) & __hle2_mask(x, hi2);
+        mnacc = as_u32(__hmin2(as_h2(mnacc), as_h2(lop3_sel(v[k], m, 0x7C007C00u))));
+        mxacc = as_u32(__hmax2(as_h2(mxacc), as_h2(lop3_sel(v[k], m, 0xFC00FC00u))));
+        bits = lop3_and_or(m, 0x00010001u << k, bits);
+        if (k & 1) bm[k >> 1] = prmt(prev, m, 0x6420u);
+        prev = m;
+    }
+    inl = bits;
+    mn2 = as_h2(mnacc);
+    mx2 = as_h2(mxacc);
+}
+
+template <int BYTES>
+__device__ __forceinline__ void store_words(uint8_t* dst, const uint32_t* w, int nwords) {
+    // nwords * 4 bytes to dst, which is BYTES-aligned (BYTES in {4, 8, 16})
+    if (BYTES == 16 && nwords % 4 == 0) {
+        for (int i = 0; i < nwords; i += 4) *reinterpret_cast<uint4*>(dst + 4 * i) = make_uint4(w[i], w[i + 1], w[i + 2], w[i + 3]);
+    } else if (BYTES >= 8 && nwords % 2 == 0) {
+        for (int i = 0; i < nwords; i += 2) *reinterpret_cast<uint2*>(dst + 4 * i) = make_uint2(w[i], w[i + 1]);
+    } else {
+        for (int i = 0; i < nwords; ++i) *reinterpret_cast<uint32_t*>(dst + 4 * i) = w[i];
+    }
+}
+
+// One CTA = one tile of 64 tokens of one (b,h); P = D/32 lanes own a token, each lane 32
+// consecutive channels (64 bytes) of K and of V, kept in registers across all phases.
 template <int D, bool SELECT_ONLY>
-__global__ void __launch_bounds__(256) quant_kernel(const QuantArgs a) {
-    constexpr int G = D / 4;         // lanes per token
-    constexpr int TPW = 32 / G;      // tokens handled concurrently by a warp
-    constexpr int NI = 8 / TPW;      // iterations: 8 token slots per warp
+__global__ void __launch_bounds__(2 * D) quant_kernel(const QuantArgs a) {
+    constexpr int P = D / 32;            // lanes per token
+    constexpr int ALIGN = D / 8 >= 16 ? 16 : D / 8;  // alignment of a token's bytes inside a tile
     const int bh = blockIdx.y;
     const int tile = a.first_tile + blockIdx.x;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = lane % G, sub = lane / G;
-    const unsigned gmask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (sub * G));
-    const unsigned lt_in_group = gmask & ((1u << lane) - 1u);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int slot = tid / P, p = tid % P;
 
-    // new-token index range of this tile
     const int abs_lo = max(tile * QAQ_TILE, a.t_old + a.tok_lo);
     const int abs_hi = min((tile + 1) * QAQ_TILE, a.t_old + a.tok_hi);
-    const int s_lo = abs_lo - tile * QAQ_TILE, s_hi = abs_hi - tile * QAQ_TILE;  // slots in the tile
+    const int s_lo = abs_lo - tile * QAQ_TILE, s_hi = abs_hi - tile * QAQ_TILE;
+    const bool valid = slot >= s_lo && slot < s_hi;
+    const int tn = tile * QAQ_TILE + slot - a.t_old;  // index among the new tokens
 
-    __shared__ float s_shat[QAQ_TILE];
-    __shared__ uint8_t s_bits[2][QAQ_TILE];
-    __shared__ float s_mn[2][QAQ_TILE], s_mx[2][QAQ_TILE];
+    __shared__ float s_part[P][QAQ_TILE];
+    __shared__ uint8_t s_nv[QAQ_TILE];
     __shared__ uint32_t s_len[2][QAQ_TILE];   // bytes, then exclusive byte offsets
     __shared__ uint32_t s_cnt[2][QAQ_TILE];   // outlier counts, then exclusive offsets
     __shared__ uint32_t s_base[2], s_obase[2], s_olimit[2];
     __shared__ int s_skip;
 
     const float* thr = a.thr + (size_t)bh * 4;
-    const float loK = thr[0], hiK = thr[1], loV = thr[2], hiV = thr[3];
     const bool given = a.bitsK != nullptr;
 
-    // ---- phase 0: attention window (max of the valid score rows of each token)
-    if (threadIdx.x < QAQ_TILE) {
-        const int slot = threadIdx.x;
-        float m = __int_as_float(0x7f800000);  // +inf: no score seen
-        if (!given && slot >= s_lo && slot < s_hi) {
-            const int tn = tile * QAQ_TILE + slot - a.t_old;
-            int nv = a.nvalid[(size_t)bh * a.n_new + tn];
-            nv = nv < a.W ? nv : a.W;
-            if (nv > 0) {
-                const float* r = a.ring + (size_t)bh * a.W * a.n_new + tn;
-                m = r[0];
-                for (int i = 1; i < nv; ++i) m = fmaxf(m, r[(size_t)i * a.n_new]);
+    // ---- loads first (independent of everything else)
+    const int b_idx = bh / a.H, h_idx = bh % a.H;
+    uint32_t vk[16], vv[16];
+    {
+        const __half* Kr = a.K + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh + (size_t)(valid ? tn : 0) * a.st + 32 * p;
+        const __half* Vr = a.V + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh + (size_t)(valid ? tn : 0) * a.st + 32 * p;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint4 x = make_uint4(0, 0, 0, 0), y = make_uint4(0, 0, 0, 0);
+            if (valid) {
+                x = *reinterpret_cast<const uint4*>(Kr + 8 * i);
+                y = *reinterpret_cast<const uint4*>(Vr + 8 * i);
             }
+            vk[4 * i] = x.x; vk[4 * i + 1] = x.y; vk[4 * i + 2] = x.z; vk[4 * i + 3] = x.w;
+            vv[4 * i] = y.x; vv[4 * i + 1] = y.y; vv[4 * i + 2] = y.z; vv[4 * i + 3] = y.w;
         }
-        s_shat[slot] = m;
-        s_len[0][slot] = 0; s_len[1][slot] = 0; s_cnt[0][slot] = 0; s_cnt[1][slot] = 0;
-        s_bits[0][slot] = 0; s_bits[1][slot] = 0;
+    }
+
+    // ---- phase 0: attention window; P threads share the rows of one token
+    {
+        const int g = tid / QAQ_TILE, tok = tid % QAQ_TILE;
+        float m = __int_as_float(0xff800000);
+        int nv = 0;
+        if (!given && tok >= s_lo && tok < s_hi) {
+            const int t2 = tile * QAQ_TILE + tok - a.t_old;
+            nv = a.nvalid[(size_t)bh * a.n_new + t2];
+            nv = nv < a.W ? nv : a.W;
+            const float* r = a.ring + (size_t)bh * a.W * a.n_new + t2;
+            for (int i = g; i < nv; i += P) m = fmaxf(m, r[(size_t)i * a.n_new]);
+        }
+        s_part[g][tok] = m;
+        if (g == 0) {
+            s_nv[tok] = (uint8_t)nv;
+            s_len[0][tok] = 0; s_len[1][tok] = 0; s_cnt[0][tok] = 0; s_cnt[1][tok] = 0;
+        }
     }
     __syncthreads();
 
-    // ---- phase 1: load, outlier flags, masked range, widths
-    const int b_idx = bh / a.H, h_idx = bh % a.H;
-    const __half* Kb = a.K + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
-    const __half* Vb = a.V + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
-    uint2 rawK[NI], rawV[NI];
+    // ---- phase 1: outlier masks, range of the rest, widths
+    uint32_t bm[2][8], inl[2];
+    float mnf[2], mxf[2];
+    int Bx[2];
 #pragma unroll
-    for (int j = 0; j < NI; ++j) {
-        const int slot = warp * 8 + j * TPW + sub;
-        const bool valid = slot >= s_lo && slot < s_hi;
-        rawK[j] = make_uint2(0, 0); rawV[j] = make_uint2(0, 0);
-        if (valid) {
-            const size_t tn = (size_t)(tile * QAQ_TILE + slot - a.t_old);
-            rawK[j] = *reinterpret_cast<const uint2*>(Kb + tn * a.st + 4 * g);
-            rawV[j] = *reinterpret_cast<const uint2*>(Vb + tn * a.st + 4 * g);
-        }
-    }
+    for (int x = 0; x < 2; ++x) {
+        // thresholds as binary16 bounds that decide exactly like the binary32 ones on binary16 data
+        const __half lo = __float2half_ru(thr[2 * x]), hi = __float2half_rd(thr[2 * x + 1]);
+        __half2 mn2, mx2;
+        analyze32(x ? vv : vk, __half2half2(lo), __half2half2(hi), bm[x], inl[x], mn2, mx2);
+        const __half lmin = __hmin(__low2half(mn2), __high2half(mn2));
+        const __half lmax = __hmax(__low2half(mx2), __high2half(mx2));
+        __half2 pk = __halves2half2(lmin, __hneg(lmax));
 #pragma unroll
-    for (int j = 0; j < NI; ++j) {
-        const int slot = warp * 8 + j * TPW + sub;
-        const bool valid = slot >= s_lo && slot < s_hi;
+        for (int o = 1; o < P; o <<= 1) pk = __hmin2(pk, as_h2(__shfl_xor_sync(0xFFFFFFFFu, as_u32(pk), o)));
+        float mn = __low2float(pk), mx = -__high2float(pk);
+        if (mn > mx) { mn = 0.f; mx = 0.f; }   // no entry inside [lo, hi]
+        uint32_t cnt = 32u - (uint32_t)__popc(inl[x]);
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
-            const uint2 raw = x ? rawV[j] : rawK[j];
-            const float lo = x ? loV : loK, hi = x ? hiV : hiK;
-            const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
-            const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
-            const float xv[4] = {f01.x, f01.y, f23.x, f23.y};
-            float mn = __int_as_float(0x7f800000), mx = __int_as_float(0xff800000);
-            unsigned cnt = 0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const bool o = !(lo <= xv[i] && xv[i] <= hi);
-                if (!o) { mn = fminf(mn, xv[i]); mx = fmaxf(mx, xv[i]); }
-                cnt += __popc(__ballot_sync(0xFFFFFFFFu, o && valid) & gmask);
-            }
-#pragma unroll
-            for (int d = 1; d < G; d <<= 1) {
-                mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, d));
-                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, d));
-            }
-            if (mn > mx) { mn = 0.f; mx = 0.f; }  // no non-outlier entry
-            int B;
-            if (given) {
-                B = valid ? (x ? a.bitsV : a.bitsK)[(size_t)bh * a.n_new + (tile * QAQ_TILE + slot - a.t_old)] : 0;
+        for (int o = 1; o < P; o <<= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
+        int B;
+        if (given) {
+            B = valid ? (x ? a.bitsV : a.bitsK)[(size_t)bh * a.n_new + tn] : 0;
+            B = B < 1 ? 1 : (B > 8 ? 8 : B);
+        } else {
+            const float r = __fsub_rn(mx, mn);
+            if (x == 0) {
+                B = ladder(r, a.cK, a.bmin, a.bmax);
             } else {
-                const float r = __fsub_rn(mx, mn);
-                if (x == 0) {
-                    B = ladder(r, a.cK, a.bmin, a.bmax);
-                } else {
-                    const float sh = s_shat[slot & (QAQ_TILE - 1)];
-                    B = isinf(sh) ? a.bmax : ladder(__fmul_rn(r, sh), a.cV, a.bmin, a.bmax);
-                }
+                float sh = __int_as_float(0xff800000);
+#pragma unroll
+                for (int g = 0; g < P; ++g) sh = fmaxf(sh, s_part[g][slot]);
+                B = (s_nv[slot] == 0) ? a.bmax : ladder(__fmul_rn(r, sh), a.cV, a.bmin, a.bmax);
             }
-            if (valid && g == 0) {
-                s_bits[x][slot] = (uint8_t)B;
-                s_mn[x][slot] = mn; s_mx[x][slot] = mx;
-                s_len[x][slot] = (uint32_t)(D * B / 8);
-                s_cnt[x][slot] = cnt;
-                if (SELECT_ONLY) (x ? a.out_bitsV : a.out_bitsK)[(size_t)bh * a.n_new + (tile * QAQ_TILE + slot - a.t_old)] = (uint8_t)B;
-            }
+        }
+        mnf[x] = mn; mxf[x] = mx; Bx[x] = B;
+        if (valid && p == 0) {
+            s_len[x][slot] = (uint32_t)(D * B / 8);
+            s_cnt[x][slot] = cnt;
+            if (SELECT_ONLY) (x ? a.out_bitsV : a.out_bitsK)[(size_t)bh * a.n_new + tn] = (uint8_t)B;
         }
     }
     if (SELECT_ONLY) return;
@@ -168,7 +232,6 @@ __global__ void __launch_bounds__(256) quant_kernel(const QuantArgs a) {
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
             const TensorStore& ts = x ? a.v : a.k;
-            // two slots per lane: (lane, lane + 32)
             uint32_t l0 = s_len[x][lane], l1 = s_len[x][lane + 32];
             uint32_t c0 = s_cnt[x][lane], c1 = s_cnt[x][lane + 32];
             uint32_t il0 = l0, il1 = l1, ic0 = c0, ic1 = c1;
@@ -185,7 +248,6 @@ __global__ void __launch_bounds__(256) quant_kernel(const QuantArgs a) {
             if (lane == 0) {
                 const uint32_t bytes = tot0 + tot1, cnt = ctot0 + ctot1;
                 const size_t ti = (size_t)bh * a.ntiles + tile;
-                // packed codes
                 uint32_t base;
                 if (whole) {
                     base = atomicAdd(&ts.pool_end[bh], (bytes + 15u) & ~15u);
@@ -200,7 +262,6 @@ __global__ void __launch_bounds__(256) quant_kernel(const QuantArgs a) {
                 if (starts) { ts.tile_off[ti] = base; ts.tile_nbytes[ti] = bytes; }
                 else ts.tile_nbytes[ti] += bytes;
                 s_base[x] = base;
-                // outliers
                 uint32_t obase;
                 if (whole) {
                     obase = atomicAdd(&ts.opool_end[bh], (cnt + 3u) & ~3u);
@@ -224,77 +285,91 @@ __global__ void __launch_bounds__(256) quant_kernel(const QuantArgs a) {
     __syncthreads();
     if (s_skip) return;
 
-    // ---- phase 3: codes, planes, stores
-    const int p = g >> 3, r = g & 7;
+    // ---- phase 3: codes, planes, stores, outlier list
 #pragma unroll
-    for (int j = 0; j < NI; ++j) {
-        const int slot = warp * 8 + j * TPW + sub;
-        const bool valid = slot >= s_lo && slot < s_hi;
-        const int sl = slot & (QAQ_TILE - 1);
+    for (int x = 0; x < 2; ++x) {
+        const TensorStore& ts = x ? a.v : a.k;
+        const uint32_t (&v)[16] = x ? vv : vk;
+        const int B = valid ? Bx[x] : 0;
+        const float mn = mnf[x], mx = mxf[x];
+        const float step = __fmul_rn(__fsub_rn(mx, mn), __int_as_float((127 - B) << 23));
+        const float inv = step > 0.f ? __fdiv_rn(1.0f, step) : 0.f;
+        const float topf = (float)((1 << B) - 1);
+        // codes of channels 4j..4j+3 in the byte lanes of creg[j]
+        uint32_t creg[8];
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
-            const TensorStore& ts = x ? a.v : a.k;
-            const uint2 raw = x ? rawV[j] : rawK[j];
-            const float lo = x ? loV : loK, hi = x ? hiV : hiK;
-            const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
-            const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
-            const float xv[4] = {f01.x, f01.y, f23.x, f23.y};
-            const unsigned short hv[4] = {(unsigned short)(raw.x & 0xFFFF), (unsigned short)(raw.x >> 16),
-                                          (unsigned short)(raw.y & 0xFFFF), (unsigned short)(raw.y >> 16)};
-            const int B = valid ? s_bits[x][sl] : 0;
-            const float mn = valid ? s_mn[x][sl] : 0.f, mx = valid ? s_mx[x][sl] : 0.f;
-            const float step = __fmul_rn(__fsub_rn(mx, mn), __int_as_float((127 - B) << 23));
-            const float inv = step > 0.f ? __fdiv_rn(1.0f, step) : 0.f;
-            const int top = (1 << B) - 1;
-            uint32_t reg = 0;
-            bool o[4];
-            unsigned bal[4];
+        for (int j = 0; j < 8; ++j) {
+            uint32_t f[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                o[i] = !(lo <= xv[i] && xv[i] <= hi);
-                int c = 0;
-                if (!o[i]) {
-                    c = __float2int_rd(__fmul_rn(__fsub_rn(xv[i], mn), inv));
-                    c = c > top ? top : c;
-                    c = c < 0 ? 0 : c;
-                }
-                reg |= (uint32_t)c << (8 * i);
-                bal[i] = __ballot_sync(0xFFFFFFFFu, o[i] && valid);
+                const uint32_t pair = v[2 * j + (i >> 1)];
+                const unsigned short h = (i & 1) ? (unsigned short)(pair >> 16) : (unsigned short)(pair & 0xFFFF);
+                float t = __fmul_rn(sub_f32_f16(h, mn), inv);
+                t = fminf(t, topf);
+                f[i] = __float_as_uint(__fadd_rd(t, 8388608.0f));   // 2^23 + floor(t): the code is the low byte
             }
-            // planes, widest first
-            uint8_t* tok = ts.codes + (size_t)bh * a.pool_bytes + s_base[x] + s_len[x][sl];
+            creg[j] = prmt(prmt(f[0], f[1], 0x0040u), prmt(f[2], f[3], 0x0040u), 0x5410u) & bm[x][j];
+        }
+        uint8_t* tok = ts.codes + (size_t)bh * a.pool_bytes + s_base[x] + s_len[x][slot & (QAQ_TILE - 1)];
+        if (B & 8) {
+            store_words<ALIGN>(tok + p * 32, creg, 8);
+        }
+        if (B & 4) {
+            const int sh = B & 3;
+            uint32_t w[4];
 #pragma unroll
-            for (int w = 8; w >= 1; w >>= 1) {
-                const int per = 8 / w;                 // slots per byte lane
-                const int m = r & (per - 1);
-                const int shift = B & (w - 1);
-                uint32_t word = ((reg >> shift) & (0x01010101u * ((1u << w) - 1u))) << (w * m);
+            for (int j = 0; j < 4; ++j)
+                w[j] = ((creg[2 * j] >> sh) & 0x0F0F0F0Fu) | (((creg[2 * j + 1] >> sh) & 0x0F0F0F0Fu) << 4);
+            store_words<ALIGN>(tok + (B & 8) * (D / 8) + p * 16, w, 4);
+        }
+        if (B & 2) {
+            const int sh = B & 1;
+            uint32_t w[2];
 #pragma unroll
-                for (int d = 1; d < per; d <<= 1) word |= __shfl_xor_sync(0xFFFFFFFFu, word, d);
-                if (valid && (B & w) && m == 0) {
-                    const int plane_base = (B & ~((w << 1) - 1)) * (D / 8);
-                    *reinterpret_cast<uint32_t*>(tok + plane_base + 4 * (p * w + ((r * w) >> 3))) = word;
-                }
+            for (int j = 0; j < 2; ++j) {
+                uint32_t acc = 0;
+#pragma unroll
+                for (int m = 0; m < 4; ++m) acc |= ((creg[4 * j + m] >> sh) & 0x03030303u) << (2 * m);
+                w[j] = acc;
             }
-            // outliers in (token, channel) order
-            uint32_t before = 0;
+            store_words<(ALIGN > 8 ? 8 : ALIGN)>(tok + (B & 12) * (D / 8) + p * 8, w, 2);
+        }
+        if (B & 1) {
+            uint32_t acc = 0;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) before += __popc(bal[i] & lt_in_group);
-            uint32_t pos = s_obase[x] + s_cnt[x][sl] + before;
+            for (int m = 0; m < 8; ++m) acc |= (creg[m] & 0x01010101u) << m;
+            *reinterpret_cast<uint32_t*>(tok + (B & 14) * (D / 8) + p * 4) = acc;
+        }
+        // outliers in (token, channel) order: entries of lanes p' < p come first
+        uint32_t ob = valid ? ~inl[x] : 0u;
+        const uint32_t mine = (uint32_t)__popc(ob);
+        uint32_t before = 0;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                if (o[i] && valid) {
-                    if (pos < s_olimit[x])
-                        ts.outl[(size_t)bh * a.ocap + pos] = (uint32_t)hv[i] | ((uint32_t)(4 * g + i) << 16) | ((uint32_t)sl << 24);
-                    ++pos;
-                }
+        for (int d = 1; d < P; ++d) {
+            const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, mine, d);
+            if (p >= d) before += o;
+        }
+        if (ob) {
+            const uint32_t all = ob;
+            const uint32_t pos0 = s_obase[x] + s_cnt[x][slot & (QAQ_TILE - 1)] + before;
+            const __half* row = (x ? a.V : a.K) + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh + (size_t)tn * a.st + 32 * p;
+            while (ob) {
+                const int bit = __ffs(ob) - 1;
+                ob &= ob - 1;
+                const int k = bit & 15, hi = bit >> 4;
+                const int c = 2 * k + hi;                                   // channel inside the lane's 32
+                // entries of lower channels: pairs k' < k, plus channel 2k when this is 2k+1
+                const uint32_t lower = (((1u << k) - 1u) * 0x00010001u) | (hi ? (1u << k) : 0u);
+                const uint32_t pos = pos0 + (uint32_t)__popc(all & lower);
+                if (pos < s_olimit[x])
+                    ts.outl[(size_t)bh * a.ocap + pos] = (uint32_t)__half_as_ushort(row[c]) | ((uint32_t)(32 * p + c) << 16) |
+                                                          ((uint32_t)(slot & (QAQ_TILE - 1)) << 24);
             }
-            if (valid && g == 0) {
-                const size_t t = (size_t)bh * a.tmax_pad + (size_t)tile * QAQ_TILE + sl;
-                ts.bits[t] = (uint8_t)B;
-                ts.mnmx[t] = (uint32_t)__half_as_ushort(__float2half_rn(mn)) |
-                             ((uint32_t)__half_as_ushort(__float2half_rn(mx)) << 16);
-            }
+        }
+        if (valid && p == 0) {
+            const size_t t = (size_t)bh * a.tmax_pad + (size_t)tile * QAQ_TILE + slot;
+            ts.bits[t] = (uint8_t)B;
+            ts.mnmx[t] = (uint32_t)__half_as_ushort(__float2half_rn(mn)) | ((uint32_t)__half_as_ushort(__float2half_rn(mx)) << 16);
         }
     }
 }
@@ -302,8 +377,8 @@ __global__ void __launch_bounds__(256) quant_kernel(const QuantArgs a) {
 template <bool SELECT_ONLY>
 qaq_status launch(int D, dim3 grid, const QuantArgs& a, cudaStream_t s) {
     switch (D) {
-        case 32: quant_kernel<32, SELECT_ONLY><<<grid, 256, 0, s>>>(a); break;
-        case 64: quant_kernel<64, SELECT_ONLY><<<grid, 256, 0, s>>>(a); break;
+        case 32: quant_kernel<32, SELECT_ONLY><<<grid, 64, 0, s>>>(a); break;
+        case 64: quant_kernel<64, SELECT_ONLY><<<grid, 128, 0, s>>>(a); break;
         case 128: quant_kernel<128, SELECT_ONLY><<<grid, 256, 0, s>>>(a); break;
         default: return QAQ_ERR_UNSUPPORTED_SHAPE;
     }
@@ -313,8 +388,8 @@ qaq_status launch(int D, dim3 grid, const QuantArgs& a, cudaStream_t s) {
 
 qaq_status check_dense(const void* K, const void* V, long sb, long sh, long st, int D) {
     if (!K || !V) return QAQ_ERR_INVALID_ARG;
-    if (((uintptr_t)K & 7) || ((uintptr_t)V & 7)) return QAQ_ERR_INVALID_ARG;  // 8-byte vector loads
-    if (st < D || (sb & 3) || (sh & 3) || (st & 3) || sb < 0 || sh < 0) return QAQ_ERR_INVALID_ARG;
+    if (((uintptr_t)K & 15) || ((uintptr_t)V & 15)) return QAQ_ERR_INVALID_ARG;  // 16-byte vector loads
+    if (st < D || (sb & 7) || (sh & 7) || (st & 7) || sb < 0 || sh < 0) return QAQ_ERR_INVALID_ARG;
     return QAQ_OK;
 }
 
