@@ -82,21 +82,21 @@ __device__ __forceinline__ float sub_f32_f16(unsigned short x, float c) {
 }
 
 // One lane's 32 channels of one token and tensor: outlier masks, masked min / max.
-//   v[k] holds channels 2k, 2k+1 (binary16 pairs).
-//   bm[j]  : byte j' of bm[j] = 0xFF iff channel 4j+j' is NOT an outlier
-//   inl    : bit k = channel 2k is an inlier, bit 16+k = channel 2k+1 is an inlier
-__device__ __forceinline__ void analyze32(const uint32_t (&v)[16], __half2 lo2, __half2 hi2, uint32_t (&bm)[8],
-                                          uint32_t& inl, __half2& mn2, __half2& mx2) {
-    uint32_t mnacc = 0x7C007C00u, mxacc = 0xFC00FC00u, bits = 0, prev = 0;
+//   v[k] holds channels 2k, 2k+1 (binary16 pairs).  On return every outlier entry of v has
+//   been replaced by -inf: in the code computation that yields code byte 0 without a mask
+//   (the outlier's own value is re-read from memory when its list entry is written).
+//   inl : bit k = channel 2k is an inlier, bit 16+k = channel 2k+1 is an inlier
+__device__ __forceinline__ void analyze32(uint32_t (&v)[16], __half2 lo2, __half2 hi2, uint32_t& inl, __half2& mn2,
+                                          __half2& mx2) {
+    uint32_t mnacc = 0x7C007C00u, mxacc = 0xFC00FC00u, bits = 0;
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
         const __half2 x = as_h2(v[k]);
         const uint32_t m = __hge2_mask(x, lo2) & __hle2_mask(x, hi2);
         mnacc = as_u32(__hmin2(as_h2(mnacc), as_h2(lop3_sel(v[k], m, 0x7C007C00u))));
-        mxacc = as_u32(__hmax2(as_h2(mxacc), as_h2(lop3_sel(v[k], m, 0xFC00FC00u))));
+        v[k] = lop3_sel(v[k], m, 0xFC00FC00u);
+        mxacc = as_u32(__hmax2(as_h2(mxacc), as_h2(v[k])));
         bits = lop3_and_or(m, 0x00010001u << k, bits);
-        if (k & 1) bm[k >> 1] = prmt(prev, m, 0x6420u);
-        prev = m;
     }
     inl = bits;
     mn2 = as_h2(mnacc);
@@ -118,7 +118,7 @@ __device__ __forceinline__ void store_words(uint8_t* dst, const uint32_t* w, int
 // One CTA = one tile of 64 tokens of one (b,h); P = D/32 lanes own a token, each lane 32
 // consecutive channels (64 bytes) of K and of V, kept in registers across all phases.
 template <int D, bool SELECT_ONLY>
-__global__ void __launch_bounds__(2 * D) quant_kernel(const QuantArgs a) {
+__global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const QuantArgs a) {
     constexpr int P = D / 32;            // lanes per token
     constexpr int ALIGN = D / 8 >= 16 ? 16 : D / 8;  // alignment of a token's bytes inside a tile
     const int bh = blockIdx.y;
@@ -181,7 +181,7 @@ __global__ void __launch_bounds__(2 * D) quant_kernel(const QuantArgs a) {
     __syncthreads();
 
     // ---- phase 1: outlier masks, range of the rest, widths
-    uint32_t bm[2][8], inl[2];
+    uint32_t inl[2];
     float mnf[2], mxf[2];
     int Bx[2];
 #pragma unroll
@@ -189,7 +189,7 @@ __global__ void __launch_bounds__(2 * D) quant_kernel(const QuantArgs a) {
         // thresholds as binary16 bounds that decide exactly like the binary32 ones on binary16 data
         const __half lo = __float2half_ru(thr[2 * x]), hi = __float2half_rd(thr[2 * x + 1]);
         __half2 mn2, mx2;
-        analyze32(x ? vv : vk, __half2half2(lo), __half2half2(hi), bm[x], inl[x], mn2, mx2);
+        analyze32(x ? vv : vk, __half2half2(lo), __half2half2(hi), inl[x], mn2, mx2);
         const __half lmin = __hmin(__low2half(mn2), __high2half(mn2));
         const __half lmax = __hmax(__low2half(mx2), __high2half(mx2));
         __half2 pk = __halves2half2(lmin, __hneg(lmax));
@@ -294,7 +294,8 @@ __global__ void __launch_bounds__(2 * D) quant_kernel(const QuantArgs a) {
         const float mn = mnf[x], mx = mxf[x];
         const float step = __fmul_rn(__fsub_rn(mx, mn), __int_as_float((127 - B) << 23));
         const float inv = step > 0.f ? __fdiv_rn(1.0f, step) : 0.f;
-        const float topf = (float)((1 << B) - 1);
+        // zero step (constant token): every code is 0, and -inf * 0 = NaN must not clamp to the top code
+        const float topf = step > 0.f ? (float)((1 << B) - 1) : 0.f;
         // codes of channels 4j..4j+3 in the byte lanes of creg[j]
         uint32_t creg[8];
 #pragma unroll
@@ -304,11 +305,11 @@ __global__ void __launch_bounds__(2 * D) quant_kernel(const QuantArgs a) {
             for (int i = 0; i < 4; ++i) {
                 const uint32_t pair = v[2 * j + (i >> 1)];
                 const unsigned short h = (i & 1) ? (unsigned short)(pair >> 16) : (unsigned short)(pair & 0xFFFF);
-                float t = __fmul_rn(sub_f32_f16(h, mn), inv);
+                float t = __fmul_rn(sub_f32_f16(h, mn), inv);            // -inf for an outlier
                 t = fminf(t, topf);
-                f[i] = __float_as_uint(__fadd_rd(t, 8388608.0f));   // 2^23 + floor(t): the code is the low byte
+                f[i] = __float_as_uint(__fadd_rd(t, 8388608.0f));   // 2^23 + floor(t): the code is the low byte (0 for -inf)
             }
-            creg[j] = prmt(prmt(f[0], f[1], 0x0040u), prmt(f[2], f[3], 0x0040u), 0x5410u) & bm[x][j];
+            creg[j] = prmt(prmt(f[0], f[1], 0x0040u), prmt(f[2], f[3], 0x0040u), 0x5410u);
         }
         uint8_t* tok = ts.codes + (size_t)bh * a.pool_bytes + s_base[x] + s_len[x][slot & (QAQ_TILE - 1)];
         if (B & 8) {
