@@ -14,17 +14,18 @@
 // word of codes (already one field per byte lane after a mask) feeds two dp4a.  The sums
 // are exact integers; the fixed-point error of q is below 2^-16 of max|q|.
 //
-// One CTA = one (b,h) and one split; per tile of QAQ_TILE tokens the packed bytes, the
-// metadata and the outlier entries are staged in shared memory with cp.async (two
-// buffers).  A (token, plane) pair is one work item, handled by head_dim/32 lanes; items
-// are sorted by plane width so the lanes of a warp run the same extraction code.
+// One CTA = one (b,h) and one split of its tiles; each warp works through whole tiles
+// (QAQ_TILE tokens) on its own, with its own running max / sum / accumulators and no CTA
+// barrier in the tile loop; warps are merged once at the end.  A (token, plane) pair is one
+// work item, handled by head_dim/32 lanes that read their words of the plane straight from
+// global memory (every packed byte is read once, by one lane); items are grouped by plane
+// width so that the lanes of a warp run the same extraction code.
 #include "qaq_internal.cuh"
 
 namespace {
 
-constexpr int DEC_THREADS = 256;
-constexpr int DEC_WARPS = DEC_THREADS / 32;
-constexpr int OSTAGE = 512;  // outlier entries staged per tile and tensor; the rest is read from global
+constexpr int DEC_WARPS = 4;
+constexpr int DEC_THREADS = DEC_WARPS * 32;
 
 struct DecArgs {
     TensorStore k, v;
@@ -41,14 +42,6 @@ struct DecArgs {
     float* scores;     // [BH][T] or null
 };
 
-__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
-    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
-
 __device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {  // unsigned bytes x signed bytes
     int d;
     asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
@@ -60,9 +53,30 @@ __device__ __forceinline__ int dp4a_uu(uint32_t a, uint32_t b, int c) {  // unsi
     return d;
 }
 
+// W words (4*W bytes) of a plane from global memory; the address is ALIGN-byte aligned
+template <int W, int ALIGN>
+__device__ __forceinline__ void load_words(const uint8_t* __restrict__ p, uint32_t (&w)[8]) {
+    if (ALIGN == 16 && W % 4 == 0) {
+#pragma unroll
+        for (int i = 0; i < W; i += 4) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(p + 4 * i));
+            w[i] = v.x; w[i + 1] = v.y; w[i + 2] = v.z; w[i + 3] = v.w;
+        }
+    } else if (ALIGN >= 8 && W % 2 == 0) {
+#pragma unroll
+        for (int i = 0; i < W; i += 2) {
+            const uint2 v = __ldg(reinterpret_cast<const uint2*>(p + 4 * i));
+            w[i] = v.x; w[i + 1] = v.y;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < W; ++i) w[i] = __ldg(reinterpret_cast<const uint32_t*>(p + 4 * i));
+    }
+}
+
 // integer dot product of one lane's 32 channels of a w-bit plane with q (hi/lo bytes)
 template <int W>
-__device__ __forceinline__ int plane_dot(const uint32_t* __restrict__ words, const uint32_t (&qh)[8], const uint32_t (&ql)[8]) {
+__device__ __forceinline__ int plane_dot(const uint32_t (&words)[8], const uint32_t (&qh)[8], const uint32_t (&ql)[8]) {
     constexpr int PER = 8 / W;
     constexpr uint32_t MASK = 0x01010101u * ((1u << W) - 1u);
     int ah = 0, al = 0;
@@ -81,7 +95,7 @@ __device__ __forceinline__ int plane_dot(const uint32_t* __restrict__ words, con
 
 // acc[r][i] += wt * (1 + f/2^W) for the lane's 32 channels of a w-bit plane
 template <int W>
-__device__ __forceinline__ void plane_axpy(const uint32_t* __restrict__ words, float wt, float (&acc)[8][4]) {
+__device__ __forceinline__ void plane_axpy(const uint32_t (&words)[8], float wt, float (&acc)[8][4]) {
     constexpr int PER = 8 / W;
     constexpr uint32_t MASK = ((1u << W) - 1u) << (23 - W);
 #pragma unroll
@@ -91,8 +105,6 @@ __device__ __forceinline__ void plane_axpy(const uint32_t* __restrict__ words, f
         for (int m = 0; m < PER; ++m) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                constexpr int dummy = 0;
-                (void)dummy;
                 const int pos = 8 * i + W * m;
                 const uint32_t sh = (pos + W <= 23) ? (wd << (23 - W - pos)) : (wd >> (pos + W - 23));
                 const float xf = __uint_as_float((sh & MASK) | 0x3F800000u);
@@ -102,52 +114,104 @@ __device__ __forceinline__ void plane_axpy(const uint32_t* __restrict__ words, f
     }
 }
 
+// per-warp scratch for the tile a warp is working on
 template <int D>
-struct DecSmem {
-    alignas(16) uint8_t codes[2][2][QAQ_TILE * D + 32];  // [buffer][tensor]
-    alignas(16) uint32_t outl[2][2][OSTAGE];
-    alignas(16) uint8_t bits[2][2][QAQ_TILE];
-    alignas(16) uint32_t mnmx[2][2][QAQ_TILE];
-    uint32_t table[3][8];       // per tile: off, nbytes, ooff, ocnt for K then V
-    uint32_t tokoff[2][QAQ_TILE];
+struct WarpScratch {
     float step[2][QAQ_TILE];
     float mid[2][QAQ_TILE];     // min + step/2
-    int dot[QAQ_TILE];
-    float ocorr[QAQ_TILE];
-    float logit[QAQ_TILE];
+    float ocorr[QAQ_TILE];      // sum over a token's key outliers of q_ch * (x - mid)
     float p[QAQ_TILE];
-    uint8_t item[2][3 * QAQ_TILE];  // token | class << 6, sorted by class (0:w=8 .. 3:w=1)
-    int nitem[2];
-    float qf[D];
-    float vout[D];
-    float accsum[D];
-    float red[DEC_WARPS];
-    float red2[DEC_WARPS];
-    float qscale, qsum;
+    float vout[D];              // value-outlier corrections
+    int dot[QAQ_TILE];
+    uint16_t tokoff[2][QAQ_TILE];
+    uint8_t bits[2][QAQ_TILE];
+    uint8_t item[2][3 * QAQ_TILE];  // token indices, grouped by plane width (8, 4, 2, 1)
 };
 
 template <int D>
+struct DecSmem {
+    WarpScratch<D> ws[DEC_WARPS];
+    float qf[D];
+    float macc[DEC_WARPS][D];
+    float mm[DEC_WARPS], ml[DEC_WARPS];
+    float red[DEC_WARPS], red2[DEC_WARPS];
+    float qscale, qsum;
+};
+
+// One item pass of the key side: every group of P lanes takes one (token, plane) item.
+template <int D, int W, int ALIGN>
+__device__ __forceinline__ void k_items(WarpScratch<D>& ws, const uint8_t* __restrict__ tile, int first, int n,
+                                        const uint32_t (&qh)[8], const uint32_t (&ql)[8], int part, int sub) {
+    constexpr int P = D / 32, IPW = 32 / P;
+    for (int i0 = 0; i0 < n; i0 += 2 * IPW) {
+        uint32_t w0[8], w1[8];
+        const int ia = i0 + sub, ib = i0 + IPW + sub;
+        const bool va = ia < n, vb = ib < n;
+        const int ta = va ? ws.item[0][first + ia] : 0, tb = vb ? ws.item[0][first + ib] : 0;
+        const int Ba = ws.bits[0][ta], Bb = ws.bits[0][tb];
+        if (va) load_words<W, ALIGN>(tile + ws.tokoff[0][ta] + (Ba & ~(2 * W - 1)) * (D / 8) + part * 4 * W, w0);
+        if (vb) load_words<W, ALIGN>(tile + ws.tokoff[0][tb] + (Bb & ~(2 * W - 1)) * (D / 8) + part * 4 * W, w1);
+        int da = va ? plane_dot<W>(w0, qh, ql) : 0;
+        int db = vb ? plane_dot<W>(w1, qh, ql) : 0;
+#pragma unroll
+        for (int o = 1; o < P; o <<= 1) {
+            da += __shfl_xor_sync(0xFFFFFFFFu, da, o);
+            db += __shfl_xor_sync(0xFFFFFFFFu, db, o);
+        }
+        if (part == 0) {
+            if (va) atomicAdd(&ws.dot[ta], da << (Ba & (W - 1)));
+            if (vb) atomicAdd(&ws.dot[tb], db << (Bb & (W - 1)));
+        }
+    }
+}
+
+template <int D, int W, int ALIGN>
+__device__ __forceinline__ void v_items(WarpScratch<D>& ws, const uint8_t* __restrict__ tile, int first, int n,
+                                        float (&acc)[8][4], float& offs, int part, int sub) {
+    constexpr int P = D / 32, IPW = 32 / P;
+    for (int i0 = 0; i0 < n; i0 += 2 * IPW) {
+        uint32_t w0[8], w1[8];
+        const int ia = i0 + sub, ib = i0 + IPW + sub;
+        const bool va = ia < n, vb = ib < n;
+        const int ta = va ? ws.item[1][first + ia] : 0, tb = vb ? ws.item[1][first + ib] : 0;
+        const int Ba = ws.bits[1][ta], Bb = ws.bits[1][tb];
+        if (va) load_words<W, ALIGN>(tile + ws.tokoff[1][ta] + (Ba & ~(2 * W - 1)) * (D / 8) + part * 4 * W, w0);
+        if (vb) load_words<W, ALIGN>(tile + ws.tokoff[1][tb] + (Bb & ~(2 * W - 1)) * (D / 8) + part * 4 * W, w1);
+        if (va) {   // p_t * step_t * 2^shift * f = wt * (f / 2^W)
+            const float wt = ws.p[ta] * ws.step[1][ta] * __int_as_float((127 + (Ba & (W - 1)) + W) << 23);
+            plane_axpy<W>(w0, wt, acc);
+            offs += wt;
+        }
+        if (vb) {
+            const float wt = ws.p[tb] * ws.step[1][tb] * __int_as_float((127 + (Bb & (W - 1)) + W) << 23);
+            plane_axpy<W>(w1, wt, acc);
+            offs += wt;
+        }
+    }
+}
+
+// One CTA = one (b,h) and one split of its tiles; every warp works through whole tiles on
+// its own (own running max / sum / accumulators), the warps are merged once at the end.
+template <int D>
 __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(const DecArgs a) {
     constexpr int P = D / 32;        // lanes per item
-    constexpr int IPW = 32 / P;      // items per warp pass
+    constexpr int ALIGN = D / 8 >= 16 ? 16 : D / 8;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DecSmem<D>& sm = *reinterpret_cast<DecSmem<D>*>(smem_raw);
     const int bh = blockIdx.y, split = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int part = lane % P, sub = lane / P;
+    WarpScratch<D>& ws = sm.ws[warp];
 
     const int ntiles = (a.T + QAQ_TILE - 1) / QAQ_TILE;
     const int per_split = (ntiles + a.nsplit - 1) / a.nsplit;
     const int tile_lo = split * per_split, tile_hi = min(ntiles, tile_lo + per_split);
-    const int n_my = max(0, tile_hi - tile_lo);
 
     // ---- q: float copy, fixed-point bytes per lane
     float qmax = 0.f, qs = 0.f;
     for (int d = tid; d < D; d += DEC_THREADS) {
         const float f = __half2float(a.q[(size_t)bh * D + d]);
         sm.qf[d] = f;
-        sm.vout[d] = 0.f;
-        sm.accsum[d] = 0.f;
         qmax = fmaxf(qmax, fabsf(f));
         qs += f;
     }
@@ -157,6 +221,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(const DecArgs a) {
         qs += __shfl_xor_sync(0xFFFFFFFFu, qs, o);
     }
     if (lane == 0) { sm.red[warp] = qmax; sm.red2[warp] = qs; }
+    for (int d = lane; d < D; d += 32) ws.vout[d] = 0.f;
     __syncthreads();
     if (tid == 0) {
         float m = 0.f, s = 0.f;
@@ -188,74 +253,59 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(const DecArgs a) {
         for (int i = 0; i < 4; ++i) acc[r][i] = 0.f;
     float offs = 0.f;        // sum of the weights this lane applied (the "1 +" of the magic floats)
     float m_run = __int_as_float(0xff800000), l_run = 0.f;
-    float c_run = 0.f;       // thread-per-token part of sum_t p_t (min_t + step_t/2)
+    float c_run = 0.f;       // per-lane part of sum_t p_t (min_t + step_t/2)
 
     const size_t trow = (size_t)bh * a.ntiles_max;
-    auto load_table = [&](int it) {  // it: index among my tiles
-        if (tid < 8 && it < n_my) {
-            const TensorStore& ts = (tid >= 4) ? a.v : a.k;
-            const size_t ti = trow + tile_lo + it;
-            const int f = tid & 3;
-            sm.table[it % 3][tid] = f == 0 ? ts.tile_off[ti] : f == 1 ? ts.tile_nbytes[ti] : f == 2 ? ts.tile_ooff[ti] : ts.tile_ocnt[ti];
+    const size_t mrow = (size_t)bh * a.tmax_pad;
+
+    // metadata of a tile: table entries in lanes 0..7, per-token width / min / max of tokens lane, lane + 32
+    uint32_t tbv = 0, bits4 = 0, mmv[4] = {0, 0, 0, 0};
+    auto fetch_meta = [&](int tile) {
+        if (tile < tile_hi) {
+            const size_t ti = trow + tile;
+            if (lane < 8) {
+                const TensorStore& ts = (lane >= 4) ? a.v : a.k;
+                const int f = lane & 3;
+                tbv = f == 0 ? ts.tile_off[ti] : f == 1 ? ts.tile_nbytes[ti] : f == 2 ? ts.tile_ooff[ti] : ts.tile_ocnt[ti];
+            }
+            const size_t t0 = mrow + (size_t)tile * QAQ_TILE + lane;
+            bits4 = (uint32_t)a.k.bits[t0] | ((uint32_t)a.k.bits[t0 + 32] << 8) | ((uint32_t)a.v.bits[t0] << 16) |
+                    ((uint32_t)a.v.bits[t0 + 32] << 24);
+            mmv[0] = a.k.mnmx[t0]; mmv[1] = a.k.mnmx[t0 + 32]; mmv[2] = a.v.mnmx[t0]; mmv[3] = a.v.mnmx[t0 + 32];
         }
     };
-    auto issue_tile = [&](int it) {  // cp.async of tile `it` into buffer it & 1
-        const int buf = it & 1;
-        const uint32_t* tb = sm.table[it % 3];
-        const int tile = tile_lo + it;
+    fetch_meta(tile_lo + warp);
+
+    for (int tile = tile_lo + warp; tile < tile_hi; tile += DEC_WARPS) {
+        // ---- take over the prefetched metadata, start the next tile's
+        const uint32_t offK = __shfl_sync(0xFFFFFFFFu, tbv, 0), ooK = __shfl_sync(0xFFFFFFFFu, tbv, 2), ocK = __shfl_sync(0xFFFFFFFFu, tbv, 3);
+        const uint32_t offV = __shfl_sync(0xFFFFFFFFu, tbv, 4), ooV = __shfl_sync(0xFFFFFFFFu, tbv, 6), ocV = __shfl_sync(0xFFFFFFFFu, tbv, 7);
+        const uint32_t cb4 = bits4;
+        const uint32_t cm[4] = {mmv[0], mmv[1], mmv[2], mmv[3]};
+        fetch_meta(tile + DEC_WARPS);
+
+        // ---- per-token scalars, byte offsets, item lists (tokens lane and lane + 32)
+        int ncls[2][4];
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
-            const TensorStore& ts = x ? a.v : a.k;
-            const uint8_t* src = ts.codes + (size_t)bh * a.pool_bytes + tb[4 * x + 0];
-            const int n16 = (int)((tb[4 * x + 1] + 15u) >> 4);
-            for (int i = tid; i < n16; i += DEC_THREADS) cp_async16(&sm.codes[buf][x][16 * i], src + 16 * i);
-            const uint32_t* osrc = ts.outl + (size_t)bh * a.ocap + tb[4 * x + 2];
-            const int o16 = (int)((min(tb[4 * x + 3], (uint32_t)OSTAGE) + 3u) >> 2);
-            for (int i = tid; i < o16; i += DEC_THREADS) cp_async16(&sm.outl[buf][x][4 * i], osrc + 4 * i);
-            const size_t t0 = (size_t)bh * a.tmax_pad + (size_t)tile * QAQ_TILE;
-            if (tid < QAQ_TILE / 16) cp_async16(&sm.bits[buf][x][16 * tid], ts.bits + t0 + 16 * tid);
-            if (tid >= 32 && tid < 32 + QAQ_TILE / 4) cp_async16(&sm.mnmx[buf][x][4 * (tid - 32)], ts.mnmx + t0 + 4 * (tid - 32));
-        }
-    };
-
-    load_table(0);
-    load_table(1);
-    __syncthreads();
-    if (n_my > 0) issue_tile(0);
-    cp_async_commit();
-
-    for (int it = 0; it < n_my; ++it) {
-        const int buf = it & 1;
-        const int tile = tile_lo + it;
-        if (it + 1 < n_my) issue_tile(it + 1);
-        cp_async_commit();
-        load_table(it + 2);
-        cp_async_wait<1>();
-        __syncthreads();
-        const uint32_t* tb = sm.table[it % 3];
-
-        // ---- per-token scalars, byte offsets, work items (warp 0: K, warp 1: V)
-        if (warp < 2) {
-            const int x = warp;
-            int cls_cnt_lo[4], cls_cnt_hi[4];
             uint32_t len[2];
             int Bv[2];
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const int slot = lane + 32 * e;
                 const bool valid = tile * QAQ_TILE + slot < a.T;
-                const int B = valid ? sm.bits[buf][x][slot] : 0;
+                const int B = valid ? (int)((cb4 >> (16 * x + 8 * e)) & 0xFF) : 0;
                 Bv[e] = B;
                 len[e] = (uint32_t)(D * B / 8);
-                const uint32_t mm = sm.mnmx[buf][x][slot];
-                const float mn = __half2float(__ushort_as_half((unsigned short)(mm & 0xFFFF)));
-                const float mx = __half2float(__ushort_as_half((unsigned short)(mm >> 16)));
+                const uint32_t mmw = cm[2 * x + e];
+                const float mn = __half2float(__ushort_as_half((unsigned short)(mmw & 0xFFFF)));
+                const float mx = __half2float(__ushort_as_half((unsigned short)(mmw >> 16)));
                 const float st = __fmul_rn(__fsub_rn(mx, mn), __int_as_float((127 - B) << 23));
-                sm.step[x][slot] = valid ? st : 0.f;
-                sm.mid[x][slot] = valid ? fmaf(0.5f, st, mn) : 0.f;
-                if (x == 0) { sm.dot[slot] = 0; sm.ocorr[slot] = 0.f; }
+                ws.step[x][slot] = valid ? st : 0.f;
+                ws.mid[x][slot] = valid ? fmaf(0.5f, st, mn) : 0.f;
+                ws.bits[x][slot] = (uint8_t)B;
+                if (x == 0) { ws.dot[slot] = 0; ws.ocorr[slot] = 0.f; }
             }
-            // exclusive scan of byte lengths in token order
             uint32_t i0 = len[0], i1 = len[1];
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
@@ -263,148 +313,108 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(const DecArgs a) {
                 if (lane >= d) { i0 += t0; i1 += t1; }
             }
             const uint32_t tot0 = __shfl_sync(0xFFFFFFFFu, i0, 31);
-            sm.tokoff[x][lane] = i0 - len[0];
-            sm.tokoff[x][lane + 32] = tot0 + i1 - len[1];
-            // items sorted by class: class c <-> plane width 8 >> c
+            ws.tokoff[x][lane] = (uint16_t)(i0 - len[0]);
+            ws.tokoff[x][lane + 32] = (uint16_t)(tot0 + i1 - len[1]);
             int base = 0;
+            const unsigned lt = (1u << lane) - 1u;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int w = 8 >> c;
                 const unsigned b0 = __ballot_sync(0xFFFFFFFFu, (Bv[0] & w) != 0);
                 const unsigned b1 = __ballot_sync(0xFFFFFFFFu, (Bv[1] & w) != 0);
-                const unsigned lt = (1u << lane) - 1u;
-                if (Bv[0] & w) sm.item[x][base + __popc(b0 & lt)] = (uint8_t)(lane | (c << 6));
-                if (Bv[1] & w) sm.item[x][base + __popc(b0) + __popc(b1 & lt)] = (uint8_t)((lane + 32) | (c << 6));
-                base += __popc(b0) + __popc(b1);
-                cls_cnt_lo[c] = 0; cls_cnt_hi[c] = 0;
+                if (Bv[0] & w) ws.item[x][base + __popc(b0 & lt)] = (uint8_t)lane;
+                if (Bv[1] & w) ws.item[x][base + __popc(b0) + __popc(b1 & lt)] = (uint8_t)(lane + 32);
+                ncls[x][c] = __popc(b0) + __popc(b1);
+                base += ncls[x][c];
             }
-            (void)cls_cnt_lo; (void)cls_cnt_hi;
-            if (lane == 0) sm.nitem[x] = base;
         }
-        __syncthreads();
+        __syncwarp();
 
-        // ---- K: integer dot products per (token, plane) item, outlier corrections
+        // ---- K: integer dot products per (token, plane), outlier corrections
         {
-            const int n = sm.nitem[0];
-            const uint8_t* cbuf = sm.codes[buf][0];
-            for (int base = warp * IPW; base < n; base += DEC_WARPS * IPW) {
-                const int idx = base + sub;
-                const bool valid = idx < n;
-                const int itv = valid ? sm.item[0][idx] : 0;
-                const int tok = itv & 63, cls = itv >> 6;
-                const int B = sm.bits[buf][0][tok];
-                int dot = 0, shift = 0;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (__ballot_sync(0xFFFFFFFFu, valid && cls == c) == 0) continue;
-                    if (valid && cls == c) {
-                        constexpr int dummy = 0; (void)dummy;
-                        const int w = 8 >> c;
-                        const int plane_base = (B & ~((w << 1) - 1)) * (D / 8);
-                        const uint32_t* words = reinterpret_cast<const uint32_t*>(cbuf + sm.tokoff[0][tok] + plane_base + part * 4 * w);
-                        shift = B & (w - 1);
-                        if (c == 0) dot = plane_dot<8>(words, qh, ql);
-                        else if (c == 1) dot = plane_dot<4>(words, qh, ql);
-                        else if (c == 2) dot = plane_dot<2>(words, qh, ql);
-                        else dot = plane_dot<1>(words, qh, ql);
-                    }
-                }
-#pragma unroll
-                for (int o = 1; o < P; o <<= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, o);
-                if (valid && part == 0) atomicAdd(&sm.dot[tok], dot << shift);
-            }
-            const uint32_t no = tb[3];
-            const uint32_t* og = a.k.outl + (size_t)bh * a.ocap + tb[2];
-            for (uint32_t e = tid; e < no; e += DEC_THREADS) {
-                const uint32_t v = e < OSTAGE ? sm.outl[buf][0][e] : og[e];
+            const uint8_t* tk = a.k.codes + (size_t)bh * a.pool_bytes + offK;
+            int first = 0;
+            k_items<D, 8, ALIGN>(ws, tk, first, ncls[0][0], qh, ql, part, sub); first += ncls[0][0];
+            k_items<D, 4, ALIGN>(ws, tk, first, ncls[0][1], qh, ql, part, sub); first += ncls[0][1];
+            k_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, tk, first, ncls[0][2], qh, ql, part, sub); first += ncls[0][2];
+            k_items<D, 1, 4>(ws, tk, first, ncls[0][3], qh, ql, part, sub);
+            const uint32_t* og = a.k.outl + (size_t)bh * a.ocap + ooK;
+            for (uint32_t e = lane; e < ocK; e += 32) {
+                const uint32_t v = __ldg(og + e);
                 const int tok = v >> 24, ch = (v >> 16) & 0xFF;
                 const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
-                atomicAdd(&sm.ocorr[tok], sm.qf[ch] * (val - sm.mid[0][tok]));
+                atomicAdd(&ws.ocorr[tok], sm.qf[ch] * (val - ws.mid[0][tok]));
             }
         }
-        __syncthreads();
+        __syncwarp();
 
-        // ---- logits, tile maximum
-        float logit = __int_as_float(0xff800000);
-        if (tid < QAQ_TILE) {
-            const int t = tile * QAQ_TILE + tid;
-            if (t < a.T) {
-                const float qk = fmaf(qscale * sm.step[0][tid], (float)sm.dot[tid], fmaf(sm.mid[0][tid], qsum, sm.ocorr[tid]));
-                logit = a.scale * qk;
-                if (a.scores) a.scores[(size_t)bh * a.T + t] = logit;
+        // ---- logits of tokens lane, lane + 32; running max / sum; weights
+        {
+            float lg[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int slot = lane + 32 * e;
+                const int t = tile * QAQ_TILE + slot;
+                lg[e] = __int_as_float(0xff800000);
+                if (t < a.T) {
+                    const float qk = fmaf(qscale * ws.step[0][slot], (float)ws.dot[slot], fmaf(ws.mid[0][slot], qsum, ws.ocorr[slot]));
+                    lg[e] = a.scale * qk;
+                    if (a.scores) a.scores[(size_t)bh * a.T + t] = lg[e];
+                }
             }
-            float m = logit;
+            float m = fmaxf(lg[0], lg[1]);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-            if (lane == 0) sm.red[warp] = m;
-        }
-        __syncthreads();
-        const float m_new = fmaxf(m_run, fmaxf(sm.red[0], sm.red[1]));
-        const float alpha = __expf(m_run - m_new);   // 0 on the first tile (m_run = -inf)
-        m_run = m_new;
-        if (alpha != 1.0f) {
+            const float m_new = fmaxf(m_run, m);
+            const float alpha = __expf(m_run - m_new);   // 0 on the first tile (m_run = -inf)
+            m_run = m_new;
+            if (alpha != 1.0f) {
 #pragma unroll
-            for (int r = 0; r < 8; ++r)
+                for (int r = 0; r < 8; ++r)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[r][i] *= alpha;
-            offs *= alpha;
-            c_run *= alpha;
-            for (int d = tid; d < D; d += DEC_THREADS) sm.vout[d] *= alpha;
-        }
-        if (tid < QAQ_TILE) {
-            const float p = __expf(logit - m_new);   // 0 for slots beyond T
-            sm.p[tid] = p;
-            c_run = fmaf(p, sm.mid[1][tid], c_run);
-            float s = p;
+                    for (int i = 0; i < 4; ++i) acc[r][i] *= alpha;
+                offs *= alpha;
+                c_run *= alpha;
+                for (int d = lane; d < D; d += 32) ws.vout[d] *= alpha;
+            }
+            float s = 0.f;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int slot = lane + 32 * e;
+                const float p = __expf(lg[e] - m_new);   // 0 for slots beyond T
+                ws.p[slot] = p;
+                c_run = fmaf(p, ws.mid[1][slot], c_run);
+                s += p;
+            }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-            if (lane == 0) sm.red2[warp] = s;
+            l_run = l_run * alpha + s;
         }
-        __syncthreads();
-        l_run = l_run * alpha + sm.red2[0] + sm.red2[1];
+        __syncwarp();
 
         // ---- V: weighted accumulation of raw codes, outlier corrections
         {
-            const int n = sm.nitem[1];
-            const uint8_t* cbuf = sm.codes[buf][1];
-            for (int base = warp * IPW; base < n; base += DEC_WARPS * IPW) {
-                const int idx = base + sub;
-                const bool valid = idx < n;
-                const int itv = valid ? sm.item[1][idx] : 0;
-                const int tok = itv & 63, cls = itv >> 6;
-                const int B = sm.bits[buf][1][tok];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (__ballot_sync(0xFFFFFFFFu, valid && cls == c) == 0) continue;
-                    if (valid && cls == c) {
-                        const int w = 8 >> c;
-                        const int plane_base = (B & ~((w << 1) - 1)) * (D / 8);
-                        const uint32_t* words = reinterpret_cast<const uint32_t*>(cbuf + sm.tokoff[1][tok] + plane_base + part * 4 * w);
-                        const int shift = B & (w - 1);
-                        // p_t * step_t * 2^shift * f = wt * (f / 2^w)
-                        const float wt = sm.p[tok] * sm.step[1][tok] * __int_as_float((127 + shift + w) << 23);
-                        if (c == 0) plane_axpy<8>(words, wt, acc);
-                        else if (c == 1) plane_axpy<4>(words, wt, acc);
-                        else if (c == 2) plane_axpy<2>(words, wt, acc);
-                        else plane_axpy<1>(words, wt, acc);
-                        offs += wt;
-                    }
-                }
-            }
-            const uint32_t no = tb[7];
-            const uint32_t* og = a.v.outl + (size_t)bh * a.ocap + tb[6];
-            for (uint32_t e = tid; e < no; e += DEC_THREADS) {
-                const uint32_t v = e < OSTAGE ? sm.outl[buf][1][e] : og[e];
+            const uint8_t* tv = a.v.codes + (size_t)bh * a.pool_bytes + offV;
+            int first = 0;
+            v_items<D, 8, ALIGN>(ws, tv, first, ncls[1][0], acc, offs, part, sub); first += ncls[1][0];
+            v_items<D, 4, ALIGN>(ws, tv, first, ncls[1][1], acc, offs, part, sub); first += ncls[1][1];
+            v_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, tv, first, ncls[1][2], acc, offs, part, sub); first += ncls[1][2];
+            v_items<D, 1, 4>(ws, tv, first, ncls[1][3], acc, offs, part, sub);
+            const uint32_t* og = a.v.outl + (size_t)bh * a.ocap + ooV;
+            for (uint32_t e = lane; e < ocV; e += 32) {
+                const uint32_t v = __ldg(og + e);
                 const int tok = v >> 24, ch = (v >> 16) & 0xFF;
                 const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
-                atomicAdd(&sm.vout[ch], sm.p[tok] * (val - sm.mid[1][tok]));
+                atomicAdd(&ws.vout[ch], ws.p[tok] * (val - ws.mid[1][tok]));
             }
         }
-        __syncthreads();
+        __syncwarp();
     }
-    cp_async_wait<0>();
 
-    // ---- CTA reduction: lanes with the same part over the warp, then warps through smem
+    // ---- warp result: lanes with the same part hold partial sums of the same channels
+    float cs = c_run;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cs += __shfl_xor_sync(0xFFFFFFFFu, cs, o);
 #pragma unroll
     for (int r = 0; r < 8; ++r)
 #pragma unroll
@@ -412,18 +422,29 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(const DecArgs a) {
             float v = acc[r][i] - offs;
 #pragma unroll
             for (int o = P; o < 32; o <<= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-            if (sub == 0) atomicAdd(&sm.accsum[32 * part + 4 * r + i], v);
+            if (sub == 0) sm.macc[warp][32 * part + 4 * r + i] = v + ws.vout[32 * part + 4 * r + i] + cs;
         }
-    float cs = c_run;
+    if (lane == 0) { sm.mm[warp] = m_run; sm.ml[warp] = l_run; }
+    __syncthreads();
+    // ---- merge the warps (log-sum-exp) into this split's partial
+    float M = __int_as_float(0xff800000);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) cs += __shfl_xor_sync(0xFFFFFFFFu, cs, o);
-    __syncthreads();
-    if (lane == 0) sm.red[warp] = cs;
-    __syncthreads();
-    const float cterm = sm.red[0] + sm.red[1];
+    for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, sm.mm[w]);
     float* dst = a.part + ((size_t)bh * a.nsplit + split) * (D + 2);
-    for (int d = tid; d < D; d += DEC_THREADS) dst[d] = sm.accsum[d] + sm.vout[d] + cterm;
-    if (tid == 0) { dst[D] = m_run; dst[D + 1] = l_run; }
+    float L = 0.f;
+    float wgt[DEC_WARPS];
+#pragma unroll
+    for (int w = 0; w < DEC_WARPS; ++w) {
+        wgt[w] = (sm.mm[w] == __int_as_float(0xff800000)) ? 0.f : __expf(sm.mm[w] - M);
+        L = fmaf(wgt[w], sm.ml[w], L);
+    }
+    for (int d = tid; d < D; d += DEC_THREADS) {
+        float x = 0.f;
+#pragma unroll
+        for (int w = 0; w < DEC_WARPS; ++w) x = fmaf(wgt[w], sm.macc[w][d], x);
+        dst[d] = x;
+    }
+    if (tid == 0) { dst[D] = M; dst[D + 1] = L; }
 }
 
 // log-sum-exp merge of the split partials -> X, and (max, sum) for the score row
@@ -456,9 +477,9 @@ __global__ void scores_kernel(float* scores, const float* ml, int T) {
 }
 
 int pick_nsplit(int BH, int ntiles) {
-    // enough CTAs for ~4 per SM on 148 SMs, at least 4 tiles per CTA where possible
-    int want = (148 * 4 + BH - 1) / BH;
-    int cap = ntiles / 4 > 0 ? ntiles / 4 : 1;
+    // about 16 warps per SM on 148 SMs in total (4 warps per CTA), at least one tile per warp
+    int want = (148 * 16 + 2 * BH) / (DEC_WARPS * BH);
+    int cap = ntiles / DEC_WARPS > 0 ? ntiles / DEC_WARPS : 1;
     int n = want < cap ? want : cap;
     if (n < 1) n = 1;
     if (n > 64) n = 64;
@@ -467,12 +488,9 @@ int pick_nsplit(int BH, int ntiles) {
 
 template <int D>
 qaq_status run_decode(const DecArgs& a, int BH, cudaStream_t s) {
-    static bool attr_done = false;
     const size_t smem = sizeof(DecSmem<D>);
-    if (!attr_done) {
+    if (smem > 48 * 1024)
         QAQ_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_done = true;
-    }
     decode_kernel<D><<<dim3(a.nsplit, BH), DEC_THREADS, smem, s>>>(a);
     merge_kernel<D><<<BH, D, 0, s>>>(a);
     if (a.scores) {
