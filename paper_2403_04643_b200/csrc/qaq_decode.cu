@@ -123,9 +123,10 @@ struct WarpScratch {
     float p[QAQ_TILE];
     float vout[D];              // value-outlier corrections
     int dot[QAQ_TILE];
-    uint16_t tokoff[2][QAQ_TILE];
-    uint8_t bits[2][QAQ_TILE];
-    uint8_t item[2][3 * QAQ_TILE];  // token indices, grouped by plane width (8, 4, 2, 1)
+    float wv[QAQ_TILE];         // p_t * step_t of the value side
+    // work items grouped by plane width (8, 4, 2, 1):
+    //   byte offset of the plane inside the tile | shift of the piece << 16 | token << 24
+    uint32_t item[2][3 * QAQ_TILE];
 };
 
 template <int D>
@@ -138,7 +139,7 @@ struct DecSmem {
     float qscale, qsum;
 };
 
-// One item pass of the key side: every group of P lanes takes one (token, plane) item.
+// One pass over the key-side items of one plane width: a group of P lanes per item.
 template <int D, int W, int ALIGN>
 __device__ __forceinline__ void k_items(WarpScratch<D>& ws, const uint8_t* __restrict__ tile, int first, int n,
                                         const uint32_t (&qh)[8], const uint32_t (&ql)[8], int part, int sub) {
@@ -147,10 +148,9 @@ __device__ __forceinline__ void k_items(WarpScratch<D>& ws, const uint8_t* __res
         uint32_t w0[8], w1[8];
         const int ia = i0 + sub, ib = i0 + IPW + sub;
         const bool va = ia < n, vb = ib < n;
-        const int ta = va ? ws.item[0][first + ia] : 0, tb = vb ? ws.item[0][first + ib] : 0;
-        const int Ba = ws.bits[0][ta], Bb = ws.bits[0][tb];
-        if (va) load_words<W, ALIGN>(tile + ws.tokoff[0][ta] + (Ba & ~(2 * W - 1)) * (D / 8) + part * 4 * W, w0);
-        if (vb) load_words<W, ALIGN>(tile + ws.tokoff[0][tb] + (Bb & ~(2 * W - 1)) * (D / 8) + part * 4 * W, w1);
+        const uint32_t da_ = va ? ws.item[0][first + ia] : 0u, db_ = vb ? ws.item[0][first + ib] : 0u;
+        if (va) load_words<W, ALIGN>(tile + (da_ & 0xFFFFu) + part * 4 * W, w0);
+        if (vb) load_words<W, ALIGN>(tile + (db_ & 0xFFFFu) + part * 4 * W, w1);
         int da = va ? plane_dot<W>(w0, qh, ql) : 0;
         int db = vb ? plane_dot<W>(w1, qh, ql) : 0;
 #pragma unroll
@@ -159,8 +159,8 @@ __device__ __forceinline__ void k_items(WarpScratch<D>& ws, const uint8_t* __res
             db += __shfl_xor_sync(0xFFFFFFFFu, db, o);
         }
         if (part == 0) {
-            if (va) atomicAdd(&ws.dot[ta], da << (Ba & (W - 1)));
-            if (vb) atomicAdd(&ws.dot[tb], db << (Bb & (W - 1)));
+            if (va) atomicAdd(&ws.dot[da_ >> 24], da << ((da_ >> 16) & 7));
+            if (vb) atomicAdd(&ws.dot[db_ >> 24], db << ((db_ >> 16) & 7));
         }
     }
 }
@@ -173,17 +173,16 @@ __device__ __forceinline__ void v_items(WarpScratch<D>& ws, const uint8_t* __res
         uint32_t w0[8], w1[8];
         const int ia = i0 + sub, ib = i0 + IPW + sub;
         const bool va = ia < n, vb = ib < n;
-        const int ta = va ? ws.item[1][first + ia] : 0, tb = vb ? ws.item[1][first + ib] : 0;
-        const int Ba = ws.bits[1][ta], Bb = ws.bits[1][tb];
-        if (va) load_words<W, ALIGN>(tile + ws.tokoff[1][ta] + (Ba & ~(2 * W - 1)) * (D / 8) + part * 4 * W, w0);
-        if (vb) load_words<W, ALIGN>(tile + ws.tokoff[1][tb] + (Bb & ~(2 * W - 1)) * (D / 8) + part * 4 * W, w1);
+        const uint32_t da_ = va ? ws.item[1][first + ia] : 0u, db_ = vb ? ws.item[1][first + ib] : 0u;
+        if (va) load_words<W, ALIGN>(tile + (da_ & 0xFFFFu) + part * 4 * W, w0);
+        if (vb) load_words<W, ALIGN>(tile + (db_ & 0xFFFFu) + part * 4 * W, w1);
         if (va) {   // p_t * step_t * 2^shift * f = wt * (f / 2^W)
-            const float wt = ws.p[ta] * ws.step[1][ta] * __int_as_float((127 + (Ba & (W - 1)) + W) << 23);
+            const float wt = ws.wv[da_ >> 24] * __int_as_float((127 + W) << 23) * __int_as_float((127 + ((da_ >> 16) & 7)) << 23);
             plane_axpy<W>(w0, wt, acc);
             offs += wt;
         }
         if (vb) {
-            const float wt = ws.p[tb] * ws.step[1][tb] * __int_as_float((127 + (Bb & (W - 1)) + W) << 23);
+            const float wt = ws.wv[db_ >> 24] * __int_as_float((127 + W) << 23) * __int_as_float((127 + ((db_ >> 16) & 7)) << 23);
             plane_axpy<W>(w1, wt, acc);
             offs += wt;
         }
@@ -193,7 +192,7 @@ __device__ __forceinline__ void v_items(WarpScratch<D>& ws, const uint8_t* __res
 // One CTA = one (b,h) and one split of its tiles; every warp works through whole tiles on
 // its own (own running max / sum / accumulators), the warps are merged once at the end.
 template <int D>
-__global__ void __launch_bounds__(DEC_THREADS) decode_kernel(const DecArgs a) {
+__global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a) {
     constexpr int P = D / 32;        // lanes per item
     constexpr int ALIGN = D / 8 >= 16 ? 16 : D / 8;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -258,31 +257,51 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(const DecArgs a) {
     const size_t trow = (size_t)bh * a.ntiles_max;
     const size_t mrow = (size_t)bh * a.tmax_pad;
 
-    // metadata of a tile: table entries in lanes 0..7, per-token width / min / max of tokens lane, lane + 32
-    uint32_t tbv = 0, bits4 = 0, mmv[4] = {0, 0, 0, 0};
-    auto fetch_meta = [&](int tile) {
-        if (tile < tile_hi) {
+    // Metadata runs ahead of the work: the tile table (lanes 0..7) two tiles ahead, the
+    // per-token width / min / max (tokens lane, lane + 32) one tile ahead, and the packed
+    // bytes of the next tile are pulled into L1 while the current tile is processed.
+    uint32_t tb_next = 0, tb_next2 = 0, bits4 = 0, mmv[4] = {0, 0, 0, 0};
+    auto fetch_table = [&](int tile) -> uint32_t {
+        uint32_t v = 0;
+        if (tile < tile_hi && lane < 8) {
+            const TensorStore& ts = (lane >= 4) ? a.v : a.k;
             const size_t ti = trow + tile;
-            if (lane < 8) {
-                const TensorStore& ts = (lane >= 4) ? a.v : a.k;
-                const int f = lane & 3;
-                tbv = f == 0 ? ts.tile_off[ti] : f == 1 ? ts.tile_nbytes[ti] : f == 2 ? ts.tile_ooff[ti] : ts.tile_ocnt[ti];
-            }
+            const int f = lane & 3;
+            v = f == 0 ? ts.tile_off[ti] : f == 1 ? ts.tile_nbytes[ti] : f == 2 ? ts.tile_ooff[ti] : ts.tile_ocnt[ti];
+        }
+        return v;
+    };
+    auto fetch_tokens = [&](int tile) {
+        if (tile < tile_hi) {
             const size_t t0 = mrow + (size_t)tile * QAQ_TILE + lane;
             bits4 = (uint32_t)a.k.bits[t0] | ((uint32_t)a.k.bits[t0 + 32] << 8) | ((uint32_t)a.v.bits[t0] << 16) |
                     ((uint32_t)a.v.bits[t0 + 32] << 24);
             mmv[0] = a.k.mnmx[t0]; mmv[1] = a.k.mnmx[t0 + 32]; mmv[2] = a.v.mnmx[t0]; mmv[3] = a.v.mnmx[t0 + 32];
         }
     };
-    fetch_meta(tile_lo + warp);
+    auto prefetch_codes = [&](uint32_t tb) {   // tb: table registers of the tile to prefetch
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            const uint32_t off = __shfl_sync(0xFFFFFFFFu, tb, 4 * x), nb = __shfl_sync(0xFFFFFFFFu, tb, 4 * x + 1);
+            const uint8_t* src = (x ? a.v.codes : a.k.codes) + (size_t)bh * a.pool_bytes + off;
+            for (uint32_t o = lane * 128u; o < nb; o += 32u * 128u) asm volatile("prefetch.global.L1 [%0];" ::"l"(src + o));
+        }
+    };
+    uint32_t tb_cur = fetch_table(tile_lo + warp);
+    tb_next = fetch_table(tile_lo + warp + DEC_WARPS);
+    fetch_tokens(tile_lo + warp);
 
     for (int tile = tile_lo + warp; tile < tile_hi; tile += DEC_WARPS) {
-        // ---- take over the prefetched metadata, start the next tile's
-        const uint32_t offK = __shfl_sync(0xFFFFFFFFu, tbv, 0), ooK = __shfl_sync(0xFFFFFFFFu, tbv, 2), ocK = __shfl_sync(0xFFFFFFFFu, tbv, 3);
-        const uint32_t offV = __shfl_sync(0xFFFFFFFFu, tbv, 4), ooV = __shfl_sync(0xFFFFFFFFu, tbv, 6), ocV = __shfl_sync(0xFFFFFFFFu, tbv, 7);
+        // ---- take over the metadata fetched earlier, start the fetches for the tiles ahead
+        const uint32_t offK = __shfl_sync(0xFFFFFFFFu, tb_cur, 0), ooK = __shfl_sync(0xFFFFFFFFu, tb_cur, 2), ocK = __shfl_sync(0xFFFFFFFFu, tb_cur, 3);
+        const uint32_t offV = __shfl_sync(0xFFFFFFFFu, tb_cur, 4), ooV = __shfl_sync(0xFFFFFFFFu, tb_cur, 6), ocV = __shfl_sync(0xFFFFFFFFu, tb_cur, 7);
         const uint32_t cb4 = bits4;
         const uint32_t cm[4] = {mmv[0], mmv[1], mmv[2], mmv[3]};
-        fetch_meta(tile + DEC_WARPS);
+        tb_next2 = fetch_table(tile + 2 * DEC_WARPS);
+        fetch_tokens(tile + DEC_WARPS);
+        if (tile + DEC_WARPS < tile_hi) prefetch_codes(tb_next);
+        tb_cur = tb_next;
+        tb_next = tb_next2;
 
         // ---- per-token scalars, byte offsets, item lists (tokens lane and lane + 32)
         int ncls[2][4];
@@ -303,7 +322,6 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(const DecArgs a) {
                 const float st = __fmul_rn(__fsub_rn(mx, mn), __int_as_float((127 - B) << 23));
                 ws.step[x][slot] = valid ? st : 0.f;
                 ws.mid[x][slot] = valid ? fmaf(0.5f, st, mn) : 0.f;
-                ws.bits[x][slot] = (uint8_t)B;
                 if (x == 0) { ws.dot[slot] = 0; ws.ocorr[slot] = 0.f; }
             }
             uint32_t i0 = len[0], i1 = len[1];
@@ -313,8 +331,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(const DecArgs a) {
                 if (lane >= d) { i0 += t0; i1 += t1; }
             }
             const uint32_t tot0 = __shfl_sync(0xFFFFFFFFu, i0, 31);
-            ws.tokoff[x][lane] = (uint16_t)(i0 - len[0]);
-            ws.tokoff[x][lane + 32] = (uint16_t)(tot0 + i1 - len[1]);
+            const uint32_t toff[2] = {i0 - len[0], tot0 + i1 - len[1]};
             int base = 0;
             const unsigned lt = (1u << lane) - 1u;
 #pragma unroll
@@ -322,8 +339,14 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(const DecArgs a) {
                 const int w = 8 >> c;
                 const unsigned b0 = __ballot_sync(0xFFFFFFFFu, (Bv[0] & w) != 0);
                 const unsigned b1 = __ballot_sync(0xFFFFFFFFu, (Bv[1] & w) != 0);
-                if (Bv[0] & w) ws.item[x][base + __popc(b0 & lt)] = (uint8_t)lane;
-                if (Bv[1] & w) ws.item[x][base + __popc(b0) + __popc(b1 & lt)] = (uint8_t)(lane + 32);
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    if (Bv[e] & w) {
+                        const uint32_t plane = toff[e] + (uint32_t)((Bv[e] & ~(2 * w - 1)) * (D / 8));
+                        const uint32_t desc = plane | ((uint32_t)(Bv[e] & (w - 1)) << 16) | ((uint32_t)(lane + 32 * e) << 24);
+                        ws.item[x][base + (e ? __popc(b0) + __popc(b1 & lt) : __popc(b0 & lt))] = desc;
+                    }
+                }
                 ncls[x][c] = __popc(b0) + __popc(b1);
                 base += ncls[x][c];
             }
@@ -383,6 +406,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(const DecArgs a) {
                 const int slot = lane + 32 * e;
                 const float p = __expf(lg[e] - m_new);   // 0 for slots beyond T
                 ws.p[slot] = p;
+                ws.wv[slot] = p * ws.step[1][slot];
                 c_run = fmaf(p, ws.mid[1][slot], c_run);
                 s += p;
             }
