@@ -172,7 +172,7 @@ qaq_status qaq_decode_attention_host(qaq_cache* c, const void* q, float softmax_
  * until the process exits).  The call performs no cudaMalloc/cudaFree and uses no
  * allocating library routine; q and out are still the caller's buffers, as above.
  *
- *   - Limit: batch*heads * splits * (head_dim+2) * 4 bytes + batch*heads*8 must fit in
+ *   - Limit: batch*heads * splits * (head_dim+3) * 4 bytes + batch*heads*8 must fit in
  *     4 MiB (the split count is the one qaq_decode_attention would use; e.g. 256 (b,h) x
  *     4096 tokens x head_dim 128 needs 0.4 MiB).  Larger shapes get QAQ_ERR_WORKSPACE
  *     and nothing is launched -- use qaq_decode_attention with your own workspace.

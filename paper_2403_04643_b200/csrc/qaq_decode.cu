@@ -35,7 +35,7 @@ struct DecArgs {
     int T;
     const __half* q;
     float scale;
-    float* part;       // [BH][nsplit][D+2]
+    float* part;       // [BH][nsplit][D+3]: accumulators, running max, sum of the weights used, exact sum
     float* ml;         // [BH][2]   merged (max, sum) for score normalisation
     int nsplit;
     float* out;        // [BH][D]
@@ -53,24 +53,44 @@ __device__ __forceinline__ int dp4a_uu(uint32_t a, uint32_t b, int c) {  // unsi
     return d;
 }
 
-// W words (4*W bytes) of a plane from global memory; the address is ALIGN-byte aligned
+__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t c) {  // (a & b) | c
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+// acc += a * b with a, b binary16 and acc binary32 (one rounding)
+__device__ __forceinline__ void fma_f32_f16(float& acc, unsigned short a, unsigned short b) {
+    asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc) : "h"(a), "h"(b));
+}
+template <int BYTES>
+__device__ __forceinline__ void cp_async(void* smem, const void* gmem) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    if (BYTES == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem));
+    else if (BYTES == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(s), "l"(gmem));
+    else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(s), "l"(gmem));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+// W words (4*W bytes) of a plane; the address is ALIGN-byte aligned
 template <int W, int ALIGN>
 __device__ __forceinline__ void load_words(const uint8_t* __restrict__ p, uint32_t (&w)[8]) {
     if (ALIGN == 16 && W % 4 == 0) {
 #pragma unroll
         for (int i = 0; i < W; i += 4) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(p + 4 * i));
+            const uint4 v = *reinterpret_cast<const uint4*>(p + 4 * i);
             w[i] = v.x; w[i + 1] = v.y; w[i + 2] = v.z; w[i + 3] = v.w;
         }
     } else if (ALIGN >= 8 && W % 2 == 0) {
 #pragma unroll
         for (int i = 0; i < W; i += 2) {
-            const uint2 v = __ldg(reinterpret_cast<const uint2*>(p + 4 * i));
+            const uint2 v = *reinterpret_cast<const uint2*>(p + 4 * i);
             w[i] = v.x; w[i + 1] = v.y;
         }
     } else {
 #pragma unroll
-        for (int i = 0; i < W; ++i) w[i] = __ldg(reinterpret_cast<const uint32_t*>(p + 4 * i));
+        for (int i = 0; i < W; ++i) w[i] = *reinterpret_cast<const uint32_t*>(p + 4 * i);
     }
 }
 
@@ -79,54 +99,67 @@ template <int W>
 __device__ __forceinline__ int plane_dot(const uint32_t (&words)[8], const uint32_t (&qh)[8], const uint32_t (&ql)[8]) {
     constexpr int PER = 8 / W;
     constexpr uint32_t MASK = 0x01010101u * ((1u << W) - 1u);
-    int ah = 0, al = 0;
+    int ah[2] = {0, 0}, al[2] = {0, 0};
 #pragma unroll
     for (int j = 0; j < W; ++j) {
         const uint32_t wd = words[j];
 #pragma unroll
         for (int m = 0; m < PER; ++m) {
             const uint32_t f = (wd >> (W * m)) & MASK;
-            ah = dp4a_us(f, qh[PER * j + m], ah);
-            al = dp4a_uu(f, ql[PER * j + m], al);
+            const int r = PER * j + m;
+            ah[r & 1] = dp4a_us(f, qh[r], ah[r & 1]);
+            al[r & 1] = dp4a_uu(f, ql[r], al[r & 1]);
         }
     }
-    return ah * 256 + al;
+    return (ah[0] + ah[1]) * 256 + (al[0] + al[1]);
 }
 
-// acc[r][i] += wt * (1 + f/2^W) for the lane's 32 channels of a w-bit plane
+// acc[r][i] += b * (f - 2^(W-1)) for the lane's 32 channels of a w-bit plane, b = bm[m] * 2^(W*m).
+// Fields are taken two at a time (the same bit positions of the two 16-bit halves of a word) by
+// OR-ing them into the mantissa of binary16 1024: 1024 + f * 2^(W*m); subtracting 1024 +
+// 2^(W-1) * 2^(W*m) is exact and centres the code.  The products go into binary32 accumulators.
 template <int W>
-__device__ __forceinline__ void plane_axpy(const uint32_t (&words)[8], float wt, float (&acc)[8][4]) {
+__device__ __forceinline__ void plane_axpy(const uint32_t (&words)[8], const unsigned short (&bm)[8 / W], float (&acc)[8][4]) {
     constexpr int PER = 8 / W;
-    constexpr uint32_t MASK = ((1u << W) - 1u) << (23 - W);
 #pragma unroll
     for (int j = 0; j < W; ++j) {
-        const uint32_t wd = words[j];
+        const uint32_t ev = words[j];          // byte lanes 0 and 2 in the low bytes of the halves
+        const uint32_t od = words[j] >> 8;     // byte lanes 1 and 3
 #pragma unroll
         for (int m = 0; m < PER; ++m) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int pos = 8 * i + W * m;
-                const uint32_t sh = (pos + W <= 23) ? (wd << (23 - W - pos)) : (wd >> (pos + W - 23));
-                const float xf = __uint_as_float((sh & MASK) | 0x3F800000u);
-                acc[PER * j + m][i] = fmaf(wt, xf, acc[PER * j + m][i]);
-            }
+            const uint32_t mask = (((1u << W) - 1u) << (W * m)) * 0x00010001u;
+            const uint32_t cen = (0x6400u + (1u << (W - 1 + W * m))) * 0x00010001u;   // binary16 of 1024 + 2^(W-1+Wm), twice
+            const __half2 c2 = *reinterpret_cast<const __half2*>(&cen);
+            uint32_t xe = lop3_and_or(ev, mask, 0x64006400u), xo = lop3_and_or(od, mask, 0x64006400u);
+            const __half2 ye = __hsub2(*reinterpret_cast<__half2*>(&xe), c2);
+            const __half2 yo = __hsub2(*reinterpret_cast<__half2*>(&xo), c2);
+            const int r = PER * j + m;
+            fma_f32_f16(acc[r][0], __half_as_ushort(__low2half(ye)), bm[m]);
+            fma_f32_f16(acc[r][2], __half_as_ushort(__high2half(ye)), bm[m]);
+            fma_f32_f16(acc[r][1], __half_as_ushort(__low2half(yo)), bm[m]);
+            fma_f32_f16(acc[r][3], __half_as_ushort(__high2half(yo)), bm[m]);
         }
     }
 }
 
-// per-warp scratch for the tile a warp is working on
+constexpr int UNIT = QAQ_TILE / 2;   // tokens a warp handles at a time (half a tile)
+
+// per-warp scratch for the half tile a warp is working on
 template <int D>
 struct WarpScratch {
-    float step[2][QAQ_TILE];
-    float mid[2][QAQ_TILE];     // min + step/2
-    float ocorr[QAQ_TILE];      // sum over a token's key outliers of q_ch * (x - mid)
-    float p[QAQ_TILE];
+    alignas(16) uint8_t bufK[UNIT * D + 16];
+    alignas(16) uint8_t bufV[UNIT * D + 16];
+    float stepK[UNIT];
+    float midK[UNIT];           // min + step/2
+    float midV[UNIT];
+    float ocorr[UNIT];          // sum over a token's key outliers of q_ch * (x - mid)
+    float p[UNIT];
+    float wv[UNIT];             // p_t * step_t * 2^g of the value side
     float vout[D];              // value-outlier corrections
-    int dot[QAQ_TILE];
-    float wv[QAQ_TILE];         // p_t * step_t of the value side
+    int dot[UNIT];
     // work items grouped by plane width (8, 4, 2, 1):
-    //   byte offset of the plane inside the tile | shift of the piece << 16 | token << 24
-    uint32_t item[2][3 * QAQ_TILE];
+    //   byte offset of the plane inside the half tile | shift of the piece << 16 | token << 24
+    uint32_t item[2][3 * UNIT];
 };
 
 template <int D>
@@ -134,63 +167,53 @@ struct DecSmem {
     WarpScratch<D> ws[DEC_WARPS];
     float qf[D];
     float macc[DEC_WARPS][D];
-    float mm[DEC_WARPS], ml[DEC_WARPS];
+    float mm[DEC_WARPS], ml[DEC_WARPS], mlx[DEC_WARPS];
     float red[DEC_WARPS], red2[DEC_WARPS];
     float qscale, qsum;
 };
 
-// One pass over the key-side items of one plane width: a group of P lanes per item.
 template <int D, int W, int ALIGN>
-__device__ __forceinline__ void k_items(WarpScratch<D>& ws, const uint8_t* __restrict__ tile, int first, int n,
-                                        const uint32_t (&qh)[8], const uint32_t (&ql)[8], int part, int sub) {
+__device__ __forceinline__ void k_items(WarpScratch<D>& ws, int first, int n, const uint32_t (&qh)[8],
+                                        const uint32_t (&ql)[8], int part, int sub) {
     constexpr int P = D / 32, IPW = 32 / P;
-    for (int i0 = 0; i0 < n; i0 += 2 * IPW) {
-        uint32_t w0[8], w1[8];
-        const int ia = i0 + sub, ib = i0 + IPW + sub;
-        const bool va = ia < n, vb = ib < n;
-        const uint32_t da_ = va ? ws.item[0][first + ia] : 0u, db_ = vb ? ws.item[0][first + ib] : 0u;
-        if (va) load_words<W, ALIGN>(tile + (da_ & 0xFFFFu) + part * 4 * W, w0);
-        if (vb) load_words<W, ALIGN>(tile + (db_ & 0xFFFFu) + part * 4 * W, w1);
-        int da = va ? plane_dot<W>(w0, qh, ql) : 0;
-        int db = vb ? plane_dot<W>(w1, qh, ql) : 0;
+    for (int i0 = 0; i0 < n; i0 += IPW) {
+        uint32_t w0[8];
+        const int ia = i0 + sub;
+        const bool va = ia < n;
+        const uint32_t de = va ? ws.item[0][first + ia] : 0u;
+        int da = 0;
+        if (va) {
+            load_words<W, ALIGN>(ws.bufK + (de & 0xFFFFu) + part * 4 * W, w0);
+            da = plane_dot<W>(w0, qh, ql);
+        }
 #pragma unroll
-        for (int o = 1; o < P; o <<= 1) {
-            da += __shfl_xor_sync(0xFFFFFFFFu, da, o);
-            db += __shfl_xor_sync(0xFFFFFFFFu, db, o);
-        }
-        if (part == 0) {
-            if (va) atomicAdd(&ws.dot[da_ >> 24], da << ((da_ >> 16) & 7));
-            if (vb) atomicAdd(&ws.dot[db_ >> 24], db << ((db_ >> 16) & 7));
-        }
+        for (int o = 1; o < P; o <<= 1) da += __shfl_xor_sync(0xFFFFFFFFu, da, o);
+        if (va && part == 0) atomicAdd(&ws.dot[de >> 24], da << ((de >> 16) & 7));
     }
 }
 
 template <int D, int W, int ALIGN>
-__device__ __forceinline__ void v_items(WarpScratch<D>& ws, const uint8_t* __restrict__ tile, int first, int n,
-                                        float (&acc)[8][4], float& offs, int part, int sub) {
-    constexpr int P = D / 32, IPW = 32 / P;
-    for (int i0 = 0; i0 < n; i0 += 2 * IPW) {
-        uint32_t w0[8], w1[8];
-        const int ia = i0 + sub, ib = i0 + IPW + sub;
-        const bool va = ia < n, vb = ib < n;
-        const uint32_t da_ = va ? ws.item[1][first + ia] : 0u, db_ = vb ? ws.item[1][first + ib] : 0u;
-        if (va) load_words<W, ALIGN>(tile + (da_ & 0xFFFFu) + part * 4 * W, w0);
-        if (vb) load_words<W, ALIGN>(tile + (db_ & 0xFFFFu) + part * 4 * W, w1);
-        if (va) {   // p_t * step_t * 2^shift * f = wt * (f / 2^W)
-            const float wt = ws.wv[da_ >> 24] * __int_as_float((127 + W) << 23) * __int_as_float((127 + ((da_ >> 16) & 7)) << 23);
-            plane_axpy<W>(w0, wt, acc);
-            offs += wt;
-        }
-        if (vb) {
-            const float wt = ws.wv[db_ >> 24] * __int_as_float((127 + W) << 23) * __int_as_float((127 + ((db_ >> 16) & 7)) << 23);
-            plane_axpy<W>(w1, wt, acc);
-            offs += wt;
-        }
+__device__ __forceinline__ void v_items(WarpScratch<D>& ws, int first, int n, float (&acc)[8][4], int part, int sub) {
+    constexpr int P = D / 32, IPW = 32 / P, PER = 8 / W;
+    for (int i0 = sub; i0 < n; i0 += IPW) {
+        uint32_t w0[8];
+        const uint32_t de = ws.item[1][first + i0];
+        load_words<W, ALIGN>(ws.bufV + (de & 0xFFFFu) + part * 4 * W, w0);
+        // weight of field slot m: p_t * step_t * 2^g * 2^shift / 2^(W*m), in binary16
+        const float wt = ws.wv[de >> 24] * __int_as_float((127 + ((de >> 16) & 7)) << 23);
+        unsigned short bm[PER];
+        const __half b0 = __float2half_rn(wt);
+#pragma unroll
+        for (int m = 0; m < PER; ++m) bm[m] = __half_as_ushort(__hmul(b0, __ushort_as_half((unsigned short)((15 - W * m) << 10))));
+        plane_axpy<W>(w0, bm, acc);
     }
 }
 
-// One CTA = one (b,h) and one split of its tiles; every warp works through whole tiles on
-// its own (own running max / sum / accumulators), the warps are merged once at the end.
+// One CTA = one (b,h) and one split of its tiles.  Every warp works through whole tiles on its
+// own, half a tile (32 tokens) at a time: own running max / sum / accumulators, own staging
+// buffers, no CTA barrier in the loop; the warps are merged once at the end.  The packed bytes
+// of the next half tile are copied to shared memory with cp.async while the current one is being
+// processed: the keys during the value phase, the values during the key phase.
 template <int D>
 __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a) {
     constexpr int P = D / 32;        // lanes per item
@@ -250,217 +273,271 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
     for (int r = 0; r < 8; ++r)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[r][i] = 0.f;
-    float offs = 0.f;        // sum of the weights this lane applied (the "1 +" of the magic floats)
-    float m_run = __int_as_float(0xff800000), l_run = 0.f;
-    float c_run = 0.f;       // per-lane part of sum_t p_t (min_t + step_t/2)
+    float m_run = __int_as_float(0xff800000), l_run = 0.f, lx_run = 0.f;   // lx: sum of the unperturbed p
+    float c_run = 0.f;       // per-lane part of sum_t p_t * (constant part of the token's values)
+    // The binary16 weights of the value side carry a common power-of-two factor 2^g so that the
+    // largest possible weight (range/2) sits near 2^12; g only ever decreases.
+    int g_run = 24;
 
     const size_t trow = (size_t)bh * a.ntiles_max;
     const size_t mrow = (size_t)bh * a.tmax_pad;
+    const uint8_t* poolK = a.k.codes + (size_t)bh * a.pool_bytes;
+    const uint8_t* poolV = a.v.codes + (size_t)bh * a.pool_bytes;
 
-    // Metadata runs ahead of the work: the tile table (lanes 0..7) two tiles ahead, the
-    // per-token width / min / max (tokens lane, lane + 32) one tile ahead, and the packed
-    // bytes of the next tile are pulled into L1 while the current tile is processed.
-    uint32_t tb_next = 0, tb_next2 = 0, bits4 = 0, mmv[4] = {0, 0, 0, 0};
-    auto fetch_table = [&](int tile) -> uint32_t {
-        uint32_t v = 0;
-        if (tile < tile_hi && lane < 8) {
-            const TensorStore& ts = (lane >= 4) ? a.v : a.k;
-            const size_t ti = trow + tile;
-            const int f = lane & 3;
-            v = f == 0 ? ts.tile_off[ti] : f == 1 ? ts.tile_nbytes[ti] : f == 2 ? ts.tile_ooff[ti] : ts.tile_ocnt[ti];
-        }
-        return v;
-    };
-    auto fetch_tokens = [&](int tile) {
+    // ---- tile metadata in registers: table words in lanes 0..7, widths and min/max of tokens lane, lane+32
+    struct Meta { uint32_t tb, bits4, mm[4]; };
+    auto fetch_meta = [&](int tile) {
+        Meta m;
+        m.tb = 0; m.bits4 = 0; m.mm[0] = m.mm[1] = m.mm[2] = m.mm[3] = 0;
         if (tile < tile_hi) {
+            if (lane < 8) {
+                const TensorStore& ts = (lane >= 4) ? a.v : a.k;
+                const size_t ti = trow + tile;
+                const int f = lane & 3;
+                m.tb = f == 0 ? ts.tile_off[ti] : f == 1 ? ts.tile_nbytes[ti] : f == 2 ? ts.tile_ooff[ti] : ts.tile_ocnt[ti];
+            }
             const size_t t0 = mrow + (size_t)tile * QAQ_TILE + lane;
-            bits4 = (uint32_t)a.k.bits[t0] | ((uint32_t)a.k.bits[t0 + 32] << 8) | ((uint32_t)a.v.bits[t0] << 16) |
-                    ((uint32_t)a.v.bits[t0 + 32] << 24);
-            mmv[0] = a.k.mnmx[t0]; mmv[1] = a.k.mnmx[t0 + 32]; mmv[2] = a.v.mnmx[t0]; mmv[3] = a.v.mnmx[t0 + 32];
+            m.bits4 = (uint32_t)a.k.bits[t0] | ((uint32_t)a.k.bits[t0 + 32] << 8) | ((uint32_t)a.v.bits[t0] << 16) |
+                      ((uint32_t)a.v.bits[t0 + 32] << 24);
+            m.mm[0] = a.k.mnmx[t0]; m.mm[1] = a.k.mnmx[t0 + 32]; m.mm[2] = a.v.mnmx[t0]; m.mm[3] = a.v.mnmx[t0 + 32];
         }
+        return m;
     };
-    auto prefetch_codes = [&](uint32_t tb) {   // tb: table registers of the tile to prefetch
+    // bytes of the first half (tokens 0..31) of a tile, per tensor (slots beyond T have width 0)
+    auto first_half_bytes = [&](const Meta& m, uint32_t& hK, uint32_t& hV) {
+        uint32_t k = (m.bits4 & 0xFF) * (D / 8), v = ((m.bits4 >> 16) & 0xFF) * (D / 8);
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
-            const uint32_t off = __shfl_sync(0xFFFFFFFFu, tb, 4 * x), nb = __shfl_sync(0xFFFFFFFFu, tb, 4 * x + 1);
-            const uint8_t* src = (x ? a.v.codes : a.k.codes) + (size_t)bh * a.pool_bytes + off;
-            for (uint32_t o = lane * 128u; o < nb; o += 32u * 128u) asm volatile("prefetch.global.L1 [%0];" ::"l"(src + o));
+        for (int o = 16; o > 0; o >>= 1) {
+            k += __shfl_xor_sync(0xFFFFFFFFu, k, o);
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
         }
+        hK = k; hV = v;
     };
-    uint32_t tb_cur = fetch_table(tile_lo + warp);
-    tb_next = fetch_table(tile_lo + warp + DEC_WARPS);
-    fetch_tokens(tile_lo + warp);
+    auto stage = [&](uint8_t* dst, const uint8_t* src, uint32_t nbytes) {
+        for (uint32_t o = lane * ALIGN; o < nbytes; o += 32 * ALIGN) cp_async<ALIGN>(dst + o, src + o);
+    };
 
-    for (int tile = tile_lo + warp; tile < tile_hi; tile += DEC_WARPS) {
-        // ---- take over the metadata fetched earlier, start the fetches for the tiles ahead
-        const uint32_t offK = __shfl_sync(0xFFFFFFFFu, tb_cur, 0), ooK = __shfl_sync(0xFFFFFFFFu, tb_cur, 2), ocK = __shfl_sync(0xFFFFFFFFu, tb_cur, 3);
-        const uint32_t offV = __shfl_sync(0xFFFFFFFFu, tb_cur, 4), ooV = __shfl_sync(0xFFFFFFFFu, tb_cur, 6), ocV = __shfl_sync(0xFFFFFFFFu, tb_cur, 7);
-        const uint32_t cb4 = bits4;
-        const uint32_t cm[4] = {mmv[0], mmv[1], mmv[2], mmv[3]};
-        tb_next2 = fetch_table(tile + 2 * DEC_WARPS);
-        fetch_tokens(tile + DEC_WARPS);
-        if (tile + DEC_WARPS < tile_hi) prefetch_codes(tb_next);
-        tb_cur = tb_next;
-        tb_next = tb_next2;
+    int tile = tile_lo + warp;
+    Meta cur = fetch_meta(tile);
+    Meta nxt = fetch_meta(tile + DEC_WARPS);
+    uint32_t h0K = 0, h0V = 0;
+    first_half_bytes(cur, h0K, h0V);
+    if (tile < tile_hi) {
+        stage(ws.bufK, poolK + __shfl_sync(0xFFFFFFFFu, cur.tb, 0), h0K);
+        cp_async_commit();
+        stage(ws.bufV, poolV + __shfl_sync(0xFFFFFFFFu, cur.tb, 4), h0V);
+        cp_async_commit();
+    }
 
-        // ---- per-token scalars, byte offsets, item lists (tokens lane and lane + 32)
-        int ncls[2][4];
+    for (; tile < tile_hi; tile += DEC_WARPS) {
+        const uint32_t offK = __shfl_sync(0xFFFFFFFFu, cur.tb, 0), totK = __shfl_sync(0xFFFFFFFFu, cur.tb, 1);
+        const uint32_t ooK = __shfl_sync(0xFFFFFFFFu, cur.tb, 2), ocK = __shfl_sync(0xFFFFFFFFu, cur.tb, 3);
+        const uint32_t offV = __shfl_sync(0xFFFFFFFFu, cur.tb, 4), totV = __shfl_sync(0xFFFFFFFFu, cur.tb, 5);
+        const uint32_t ooV = __shfl_sync(0xFFFFFFFFu, cur.tb, 6), ocV = __shfl_sync(0xFFFFFFFFu, cur.tb, 7);
+        const bool has_next = tile + DEC_WARPS < tile_hi;
+        uint32_t n0K = 0, n0V = 0;   // first-half bytes of the next tile
+
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+            const int t = tile * QAQ_TILE + UNIT * half + lane;   // this lane's token
+            const bool valid = t < a.T;
+            // ---- per-token scalars, byte offsets inside the half tile, item lists
+            int ncls[2][4];
+            float rngV = 0.f;
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
-            uint32_t len[2];
-            int Bv[2];
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int slot = lane + 32 * e;
-                const bool valid = tile * QAQ_TILE + slot < a.T;
-                const int B = valid ? (int)((cb4 >> (16 * x + 8 * e)) & 0xFF) : 0;
-                Bv[e] = B;
-                len[e] = (uint32_t)(D * B / 8);
-                const uint32_t mmw = cm[2 * x + e];
+            for (int x = 0; x < 2; ++x) {
+                const int B = valid ? (int)((cur.bits4 >> (16 * x + 8 * half)) & 0xFF) : 0;
+                const uint32_t len = (uint32_t)(D * B / 8);
+                const uint32_t mmw = half ? cur.mm[2 * x + 1] : cur.mm[2 * x];
                 const float mn = __half2float(__ushort_as_half((unsigned short)(mmw & 0xFFFF)));
                 const float mx = __half2float(__ushort_as_half((unsigned short)(mmw >> 16)));
-                const float st = __fmul_rn(__fsub_rn(mx, mn), __int_as_float((127 - B) << 23));
-                ws.step[x][slot] = valid ? st : 0.f;
-                ws.mid[x][slot] = valid ? fmaf(0.5f, st, mn) : 0.f;
-                if (x == 0) { ws.dot[slot] = 0; ws.ocorr[slot] = 0.f; }
+                const float rng = valid ? __fsub_rn(mx, mn) : 0.f;
+                const float st = __fmul_rn(rng, __int_as_float((127 - B) << 23));
+                const float mid = fmaf(0.5f, st, mn);
+                if (x == 0) {
+                    ws.stepK[lane] = st; ws.midK[lane] = valid ? mid : 0.f;
+                    ws.dot[lane] = 0; ws.ocorr[lane] = 0.f;
+                } else {
+                    // centred planes: piece w contributes a constant step * 2^((B & (2w-1)) - 1)
+                    float cst = 0.5f;
+#pragma unroll
+                    for (int w = 8; w >= 1; w >>= 1)
+                        if (B & w) cst += __int_as_float((127 + (B & (2 * w - 1)) - 1) << 23);
+                    ws.midV[lane] = valid ? mid : 0.f;                     // value of a zero code slot (outliers)
+                    ws.p[lane] = valid ? fmaf(cst, st, mn) : 0.f;           // constant part, picked up below
+                    ws.wv[lane] = st;                                       // step for now, weight after the softmax
+                    rngV = rng;
+                }
+                uint32_t inc = len;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                    if (lane >= d) inc += u;
+                }
+                const uint32_t toff = inc - len;
+                int base = 0;
+                const unsigned lt = (1u << lane) - 1u;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int w = 8 >> c;
+                    const unsigned bal = __ballot_sync(0xFFFFFFFFu, (B & w) != 0);
+                    if (B & w) {
+                        const uint32_t plane = toff + (uint32_t)((B & ~(2 * w - 1)) * (D / 8));
+                        ws.item[x][base + __popc(bal & lt)] = plane | ((uint32_t)(B & (w - 1)) << 16) | ((uint32_t)lane << 24);
+                    }
+                    ncls[x][c] = __popc(bal);
+                    base += ncls[x][c];
+                }
             }
-            uint32_t i0 = len[0], i1 = len[1];
+            // common exponent of the value weights
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t t0 = __shfl_up_sync(0xFFFFFFFFu, i0, d), t1 = __shfl_up_sync(0xFFFFFFFFu, i1, d);
-                if (lane >= d) { i0 += t0; i1 += t1; }
+            for (int o = 16; o > 0; o >>= 1) rngV = fmaxf(rngV, __shfl_xor_sync(0xFFFFFFFFu, rngV, o));
+            {
+                const int e = rngV > 0.f ? ((__float_as_int(rngV) >> 23) & 0xFF) - 127 : -12;
+                const int g = 12 - e;
+                if (g < g_run) {
+                    const float f = __int_as_float((127 + g - g_run) << 23);
+#pragma unroll
+                    for (int r = 0; r < 8; ++r)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) acc[r][i] *= f;
+                    g_run = g;
+                }
             }
-            const uint32_t tot0 = __shfl_sync(0xFFFFFFFFu, i0, 31);
-            const uint32_t toff[2] = {i0 - len[0], tot0 + i1 - len[1]};
-            int base = 0;
-            const unsigned lt = (1u << lane) - 1u;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const int w = 8 >> c;
-                const unsigned b0 = __ballot_sync(0xFFFFFFFFu, (Bv[0] & w) != 0);
-                const unsigned b1 = __ballot_sync(0xFFFFFFFFu, (Bv[1] & w) != 0);
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    if (Bv[e] & w) {
-                        const uint32_t plane = toff[e] + (uint32_t)((Bv[e] & ~(2 * w - 1)) * (D / 8));
-                        const uint32_t desc = plane | ((uint32_t)(Bv[e] & (w - 1)) << 16) | ((uint32_t)(lane + 32 * e) << 24);
-                        ws.item[x][base + (e ? __popc(b0) + __popc(b1 & lt) : __popc(b0 & lt))] = desc;
+            cp_async_wait<1>();     // this half's keys have landed (its values may still be in flight)
+            __syncwarp();
+
+            // ---- K: integer dot products per (token, plane), outlier corrections
+            {
+                int first = 0;
+                k_items<D, 8, ALIGN>(ws, first, ncls[0][0], qh, ql, part, sub); first += ncls[0][0];
+                k_items<D, 4, ALIGN>(ws, first, ncls[0][1], qh, ql, part, sub); first += ncls[0][1];
+                k_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, first, ncls[0][2], qh, ql, part, sub); first += ncls[0][2];
+                k_items<D, 1, 4>(ws, first, ncls[0][3], qh, ql, part, sub);
+                const uint32_t* og = a.k.outl + (size_t)bh * a.ocap + ooK;
+                for (uint32_t e = lane; e < ocK; e += 32) {
+                    const uint32_t v = __ldg(og + e);
+                    const int tok = v >> 24, ch = (v >> 16) & 0xFF;
+                    if ((tok >> 5) == half) {
+                        const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
+                        atomicAdd(&ws.ocorr[tok & 31], sm.qf[ch] * (val - ws.midK[tok & 31]));
                     }
                 }
-                ncls[x][c] = __popc(b0) + __popc(b1);
-                base += ncls[x][c];
             }
-        }
-        __syncwarp();
-
-        // ---- K: integer dot products per (token, plane), outlier corrections
-        {
-            const uint8_t* tk = a.k.codes + (size_t)bh * a.pool_bytes + offK;
-            int first = 0;
-            k_items<D, 8, ALIGN>(ws, tk, first, ncls[0][0], qh, ql, part, sub); first += ncls[0][0];
-            k_items<D, 4, ALIGN>(ws, tk, first, ncls[0][1], qh, ql, part, sub); first += ncls[0][1];
-            k_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, tk, first, ncls[0][2], qh, ql, part, sub); first += ncls[0][2];
-            k_items<D, 1, 4>(ws, tk, first, ncls[0][3], qh, ql, part, sub);
-            const uint32_t* og = a.k.outl + (size_t)bh * a.ocap + ooK;
-            for (uint32_t e = lane; e < ocK; e += 32) {
-                const uint32_t v = __ldg(og + e);
-                const int tok = v >> 24, ch = (v >> 16) & 0xFF;
-                const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
-                atomicAdd(&ws.ocorr[tok], sm.qf[ch] * (val - ws.mid[0][tok]));
+            __syncwarp();
+            // ---- the key buffer is free: start the copy of the next unit's keys
+            if (half == 0) {
+                stage(ws.bufK, poolK + offK + h0K, totK - h0K);
+            } else if (has_next) {
+                first_half_bytes(nxt, n0K, n0V);
+                stage(ws.bufK, poolK + __shfl_sync(0xFFFFFFFFu, nxt.tb, 0), n0K);
             }
-        }
-        __syncwarp();
+            cp_async_commit();
 
-        // ---- logits of tokens lane, lane + 32; running max / sum; weights
-        {
-            float lg[2];
+            // ---- logit of this lane's token; running max / sum; weights
+            {
+                float lg = __int_as_float(0xff800000);
+                if (valid) {
+                    const float qk = fmaf(qscale * ws.stepK[lane], (float)ws.dot[lane], fmaf(ws.midK[lane], qsum, ws.ocorr[lane]));
+                    lg = a.scale * qk;
+                    if (a.scores) a.scores[(size_t)bh * a.T + t] = lg;
+                }
+                float m = lg;
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int slot = lane + 32 * e;
-                const int t = tile * QAQ_TILE + slot;
-                lg[e] = __int_as_float(0xff800000);
-                if (t < a.T) {
-                    const float qk = fmaf(qscale * ws.step[0][slot], (float)ws.dot[slot], fmaf(ws.mid[0][slot], qsum, ws.ocorr[slot]));
-                    lg[e] = a.scale * qk;
-                    if (a.scores) a.scores[(size_t)bh * a.T + t] = lg[e];
+                for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+                const float m_new = fmaxf(m_run, m);
+                const float alpha = __expf(m_run - m_new);   // 0 on the first unit (m_run = -inf)
+                m_run = m_new;
+                if (alpha != 1.0f) {
+#pragma unroll
+                    for (int r = 0; r < 8; ++r)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) acc[r][i] *= alpha;
+                    c_run *= alpha;
+                    for (int d = lane; d < D; d += 32) ws.vout[d] *= alpha;
+                }
+                float p = __expf(lg - m_new);                // 0 for slots beyond T
+                float sx = p;
+                // The value weight p * step * 2^g is used in binary16.  It is rounded to 11 significant
+                // bits here, once, and p is adjusted by the same factor, so that the planes, the constant
+                // part and the softmax denominator all see the same (slightly perturbed) probability.
+                const float wfull = p * ws.wv[lane] * __int_as_float((127 + g_run) << 23);
+                const float big = __fmul_rn(wfull, 8193.0f);  // 2^13 + 1: splits off the upper 11 bits (no contraction)
+                const float wr = __fsub_rn(big, __fsub_rn(big, wfull));
+                if (wfull > 0.f) p *= __fdividef(wr, wfull);
+                ws.wv[lane] = wr;
+                c_run = fmaf(p, ws.p[lane], c_run);           // ws.p held the token's constant part
+                float s = p;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+                    sx += __shfl_xor_sync(0xFFFFFFFFu, sx, o);
+                }
+                l_run = l_run * alpha + s;
+                lx_run = lx_run * alpha + sx;
+                __syncwarp();
+                ws.p[lane] = p;
+            }
+            cp_async_wait<1>();     // this half's values have landed
+            __syncwarp();
+
+            // ---- V: weighted accumulation of centred codes, outlier corrections
+            {
+                int first = 0;
+                v_items<D, 8, ALIGN>(ws, first, ncls[1][0], acc, part, sub); first += ncls[1][0];
+                v_items<D, 4, ALIGN>(ws, first, ncls[1][1], acc, part, sub); first += ncls[1][1];
+                v_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, first, ncls[1][2], acc, part, sub); first += ncls[1][2];
+                v_items<D, 1, 4>(ws, first, ncls[1][3], acc, part, sub);
+                const uint32_t* og = a.v.outl + (size_t)bh * a.ocap + ooV;
+                for (uint32_t e = lane; e < ocV; e += 32) {
+                    const uint32_t v = __ldg(og + e);
+                    const int tok = v >> 24, ch = (v >> 16) & 0xFF;
+                    if ((tok >> 5) == half) {
+                        const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
+                        atomicAdd(&ws.vout[ch], ws.p[tok & 31] * (val - ws.midV[tok & 31]));
+                    }
                 }
             }
-            float m = fmaxf(lg[0], lg[1]);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-            const float m_new = fmaxf(m_run, m);
-            const float alpha = __expf(m_run - m_new);   // 0 on the first tile (m_run = -inf)
-            m_run = m_new;
-            if (alpha != 1.0f) {
-#pragma unroll
-                for (int r = 0; r < 8; ++r)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) acc[r][i] *= alpha;
-                offs *= alpha;
-                c_run *= alpha;
-                for (int d = lane; d < D; d += 32) ws.vout[d] *= alpha;
-            }
-            float s = 0.f;
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int slot = lane + 32 * e;
-                const float p = __expf(lg[e] - m_new);   // 0 for slots beyond T
-                ws.p[slot] = p;
-                ws.wv[slot] = p * ws.step[1][slot];
-                c_run = fmaf(p, ws.mid[1][slot], c_run);
-                s += p;
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-            l_run = l_run * alpha + s;
+            __syncwarp();
+            // ---- the value buffer is free: start the copy of the next unit's values
+            if (half == 0) stage(ws.bufV, poolV + offV + h0V, totV - h0V);
+            else if (has_next) stage(ws.bufV, poolV + __shfl_sync(0xFFFFFFFFu, nxt.tb, 4), n0V);
+            cp_async_commit();
         }
-        __syncwarp();
-
-        // ---- V: weighted accumulation of raw codes, outlier corrections
-        {
-            const uint8_t* tv = a.v.codes + (size_t)bh * a.pool_bytes + offV;
-            int first = 0;
-            v_items<D, 8, ALIGN>(ws, tv, first, ncls[1][0], acc, offs, part, sub); first += ncls[1][0];
-            v_items<D, 4, ALIGN>(ws, tv, first, ncls[1][1], acc, offs, part, sub); first += ncls[1][1];
-            v_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, tv, first, ncls[1][2], acc, offs, part, sub); first += ncls[1][2];
-            v_items<D, 1, 4>(ws, tv, first, ncls[1][3], acc, offs, part, sub);
-            const uint32_t* og = a.v.outl + (size_t)bh * a.ocap + ooV;
-            for (uint32_t e = lane; e < ocV; e += 32) {
-                const uint32_t v = __ldg(og + e);
-                const int tok = v >> 24, ch = (v >> 16) & 0xFF;
-                const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
-                atomicAdd(&ws.vout[ch], ws.p[tok] * (val - ws.mid[1][tok]));
-            }
-        }
-        __syncwarp();
+        cur = nxt;
+        h0K = n0K; h0V = n0V;
+        nxt = fetch_meta(tile + 2 * DEC_WARPS);
     }
+    cp_async_wait<0>();
 
     // ---- warp result: lanes with the same part hold partial sums of the same channels
     float cs = c_run;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) cs += __shfl_xor_sync(0xFFFFFFFFu, cs, o);
+    const float unscale = __int_as_float((127 - g_run) << 23);
 #pragma unroll
     for (int r = 0; r < 8; ++r)
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            float v = acc[r][i] - offs;
+            float v = acc[r][i];
 #pragma unroll
             for (int o = P; o < 32; o <<= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-            if (sub == 0) sm.macc[warp][32 * part + 4 * r + i] = v + ws.vout[32 * part + 4 * r + i] + cs;
+            if (sub == 0) sm.macc[warp][32 * part + 4 * r + i] = fmaf(v, unscale, ws.vout[32 * part + 4 * r + i] + cs);
         }
-    if (lane == 0) { sm.mm[warp] = m_run; sm.ml[warp] = l_run; }
+    if (lane == 0) { sm.mm[warp] = m_run; sm.ml[warp] = l_run; sm.mlx[warp] = lx_run; }
     __syncthreads();
     // ---- merge the warps (log-sum-exp) into this split's partial
     float M = __int_as_float(0xff800000);
 #pragma unroll
     for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, sm.mm[w]);
-    float* dst = a.part + ((size_t)bh * a.nsplit + split) * (D + 2);
-    float L = 0.f;
+    float* dst = a.part + ((size_t)bh * a.nsplit + split) * (D + 3);
+    float L = 0.f, LX = 0.f;
     float wgt[DEC_WARPS];
 #pragma unroll
     for (int w = 0; w < DEC_WARPS; ++w) {
         wgt[w] = (sm.mm[w] == __int_as_float(0xff800000)) ? 0.f : __expf(sm.mm[w] - M);
         L = fmaf(wgt[w], sm.ml[w], L);
+        LX = fmaf(wgt[w], sm.mlx[w], LX);
     }
     for (int d = tid; d < D; d += DEC_THREADS) {
         float x = 0.f;
@@ -468,26 +545,27 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
         for (int w = 0; w < DEC_WARPS; ++w) x = fmaf(wgt[w], sm.macc[w][d], x);
         dst[d] = x;
     }
-    if (tid == 0) { dst[D] = M; dst[D + 1] = L; }
+    if (tid == 0) { dst[D] = M; dst[D + 1] = L; dst[D + 2] = LX; }
 }
 
 // log-sum-exp merge of the split partials -> X, and (max, sum) for the score row
 template <int D>
 __global__ void merge_kernel(const DecArgs a) {
     const int bh = blockIdx.x, d = threadIdx.x;
-    const float* p = a.part + (size_t)bh * a.nsplit * (D + 2);
+    const float* p = a.part + (size_t)bh * a.nsplit * (D + 3);
     float M = __int_as_float(0xff800000);
-    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, p[s * (D + 2) + D]);
-    float L = 0.f, x = 0.f;
+    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, p[s * (D + 3) + D]);
+    float L = 0.f, LX = 0.f, x = 0.f;
     for (int s = 0; s < a.nsplit; ++s) {
-        const float m = p[s * (D + 2) + D];
+        const float m = p[s * (D + 3) + D];
         if (m == __int_as_float(0xff800000)) continue;
         const float w = __expf(m - M);
-        L = fmaf(w, p[s * (D + 2) + D + 1], L);
-        x = fmaf(w, p[s * (D + 2) + d], x);
+        L = fmaf(w, p[s * (D + 3) + D + 1], L);
+        LX = fmaf(w, p[s * (D + 3) + D + 2], LX);
+        x = fmaf(w, p[s * (D + 3) + d], x);
     }
     a.out[(size_t)bh * D + d] = L > 0.f ? x / L : 0.f;
-    if (d == 0) { a.ml[2 * bh] = M; a.ml[2 * bh + 1] = L; }
+    if (d == 0) { a.ml[2 * bh] = M; a.ml[2 * bh + 1] = LX; }
 }
 
 __global__ void scores_kernel(float* scores, const float* ml, int T) {
@@ -533,7 +611,7 @@ static const int QAQ_MAX_SPLIT = 64;
 extern "C" qaq_status qaq_decode_workspace_bytes(const qaq_cache* c, size_t* host_out) {
     if (!c || !host_out) return QAQ_ERR_INVALID_ARG;
     const size_t BH = (size_t)c->BH, D = (size_t)c->cfg.head_dim;
-    *host_out = (BH * QAQ_MAX_SPLIT * (D + 2) + BH * 2) * sizeof(float);
+    *host_out = (BH * QAQ_MAX_SPLIT * (D + 3) + BH * 2) * sizeof(float);
     return QAQ_OK;
 }
 
@@ -552,7 +630,7 @@ extern "C" qaq_status qaq_decode_attention(const qaq_cache* c, const void* q, fl
     const int ntiles = (a.T + QAQ_TILE - 1) / QAQ_TILE;
     a.nsplit = pick_nsplit(BH, ntiles);
     a.part = (float*)ws;
-    a.ml = a.part + (size_t)BH * QAQ_MAX_SPLIT * (D + 2);
+    a.ml = a.part + (size_t)BH * QAQ_MAX_SPLIT * (D + 3);
     a.out = out; a.scores = scores_out;
     cudaStream_t s = (cudaStream_t)stream;
     switch (D) {
@@ -585,8 +663,8 @@ extern "C" qaq_status qaq_decode_attention_static(const qaq_cache* c, const void
     const int T = (int)c->tokens;
     const int ntiles = (T + QAQ_TILE - 1) / QAQ_TILE;
     const int nsplit = pick_nsplit(BH, ntiles);
-    // partials [BH][nsplit][D+2] followed by the merged (max, sum) pairs [BH][2]
-    const size_t need = ((size_t)BH * nsplit * (D + 2) + (size_t)BH * 2) * sizeof(float);
+    // partials [BH][nsplit][D+3] followed by the merged (max, sum) pairs [BH][2]
+    const size_t need = ((size_t)BH * nsplit * (D + 3) + (size_t)BH * 2) * sizeof(float);
     if (need > QAQ_STATIC_SCRATCH_BYTES) return QAQ_ERR_WORKSPACE;  // shape too large for the built-in scratch
 
     int dev = -1;
@@ -615,7 +693,7 @@ extern "C" qaq_status qaq_decode_attention_static(const qaq_cache* c, const void
     // Every (b,h,split) partial and every (max,sum) pair is written before it is read, so
     // nothing in the scratch has to be cleared between calls.
     a.part = (float*)scratch;
-    a.ml = a.part + (size_t)BH * nsplit * (D + 2);
+    a.ml = a.part + (size_t)BH * nsplit * (D + 3);
     a.out = out; a.scores = nullptr;
     cudaStream_t s = (cudaStream_t)stream;
     switch (D) {
