@@ -1,128 +1,260 @@
-// S2a: exact outlier thresholds (order statistics) per (b,h) and tensor.
+// S2a: exact outlier thresholds (order statistics) per (b,h) and tensor, in one read of the data.
 //
-// binary16 patterns are mapped to 16-bit keys that sort like the values.  Two passes of
-// an 8-bit radix select find the key of rank k from below and of rank k from above:
-//   pass 1  256-bin histogram of the high key byte (shared-memory bins per CTA, merged
-//           with global atomics);
-//   pass 2  every CTA locates the two high-byte bins holding the wanted ranks, then
-//           histograms the low byte of the keys that fall into them;
-//   pass 3  one warp per (b,h,tensor) finishes the select and writes binary32 thresholds.
-// NaNs are not counted.  k = floor(alpha * N / 2), N = number of counted values.
+// Wanted: lo = k-th smallest and hi = k-th largest of the N non-NaN values, k = floor(alpha*N/2).
+// Only the two tails matter, so the bulk of the data is never histogrammed:
+//   1. thr_sample_kernel   a few tokens spread over the sequence give a bracket per tail: a value
+//                          below (above) which roughly twice the wanted tail mass lies.  Problems
+//                          small enough to be sampled completely are solved right here.
+//   2. thr_scan_kernel     the one pass over all values: entries beyond the brackets ("candidates",
+//                          a few per cent) are compacted into per-problem lists (shared-memory lists
+//                          per CTA, one global reservation per CTA and tail), NaNs are counted.
+//   3. thr_select_kernel   exact radix select of rank k inside the candidate lists.  If a bracket
+//                          turned out too tight (fewer than k+1 candidates) or a list overflowed, the
+//                          problem is redone exactly by a two-pass radix select over its data, so the
+//                          result is always the exact order statistic.
+// binary16 patterns are mapped to 16-bit keys that sort like the values.
 #include "qaq_internal.cuh"
 
 namespace {
 
-constexpr int THR_CHUNK_TOKENS = 256;  // tokens per CTA
+constexpr int SAMPLE_TOKENS = 64;
+constexpr int SCAN_TOKENS = 64;      // tokens per CTA of the scan
+constexpr int CTA_LIST = 2048;       // candidates per tail a scan CTA can hold
 
 __device__ __forceinline__ uint32_t key_of(unsigned short h) { return (h & 0x8000u) ? (uint32_t)(~h & 0xFFFFu) : (uint32_t)(h | 0x8000u); }
 __device__ __forceinline__ unsigned short half_of_key(uint32_t k) { return (k & 0x8000u) ? (unsigned short)(k & 0x7FFFu) : (unsigned short)(~k & 0xFFFFu); }
 __device__ __forceinline__ bool is_nan_bits(unsigned short h) { return (h & 0x7FFFu) > 0x7C00u; }
+__device__ __forceinline__ float float_of_key(uint32_t k) { return __half2float(__ushort_as_half(half_of_key(k))); }
+
+struct Problem {          // per (b,h,tensor), in the workspace
+    uint32_t klo, khi;    // bracket keys: candidates are keys < klo and keys > khi
+    uint32_t cnt[2];      // candidates found (may exceed the capacity: then the list is incomplete)
+    uint32_t nan;         // NaN entries seen by the scan
+    uint32_t done;        // solved by the sample kernel
+    uint32_t pad[2];
+};
 
 struct ThrArgs {
     const __half* X[2];
     long sb, sh, st;
     int H, T, D;
     double alpha;
-    uint32_t* hist1;  // [BH*2][256]
-    uint32_t* hist2;  // [BH*2][2][256]
-    float* thr;       // [BH][4]
+    Problem* prob;        // [BH*2]
+    unsigned short* list; // [BH*2][2][cap]
+    uint32_t cap;
+    float* thr;           // [BH][4]
 };
 
-// rank search in a 256-bin histogram: bin holding rank `want` (0-based), and the rank inside it
-__device__ void find_bin(const uint32_t* hist, unsigned long long want, int* bin, unsigned long long* within) {
-    unsigned long long acc = 0;
-    int b = 0;
-    for (; b < 255; ++b) {
-        unsigned long long n = hist[b];
-        if (acc + n > want) break;
-        acc += n;
+// rank select (0-based rank `want`) over n 16-bit keys readable through get(i); all threads of the
+// CTA call it; hist is 256 words of shared memory.  Two rounds of an 8-bit radix select.
+template <typename Get>
+__device__ uint32_t cta_select(Get get, uint32_t n, uint32_t want, uint32_t* hist, uint32_t* s_tmp) {
+    uint32_t prefix = 0;
+    for (int round = 0; round < 2; ++round) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
+            const uint32_t k = get(i);
+            if (k > 0xFFFFu) continue;                      // NaN marker
+            if (round == 0) atomicAdd(&hist[k >> 8], 1u);
+            else if ((k >> 8) == prefix) atomicAdd(&hist[k & 255], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t acc = 0;
+            int b = 0;
+            for (; b < 255; ++b) {
+                if (acc + hist[b] > want) break;
+                acc += hist[b];
+            }
+            s_tmp[0] = (uint32_t)b;
+            s_tmp[1] = want - acc;
+        }
+        __syncthreads();
+        if (round == 0) prefix = s_tmp[0];
+        else prefix = (prefix << 8) | s_tmp[0];
+        want = s_tmp[1];
+        __syncthreads();
     }
-    *bin = b;
-    *within = want - acc;
+    return prefix;
 }
 
-template <int PASS>
-__global__ void __launch_bounds__(256) thr_hist_kernel(const ThrArgs a) {
-    const int bhx = blockIdx.y;  // (b,h) * 2 + tensor
-    const int bh = bhx >> 1, x = bhx & 1;
-    __shared__ uint32_t sh[2][256];
-    __shared__ int s_bin[2];
-    sh[0][threadIdx.x] = 0;
-    sh[1][threadIdx.x] = 0;
-    if (PASS == 2 && threadIdx.x == 0) {
-        const uint32_t* h1 = a.hist1 + (size_t)bhx * 256;
-        unsigned long long N = 0;
-        for (int b = 0; b < 256; ++b) N += h1[b];
-        int bl = 0, bu = 0;
-        if (N > 0) {
-            unsigned long long k = (unsigned long long)floor(a.alpha * (double)N / 2.0);
-            if (k > (N - 1) / 2) k = (N - 1) / 2;
-            unsigned long long w;
-            find_bin(h1, k, &bl, &w);
-            find_bin(h1, N - 1 - k, &bu, &w);
-        }
-        s_bin[0] = bl; s_bin[1] = bu;
-    }
-    __syncthreads();
+__device__ __forceinline__ unsigned long long rank_k(double alpha, unsigned long long N) {
+    unsigned long long k = (unsigned long long)floor(alpha * (double)N / 2.0);
+    if (N > 0 && k > (N - 1) / 2) k = (N - 1) / 2;
+    return k;
+}
+
+// ---- 1. sample: brackets (or the exact answer when the sample is the whole problem)
+__global__ void __launch_bounds__(256) thr_sample_kernel(const ThrArgs a) {
+    const int bhx = blockIdx.x, bh = bhx >> 1, x = bhx & 1;
+    __shared__ unsigned short s_keys[SAMPLE_TOKENS * 128];
+    __shared__ unsigned short s_nanflag[1];
+    __shared__ uint32_t hist[256], s_tmp[2], s_cnt;
     const int b_idx = bh / a.H, h_idx = bh % a.H;
     const __half* X = a.X[x] + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
-    const int t0 = blockIdx.x * THR_CHUNK_TOKENS, t1 = min(a.T, t0 + THR_CHUNK_TOKENS);
-    const int per_tok = a.D / 4;  // uint2 (4 halves) per token
+    const int ns = a.T < SAMPLE_TOKENS ? a.T : SAMPLE_TOKENS;
+    const int M = ns * a.D;
+    if (threadIdx.x == 0) s_cnt = 0;
+    __syncthreads();
+    uint32_t nn = 0;
+    for (int i = threadIdx.x; i < M; i += blockDim.x) {
+        const int s = i / a.D, c = i % a.D;
+        const long t = (long)s * a.T / ns;                        // tokens spread over the sequence
+        const unsigned short h = __half_as_ushort(X[(size_t)t * a.st + c]);
+        s_keys[i] = h;
+        if (!is_nan_bits(h)) ++nn;
+    }
+    (void)s_nanflag;
+    atomicAdd(&s_cnt, nn);
+    __syncthreads();
+    const uint32_t Mv = s_cnt;                                     // non-NaN sample values
+    auto get = [&](uint32_t i) -> uint32_t { const unsigned short h = s_keys[i]; return is_nan_bits(h) ? 0x10000u : key_of(h); };
+    Problem* pr = a.prob + bhx;
+    const bool whole = (ns == a.T);
+    if (Mv == 0) {
+        if (threadIdx.x == 0) {
+            pr->klo = 0; pr->khi = 0xFFFF; pr->cnt[0] = pr->cnt[1] = 0; pr->nan = 0; pr->done = whole ? 1u : 0u;
+            if (whole) { a.thr[(size_t)bh * 4 + 2 * x] = 0.f; a.thr[(size_t)bh * 4 + 2 * x + 1] = 0.f; }
+        }
+        return;
+    }
+    uint32_t r_lo, r_hi;
+    if (whole) {
+        const unsigned long long k = rank_k(a.alpha, Mv);
+        r_lo = (uint32_t)k; r_hi = (uint32_t)(Mv - 1 - k);
+    } else {
+        // rank of about twice the wanted tail mass plus four standard deviations of the sample count
+        const double f2 = a.alpha * (double)Mv;                  // 2 * (alpha/2) * Mv
+        uint32_t r = (uint32_t)ceil(f2 + 4.0 * sqrt(f2 + 1.0) + 2.0);
+        if (r > (Mv - 1) / 2) r = (Mv - 1) / 2;
+        r_lo = r; r_hi = Mv - 1 - r;
+    }
+    const uint32_t klo = cta_select(get, (uint32_t)M, r_lo, hist, s_tmp);
+    const uint32_t khi = cta_select(get, (uint32_t)M, r_hi, hist, s_tmp);
+    if (threadIdx.x == 0) {
+        pr->klo = klo; pr->khi = khi; pr->cnt[0] = pr->cnt[1] = 0; pr->nan = 0; pr->done = whole ? 1u : 0u;
+        if (whole) {
+            a.thr[(size_t)bh * 4 + 2 * x] = float_of_key(klo);
+            a.thr[(size_t)bh * 4 + 2 * x + 1] = float_of_key(khi);
+        }
+    }
+}
+
+// ---- 2. the one pass over the data: compaction of the tail candidates
+__global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
+    const int bhx = blockIdx.y, bh = bhx >> 1, x = bhx & 1;
+    Problem* pr = a.prob + bhx;
+    if (pr->done) return;
+    __shared__ unsigned short s_list[2][CTA_LIST];
+    __shared__ uint32_t s_n[2], s_base[2], s_nan;
+    if (threadIdx.x < 2) s_n[threadIdx.x] = 0;
+    if (threadIdx.x == 2) s_nan = 0;
+    __syncthreads();
+    const float flo = float_of_key(pr->klo), fhi = float_of_key(pr->khi);
+    const __half2 lo2 = __float2half2_rn(flo), hi2 = __float2half2_rn(fhi);   // exact: both are binary16 values
+    const int b_idx = bh / a.H, h_idx = bh % a.H;
+    const __half* X = a.X[x] + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
+    const int t0 = blockIdx.x * SCAN_TOKENS, t1 = min(a.T, t0 + SCAN_TOKENS);
+    const int per_tok = a.D / 8;                                 // 16-byte pieces per token
     const int n = (t1 - t0) * per_tok;
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const int t = t0 + i / per_tok, c = (i % per_tok) * 4;
-        const uint2 raw = *reinterpret_cast<const uint2*>(X + (size_t)t * a.st + c);
-        const unsigned short hv[4] = {(unsigned short)(raw.x & 0xFFFF), (unsigned short)(raw.x >> 16),
-                                      (unsigned short)(raw.y & 0xFFFF), (unsigned short)(raw.y >> 16)};
+        const int t = t0 + i / per_tok, c = (i % per_tok) * 8;
+        const uint4 raw = *reinterpret_cast<const uint4*>(X + (size_t)t * a.st + c);
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        uint32_t any = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            if (is_nan_bits(hv[j])) continue;
-            const uint32_t key = key_of(hv[j]);
-            if (PASS == 1) {
-                atomicAdd(&sh[0][key >> 8], 1u);
-            } else {
-                if ((int)(key >> 8) == s_bin[0]) atomicAdd(&sh[0][key & 255], 1u);
-                if ((int)(key >> 8) == s_bin[1]) atomicAdd(&sh[1][key & 255], 1u);
+            const __half2 v = *reinterpret_cast<const __half2*>(&w[j]);
+            // candidates and NaNs: everything that is not inside [lo, hi]
+            any |= ~(__hge2_mask(v, lo2) & __hle2_mask(v, hi2));
+        }
+        if (any) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const unsigned short h = (unsigned short)((w[j >> 1] >> (16 * (j & 1))) & 0xFFFF);
+                if (is_nan_bits(h)) { atomicAdd(&s_nan, 1u); continue; }
+                const float f = __half2float(__ushort_as_half(h));
+                const int side = f < flo ? 0 : (f > fhi ? 1 : -1);
+                if (side >= 0) {
+                    const uint32_t pos = atomicAdd(&s_n[side], 1u);
+                    if (pos < CTA_LIST) s_list[side][pos] = (unsigned short)key_of(h);
+                }
             }
         }
     }
     __syncthreads();
-    if (PASS == 1) {
-        if (sh[0][threadIdx.x]) atomicAdd(&a.hist1[(size_t)bhx * 256 + threadIdx.x], sh[0][threadIdx.x]);
-    } else {
-        if (sh[0][threadIdx.x]) atomicAdd(&a.hist2[((size_t)bhx * 2 + 0) * 256 + threadIdx.x], sh[0][threadIdx.x]);
-        if (sh[1][threadIdx.x]) atomicAdd(&a.hist2[((size_t)bhx * 2 + 1) * 256 + threadIdx.x], sh[1][threadIdx.x]);
+    if (threadIdx.x < 2) s_base[threadIdx.x] = s_n[threadIdx.x] ? atomicAdd(&pr->cnt[threadIdx.x], s_n[threadIdx.x]) : 0u;
+    if (threadIdx.x == 2 && s_nan) atomicAdd(&pr->nan, s_nan);
+    __syncthreads();
+#pragma unroll
+    for (int side = 0; side < 2; ++side) {
+        const uint32_t cnt = s_n[side];
+        // a CTA list that overflowed makes the global count exceed what was stored: the select
+        // kernel sees cnt > cap or a hole and falls back; mark it by a huge count
+        if (cnt > CTA_LIST) { if (threadIdx.x == 0) atomicAdd(&pr->cnt[side], 0x40000000u); continue; }
+        unsigned short* dst = a.list + ((size_t)bhx * 2 + side) * a.cap;
+        for (uint32_t i = threadIdx.x; i < cnt; i += blockDim.x) {
+            const uint32_t pos = s_base[side] + i;
+            if (pos < a.cap) dst[pos] = s_list[side][i];
+        }
     }
 }
 
-__global__ void thr_final_kernel(const ThrArgs a, int n_problems) {
-    const int bhx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (bhx >= n_problems) return;
-    const uint32_t* h1 = a.hist1 + (size_t)bhx * 256;
-    unsigned long long N = 0;
-    for (int b = 0; b < 256; ++b) N += h1[b];
+// ---- 3. exact select among the candidates, exact fallback over the data when that is not possible
+__global__ void __launch_bounds__(256) thr_select_kernel(const ThrArgs a) {
+    const int bhx = blockIdx.x, bh = bhx >> 1, x = bhx & 1;
+    Problem* pr = a.prob + bhx;
+    if (pr->done) return;
+    __shared__ uint32_t hist[256], s_tmp[2];
+    const unsigned long long total = (unsigned long long)a.T * a.D;
+    const unsigned long long N = total - pr->nan;
     float lo = 0.f, hi = 0.f;
     if (N > 0) {
-        unsigned long long k = (unsigned long long)floor(a.alpha * (double)N / 2.0);
-        if (k > (N - 1) / 2) k = (N - 1) / 2;
-        int bl, bu, ll, lu;
-        unsigned long long wl, wu, dummy;
-        find_bin(h1, k, &bl, &wl);
-        find_bin(h1, N - 1 - k, &bu, &wu);
-        find_bin(a.hist2 + ((size_t)bhx * 2 + 0) * 256, wl, &ll, &dummy);
-        find_bin(a.hist2 + ((size_t)bhx * 2 + 1) * 256, wu, &lu, &dummy);
-        lo = __half2float(__ushort_as_half(half_of_key(((uint32_t)bl << 8) | (uint32_t)ll)));
-        hi = __half2float(__ushort_as_half(half_of_key(((uint32_t)bu << 8) | (uint32_t)lu)));
+        const unsigned long long k = rank_k(a.alpha, N);
+        const uint32_t c0 = pr->cnt[0], c1 = pr->cnt[1];
+        const bool ok = c0 > k && c1 > k && c0 <= a.cap && c1 <= a.cap;
+        if (ok) {
+            const unsigned short* l0 = a.list + ((size_t)bhx * 2 + 0) * a.cap;
+            const unsigned short* l1 = a.list + ((size_t)bhx * 2 + 1) * a.cap;
+            auto get0 = [&](uint32_t i) -> uint32_t { return l0[i]; };
+            auto get1 = [&](uint32_t i) -> uint32_t { return l1[i]; };
+            lo = float_of_key(cta_select(get0, c0, (uint32_t)k, hist, s_tmp));           // k-th smallest
+            hi = float_of_key(cta_select(get1, c1, (uint32_t)(c1 - 1 - k), hist, s_tmp)); // k-th largest
+        } else {
+            // bracket too tight or list overflow: two-pass radix select over this problem's data
+            const int b_idx = bh / a.H, h_idx = bh % a.H;
+            const __half* X = a.X[x] + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
+            const int D = a.D;
+            auto getx = [&](uint32_t i) -> uint32_t {
+                const unsigned short h = __half_as_ushort(X[(size_t)(i / D) * a.st + (i % D)]);
+                return is_nan_bits(h) ? 0x10000u : key_of(h);
+            };
+            lo = float_of_key(cta_select(getx, (uint32_t)total, (uint32_t)k, hist, s_tmp));
+            hi = float_of_key(cta_select(getx, (uint32_t)total, (uint32_t)(N - 1 - k), hist, s_tmp));
+        }
     }
-    a.thr[(size_t)(bhx >> 1) * 4 + (bhx & 1) * 2 + 0] = lo;
-    a.thr[(size_t)(bhx >> 1) * 4 + (bhx & 1) * 2 + 1] = hi;
+    if (threadIdx.x == 0) {
+        a.thr[(size_t)bh * 4 + 2 * x] = lo;
+        a.thr[(size_t)bh * 4 + 2 * x + 1] = hi;
+    }
+}
+
+uint32_t list_capacity(const qaq_config* cfg, int n_tokens) {
+    // expected candidates per tail: (alpha + margin) * N; keep twice that, at least 4096
+    const double N = (double)n_tokens * cfg->head_dim;
+    double want = 2.0 * (cfg->outlier_frac * N + 8.0 * sqrt(cfg->outlier_frac * N + 64.0) + 64.0) + 4096.0;
+    if (want > N) want = N;
+    uint32_t cap = (uint32_t)want;
+    return (cap + 63u) & ~63u;
 }
 
 }  // namespace
 
 extern "C" qaq_status qaq_thresholds_workspace_bytes(const qaq_config* cfg, size_t* host_out) {
-    if (!cfg || !host_out || cfg->batch < 1 || cfg->heads < 1) return QAQ_ERR_INVALID_ARG;
-    *host_out = (size_t)cfg->batch * cfg->heads * 2 * 3 * 256 * sizeof(uint32_t);
+    if (!cfg || !host_out || cfg->batch < 1 || cfg->heads < 1 || cfg->max_tokens < 1) return QAQ_ERR_INVALID_ARG;
+    const size_t P = (size_t)cfg->batch * cfg->heads * 2;
+    *host_out = P * sizeof(Problem) + P * 2 * (size_t)list_capacity(cfg, cfg->max_tokens) * sizeof(unsigned short) + 256;
     return QAQ_OK;
 }
 
@@ -132,7 +264,8 @@ extern "C" qaq_status qaq_outlier_thresholds(const qaq_config* cfg, const void* 
     if (!cfg || !K || !V || !thr || !ws || n_tokens < 1) return QAQ_ERR_INVALID_ARG;
     if (!qaq_dim_ok(cfg->head_dim)) return QAQ_ERR_UNSUPPORTED_SHAPE;
     if (!(cfg->outlier_frac >= 0.0 && cfg->outlier_frac <= 1.0)) return QAQ_ERR_INVALID_ARG;
-    if (((uintptr_t)K & 7) || ((uintptr_t)V & 7) || (stride_b & 3) || (stride_h & 3) || (stride_t & 3) ||
+    if ((double)n_tokens * cfg->head_dim >= 4.0e9) return QAQ_ERR_UNSUPPORTED_SHAPE;
+    if (((uintptr_t)K & 15) || ((uintptr_t)V & 15) || (stride_b & 7) || (stride_h & 7) || (stride_t & 7) ||
         stride_t < cfg->head_dim)
         return QAQ_ERR_INVALID_ARG;
     size_t need = 0;
@@ -144,14 +277,20 @@ extern "C" qaq_status qaq_outlier_thresholds(const qaq_config* cfg, const void* 
     a.X[0] = (const __half*)K; a.X[1] = (const __half*)V;
     a.sb = stride_b; a.sh = stride_h; a.st = stride_t;
     a.H = cfg->heads; a.T = n_tokens; a.D = cfg->head_dim; a.alpha = cfg->outlier_frac;
-    a.hist1 = (uint32_t*)ws;
-    a.hist2 = a.hist1 + (size_t)BH * 2 * 256;
+    a.prob = (Problem*)ws;
+    // the candidate lists take whatever the workspace offers beyond the problem records
+    const size_t head = ((size_t)BH * 2 * sizeof(Problem) + 255) / 256 * 256;
+    const size_t per_list = (ws_bytes - head) / ((size_t)BH * 4 * sizeof(unsigned short));
+    a.cap = (uint32_t)(per_list > 0x3FFFFFC0u ? 0x3FFFFFC0u : per_list) & ~63u;
+    if (a.cap < 64) return QAQ_ERR_WORKSPACE;
+    a.list = (unsigned short*)((char*)ws + head);
     a.thr = thr;
-    QAQ_CUDA_TRY(cudaMemsetAsync(ws, 0, need, s));
-    dim3 grid((n_tokens + THR_CHUNK_TOKENS - 1) / THR_CHUNK_TOKENS, BH * 2);
-    thr_hist_kernel<1><<<grid, 256, 0, s>>>(a);
-    thr_hist_kernel<2><<<grid, 256, 0, s>>>(a);
-    thr_final_kernel<<<(BH * 2 + 63) / 64, 64, 0, s>>>(a, BH * 2);
+    thr_sample_kernel<<<BH * 2, 256, 0, s>>>(a);
+    if (n_tokens > SAMPLE_TOKENS) {
+        dim3 grid((n_tokens + SCAN_TOKENS - 1) / SCAN_TOKENS, BH * 2);
+        thr_scan_kernel<<<grid, 256, 0, s>>>(a);
+        thr_select_kernel<<<BH * 2, 256, 0, s>>>(a);
+    }
     QAQ_CUDA_TRY(cudaGetLastError());
     return QAQ_OK;
 }
