@@ -147,40 +147,55 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
     Problem* pr = a.prob + bhx;
     if (pr->done) return;
     __shared__ unsigned short s_list[2][CTA_LIST];
-    __shared__ uint32_t s_n[2], s_base[2], s_nan;
+    __shared__ uint4 s_flag[SCAN_TOKENS * 16];                    // 16-byte pieces with something outside [lo, hi]
+    __shared__ uint32_t s_n[2], s_base[2], s_nan, s_nflag;
     if (threadIdx.x < 2) s_n[threadIdx.x] = 0;
     if (threadIdx.x == 2) s_nan = 0;
+    if (threadIdx.x == 3) s_nflag = 0;
     __syncthreads();
     const float flo = float_of_key(pr->klo), fhi = float_of_key(pr->khi);
     const __half2 lo2 = __float2half2_rn(flo), hi2 = __float2half2_rn(fhi);   // exact: both are binary16 values
     const int b_idx = bh / a.H, h_idx = bh % a.H;
     const __half* X = a.X[x] + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
     const int t0 = blockIdx.x * SCAN_TOKENS, t1 = min(a.T, t0 + SCAN_TOKENS);
-    const int per_tok = a.D / 8;                                 // 16-byte pieces per token
-    const int n = (t1 - t0) * per_tok;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const int t = t0 + i / per_tok, c = (i % per_tok) * 8;
-        const uint4 raw = *reinterpret_cast<const uint4*>(X + (size_t)t * a.st + c);
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-        uint32_t any = 0;
+    const int tok_shift = 31 - __clz(a.D / 8);                   // 16-byte pieces per token is a power of two
+    const int n = (t1 - t0) << tok_shift;
+    for (int i0 = 0; i0 < n; i0 += 4 * 256) {
+        // four independent 16-byte loads per thread before any of them is looked at
+        uint4 raw[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const __half2 v = *reinterpret_cast<const __half2*>(&w[j]);
-            // candidates and NaNs: everything that is not inside [lo, hi]
-            any |= ~(__hge2_mask(v, lo2) & __hle2_mask(v, hi2));
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * 256 + threadIdx.x;
+            raw[u] = make_uint4(0, 0, 0, 0);
+            if (i < n) raw[u] = *reinterpret_cast<const uint4*>(X + (size_t)(t0 + (i >> tok_shift)) * a.st + ((i & ((1 << tok_shift) - 1)) << 3));
         }
-        if (any) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const unsigned short h = (unsigned short)((w[j >> 1] >> (16 * (j & 1))) & 0xFFFF);
-                if (is_nan_bits(h)) { atomicAdd(&s_nan, 1u); continue; }
-                const float f = __half2float(__ushort_as_half(h));
-                const int side = f < flo ? 0 : (f > fhi ? 1 : -1);
-                if (side >= 0) {
-                    const uint32_t pos = atomicAdd(&s_n[side], 1u);
-                    if (pos < CTA_LIST) s_list[side][pos] = (unsigned short)key_of(h);
-                }
+        for (int u = 0; u < 4; ++u) {
+            // cheap filter: almost all entries are inside [lo, hi]; a 16-byte piece holding anything
+            // else is set aside and looked at entry by entry afterwards, with all lanes busy
+            const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+            bool inside = true;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const __half2 v = *reinterpret_cast<const __half2*>(&w[j]);
+                inside = inside && __hbge2(v, lo2) && __hble2(v, hi2);
             }
+            if (!inside && i0 + u * 256 + (int)threadIdx.x < n) s_flag[atomicAdd(&s_nflag, 1u)] = raw[u];
+        }
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < s_nflag; i += blockDim.x) {
+        const uint4 r = s_flag[i];
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const unsigned short h = (unsigned short)((w[j >> 1] >> (16 * (j & 1))) & 0xFFFF);
+            const float f = __half2float(__ushort_as_half(h));
+            if (f >= flo && f <= fhi) continue;
+            if (is_nan_bits(h)) { atomicAdd(&s_nan, 1u); continue; }
+            const int side = f < flo ? 0 : 1;
+            const uint32_t pos = atomicAdd(&s_n[side], 1u);
+            if (pos < CTA_LIST) s_list[side][pos] = (unsigned short)key_of(h);
         }
     }
     __syncthreads();
