@@ -115,12 +115,33 @@ __device__ __forceinline__ void store_words(uint8_t* dst, const uint32_t* w, int
     }
 }
 
+// space from a (b,h) pool: `whole` tiles take a rounded-up amount in one atomic; a tile that is
+// being continued takes the exact amount and is padded to the unit when it closes
+__device__ __forceinline__ uint32_t pool_take(uint32_t* pool, uint32_t amount, uint32_t unit_mask, bool whole, bool closes) {
+    uint32_t base;
+    if (whole) {
+        base = atomicAdd(pool, (amount + unit_mask) & ~unit_mask);
+    } else {
+        base = atomicAdd(pool, amount);
+        if (closes) {
+            const uint32_t pad = (0u - (base + amount)) & unit_mask;
+            if (pad) atomicAdd(pool, pad);
+        }
+    }
+    return base;
+}
+
 // One CTA = one tile of 64 tokens of one (b,h); P = D/32 lanes own a token, each lane 32
 // consecutive channels (64 bytes) of K and of V, kept in registers across all phases.
+// Order of work (barriers in brackets): loads, attention window, outlier masks and ranges
+// [0] widths [A] warp 0 scans the tile and takes pool space with four atomics in flight at once
+// while every warp computes its codes [B] planes into a shared-memory image of the tile
+// [C] the image goes out with 16-byte stores; outlier entries and per-token metadata follow.
 template <int D, bool SELECT_ONLY>
 __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const QuantArgs a) {
     constexpr int P = D / 32;            // lanes per token
     constexpr int ALIGN = D / 8 >= 16 ? 16 : D / 8;  // alignment of a token's bytes inside a tile
+    constexpr int NT = 2 * D;            // threads
     const int bh = blockIdx.y;
     const int tile = a.first_tile + blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -136,8 +157,9 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
     __shared__ uint8_t s_nv[QAQ_TILE];
     __shared__ uint32_t s_len[2][QAQ_TILE];   // bytes, then exclusive byte offsets
     __shared__ uint32_t s_cnt[2][QAQ_TILE];   // outlier counts, then exclusive offsets
-    __shared__ uint32_t s_base[2], s_obase[2], s_olimit[2];
+    __shared__ uint32_t s_tot[2], s_base[2], s_obase[2], s_olimit[2];
     __shared__ int s_skip;
+    __shared__ __align__(16) uint8_t s_img[SELECT_ONLY ? 1 : 2][SELECT_ONLY ? 16 : QAQ_TILE * D];  // packed tile, K and V
 
     const float* thr = a.thr + (size_t)bh * 4;
     const bool given = a.bitsK != nullptr;
@@ -160,7 +182,7 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
         }
     }
 
-    // ---- phase 0: attention window; P threads share the rows of one token
+    // ---- attention window; P threads share the rows of one token
     {
         const int g = tid / QAQ_TILE, tok = tid % QAQ_TILE;
         float m = __int_as_float(0xff800000);
@@ -178,12 +200,10 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
             s_len[0][tok] = 0; s_len[1][tok] = 0; s_cnt[0][tok] = 0; s_cnt[1][tok] = 0;
         }
     }
-    __syncthreads();
 
-    // ---- phase 1: outlier masks, range of the rest, widths
-    uint32_t inl[2];
+    // ---- outlier masks and range of the rest (register work, needs nothing from shared memory)
+    uint32_t inl[2], cntx[2];
     float mnf[2], mxf[2];
-    int Bx[2];
 #pragma unroll
     for (int x = 0; x < 2; ++x) {
         // thresholds as binary16 bounds that decide exactly like the binary32 ones on binary16 data
@@ -200,12 +220,20 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
         uint32_t cnt = 32u - (uint32_t)__popc(inl[x]);
 #pragma unroll
         for (int o = 1; o < P; o <<= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
+        mnf[x] = mn; mxf[x] = mx; cntx[x] = cnt;
+    }
+    __syncthreads();   // [0] window partials visible
+
+    // ---- widths
+    int Bx[2];
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
         int B;
         if (given) {
             B = valid ? (x ? a.bitsV : a.bitsK)[(size_t)bh * a.n_new + tn] : 0;
             B = B < 1 ? 1 : (B > 8 ? 8 : B);
         } else {
-            const float r = __fsub_rn(mx, mn);
+            const float r = __fsub_rn(mxf[x], mnf[x]);
             if (x == 0) {
                 B = ladder(r, a.cK, a.bmin, a.bmax);
             } else {
@@ -215,23 +243,23 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
                 B = (s_nv[slot] == 0) ? a.bmax : ladder(__fmul_rn(r, sh), a.cV, a.bmin, a.bmax);
             }
         }
-        mnf[x] = mn; mxf[x] = mx; Bx[x] = B;
+        Bx[x] = valid ? B : 0;
         if (valid && p == 0) {
             s_len[x][slot] = (uint32_t)(D * B / 8);
-            s_cnt[x][slot] = cnt;
+            s_cnt[x][slot] = cntx[x];
             if (SELECT_ONLY) (x ? a.out_bitsV : a.out_bitsK)[(size_t)bh * a.n_new + tn] = (uint8_t)B;
         }
     }
     if (SELECT_ONLY) return;
-    __syncthreads();
+    __syncthreads();   // [A] byte lengths and outlier counts visible
 
-    // ---- phase 2: scans over the tile and pool allocation
+    // ---- warp 0: scans over the tile; lanes 0..3 each take space from one pool (four atomics in flight)
+    const bool starts = (s_lo == 0), closes = (s_hi == QAQ_TILE), whole = starts && closes;
+    uint32_t my_base = 0, my_amount = 0;
     if (warp == 0) {
-        const bool starts = (s_lo == 0), closes = (s_hi == QAQ_TILE), whole = starts && closes;
-        if (lane == 0) s_skip = 0;
+        uint32_t amount[2][2];   // [tensor][0: bytes, 1: outliers]
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
-            const TensorStore& ts = x ? a.v : a.k;
             uint32_t l0 = s_len[x][lane], l1 = s_len[x][lane + 32];
             uint32_t c0 = s_cnt[x][lane], c1 = s_cnt[x][lane + 32];
             uint32_t il0 = l0, il1 = l1, ic0 = c0, ic1 = c1;
@@ -245,59 +273,28 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
             const uint32_t ctot0 = __shfl_sync(0xFFFFFFFFu, ic0, 31), ctot1 = __shfl_sync(0xFFFFFFFFu, ic1, 31);
             s_len[x][lane] = il0 - l0; s_len[x][lane + 32] = tot0 + il1 - l1;
             s_cnt[x][lane] = ic0 - c0; s_cnt[x][lane + 32] = ctot0 + ic1 - c1;
-            if (lane == 0) {
-                const uint32_t bytes = tot0 + tot1, cnt = ctot0 + ctot1;
-                const size_t ti = (size_t)bh * a.ntiles + tile;
-                uint32_t base;
-                if (whole) {
-                    base = atomicAdd(&ts.pool_end[bh], (bytes + 15u) & ~15u);
-                } else {
-                    base = atomicAdd(&ts.pool_end[bh], bytes);
-                    if (closes) {
-                        const uint32_t pad = (0u - (base + bytes)) & 15u;
-                        if (pad) atomicAdd(&ts.pool_end[bh], pad);
-                    }
-                }
-                if ((size_t)base + bytes + 16 > a.pool_bytes) { atomicMax(a.status, (int)QAQ_ERR_CAPACITY); s_skip = 1; }
-                if (starts) { ts.tile_off[ti] = base; ts.tile_nbytes[ti] = bytes; }
-                else ts.tile_nbytes[ti] += bytes;
-                s_base[x] = base;
-                uint32_t obase;
-                if (whole) {
-                    obase = atomicAdd(&ts.opool_end[bh], (cnt + 3u) & ~3u);
-                } else {
-                    obase = atomicAdd(&ts.opool_end[bh], cnt);
-                    if (closes) {
-                        const uint32_t pad = (0u - (obase + cnt)) & 3u;
-                        if (pad) atomicAdd(&ts.opool_end[bh], pad);
-                    }
-                }
-                const uint32_t room = obase + 8 < a.ocap ? a.ocap - 8 - obase : 0;  // 8 entries of read-ahead margin
-                const uint32_t stored = cnt < room ? cnt : room;
-                if (stored < cnt) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
-                if (starts) { ts.tile_ooff[ti] = obase; ts.tile_ocnt[ti] = stored; }
-                else ts.tile_ocnt[ti] += stored;
-                s_obase[x] = obase;
-                s_olimit[x] = obase + stored;
-            }
+            amount[x][0] = tot0 + tot1; amount[x][1] = ctot0 + ctot1;
+            if (lane == 0) s_tot[x] = amount[x][0];
+        }
+        if (lane < 4) {
+            const int x = lane >> 1, pool = lane & 1;
+            const TensorStore& ts = x ? a.v : a.k;
+            my_amount = amount[x][pool];
+            my_base = pool_take(pool ? &ts.opool_end[bh] : &ts.pool_end[bh], my_amount, pool ? 3u : 15u, whole, closes);
         }
     }
-    __syncthreads();
-    if (s_skip) return;
 
-    // ---- phase 3: codes, planes, stores, outlier list
+    // ---- codes (every warp; needs only registers): channels 4j..4j+3 in the byte lanes of creg[j]
+    uint32_t cregs[2][8];
 #pragma unroll
     for (int x = 0; x < 2; ++x) {
-        const TensorStore& ts = x ? a.v : a.k;
         const uint32_t (&v)[16] = x ? vv : vk;
-        const int B = valid ? Bx[x] : 0;
-        const float mn = mnf[x], mx = mxf[x];
-        const float step = __fmul_rn(__fsub_rn(mx, mn), __int_as_float((127 - B) << 23));
+        const int B = Bx[x];
+        const float mn = mnf[x];
+        const float step = __fmul_rn(__fsub_rn(mxf[x], mn), __int_as_float((127 - B) << 23));
         const float inv = step > 0.f ? __fdiv_rn(1.0f, step) : 0.f;
         // zero step (constant token): every code is 0, and -inf * 0 = NaN must not clamp to the top code
         const float topf = step > 0.f ? (float)((1 << B) - 1) : 0.f;
-        // codes of channels 4j..4j+3 in the byte lanes of creg[j]
-        uint32_t creg[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             uint32_t f[4];
@@ -309,9 +306,17 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
                 t = fminf(t, topf);
                 f[i] = __float_as_uint(__fadd_rd(t, 8388608.0f));   // 2^23 + floor(t): the code is the low byte (0 for -inf)
             }
-            creg[j] = prmt(prmt(f[0], f[1], 0x0040u), prmt(f[2], f[3], 0x0040u), 0x5410u);
+            cregs[x][j] = prmt(prmt(f[0], f[1], 0x0040u), prmt(f[2], f[3], 0x0040u), 0x5410u);
         }
-        uint8_t* tok = ts.codes + (size_t)bh * a.pool_bytes + s_base[x] + s_len[x][slot & (QAQ_TILE - 1)];
+    }
+    __syncthreads();   // [B] offsets inside the tile visible
+
+    // ---- planes into the shared-memory image of the tile
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+        const uint32_t (&creg)[8] = cregs[x];
+        const int B = Bx[x];
+        uint8_t* tok = s_img[x] + s_len[x][slot & (QAQ_TILE - 1)];
         if (B & 8) {
             store_words<ALIGN>(tok + p * 32, creg, 8);
         }
@@ -341,6 +346,42 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
             for (int m = 0; m < 8; ++m) acc |= (creg[m] & 0x01010101u) << m;
             *reinterpret_cast<uint32_t*>(tok + (B & 14) * (D / 8) + p * 4) = acc;
         }
+    }
+    // ---- allocation results (the atomics were issued before the codes were computed)
+    if (warp == 0 && lane < 4) {
+        const int x = lane >> 1, pool = lane & 1;
+        const TensorStore& ts = x ? a.v : a.k;
+        const size_t ti = (size_t)bh * a.ntiles + tile;
+        if (lane == 0) s_skip = 0;
+        if (pool == 0) {
+            if ((size_t)my_base + my_amount + 16 > a.pool_bytes) { atomicMax(a.status, (int)QAQ_ERR_CAPACITY); s_skip = 1; }
+            if (starts) { ts.tile_off[ti] = my_base; ts.tile_nbytes[ti] = my_amount; }
+            else ts.tile_nbytes[ti] += my_amount;
+            s_base[x] = my_base;
+        } else {
+            const uint32_t room = my_base + 8 < a.ocap ? a.ocap - 8 - my_base : 0;  // 8 entries of read-ahead margin
+            const uint32_t stored = my_amount < room ? my_amount : room;
+            if (stored < my_amount) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
+            if (starts) { ts.tile_ooff[ti] = my_base; ts.tile_ocnt[ti] = stored; }
+            else ts.tile_ocnt[ti] += stored;
+            s_obase[x] = my_base;
+            s_olimit[x] = my_base + stored;
+        }
+    }
+    __syncthreads();   // [C] image complete, pool positions known
+    if (s_skip) return;
+
+    // ---- the image goes out with vector stores; outlier list; per-token metadata
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+        const TensorStore& ts = x ? a.v : a.k;
+        uint8_t* dst = ts.codes + (size_t)bh * a.pool_bytes + s_base[x];
+        const uint32_t nb = s_tot[x];
+        for (uint32_t o = tid * ALIGN; o < nb; o += NT * ALIGN) {
+            if (ALIGN == 16) *reinterpret_cast<uint4*>(dst + o) = *reinterpret_cast<const uint4*>(s_img[x] + o);
+            else if (ALIGN == 8) *reinterpret_cast<uint2*>(dst + o) = *reinterpret_cast<const uint2*>(s_img[x] + o);
+            else *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(s_img[x] + o);
+        }
         // outliers in (token, channel) order: entries of lanes p' < p come first
         uint32_t ob = valid ? ~inl[x] : 0u;
         const uint32_t mine = (uint32_t)__popc(ob);
@@ -369,8 +410,8 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
         }
         if (valid && p == 0) {
             const size_t t = (size_t)bh * a.tmax_pad + (size_t)tile * QAQ_TILE + slot;
-            ts.bits[t] = (uint8_t)B;
-            ts.mnmx[t] = (uint32_t)__half_as_ushort(__float2half_rn(mn)) | ((uint32_t)__half_as_ushort(__float2half_rn(mx)) << 16);
+            ts.bits[t] = (uint8_t)Bx[x];
+            ts.mnmx[t] = (uint32_t)__half_as_ushort(__float2half_rn(mnf[x])) | ((uint32_t)__half_as_ushort(__float2half_rn(mxf[x])) << 16);
         }
     }
 }
