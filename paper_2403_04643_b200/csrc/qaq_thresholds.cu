@@ -46,29 +46,53 @@ struct ThrArgs {
 };
 
 // rank select (0-based rank `want`) over n 16-bit keys readable through get(i); all threads of the
-// CTA call it; hist is 256 words of shared memory.  Two rounds of an 8-bit radix select.
+// CTA (256) call it; hist is 8 x 256 words of shared memory (one histogram per warp, so that hot
+// bins are contended inside a warp only).  Two rounds of an 8-bit radix select; the bin holding the
+// wanted rank is found by warp 0 with a prefix sum over the 256 bins (8 per lane).
 template <typename Get>
 __device__ uint32_t cta_select(Get get, uint32_t n, uint32_t want, uint32_t* hist, uint32_t* s_tmp) {
     uint32_t prefix = 0;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint32_t* mine = hist + 256 * warp;
     for (int round = 0; round < 2; ++round) {
-        for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+        for (int i = threadIdx.x; i < 8 * 256; i += blockDim.x) hist[i] = 0;
         __syncthreads();
         for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
             const uint32_t k = get(i);
             if (k > 0xFFFFu) continue;                      // NaN marker
-            if (round == 0) atomicAdd(&hist[k >> 8], 1u);
-            else if ((k >> 8) == prefix) atomicAdd(&hist[k & 255], 1u);
+            if (round == 0) atomicAdd(&mine[k >> 8], 1u);
+            else if ((k >> 8) == prefix) atomicAdd(&mine[k & 255], 1u);
         }
         __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t acc = 0;
-            int b = 0;
-            for (; b < 255; ++b) {
-                if (acc + hist[b] > want) break;
-                acc += hist[b];
+        if (warp == 0) {
+            uint32_t c[8], tot = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                uint32_t v = 0;
+#pragma unroll
+                for (int w = 0; w < 8; ++w) v += hist[256 * w + 8 * lane + j];
+                c[j] = v; tot += v;
             }
-            s_tmp[0] = (uint32_t)b;
-            s_tmp[1] = want - acc;
+            uint32_t inc = tot;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                if (lane >= d) inc += t;
+            }
+            uint32_t acc = inc - tot;                       // keys in the bins before this lane's eight
+            const uint32_t all = __shfl_sync(0xFFFFFFFFu, inc, 31);
+            const uint32_t w2 = want < all ? want : (all ? all - 1 : 0);   // defensive clamp
+            if (tot > 0 && w2 >= acc && w2 < acc + tot) {   // exactly one lane
+                int bsel = 0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (w2 >= acc + c[j] && j < 7) { acc += c[j]; bsel = j + 1; }
+                    else break;
+                }
+                s_tmp[0] = (uint32_t)(8 * lane + bsel);
+                s_tmp[1] = w2 - acc;
+            }
+            if (all == 0 && lane == 0) { s_tmp[0] = 0; s_tmp[1] = 0; }
         }
         __syncthreads();
         if (round == 0) prefix = s_tmp[0];
@@ -88,9 +112,9 @@ __device__ __forceinline__ unsigned long long rank_k(double alpha, unsigned long
 // ---- 1. sample: brackets (or the exact answer when the sample is the whole problem)
 __global__ void __launch_bounds__(256) thr_sample_kernel(const ThrArgs a) {
     const int bhx = blockIdx.x, bh = bhx >> 1, x = bhx & 1;
-    __shared__ unsigned short s_keys[SAMPLE_TOKENS * 128];
+    __shared__ __align__(16) unsigned short s_keys[SAMPLE_TOKENS * 128];
     __shared__ unsigned short s_nanflag[1];
-    __shared__ uint32_t hist[256], s_tmp[2], s_cnt;
+    __shared__ uint32_t hist[8 * 256], s_tmp[2], s_cnt;
     const int b_idx = bh / a.H, h_idx = bh % a.H;
     const __half* X = a.X[x] + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
     const int ns = a.T < SAMPLE_TOKENS ? a.T : SAMPLE_TOKENS;
@@ -98,12 +122,15 @@ __global__ void __launch_bounds__(256) thr_sample_kernel(const ThrArgs a) {
     if (threadIdx.x == 0) s_cnt = 0;
     __syncthreads();
     uint32_t nn = 0;
-    for (int i = threadIdx.x; i < M; i += blockDim.x) {
-        const int s = i / a.D, c = i % a.D;
+    for (int i = threadIdx.x; i < M / 8; i += blockDim.x) {    // 16-byte pieces
+        const int s = (i * 8) / a.D, c = (i * 8) % a.D;
         const long t = (long)s * a.T / ns;                        // tokens spread over the sequence
-        const unsigned short h = __half_as_ushort(X[(size_t)t * a.st + c]);
-        s_keys[i] = h;
-        if (!is_nan_bits(h)) ++nn;
+        const uint4 r = *reinterpret_cast<const uint4*>(X + (size_t)t * a.st + c);
+        *reinterpret_cast<uint4*>(&s_keys[8 * i]) = r;
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (!is_nan_bits((unsigned short)((w[j >> 1] >> (16 * (j & 1))) & 0xFFFF))) ++nn;
     }
     (void)s_nanflag;
     atomicAdd(&s_cnt, nn);
@@ -187,13 +214,21 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
     for (uint32_t i = threadIdx.x; i < s_nflag; i += blockDim.x) {
         const uint4 r = s_flag[i];
         const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+        // bit j / 16 + j: low / high half of word j is not inside [lo, hi] (a candidate or a NaN)
+        uint32_t out = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const unsigned short h = (unsigned short)((w[j >> 1] >> (16 * (j & 1))) & 0xFFFF);
-            const float f = __half2float(__ushort_as_half(h));
-            if (f >= flo && f <= fhi) continue;
+        for (int j = 0; j < 4; ++j) {
+            const __half2 v = *reinterpret_cast<const __half2*>(&w[j]);
+            out |= (~(__hge2_mask(v, lo2) & __hle2_mask(v, hi2)) & 0x00010001u) << j;
+        }
+        while (out) {
+            const int bit = __ffs(out) - 1;
+            out &= out - 1;
+            const int j = bit & 3;
+            const uint32_t wj = (j & 2) ? ((j & 1) ? w[3] : w[2]) : ((j & 1) ? w[1] : w[0]);
+            const unsigned short h = (unsigned short)((bit >> 4) ? (wj >> 16) : (wj & 0xFFFF));
             if (is_nan_bits(h)) { atomicAdd(&s_nan, 1u); continue; }
-            const int side = f < flo ? 0 : 1;
+            const int side = __half2float(__ushort_as_half(h)) < flo ? 0 : 1;   // outside [lo, hi]: below lo or above hi
             const uint32_t pos = atomicAdd(&s_n[side], 1u);
             if (pos < CTA_LIST) s_list[side][pos] = (unsigned short)key_of(h);
         }
@@ -221,7 +256,7 @@ __global__ void __launch_bounds__(256) thr_select_kernel(const ThrArgs a) {
     const int bhx = blockIdx.x, bh = bhx >> 1, x = bhx & 1;
     Problem* pr = a.prob + bhx;
     if (pr->done) return;
-    __shared__ uint32_t hist[256], s_tmp[2];
+    __shared__ uint32_t hist[8 * 256], s_tmp[2];
     const unsigned long long total = (unsigned long long)a.T * a.D;
     const unsigned long long N = total - pr->nan;
     float lo = 0.f, hi = 0.f;
@@ -256,9 +291,9 @@ __global__ void __launch_bounds__(256) thr_select_kernel(const ThrArgs a) {
 }
 
 uint32_t list_capacity(const qaq_config* cfg, int n_tokens) {
-    // expected candidates per tail: (alpha + margin) * N; keep twice that, at least 4096
+    // expected candidates per tail: (alpha + margin) * N; keep three times that, at least 4096
     const double N = (double)n_tokens * cfg->head_dim;
-    double want = 2.0 * (cfg->outlier_frac * N + 8.0 * sqrt(cfg->outlier_frac * N + 64.0) + 64.0) + 4096.0;
+    double want = 3.0 * (cfg->outlier_frac * N + 8.0 * sqrt(cfg->outlier_frac * N + 64.0) + 64.0) + 4096.0;
     if (want > N) want = N;
     uint32_t cap = (uint32_t)want;
     return (cap + 63u) & ~63u;
