@@ -207,7 +207,16 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
                 const __half2 v = *reinterpret_cast<const __half2*>(&w[j]);
                 inside = inside && __hbge2(v, lo2) && __hble2(v, hi2);
             }
-            if (!inside && i0 + u * 256 + (int)threadIdx.x < n) s_flag[atomicAdd(&s_nflag, 1u)] = raw[u];
+            // one shared-memory reservation per warp for its flagged pieces
+            const bool flag = !inside && i0 + u * 256 + (int)threadIdx.x < n;
+            const unsigned bal = __ballot_sync(0xFFFFFFFFu, flag);
+            if (bal) {
+                const int lane = threadIdx.x & 31;
+                uint32_t base = 0;
+                if (lane == 0) base = atomicAdd(&s_nflag, (uint32_t)__popc(bal));
+                base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                if (flag) s_flag[base + __popc(bal & ((1u << lane) - 1u))] = raw[u];
+            }
         }
     }
     __syncthreads();
