@@ -176,6 +176,7 @@ def main():
         raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
     from paper_2403_04643_b200 import qaq
     from paper_2403_04643_b200.calibrate import calibrate
+    from paper_2403_04643_b200 import dist as qdist
     qaq.lib()
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -187,7 +188,7 @@ def main():
     scale = 1.0 / math.sqrt(D)
     cfg = qaq.make_config(wl.batch, wl.heads, D, T, wl.bits_min, wl.bits_max, W, wl.alpha)
     # ---- resident inputs (each rank its own batch: seed offset by rank)
-    wl_r = synth.scaled(wl, seed=wl.seed + 7777 * rank)
+    wl_r = synth.scaled(wl, seed=qdist.rank_seed(wl.seed, rank))
     layers = []
     for l in range(L):
         K, V = synth.make_kv(wl_r, l, device=dev)
@@ -220,16 +221,13 @@ def main():
         return e
 
     def barrier():
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
-        torch.cuda.synchronize()
+        qdist.barrier(dev)
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()          # started before the warm-up: nvidia-smi needs a moment to come up
     for _ in range(args.warmup):
         step()
     barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     timers = {"thr": ([], []), "quant": ([], []), "dec": ([], [])}
     e0 = ev()
     for _ in range(args.steps):
@@ -237,12 +235,7 @@ def main():
     e1 = ev()
     barrier()
     clocks = sampler.stop()
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total, _ = qdist.aggregate(e0.elapsed_time(e1), 1.0, dev)     # slowest rank
     ms_step = ms_total / args.steps
     stage_ms = {k: sum(a.elapsed_time(b) for a, b in zip(*v)) / len(v[0]) for k, v in timers.items()}
 
@@ -304,12 +297,7 @@ def main():
             e2e_step()
         b = ev()
         barrier()
-        ms_e2e = a.elapsed_time(b) / n_e2e
-        if world > 1:
-            import torch.distributed as dist
-            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e, _ = qdist.aggregate(a.elapsed_time(b) / n_e2e, 1.0, dev)
         h2d = L * (hK.numel() * 2 * 2 + hr.numel() * 4 + hn.numel() + ht.numel() * 4 + hq.numel() * 2)
         e2e_bytes = L * (ab["quantize"] + ab["decode"])
         out["e2e"] = {"value": round(world * e2e_bytes / (ms_e2e * 1e-3) / 1e9, 2), "unit": "GB/s",
