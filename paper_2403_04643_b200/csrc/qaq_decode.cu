@@ -143,6 +143,7 @@ __device__ __forceinline__ void plane_axpy(const uint32_t (&words)[8], const uns
 }
 
 constexpr int UNIT = QAQ_TILE / 2;   // tokens a warp handles at a time (half a tile)
+constexpr int OSTAGE = 192;          // outlier entries per tile and tensor staged in shared memory
 
 // per-warp scratch for the half tile a warp is working on
 template <int D>
@@ -160,6 +161,7 @@ struct WarpScratch {
     // work items grouped by plane width (8, 4, 2, 1):
     //   byte offset of the plane inside the half tile | shift of the piece << 16 | token << 24
     uint32_t item[2][3 * UNIT];
+    alignas(16) uint32_t outl[2][OSTAGE];   // the tile's outlier entries (K, V); longer lists continue in global memory
 };
 
 template <int D>
@@ -317,6 +319,11 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
         for (uint32_t o = lane * ALIGN; o < nbytes; o += 32 * ALIGN) cp_async<ALIGN>(dst + o, src + o);
     };
 
+    auto stage_outl = [&](int x, uint32_t first, uint32_t count) {   // entries are 4 bytes, lists start 16-byte aligned
+        const uint32_t* src = (x ? a.v.outl : a.k.outl) + (size_t)bh * a.ocap + first;
+        const uint32_t n16 = ((count < (uint32_t)OSTAGE ? count : (uint32_t)OSTAGE) + 3u) >> 2;
+        for (uint32_t o = lane; o < n16; o += 32) cp_async<16>(&ws.outl[x][4 * o], src + 4 * o);
+    };
     int tile = tile_lo + warp;
     Meta cur = fetch_meta(tile);
     Meta nxt = fetch_meta(tile + DEC_WARPS);
@@ -324,8 +331,10 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
     first_half_bytes(cur, h0K, h0V);
     if (tile < tile_hi) {
         stage(ws.bufK, poolK + __shfl_sync(0xFFFFFFFFu, cur.tb, 0), h0K);
+        stage_outl(0, __shfl_sync(0xFFFFFFFFu, cur.tb, 2), __shfl_sync(0xFFFFFFFFu, cur.tb, 3));
         cp_async_commit();
         stage(ws.bufV, poolV + __shfl_sync(0xFFFFFFFFu, cur.tb, 4), h0V);
+        stage_outl(1, __shfl_sync(0xFFFFFFFFu, cur.tb, 6), __shfl_sync(0xFFFFFFFFu, cur.tb, 7));
         cp_async_commit();
     }
 
@@ -336,6 +345,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
         const uint32_t ooV = __shfl_sync(0xFFFFFFFFu, cur.tb, 6), ocV = __shfl_sync(0xFFFFFFFFu, cur.tb, 7);
         const bool has_next = tile + DEC_WARPS < tile_hi;
         uint32_t n0K = 0, n0V = 0;   // first-half bytes of the next tile
+        uint32_t resumeK = 0, resumeV = 0;   // where half 1 resumes in the tile's outlier lists
 
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
@@ -414,15 +424,22 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
                 k_items<D, 4, ALIGN>(ws, first, ncls[0][1], qh, ql, part, sub); first += ncls[0][1];
                 k_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, first, ncls[0][2], qh, ql, part, sub); first += ncls[0][2];
                 k_items<D, 1, 4>(ws, first, ncls[0][3], qh, ql, part, sub);
+                // the tile's outlier entries are sorted by token: half 0 stops at the first batch that lies
+                // entirely in tokens >= 32, half 1 resumes there
                 const uint32_t* og = a.k.outl + (size_t)bh * a.ocap + ooK;
-                for (uint32_t e = lane; e < ocK; e += 32) {
-                    const uint32_t v = __ldg(og + e);
+                uint32_t e0 = half ? resumeK : 0u;
+                for (; e0 < ocK; e0 += 32) {
+                    const uint32_t e = e0 + lane;
+                    const uint32_t v = e < ocK ? (e < (uint32_t)OSTAGE ? ws.outl[0][e] : __ldg(og + e)) : 0xFF000000u;
                     const int tok = v >> 24, ch = (v >> 16) & 0xFF;
-                    if ((tok >> 5) == half) {
+                    if (half == 0 && __all_sync(0xFFFFFFFFu, tok >= UNIT)) break;
+                    if (e < ocK && (tok >> 5) == half) {
                         const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
                         atomicAdd(&ws.ocorr[tok & 31], sm.qf[ch] * (val - ws.midK[tok & 31]));
                     }
+                    if (half == 0 && __any_sync(0xFFFFFFFFu, tok >= UNIT)) break;   // this batch straddles the halves
                 }
+                if (half == 0) resumeK = e0 < ocK ? e0 : ocK;
             }
             __syncwarp();
             // ---- the key buffer is free: start the copy of the next unit's keys
@@ -431,6 +448,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
             } else if (has_next) {
                 first_half_bytes(nxt, n0K, n0V);
                 stage(ws.bufK, poolK + __shfl_sync(0xFFFFFFFFu, nxt.tb, 0), n0K);
+                stage_outl(0, __shfl_sync(0xFFFFFFFFu, nxt.tb, 2), __shfl_sync(0xFFFFFFFFu, nxt.tb, 3));
             }
             cp_async_commit();
 
@@ -489,19 +507,27 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
                 v_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, first, ncls[1][2], acc, part, sub); first += ncls[1][2];
                 v_items<D, 1, 4>(ws, first, ncls[1][3], acc, part, sub);
                 const uint32_t* og = a.v.outl + (size_t)bh * a.ocap + ooV;
-                for (uint32_t e = lane; e < ocV; e += 32) {
-                    const uint32_t v = __ldg(og + e);
+                uint32_t e0 = half ? resumeV : 0u;
+                for (; e0 < ocV; e0 += 32) {
+                    const uint32_t e = e0 + lane;
+                    const uint32_t v = e < ocV ? (e < (uint32_t)OSTAGE ? ws.outl[1][e] : __ldg(og + e)) : 0xFF000000u;
                     const int tok = v >> 24, ch = (v >> 16) & 0xFF;
-                    if ((tok >> 5) == half) {
+                    if (half == 0 && __all_sync(0xFFFFFFFFu, tok >= UNIT)) break;
+                    if (e < ocV && (tok >> 5) == half) {
                         const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
                         atomicAdd(&ws.vout[ch], ws.p[tok & 31] * (val - ws.midV[tok & 31]));
                     }
+                    if (half == 0 && __any_sync(0xFFFFFFFFu, tok >= UNIT)) break;
                 }
+                if (half == 0) resumeV = e0 < ocV ? e0 : ocV;
             }
             __syncwarp();
             // ---- the value buffer is free: start the copy of the next unit's values
             if (half == 0) stage(ws.bufV, poolV + offV + h0V, totV - h0V);
-            else if (has_next) stage(ws.bufV, poolV + __shfl_sync(0xFFFFFFFFu, nxt.tb, 4), n0V);
+            else if (has_next) {
+                stage(ws.bufV, poolV + __shfl_sync(0xFFFFFFFFu, nxt.tb, 4), n0V);
+                stage_outl(1, __shfl_sync(0xFFFFFFFFu, nxt.tb, 6), __shfl_sync(0xFFFFFFFFu, nxt.tb, 7));
+            }
             cp_async_commit();
         }
         cur = nxt;
