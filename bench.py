@@ -31,6 +31,10 @@ import torch  # noqa: E402
 
 from paper_2403_04643_b200 import synth  # noqa: E402
 
+# DRAM bytes (read + write) per launch from an ncu capture of the C3 layer shape (profiles/kernels_C3_layer.md);
+# only valid for that shape and for the kernels as they were when the capture was taken.
+NCU_TRAFFIC = {("C3", "quant"): 672.9e6 + 128.4e6, ("C3", "decode"): 140.5e6 + 1.8e6}
+
 METRIC = "QAQ quantize GB/s + packed decode-attn tokens/s, % of B200 HBM peak"
 QNORM2 = 1.16   # stand-in for the upper-10% quantile of sum_d (q_d / sqrt(D))^2 of N(0,1) queries
 
@@ -269,9 +273,9 @@ def main():
         },
         "roofline": {"kernel": "quant_kernel (fused select + outlier split + quantize + pack)", "bound": "hbm",
                      "achieved": round(quant_gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(quant_gbs / peak, 3),
-                     "traffic": None, "peak_kind": peak_kind, "bytes_per_launch": ab["quantize"]},
+                     "traffic": NCU_TRAFFIC.get((args.workload, "quant")), "peak_kind": peak_kind, "bytes_per_launch": ab["quantize"]},
         "roofline_decode": {"kernel": "decode_kernel (+ merge)", "bound": "hbm", "achieved": round(dec_gbs, 1), "peak": peak,
-                            "unit": "GB/s", "frac": round(dec_gbs / peak, 3), "traffic": None, "peak_kind": peak_kind,
+                            "unit": "GB/s", "frac": round(dec_gbs / peak, 3), "traffic": NCU_TRAFFIC.get((args.workload, "decode")), "peak_kind": peak_kind,
                             "bytes_per_launch": ab["decode"]},
         "gpu_launches": args.steps * L * 6,
         "clocks": clocks,
