@@ -159,6 +159,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (0 = the workload's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -309,6 +310,11 @@ def main():
                       "steps": n_e2e, "note": "quantize_append_host + decode_attention_host per layer; thresholds resident"}
 
     # ---- CPU oracle beside it (rank 0, N = 1 only): a bounded sample of the same workload
+    # ---- the other 7B-shaped configurations, for context (rank 0, one GPU): one layer at batch 1 (launch-latency
+    # regime) and the long-context cache (values of tokens beyond the prefill stay at 8 bits: no score seen yet)
+    if rank == 0 and world == 1 and not args.no_extras:
+        out["extras"] = extras(qaq, calibrate, dev, peak, hyper_qn)
+
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(wl, (sS, sX, hyper_qn))
 
@@ -318,6 +324,70 @@ def main():
         import torch.distributed as dist
         dist.destroy_process_group()
     return 0
+
+
+def _time_us(fn, reps):
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record(); torch.cuda.synchronize()
+    return a.elapsed_time(b) * 1e3 / reps
+
+
+def extras(qaq, calibrate, dev, peak, qn):
+    res = {}
+    for name, wl, T, prefill in (("C2_layer_batch1", synth.CONFIGS["C2"], 4096, 4096),
+                                 ("C5_long_context", synth.CONFIGS["C5"], 131072, 32768)):
+        D, BH, W = wl.head_dim, wl.bh, wl.window
+        wlx = synth.scaled(wl, tokens=T, grow_to=0)
+        K, V = synth.make_kv(wlx, 0, device=dev)
+        q = synth.make_query(wlx, 0, device=dev)
+        ring, nv = synth.make_score_ring(wlx, 0, device=dev)
+        nv[:, :, prefill:] = 0                       # tokens appended after the prefill have no score yet
+        cfg = qaq.make_config(wl.batch, wl.heads, D, T + 64, wl.bits_min, wl.bits_max, W, wl.alpha)
+        thr = qaq.qaq_outlier_thresholds(cfg, K[:, :, :prefill], V[:, :, :prefill])
+        _, _, pol = calibrate(cfg, K[:, :, :prefill], V[:, :, :prefill], ring[:, :, :, :prefill].contiguous(),
+                              nv[:, :, :prefill].contiguous(), thr, prefill, qn)
+        cache = qaq.Cache(cfg)
+        outb = torch.empty((BH, D), dtype=torch.float32, device=dev)
+        scale = 1.0 / math.sqrt(D)
+
+        def fill():
+            cache.reset()
+            qaq.qaq_quantize_append(cache, K, V, thr, policy=pol, ring=ring, nvalid=nv)
+        us_q = _time_us(fill, 5)
+        us_d = _time_us(lambda: qaq.qaq_decode_attention(cache, q, scale, out=outb), 20)
+        st = qaq.qaq_cache_stats(cache)
+        ab = algorithmic_bytes(wlx, st)
+        # one-token append + decode, the streaming step
+        k1, v1 = K[:, :, :1].contiguous(), V[:, :, :1].contiguous()
+        r1, n1 = ring[:, :, :, :1].contiguous(), torch.zeros((wl.batch, wl.heads, 1), dtype=torch.uint8, device=dev)
+        t_now = cache.tokens
+        reps = min(32, cfg.max_tokens - t_now)
+
+        def stream():
+            qaq.qaq_quantize_append(cache, k1, v1, thr, policy=pol, ring=r1, nvalid=n1)
+            qaq.qaq_decode_attention(cache, q, scale, out=outb)
+        torch.cuda.synchronize()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            stream()
+        b.record(); torch.cuda.synchronize()
+        us_s = a.elapsed_time(b) * 1e3 / reps
+        res[name] = {"tokens": T, "bh": BH, "quantize_us": round(us_q, 1), "quantize_gbs": round(ab["quantize"] / us_q / 1e3, 1),
+                     "decode_us": round(us_d, 1), "decode_gbs": round(ab["decode"] / us_d / 1e3, 1),
+                     "decode_frac_of_hbm": round(ab["decode"] / us_d / 1e3 / peak, 3),
+                     "cached_tokens_per_s": round(wl.batch * T / (us_d * 1e-6), 1),
+                     "append1_plus_decode_us": round(us_s, 1),
+                     "mean_bits": [round(st.code_bytes[0] * 8 / (BH * T * D), 2), round(st.code_bytes[1] * 8 / (BH * T * D), 2)]}
+        del cache, K, V, ring
+        torch.cuda.empty_cache()
+    return res
 
 
 def cpu_baseline(wl, hyper, budget_s=20.0):
