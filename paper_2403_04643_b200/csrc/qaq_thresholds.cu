@@ -201,12 +201,14 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
             // cheap filter: almost all entries are inside [lo, hi]; a 16-byte piece holding anything
             // else is set aside and looked at entry by entry afterwards, with all lanes busy
             const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
-            // pair-wise min and max over the four words (NaN-propagating), then two compares
-            const __half2 v0 = *reinterpret_cast<const __half2*>(&w[0]), v1 = *reinterpret_cast<const __half2*>(&w[1]);
-            const __half2 v2 = *reinterpret_cast<const __half2*>(&w[2]), v3 = *reinterpret_cast<const __half2*>(&w[3]);
-            const __half2 mn = __hmin2_nan(__hmin2_nan(v0, v1), __hmin2_nan(v2, v3));
-            const __half2 mx = __hmax2_nan(__hmax2_nan(v0, v1), __hmax2_nan(v2, v3));
-            const bool inside = __hbge2(mn, lo2) && __hble2(mx, hi2);
+            // all-ones iff every entry of the piece is inside [lo, hi] (a NaN compares false)
+            uint32_t all_in = 0xFFFFFFFFu;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const __half2 v = *reinterpret_cast<const __half2*>(&w[j]);
+                all_in &= __hge2_mask(v, lo2) & __hle2_mask(v, hi2);
+            }
+            const bool inside = all_in == 0xFFFFFFFFu;
             // one shared-memory reservation per warp for its flagged pieces
             const bool flag = !inside && i0 + u * 256 + (int)threadIdx.x < n;
             const unsigned bal = __ballot_sync(0xFFFFFFFFu, flag);
