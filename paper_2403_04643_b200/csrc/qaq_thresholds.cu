@@ -18,8 +18,9 @@
 namespace {
 
 constexpr int SAMPLE_TOKENS = 64;
-constexpr int SCAN_TOKENS = 64;      // tokens per CTA of the scan
-constexpr int CTA_LIST = 2048;       // candidates per tail a scan CTA can hold
+constexpr int SCAN_TOKENS = 256;     // tokens per CTA of the scan
+constexpr int CHUNK_PIECES = 4 * 256; // 16-byte pieces looked at between two barriers (four per thread)
+constexpr int CTA_LIST = 4096;       // candidates per tail a scan CTA can hold
 
 __device__ __forceinline__ uint32_t key_of(unsigned short h) { return (h & 0x8000u) ? (uint32_t)(~h & 0xFFFFu) : (uint32_t)(h | 0x8000u); }
 __device__ __forceinline__ unsigned short half_of_key(uint32_t k) { return (k & 0x8000u) ? (unsigned short)(k & 0x7FFFu) : (unsigned short)(~k & 0xFFFFu); }
@@ -174,7 +175,7 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
     Problem* pr = a.prob + bhx;
     if (pr->done) return;
     __shared__ unsigned short s_list[2][CTA_LIST];
-    __shared__ uint4 s_flag[SCAN_TOKENS * 16];                    // 16-byte pieces with something outside [lo, hi]
+    __shared__ uint4 s_flag[CHUNK_PIECES];                    // 16-byte pieces with something outside [lo, hi]
     __shared__ uint32_t s_n[2], s_base[2], s_nan, s_nflag;
     if (threadIdx.x < 2) s_n[threadIdx.x] = 0;
     if (threadIdx.x == 2) s_nan = 0;
@@ -220,7 +221,6 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
                 if (flag) s_flag[base + __popc(bal & ((1u << lane) - 1u))] = raw[u];
             }
         }
-    }
     __syncthreads();
     for (uint32_t i = threadIdx.x; i < s_nflag; i += blockDim.x) {
         const uint4 r = s_flag[i];
@@ -245,6 +245,9 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
         }
     }
     __syncthreads();
+    if (threadIdx.x == 0) s_nflag = 0;   // the next chunk starts an empty list of flagged pieces
+    __syncthreads();
+    }   // chunks
     if (threadIdx.x < 2) s_base[threadIdx.x] = s_n[threadIdx.x] ? atomicAdd(&pr->cnt[threadIdx.x], s_n[threadIdx.x]) : 0u;
     if (threadIdx.x == 2 && s_nan) atomicAdd(&pr->nan, s_nan);
     __syncthreads();
