@@ -14,7 +14,8 @@
 // word of codes (already one field per byte lane after a mask) feeds two dp4a.  The sums
 // are exact integers; the fixed-point error of q is below 2^-16 of max|q|.
 //
-// One CTA = one (b,h) and one split of its tiles; each warp works through whole tiles
+// One CTA = one run of consecutive tiles of the flattened (b,h, tile) sequence (runs of equal
+// length, so every SM gets the same amount of work); each warp works through whole tiles
 // (QAQ_TILE tokens) on its own, with its own running max / sum / accumulators and no CTA
 // barrier in the tile loop; warps are merged once at the end.  A (token, plane) pair is one
 // work item, handled by head_dim/32 lanes that read their words of the plane straight from
@@ -35,9 +36,9 @@ struct DecArgs {
     int T;
     const __half* q;
     float scale;
-    float* part;       // [BH][nsplit][D+3]: accumulators, running max, sum of the weights used, exact sum
+    float* part;       // [ncta][2][D+3]: accumulators, running max, sum of the weights used, exact sum
     float* ml;         // [BH][2]   merged (max, sum) for score normalisation
-    int nsplit;
+    int BH, run, ncta; // (b,h) count; tiles per CTA of the flattened (b,h, tile) sequence; CTAs
     float* out;        // [BH][D]
     float* scores;     // [BH][T] or null
 };
@@ -211,7 +212,8 @@ __device__ __forceinline__ void v_items(WarpScratch<D>& ws, int first, int n, fl
     }
 }
 
-// One CTA = one (b,h) and one split of its tiles.  Every warp works through whole tiles on its
+// One CTA = one run of consecutive tiles, which meets one or two (b,h): the body below runs once
+// per (b,h) segment and leaves one partial per segment.  Every warp works through whole tiles on its
 // own, half a tile (32 tokens) at a time: own running max / sum / accumulators, own staging
 // buffers, no CTA barrier in the loop; the warps are merged once at the end.  The packed bytes
 // of the next half tile are copied to shared memory with cp.async while the current one is being
@@ -222,14 +224,21 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
     constexpr int ALIGN = D / 8 >= 16 ? 16 : D / 8;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DecSmem<D>& sm = *reinterpret_cast<DecSmem<D>*>(smem_raw);
-    const int bh = blockIdx.y, split = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int part = lane % P, sub = lane / P;
     WarpScratch<D>& ws = sm.ws[warp];
 
+#pragma unroll 1
+    for (int seg = 0; seg < 2; ++seg) {
+    // this CTA's run of the flattened (b,h, tile) sequence; it touches at most two (b,h).  The block
+    // index is read afresh for each segment so that none of this stays in registers over the tile loop.
+    int cta;
+    asm volatile("mov.u32 %0, %%ctaid.x;" : "=r"(cta));
     const int ntiles = (a.T + QAQ_TILE - 1) / QAQ_TILE;
-    const int per_split = (ntiles + a.nsplit - 1) / a.nsplit;
-    const int tile_lo = split * per_split, tile_hi = min(ntiles, tile_lo + per_split);
+    const int flat_lo = cta * a.run, flat_hi = min(a.BH * ntiles, flat_lo + a.run);
+    const int bh = flat_lo / ntiles + seg;
+    const int tile_lo = max(flat_lo, bh * ntiles) - bh * ntiles, tile_hi = min(flat_hi, (bh + 1) * ntiles) - bh * ntiles;
+    if (tile_lo >= tile_hi) continue;   // the same for every thread of the CTA
 
     // ---- q: float copy, fixed-point bytes per lane
     float qmax = 0.f, qs = 0.f;
@@ -552,11 +561,11 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
         }
     if (lane == 0) { sm.mm[warp] = m_run; sm.ml[warp] = l_run; sm.mlx[warp] = lx_run; }
     __syncthreads();
-    // ---- merge the warps (log-sum-exp) into this split's partial
+    // ---- merge the warps (log-sum-exp) into this segment's partial
     float M = __int_as_float(0xff800000);
 #pragma unroll
     for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, sm.mm[w]);
-    float* dst = a.part + ((size_t)bh * a.nsplit + split) * (D + 3);
+    float* dst = a.part + (size_t)(2 * cta + seg) * (D + 3);
     float L = 0.f, LX = 0.f;
     float wgt[DEC_WARPS];
 #pragma unroll
@@ -572,23 +581,30 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
         dst[d] = x;
     }
     if (tid == 0) { dst[D] = M; dst[D + 1] = L; dst[D + 2] = LX; }
+    __syncthreads();   // the shared arrays are reused by the second segment
+    }
 }
 
-// log-sum-exp merge of the split partials -> X, and (max, sum) for the score row
+// log-sum-exp merge of the partials -> X, and (max, sum) for the score row
 template <int D>
 __global__ void merge_kernel(const DecArgs a) {
     const int bh = blockIdx.x, d = threadIdx.x;
-    const float* p = a.part + (size_t)bh * a.nsplit * (D + 3);
+    // the CTAs of decode_kernel whose runs meet this (b,h); a CTA's first segment has slot 0
+    const int ntiles = (a.T + QAQ_TILE - 1) / QAQ_TILE;
+    const int c_lo = (bh * ntiles) / a.run, c_hi = ((bh + 1) * ntiles - 1) / a.run;
+    // only the first of them can have begun in the (b,h) before
+    auto slot = [&](int c) { return a.part + (size_t)(2 * c + (c * a.run < bh * ntiles ? 1 : 0)) * (D + 3); };
     float M = __int_as_float(0xff800000);
-    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, p[s * (D + 3) + D]);
+    for (int c = c_lo; c <= c_hi; ++c) M = fmaxf(M, slot(c)[D]);
     float L = 0.f, LX = 0.f, x = 0.f;
-    for (int s = 0; s < a.nsplit; ++s) {
-        const float m = p[s * (D + 3) + D];
+    for (int c = c_lo; c <= c_hi; ++c) {
+        const float* p = slot(c);
+        const float m = p[D];
         if (m == __int_as_float(0xff800000)) continue;
         const float w = __expf(m - M);
-        L = fmaf(w, p[s * (D + 3) + D + 1], L);
-        LX = fmaf(w, p[s * (D + 3) + D + 2], LX);
-        x = fmaf(w, p[s * (D + 3) + d], x);
+        L = fmaf(w, p[D + 1], L);
+        LX = fmaf(w, p[D + 2], LX);
+        x = fmaf(w, p[d], x);
     }
     a.out[(size_t)bh * D + d] = L > 0.f ? x / L : 0.f;
     if (d == 0) { a.ml[2 * bh] = M; a.ml[2 * bh + 1] = LX; }
@@ -604,22 +620,31 @@ __global__ void scores_kernel(float* scores, const float* ml, int T) {
     }
 }
 
-int pick_nsplit(int BH, int ntiles) {
-    // about 16 warps per SM on 148 SMs in total (4 warps per CTA), at least one tile per warp
-    int want = (148 * 16 + 2 * BH) / (DEC_WARPS * BH);
-    int cap = ntiles / DEC_WARPS > 0 ? ntiles / DEC_WARPS : 1;
-    int n = want < cap ? want : cap;
-    if (n < 1) n = 1;
-    if (n > 64) n = 64;
-    return n;
+// The flattened sequence of BH * ntiles tiles is cut into runs of `run` consecutive tiles, one CTA
+// each: enough CTAs to fill every SM (148 SMs, 4 resident CTAs each) evenly, at least one tile per
+// warp where there are that many, and never more than one (b,h) boundary inside a run.
+constexpr int DEC_SLOTS = 148 * 4;
+struct DecPlan { int run, ncta; };
+DecPlan plan_decode(int BH, int ntiles) {
+    const long long total = (long long)BH * ntiles;
+    long long run = (total + DEC_SLOTS - 1) / DEC_SLOTS;
+    const int floor_run = ntiles < DEC_WARPS ? ntiles : DEC_WARPS;
+    if (run < floor_run) run = floor_run;
+    if (run > ntiles) run = ntiles;
+    DecPlan p;
+    p.run = (int)run;
+    p.ncta = (int)((total + run - 1) / run);
+    return p;
 }
+// floats of workspace for the partials (two slots per CTA) and the merged (max, sum) pairs
+size_t decode_ws_floats(int BH, int ncta, int D) { return (size_t)2 * ncta * (D + 3) + (size_t)BH * 2; }
 
 template <int D>
 qaq_status run_decode(const DecArgs& a, int BH, cudaStream_t s) {
     const size_t smem = sizeof(DecSmem<D>);
     if (smem > 48 * 1024)
         QAQ_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    decode_kernel<D><<<dim3(a.nsplit, BH), DEC_THREADS, smem, s>>>(a);
+    decode_kernel<D><<<a.ncta, DEC_THREADS, smem, s>>>(a);
     merge_kernel<D><<<BH, D, 0, s>>>(a);
     if (a.scores) {
         int gx = (a.T + 1023) / 1024;
@@ -632,12 +657,11 @@ qaq_status run_decode(const DecArgs& a, int BH, cudaStream_t s) {
 
 }  // namespace
 
-static const int QAQ_MAX_SPLIT = 64;
-
 extern "C" qaq_status qaq_decode_workspace_bytes(const qaq_cache* c, size_t* host_out) {
     if (!c || !host_out) return QAQ_ERR_INVALID_ARG;
-    const size_t BH = (size_t)c->BH, D = (size_t)c->cfg.head_dim;
-    *host_out = (BH * QAQ_MAX_SPLIT * (D + 3) + BH * 2) * sizeof(float);
+    // plan_decode never uses more CTAs than max(DEC_SLOTS, BH), whatever the token count
+    const int ncta_max = c->BH > DEC_SLOTS ? c->BH : DEC_SLOTS;
+    *host_out = decode_ws_floats(c->BH, ncta_max, c->cfg.head_dim) * sizeof(float);
     return QAQ_OK;
 }
 
@@ -654,9 +678,10 @@ extern "C" qaq_status qaq_decode_attention(const qaq_cache* c, const void* q, fl
     a.tmax_pad = c->tmax_pad; a.ntiles_max = c->ntiles; a.T = (int)c->tokens;
     a.q = (const __half*)q; a.scale = softmax_scale;
     const int ntiles = (a.T + QAQ_TILE - 1) / QAQ_TILE;
-    a.nsplit = pick_nsplit(BH, ntiles);
+    const DecPlan plan = plan_decode(BH, ntiles);
+    a.BH = BH; a.run = plan.run; a.ncta = plan.ncta;
     a.part = (float*)ws;
-    a.ml = a.part + (size_t)BH * QAQ_MAX_SPLIT * (D + 3);
+    a.ml = a.part + (size_t)2 * plan.ncta * (D + 3);
     a.out = out; a.scores = scores_out;
     cudaStream_t s = (cudaStream_t)stream;
     switch (D) {
@@ -688,9 +713,9 @@ extern "C" qaq_status qaq_decode_attention_static(const qaq_cache* c, const void
     const int D = c->cfg.head_dim, BH = c->BH;
     const int T = (int)c->tokens;
     const int ntiles = (T + QAQ_TILE - 1) / QAQ_TILE;
-    const int nsplit = pick_nsplit(BH, ntiles);
-    // partials [BH][nsplit][D+3] followed by the merged (max, sum) pairs [BH][2]
-    const size_t need = ((size_t)BH * nsplit * (D + 3) + (size_t)BH * 2) * sizeof(float);
+    const DecPlan plan = plan_decode(BH, ntiles);
+    // partials [ncta][2][D+3] followed by the merged (max, sum) pairs [BH][2]
+    const size_t need = decode_ws_floats(BH, plan.ncta, D) * sizeof(float);
     if (need > QAQ_STATIC_SCRATCH_BYTES) return QAQ_ERR_WORKSPACE;  // shape too large for the built-in scratch
 
     int dev = -1;
@@ -715,11 +740,11 @@ extern "C" qaq_status qaq_decode_attention_static(const qaq_cache* c, const void
     a.k = c->t[0]; a.v = c->t[1]; a.pool_bytes = c->pool_bytes; a.ocap = c->ocap;
     a.tmax_pad = c->tmax_pad; a.ntiles_max = c->ntiles; a.T = T;
     a.q = (const __half*)q; a.scale = softmax_scale;
-    a.nsplit = nsplit;
-    // Every (b,h,split) partial and every (max,sum) pair is written before it is read, so
-    // nothing in the scratch has to be cleared between calls.
+    a.BH = BH; a.run = plan.run; a.ncta = plan.ncta;
+    // Every partial that the merge reads and every (max,sum) pair is written before it is read,
+    // so nothing in the scratch has to be cleared between calls.
     a.part = (float*)scratch;
-    a.ml = a.part + (size_t)BH * nsplit * (D + 3);
+    a.ml = a.part + (size_t)2 * plan.ncta * (D + 3);
     a.out = out; a.scores = nullptr;
     cudaStream_t s = (cudaStream_t)stream;
     switch (D) {

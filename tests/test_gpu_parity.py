@@ -141,22 +141,31 @@ def test_single_token_and_constant_tokens():
     assert scores.cpu().numpy()[0, 0] == pytest.approx(1.0)
 
 
+def test_runs_of_tiles_that_straddle_two_heads():
+    # 3 (b,h) x 10 tiles are cut into runs of 4 tiles: the third run ends one head and begins the next
+    wl = synth.scaled(synth.CONFIGS["C2"], heads=3, tokens=600)
+    full_case(wl, HYPER["C2"])
+
+
 def test_split_count_does_not_change_the_result_beyond_rounding():
-    # same cache content decoded from caches of different length classes (different split counts)
+    # same cache content decoded with different cuts of the tile sequence (runs of 4 tiles inside a head;
+    # runs of 5 tiles, some of which straddle two heads)
     wl = synth.scaled(synth.CONFIGS["C2"], heads=2, tokens=2048)
     K, V, q, ring, nv = make_inputs(wl)
     pol = qaq.qaq_policy_from_hyper(*HYPER["C2"], 2048)
     outs = []
-    for rep in (1, 40):   # 2 (b,h) -> many splits;  80 (b,h) -> few splits
+    for rep in (1, 40):   # 2 (b,h) -> 16 runs of 4 tiles;  80 (b,h) -> 512 runs of 5 tiles
         wlr = synth.scaled(wl, batch=rep)
         Kr, Vr, qr = K.repeat(rep, 1, 1, 1), V.repeat(rep, 1, 1, 1), q.repeat(rep, 1, 1)
         rr, nr = ring.repeat(rep, 1, 1, 1), nv.repeat(rep, 1, 1)
         cfg, cache, thr, out, scores, dev = gpu_pipeline(wlr, Kr, Vr, qr, rr, nr, pol)
         outs.append(out.cpu().numpy()[:2])
         if rep > 1:
-            # replicas agree up to the order of a few float additions
-            assert np.allclose(out.cpu().numpy()[:2], out.cpu().numpy()[-2:], rtol=1e-5, atol=1e-6)
-    assert np.allclose(outs[0], outs[1], rtol=1e-4, atol=1e-5)
+            # replicas are cut at different tiles, so they agree up to the rounding of the value weights to
+            # 11 significant bits: at most 2^-12 * sum_t p_t |v_t - X|, and the attention here is peaked on
+            # a few tokens whose values differ by up to ~4, so no averaging helps
+            assert np.allclose(out.cpu().numpy()[:2], out.cpu().numpy()[-2:], rtol=0, atol=1e-3)
+    assert np.allclose(outs[0], outs[1], rtol=0, atol=1e-3)
 
 
 def test_capacity_errors_are_reported_not_faulted():

@@ -61,7 +61,7 @@ def test_static_scratch_decode_matches_workspace_decode_twice_in_a_row():
 
 
 def test_static_scratch_rejects_shapes_beyond_its_limit():
-    # 8320 (b,h) x 1 split x 131 floats is a little more than the 4 MiB built in: refused on the host, nothing launched
+    # 8320 (b,h) of one tile each: 8320 CTAs x 2 partials x 131 floats do not fit the 4 MiB built in: refused on the host, nothing launched
     B, H, D, T = 128, 65, 128, 64
     cfg = qaq.make_config(B, H, D, T, 2, 8, 1, 0.0)
     cache = qaq.Cache(cfg)
