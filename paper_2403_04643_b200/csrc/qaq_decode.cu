@@ -179,6 +179,7 @@ template <int D, int W, int ALIGN>
 __device__ __forceinline__ void k_items(WarpScratch<D>& ws, int first, int n, const uint32_t (&qh)[8],
                                         const uint32_t (&ql)[8], int part, int sub) {
     constexpr int P = D / 32, IPW = 32 / P;
+#pragma unroll 1
     for (int i0 = 0; i0 < n; i0 += IPW) {
         uint32_t w0[8];
         const int ia = i0 + sub;
@@ -198,6 +199,7 @@ __device__ __forceinline__ void k_items(WarpScratch<D>& ws, int first, int n, co
 template <int D, int W, int ALIGN>
 __device__ __forceinline__ void v_items(WarpScratch<D>& ws, int first, int n, float (&acc)[8][4], int part, int sub) {
     constexpr int P = D / 32, IPW = 32 / P, PER = 8 / W;
+#pragma unroll 1
     for (int i0 = sub; i0 < n; i0 += IPW) {
         uint32_t w0[8];
         const uint32_t de = ws.item[1][first + i0];
@@ -325,12 +327,14 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
         hK = k; hV = v;
     };
     auto stage = [&](uint8_t* dst, const uint8_t* src, uint32_t nbytes) {
+#pragma unroll 1
         for (uint32_t o = lane * ALIGN; o < nbytes; o += 32 * ALIGN) cp_async<ALIGN>(dst + o, src + o);
     };
 
     auto stage_outl = [&](int x, uint32_t first, uint32_t count) {   // entries are 4 bytes, lists start 16-byte aligned
         const uint32_t* src = (x ? a.v.outl : a.k.outl) + (size_t)bh * a.ocap + first;
         const uint32_t n16 = ((count < (uint32_t)OSTAGE ? count : (uint32_t)OSTAGE) + 3u) >> 2;
+#pragma unroll 1
         for (uint32_t o = lane; o < n16; o += 32) cp_async<16>(&ws.outl[x][4 * o], src + 4 * o);
     };
     int tile = tile_lo + warp;
@@ -437,6 +441,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
                 // entirely in tokens >= 32, half 1 resumes there
                 const uint32_t* og = a.k.outl + (size_t)bh * a.ocap + ooK;
                 uint32_t e0 = half ? resumeK : 0u;
+#pragma unroll 1
                 for (; e0 < ocK; e0 += 32) {
                     const uint32_t e = e0 + lane;
                     const uint32_t v = e < ocK ? (e < (uint32_t)OSTAGE ? ws.outl[0][e] : __ldg(og + e)) : 0xFF000000u;
@@ -517,6 +522,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
                 v_items<D, 1, 4>(ws, first, ncls[1][3], acc, part, sub);
                 const uint32_t* og = a.v.outl + (size_t)bh * a.ocap + ooV;
                 uint32_t e0 = half ? resumeV : 0u;
+#pragma unroll 1
                 for (; e0 < ocV; e0 += 32) {
                     const uint32_t e = e0 + lane;
                     const uint32_t v = e < ocV ? (e < (uint32_t)OSTAGE ? ws.outl[1][e] : __ldg(og + e)) : 0xFF000000u;
