@@ -21,6 +21,7 @@ constexpr int SAMPLE_TOKENS = 64;
 constexpr int SCAN_TOKENS = 256;     // tokens per CTA of the scan
 constexpr int CHUNK_PIECES = 4 * 256; // 16-byte pieces looked at between two barriers (four per thread)
 constexpr int CTA_LIST = 4096;       // candidates per tail a scan CTA can hold
+constexpr int SELECT_KEYS = 16384;   // candidates of one tail the select kernel keeps in shared memory
 
 __device__ __forceinline__ uint32_t key_of(unsigned short h) { return (h & 0x8000u) ? (uint32_t)(~h & 0xFFFFu) : (uint32_t)(h | 0x8000u); }
 __device__ __forceinline__ unsigned short half_of_key(uint32_t k) { return (k & 0x8000u) ? (unsigned short)(k & 0x7FFFu) : (unsigned short)(~k & 0xFFFFu); }
@@ -265,26 +266,35 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
     }
 }
 
-// ---- 3. exact select among the candidates, exact fallback over the data when that is not possible
+// ---- 3. exact select among the candidates, exact fallback over the data when that is not possible.
+// One CTA per (problem, tail): the two tails are independent order statistics.
 __global__ void __launch_bounds__(256) thr_select_kernel(const ThrArgs a) {
-    const int bhx = blockIdx.x, bh = bhx >> 1, x = bhx & 1;
+    const int bhx = blockIdx.x >> 1, side = blockIdx.x & 1, bh = bhx >> 1, x = bhx & 1;
     Problem* pr = a.prob + bhx;
     if (pr->done) return;
     __shared__ uint32_t hist[8 * 256], s_tmp[2];
+    __shared__ __align__(16) unsigned short s_keys[SELECT_KEYS];
     const unsigned long long total = (unsigned long long)a.T * a.D;
     const unsigned long long N = total - pr->nan;
-    float lo = 0.f, hi = 0.f;
+    float res = 0.f;
     if (N > 0) {
         const unsigned long long k = rank_k(a.alpha, N);
-        const uint32_t c0 = pr->cnt[0], c1 = pr->cnt[1];
-        const bool ok = c0 > k && c1 > k && c0 <= a.cap && c1 <= a.cap;
-        if (ok) {
-            const unsigned short* l0 = a.list + ((size_t)bhx * 2 + 0) * a.cap;
-            const unsigned short* l1 = a.list + ((size_t)bhx * 2 + 1) * a.cap;
-            auto get0 = [&](uint32_t i) -> uint32_t { return l0[i]; };
-            auto get1 = [&](uint32_t i) -> uint32_t { return l1[i]; };
-            lo = float_of_key(cta_select(get0, c0, (uint32_t)k, hist, s_tmp));           // k-th smallest
-            hi = float_of_key(cta_select(get1, c1, (uint32_t)(c1 - 1 - k), hist, s_tmp)); // k-th largest
+        const uint32_t c = pr->cnt[side];
+        if (c > k && c <= a.cap) {
+            // rank k from below in the low list, rank k from above in the high list
+            const uint32_t want = side == 0 ? (uint32_t)k : (uint32_t)(c - 1 - k);
+            const unsigned short* l = a.list + ((size_t)bhx * 2 + side) * a.cap;   // 16-byte aligned
+            if (c <= (uint32_t)SELECT_KEYS) {
+                // the usual case: the list fits in shared memory; bring it in with independent wide loads
+                for (uint32_t i = threadIdx.x; i < (c + 7) / 8; i += blockDim.x)
+                    reinterpret_cast<uint4*>(s_keys)[i] = reinterpret_cast<const uint4*>(l)[i];
+                __syncthreads();
+                auto gets = [&](uint32_t i) -> uint32_t { return s_keys[i]; };
+                res = float_of_key(cta_select(gets, c, want, hist, s_tmp));
+            } else {
+                auto getg = [&](uint32_t i) -> uint32_t { return l[i]; };
+                res = float_of_key(cta_select(getg, c, want, hist, s_tmp));
+            }
         } else {
             // bracket too tight or list overflow: two-pass radix select over this problem's data
             const int b_idx = bh / a.H, h_idx = bh % a.H;
@@ -294,14 +304,10 @@ __global__ void __launch_bounds__(256) thr_select_kernel(const ThrArgs a) {
                 const unsigned short h = __half_as_ushort(X[(size_t)(i / D) * a.st + (i % D)]);
                 return is_nan_bits(h) ? 0x10000u : key_of(h);
             };
-            lo = float_of_key(cta_select(getx, (uint32_t)total, (uint32_t)k, hist, s_tmp));
-            hi = float_of_key(cta_select(getx, (uint32_t)total, (uint32_t)(N - 1 - k), hist, s_tmp));
+            res = float_of_key(cta_select(getx, (uint32_t)total, side == 0 ? (uint32_t)k : (uint32_t)(N - 1 - k), hist, s_tmp));
         }
     }
-    if (threadIdx.x == 0) {
-        a.thr[(size_t)bh * 4 + 2 * x] = lo;
-        a.thr[(size_t)bh * 4 + 2 * x + 1] = hi;
-    }
+    if (threadIdx.x == 0) a.thr[(size_t)bh * 4 + 2 * x + side] = res;
 }
 
 uint32_t list_capacity(const qaq_config* cfg, int n_tokens) {
@@ -353,7 +359,7 @@ extern "C" qaq_status qaq_outlier_thresholds(const qaq_config* cfg, const void* 
     if (n_tokens > SAMPLE_TOKENS) {
         dim3 grid((n_tokens + SCAN_TOKENS - 1) / SCAN_TOKENS, BH * 2);
         thr_scan_kernel<<<grid, 256, 0, s>>>(a);
-        thr_select_kernel<<<BH * 2, 256, 0, s>>>(a);
+        thr_select_kernel<<<BH * 4, 256, 0, s>>>(a);
     }
     QAQ_CUDA_TRY(cudaGetLastError());
     return QAQ_OK;
