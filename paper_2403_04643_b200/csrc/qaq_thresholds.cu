@@ -48,61 +48,84 @@ struct ThrArgs {
 };
 
 // rank select (0-based rank `want`) over n 16-bit keys readable through get(i); all threads of the
-// CTA (256) call it; hist is 8 x 256 words of shared memory (one histogram per warp, so that hot
-// bins are contended inside a warp only).  Two rounds of an 8-bit radix select; the bin holding the
-// wanted rank is found by warp 0 with a prefix sum over the 256 bins (8 per lane).
+// CTA (256) call it; hist is 2048 words of shared memory.  Two rounds of a radix select: the upper
+// 11 bits of the key first, then the lower 5.  binary16 data piles up in a few exponents, so a
+// histogram of the upper byte alone would send most lanes of a warp to the same handful of
+// counters; 11 bits spread them over 32 bins per octave.  In round 0 every thread sums 8 bins and a
+// CTA-wide prefix sum finds the bin holding the wanted rank; round 1 has 32 bins, one per lane of
+// warp 0.
 template <typename Get>
 __device__ uint32_t cta_select(Get get, uint32_t n, uint32_t want, uint32_t* hist, uint32_t* s_tmp) {
-    uint32_t prefix = 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint32_t* mine = hist + 256 * warp;
-    for (int round = 0; round < 2; ++round) {
-        for (int i = threadIdx.x; i < 8 * 256; i += blockDim.x) hist[i] = 0;
-        __syncthreads();
-        for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
-            const uint32_t k = get(i);
-            if (k > 0xFFFFu) continue;                      // NaN marker
-            if (round == 0) atomicAdd(&mine[k >> 8], 1u);
-            else if ((k >> 8) == prefix) atomicAdd(&mine[k & 255], 1u);
-        }
-        __syncthreads();
-        if (warp == 0) {
-            uint32_t c[8], tot = 0;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                uint32_t v = 0;
-#pragma unroll
-                for (int w = 0; w < 8; ++w) v += hist[256 * w + 8 * lane + j];
-                c[j] = v; tot += v;
-            }
-            uint32_t inc = tot;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-                if (lane >= d) inc += t;
-            }
-            uint32_t acc = inc - tot;                       // keys in the bins before this lane's eight
-            const uint32_t all = __shfl_sync(0xFFFFFFFFu, inc, 31);
-            const uint32_t w2 = want < all ? want : (all ? all - 1 : 0);   // defensive clamp
-            if (tot > 0 && w2 >= acc && w2 < acc + tot) {   // exactly one lane
-                int bsel = 0;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (w2 >= acc + c[j] && j < 7) { acc += c[j]; bsel = j + 1; }
-                    else break;
-                }
-                s_tmp[0] = (uint32_t)(8 * lane + bsel);
-                s_tmp[1] = w2 - acc;
-            }
-            if (all == 0 && lane == 0) { s_tmp[0] = 0; s_tmp[1] = 0; }
-        }
-        __syncthreads();
-        if (round == 0) prefix = s_tmp[0];
-        else prefix = (prefix << 8) | s_tmp[0];
-        want = s_tmp[1];
-        __syncthreads();
+    // ---- round 0: upper 11 bits
+    for (int i = threadIdx.x; i < 2048; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
+        const uint32_t k = get(i);
+        if (k <= 0xFFFFu) atomicAdd(&hist[k >> 5], 1u);     // larger: NaN marker
     }
-    return prefix;
+    __syncthreads();
+    uint32_t c[8], tot = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { c[j] = hist[8 * threadIdx.x + j]; tot += c[j]; }
+    uint32_t inc = tot;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= d) inc += t;
+    }
+    __syncthreads();                                         // every thread has read its bins
+    if (lane == 31) hist[warp] = inc;                        // warp totals
+    __syncthreads();
+    uint32_t before = 0, all = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        const uint32_t v = hist[w];
+        if (w < warp) before += v;
+        all += v;
+    }
+    uint32_t acc = before + inc - tot;                       // keys in the bins before this thread's eight
+    const uint32_t w2 = want < all ? want : (all ? all - 1 : 0);   // defensive clamp
+    if (threadIdx.x == 0) { s_tmp[0] = 0; s_tmp[1] = 0; }    // all == 0: no key at all
+    __syncthreads();
+    if (tot > 0 && w2 >= acc && w2 < acc + tot) {            // exactly one thread
+        int bsel = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (w2 >= acc + c[j] && j < 7) { acc += c[j]; bsel = j + 1; }
+            else break;
+        }
+        s_tmp[0] = (uint32_t)(8 * threadIdx.x + bsel);
+        s_tmp[1] = w2 - acc;
+    }
+    __syncthreads();
+    const uint32_t prefix = s_tmp[0];
+    const uint32_t want1 = s_tmp[1];
+    // ---- round 1: lower 5 bits of the keys in that bin
+    if (threadIdx.x < 32) hist[threadIdx.x] = 0;
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
+        const uint32_t k = get(i);
+        if (k <= 0xFFFFu && (k >> 5) == prefix) atomicAdd(&hist[k & 31], 1u);
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t v = hist[lane];
+        uint32_t in2 = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, in2, d);
+            if (lane >= d) in2 += t;
+        }
+        const uint32_t all2 = __shfl_sync(0xFFFFFFFFu, in2, 31);
+        const uint32_t w3 = want1 < all2 ? want1 : (all2 ? all2 - 1 : 0);
+        if (all2 == 0 && lane == 0) s_tmp[0] = 0;
+        if (v > 0 && w3 >= in2 - v && w3 < in2) s_tmp[0] = (uint32_t)lane;
+    }
+    __syncthreads();
+    const uint32_t low = s_tmp[0];
+    __syncthreads();                                         // s_tmp and hist are free for the next call
+    return (prefix << 5) | low;
 }
 
 __device__ __forceinline__ unsigned long long rank_k(double alpha, unsigned long long N) {
@@ -116,7 +139,7 @@ __global__ void __launch_bounds__(256) thr_sample_kernel(const ThrArgs a) {
     const int bhx = blockIdx.x, bh = bhx >> 1, x = bhx & 1;
     __shared__ __align__(16) unsigned short s_keys[SAMPLE_TOKENS * 128];
     __shared__ unsigned short s_nanflag[1];
-    __shared__ uint32_t hist[8 * 256], s_tmp[2], s_cnt;
+    __shared__ uint32_t hist[2048], s_tmp[2], s_cnt;
     const int b_idx = bh / a.H, h_idx = bh % a.H;
     const __half* X = a.X[x] + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
     const int ns = a.T < SAMPLE_TOKENS ? a.T : SAMPLE_TOKENS;
@@ -272,7 +295,7 @@ __global__ void __launch_bounds__(256) thr_select_kernel(const ThrArgs a) {
     const int bhx = blockIdx.x >> 1, side = blockIdx.x & 1, bh = bhx >> 1, x = bhx & 1;
     Problem* pr = a.prob + bhx;
     if (pr->done) return;
-    __shared__ uint32_t hist[8 * 256], s_tmp[2];
+    __shared__ uint32_t hist[2048], s_tmp[2];
     __shared__ __align__(16) unsigned short s_keys[SELECT_KEYS];
     const unsigned long long total = (unsigned long long)a.T * a.D;
     const unsigned long long N = total - pr->nan;
