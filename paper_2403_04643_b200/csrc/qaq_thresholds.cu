@@ -128,6 +128,102 @@ __device__ uint32_t cta_select(Get get, uint32_t n, uint32_t want, uint32_t* his
     return (prefix << 5) | low;
 }
 
+// The same select for keys that sit in shared memory (16-byte aligned), read eight at a time, for
+// two ranks at once: both share the round-0 histogram and each gets 32 bins in round 1.  Every key
+// counts here, NaN patterns too: as keys they sort below -inf (sign set) or above +inf, so a caller
+// whose ranks are meant among the non-NaN values adds the number of negative NaNs to them.
+// s_tmp: 4 words.
+__device__ void cta_select_keys(const unsigned short* keys, uint32_t n, uint32_t wantA, uint32_t wantB, uint32_t* hist,
+                                uint32_t* s_tmp, uint32_t& outA, uint32_t& outB) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint4* k8 = reinterpret_cast<const uint4*>(keys);
+    const uint32_t n8 = (n + 7) / 8;
+    for (int i = threadIdx.x; i < 2048; i += blockDim.x) hist[i] = 0;
+    if (threadIdx.x < 4) s_tmp[threadIdx.x] = 0;
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < n8; i += blockDim.x) {
+        const uint4 r = k8[i];
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t k = (w[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
+            if (8 * i + j < n) atomicAdd(&hist[k >> 5], 1u);
+        }
+    }
+    __syncthreads();
+    uint32_t c[8], tot = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { c[j] = hist[8 * threadIdx.x + j]; tot += c[j]; }
+    uint32_t inc = tot;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= d) inc += t;
+    }
+    __syncthreads();
+    if (lane == 31) hist[warp] = inc;
+    __syncthreads();
+    uint32_t before = 0, all = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        const uint32_t v = hist[w];
+        if (w < warp) before += v;
+        all += v;
+    }
+    const uint32_t first = before + inc - tot;               // keys in the bins before this thread's eight
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const uint32_t want = r ? wantB : wantA;
+        const uint32_t w2 = want < all ? want : (all ? all - 1 : 0);
+        if (tot > 0 && w2 >= first && w2 < first + tot) {    // exactly one thread per rank
+            uint32_t acc = first;
+            int bsel = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (w2 >= acc + c[j] && j < 7) { acc += c[j]; bsel = j + 1; }
+                else break;
+            }
+            s_tmp[2 * r] = (uint32_t)(8 * threadIdx.x + bsel);
+            s_tmp[2 * r + 1] = w2 - acc;
+        }
+    }
+    __syncthreads();
+    const uint32_t prefA = s_tmp[0], want1A = s_tmp[1], prefB = s_tmp[2], want1B = s_tmp[3];
+    if (threadIdx.x < 64) hist[threadIdx.x] = 0;
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < n8; i += blockDim.x) {
+        const uint4 r = k8[i];
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t k = (w[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
+            if (8 * i + j < n) {
+                if ((k >> 5) == prefA) atomicAdd(&hist[k & 31], 1u);
+                if ((k >> 5) == prefB) atomicAdd(&hist[32 + (k & 31)], 1u);
+            }
+        }
+    }
+    __syncthreads();
+    if (warp < 2) {                                          // warp 0: rank A, warp 1: rank B
+        const uint32_t v = hist[32 * warp + lane];
+        uint32_t in2 = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, in2, d);
+            if (lane >= d) in2 += t;
+        }
+        const uint32_t all2 = __shfl_sync(0xFFFFFFFFu, in2, 31);
+        const uint32_t want1 = warp ? want1B : want1A;
+        const uint32_t w3 = want1 < all2 ? want1 : (all2 ? all2 - 1 : 0);
+        if (all2 == 0 && lane == 0) s_tmp[2 * warp] = 0;
+        if (v > 0 && w3 >= in2 - v && w3 < in2) s_tmp[2 * warp] = (uint32_t)lane;
+    }
+    __syncthreads();
+    outA = (prefA << 5) | s_tmp[0];
+    outB = (prefB << 5) | s_tmp[2];
+    __syncthreads();
+}
+
 __device__ __forceinline__ unsigned long long rank_k(double alpha, unsigned long long N) {
     unsigned long long k = (unsigned long long)floor(alpha * (double)N / 2.0);
     if (N > 0 && k > (N - 1) / 2) k = (N - 1) / 2;
@@ -138,30 +234,35 @@ __device__ __forceinline__ unsigned long long rank_k(double alpha, unsigned long
 __global__ void __launch_bounds__(256) thr_sample_kernel(const ThrArgs a) {
     const int bhx = blockIdx.x, bh = bhx >> 1, x = bhx & 1;
     __shared__ __align__(16) unsigned short s_keys[SAMPLE_TOKENS * 128];
-    __shared__ unsigned short s_nanflag[1];
-    __shared__ uint32_t hist[2048], s_tmp[2], s_cnt;
+    __shared__ uint32_t hist[2048], s_tmp[4], s_cnt[2];
     const int b_idx = bh / a.H, h_idx = bh % a.H;
     const __half* X = a.X[x] + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
     const int ns = a.T < SAMPLE_TOKENS ? a.T : SAMPLE_TOKENS;
     const int M = ns * a.D;
-    if (threadIdx.x == 0) s_cnt = 0;
+    if (threadIdx.x < 2) s_cnt[threadIdx.x] = 0;
     __syncthreads();
-    uint32_t nn = 0;
+    uint32_t nn = 0, nneg = 0;                                  // NaNs, NaNs with the sign set
     for (int i = threadIdx.x; i < M / 8; i += blockDim.x) {    // 16-byte pieces
         const int s = (i * 8) / a.D, c = (i * 8) % a.D;
         const long t = (long)s * a.T / ns;                        // tokens spread over the sequence
         const uint4 r = *reinterpret_cast<const uint4*>(X + (size_t)t * a.st + c);
-        *reinterpret_cast<uint4*>(&s_keys[8 * i]) = r;
-        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+        uint32_t w[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if (!is_nan_bits((unsigned short)((w[j >> 1] >> (16 * (j & 1))) & 0xFFFF))) ++nn;
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t mag = w[j] & 0x7FFF7FFFu;
+            const uint32_t nan_lo = (mag & 0xFFFFu) > 0x7C00u, nan_hi = (mag >> 16) > 0x7C00u;
+            nn += nan_lo + nan_hi;
+            nneg += (nan_lo & (w[j] >> 15)) + (nan_hi & (w[j] >> 31));
+            // keys of both halves: a set sign flips all 16 bits, a clear one only the sign bit
+            const uint32_t neg = ((w[j] >> 15) & 0x00010001u) * 0xFFFFu;
+            w[j] ^= neg | 0x80008000u;
+        }
+        *reinterpret_cast<uint4*>(&s_keys[8 * i]) = make_uint4(w[0], w[1], w[2], w[3]);
     }
-    (void)s_nanflag;
-    atomicAdd(&s_cnt, nn);
+    if (nn) { atomicAdd(&s_cnt[0], nn); atomicAdd(&s_cnt[1], nneg); }
     __syncthreads();
-    const uint32_t Mv = s_cnt;                                     // non-NaN sample values
-    auto get = [&](uint32_t i) -> uint32_t { const unsigned short h = s_keys[i]; return is_nan_bits(h) ? 0x10000u : key_of(h); };
+    const uint32_t Mv = (uint32_t)M - s_cnt[0];                    // non-NaN sample values
+    const uint32_t n_neg_nan = s_cnt[1];
     Problem* pr = a.prob + bhx;
     const bool whole = (ns == a.T);
     if (Mv == 0) {
@@ -182,8 +283,8 @@ __global__ void __launch_bounds__(256) thr_sample_kernel(const ThrArgs a) {
         if (r > (Mv - 1) / 2) r = (Mv - 1) / 2;
         r_lo = r; r_hi = Mv - 1 - r;
     }
-    const uint32_t klo = cta_select(get, (uint32_t)M, r_lo, hist, s_tmp);
-    const uint32_t khi = cta_select(get, (uint32_t)M, r_hi, hist, s_tmp);
+    uint32_t klo, khi;
+    cta_select_keys(s_keys, (uint32_t)M, r_lo + n_neg_nan, r_hi + n_neg_nan, hist, s_tmp, klo, khi);
     if (threadIdx.x == 0) {
         pr->klo = klo; pr->khi = khi; pr->cnt[0] = pr->cnt[1] = 0; pr->nan = 0; pr->done = whole ? 1u : 0u;
         if (whole) {
@@ -295,7 +396,7 @@ __global__ void __launch_bounds__(256) thr_select_kernel(const ThrArgs a) {
     const int bhx = blockIdx.x >> 1, side = blockIdx.x & 1, bh = bhx >> 1, x = bhx & 1;
     Problem* pr = a.prob + bhx;
     if (pr->done) return;
-    __shared__ uint32_t hist[2048], s_tmp[2];
+    __shared__ uint32_t hist[2048], s_tmp[4];
     __shared__ __align__(16) unsigned short s_keys[SELECT_KEYS];
     const unsigned long long total = (unsigned long long)a.T * a.D;
     const unsigned long long N = total - pr->nan;
@@ -312,8 +413,9 @@ __global__ void __launch_bounds__(256) thr_select_kernel(const ThrArgs a) {
                 for (uint32_t i = threadIdx.x; i < (c + 7) / 8; i += blockDim.x)
                     reinterpret_cast<uint4*>(s_keys)[i] = reinterpret_cast<const uint4*>(l)[i];
                 __syncthreads();
-                auto gets = [&](uint32_t i) -> uint32_t { return s_keys[i]; };
-                res = float_of_key(cta_select(gets, c, want, hist, s_tmp));
+                uint32_t key, same;
+                cta_select_keys(s_keys, c, want, want, hist, s_tmp, key, same);
+                res = float_of_key(key);
             } else {
                 auto getg = [&](uint32_t i) -> uint32_t { return l[i]; };
                 res = float_of_key(cta_select(getg, c, want, hist, s_tmp));

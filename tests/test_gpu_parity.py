@@ -209,3 +209,25 @@ def test_c3_shaped_full_size_layer_sampled():
     wl = synth.scaled(synth.CONFIGS["C3"], layers=1)
     sel = [0, 97, 255]
     full_case(wl, HYPER["C2"], bh_sel=sel)
+
+
+@pytest.mark.parametrize("tokens", [48, 64, 1000])
+def test_thresholds_with_nans_of_both_signs(tokens):
+    # NaNs are left out of the population (the oracle's reading); 48 and 64 tokens are solved from the
+    # sample alone, 1000 tokens go through bracket, scan and select.  One head is NaN only.
+    wl = synth.scaled(synth.CONFIGS["C2"], heads=3, tokens=tokens)
+    K, V = synth.make_kv(wl, 0)
+    rng = np.random.default_rng(5)
+    Ku, Vu = u16(K).copy(), u16(V).copy()
+    for arr, frac in ((Ku, 0.02), (Vu, 0.3)):
+        m = rng.random(arr.shape) < frac
+        arr[m] = np.where(rng.random(int(m.sum())) < 0.5, 0x7E00, 0xFE01).astype(np.uint16)   # +NaN, -NaN
+    Vu[0, 2] = 0xFFFF
+    Kn = torch.from_numpy(Ku.view(np.float16)).cuda()
+    Vn = torch.from_numpy(Vu.view(np.float16)).cuda()
+    cfg = qaq.make_config(wl.batch, wl.heads, wl.head_dim, tokens, 2, 8, wl.window, wl.alpha)
+    thr = qaq.qaq_outlier_thresholds(cfg, Kn, Vn).cpu().numpy()
+    for bh in range(wl.bh):
+        b, h = divmod(bh, wl.heads)
+        want = (*oracle.thresholds(Ku[b, h], wl.alpha), *oracle.thresholds(Vu[b, h], wl.alpha))
+        assert np.array_equal(thr[bh], np.array(want, dtype=np.float32)), (bh, thr[bh], want)
