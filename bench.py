@@ -33,7 +33,7 @@ from paper_2403_04643_b200 import synth  # noqa: E402
 
 # DRAM bytes (read + write) per launch from an ncu capture of the C3 layer shape (profiles/kernels_C3_layer.md);
 # only valid for that shape and for the kernels as they were when the capture was taken.
-NCU_TRAFFIC = {("C3", "quant"): 672.9e6 + 128.4e6, ("C3", "decode"): 140.5e6 + 1.8e6}
+NCU_TRAFFIC = {("C3", "quant"): 672.9e6 + 128.4e6, ("C3", "decode"): 140.7e6 + 0.3e6}
 
 METRIC = "QAQ quantize GB/s + packed decode-attn tokens/s, % of B200 HBM peak"
 QNORM2 = 1.16   # stand-in for the upper-10% quantile of sum_d (q_d / sqrt(D))^2 of N(0,1) queries
