@@ -340,8 +340,15 @@ def _time_us(fn, reps):
 
 def extras(qaq, calibrate, dev, peak, qn):
     res = {}
-    for name, wl, T, prefill in (("C2_layer_batch1", synth.CONFIGS["C2"], 4096, 4096),
-                                 ("C5_long_context", synth.CONFIGS["C5"], 131072, 32768)):
+    c3 = synth.scaled(synth.CONFIGS["C3"], layers=1)
+    # (name, workload, tokens, prefill, target mean widths (K, V) or None, constant width or None)
+    points = (("C2_layer_batch1", synth.CONFIGS["C2"], 4096, 4096, (4.0, 3.0), None),
+              ("C5_long_context", synth.CONFIGS["C5"], 131072, 32768, (4.0, 3.0), None),
+              # low widths, the stress case for instruction issue (compression ratio near the paper's)
+              ("C3_layer_low_widths", c3, c3.tokens, c3.tokens, (2.2, 2.2), None),
+              # the comparison codec of Section 5.2: one width for every token, outliers kept apart as before
+              ("C3_layer_uniform4_with_outliers", c3, c3.tokens, c3.tokens, None, 4))
+    for name, wl, T, prefill, targets, uniform in points:
         D, BH, W = wl.head_dim, wl.bh, wl.window
         wlx = synth.scaled(wl, tokens=T, grow_to=0)
         K, V = synth.make_kv(wlx, 0, device=dev)
@@ -350,27 +357,42 @@ def extras(qaq, calibrate, dev, peak, qn):
         nv[:, :, prefill:] = 0                       # tokens appended after the prefill have no score yet
         cfg = qaq.make_config(wl.batch, wl.heads, D, T + 64, wl.bits_min, wl.bits_max, W, wl.alpha)
         thr = qaq.qaq_outlier_thresholds(cfg, K[:, :, :prefill], V[:, :, :prefill])
-        _, _, pol = calibrate(cfg, K[:, :, :prefill], V[:, :, :prefill], ring[:, :, :, :prefill].contiguous(),
-                              nv[:, :, :prefill].contiguous(), thr, prefill, qn)
+        pol, given = None, {}
+        if uniform is None:
+            _, _, pol = calibrate(cfg, K[:, :, :prefill], V[:, :, :prefill], ring[:, :, :, :prefill].contiguous(),
+                                  nv[:, :, :prefill].contiguous(), thr, prefill, qn, target_k=targets[0], target_v=targets[1])
+        else:
+            bits = torch.full((BH, T), uniform, dtype=torch.uint8, device=dev)
+            given = {"bitsK": bits, "bitsV": bits}
         cache = qaq.Cache(cfg)
         outb = torch.empty((BH, D), dtype=torch.float32, device=dev)
         scale = 1.0 / math.sqrt(D)
 
         def fill():
             cache.reset()
-            qaq.qaq_quantize_append(cache, K, V, thr, policy=pol, ring=ring, nvalid=nv)
+            if uniform is None:
+                qaq.qaq_quantize_append(cache, K, V, thr, policy=pol, ring=ring, nvalid=nv)
+            else:
+                qaq.qaq_quantize_append(cache, K, V, thr, **given)
         us_q = _time_us(fill, 5)
         us_d = _time_us(lambda: qaq.qaq_decode_attention(cache, q, scale, out=outb), 20)
         st = qaq.qaq_cache_stats(cache)
         ab = algorithmic_bytes(wlx, st)
+        if uniform is not None:     # given widths: two width bytes per token-head are read instead of the score window
+            ab["quantize"] += (2 - (4 * W + 1)) * BH * T
         # one-token append + decode, the streaming step
         k1, v1 = K[:, :, :1].contiguous(), V[:, :, :1].contiguous()
         r1, n1 = ring[:, :, :, :1].contiguous(), torch.zeros((wl.batch, wl.heads, 1), dtype=torch.uint8, device=dev)
         t_now = cache.tokens
         reps = min(32, cfg.max_tokens - t_now)
 
+        b1 = torch.full((BH, 1), uniform or 0, dtype=torch.uint8, device=dev)
+
         def stream():
-            qaq.qaq_quantize_append(cache, k1, v1, thr, policy=pol, ring=r1, nvalid=n1)
+            if uniform is None:
+                qaq.qaq_quantize_append(cache, k1, v1, thr, policy=pol, ring=r1, nvalid=n1)
+            else:
+                qaq.qaq_quantize_append(cache, k1, v1, thr, bitsK=b1, bitsV=b1)
             qaq.qaq_decode_attention(cache, q, scale, out=outb)
         torch.cuda.synchronize()
         a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
@@ -380,11 +402,13 @@ def extras(qaq, calibrate, dev, peak, qn):
         b.record(); torch.cuda.synchronize()
         us_s = a.elapsed_time(b) * 1e3 / reps
         res[name] = {"tokens": T, "bh": BH, "quantize_us": round(us_q, 1), "quantize_gbs": round(ab["quantize"] / us_q / 1e3, 1),
+                     "quantize_frac_of_hbm": round(ab["quantize"] / us_q / 1e3 / peak, 3),
                      "decode_us": round(us_d, 1), "decode_gbs": round(ab["decode"] / us_d / 1e3, 1),
                      "decode_frac_of_hbm": round(ab["decode"] / us_d / 1e3 / peak, 3),
                      "cached_tokens_per_s": round(wl.batch * T / (us_d * 1e-6), 1),
                      "append1_plus_decode_us": round(us_s, 1),
-                     "mean_bits": [round(st.code_bytes[0] * 8 / (BH * T * D), 2), round(st.code_bytes[1] * 8 / (BH * T * D), 2)]}
+                     "mean_bits": [round(st.code_bytes[0] * 8 / (BH * T * D), 2), round(st.code_bytes[1] * 8 / (BH * T * D), 2)],
+                     "cr_paper": round(st.cr_paper, 3)}
         del cache, K, V, ring
         torch.cuda.empty_cache()
     return res
