@@ -56,6 +56,7 @@ def lib():
         L.qaq_oracle_cr_paper.restype = C.c_double
         L.qaq_oracle_cr_paper.argtypes = [C.c_double, C.c_double, C.c_long, C.c_long, C.c_long, C.c_int]
         L.qaq_oracle_run_batch.restype = C.c_int
+        L.qaq_oracle_requantize_down.restype = C.c_long
         _lib = L
     return _lib
 
@@ -195,6 +196,36 @@ def quantize(x_u16, lo, hi, bits) -> QuantTensor:
                                   _p(val, C.c_uint16), C.c_long(ocap))
     assert n >= 0
     return QuantTensor(T, D, bits.copy(), mn, step, off, stream[: int(off[T])].copy(), rowptr, ch[:n].copy(), val[:n].copy())
+
+
+def reselect_bits(qt: QuantTensor, is_value: bool, ring, nvalid, c, bmin, bmax) -> np.ndarray:
+    """Widths recomputed from the stored form (range = step * 2^B) with the current window and policy scalar."""
+    out = np.empty(qt.T, np.uint8)
+    W = 0
+    ringp = nvp = None
+    if is_value:
+        ring = np.ascontiguousarray(ring, dtype=np.float32); nvalid = np.ascontiguousarray(nvalid, dtype=np.uint8)
+        W = ring.shape[0]
+        ringp, nvp = _p(ring, C.c_float), _p(nvalid, C.c_uint8)
+    lib().qaq_oracle_reselect_bits(C.c_long(qt.T), _p(np.ascontiguousarray(qt.bits), C.c_uint8),
+                                   _p(np.ascontiguousarray(qt.step), C.c_float), C.c_int(1 if is_value else 0), ringp, nvp,
+                                   C.c_int(W), C.c_float(c), C.c_int(bmin), C.c_int(bmax), _p(out, C.c_uint8))
+    return out
+
+
+def requantize_down(qt: QuantTensor, bits_req) -> QuantTensor:
+    """Every token at width min(current, requested): low code bits dropped, step scaled, the rest unchanged."""
+    req = np.ascontiguousarray(bits_req, dtype=np.uint8)
+    bits = np.empty(qt.T, np.uint8); step = np.empty(qt.T, np.float32); off = np.empty(qt.T + 1, np.uint32)
+    cap = int(qt.off[qt.T]) + 16
+    stream = np.zeros(cap, np.uint8)
+    src = np.ascontiguousarray(qt.stream) if qt.stream.size else np.zeros(1, np.uint8)
+    n = lib().qaq_oracle_requantize_down(C.c_long(qt.T), C.c_int(qt.D), _p(np.ascontiguousarray(qt.bits), C.c_uint8),
+                                         _p(np.ascontiguousarray(qt.step), C.c_float), _p(np.ascontiguousarray(qt.off), C.c_uint32),
+                                         _p(src, C.c_uint8), _p(req, C.c_uint8), _p(bits, C.c_uint8), _p(step, C.c_float),
+                                         _p(off, C.c_uint32), _p(stream, C.c_uint8), C.c_long(cap))
+    assert n >= 0
+    return QuantTensor(qt.T, qt.D, bits, qt.mn.copy(), step, off, stream[:n].copy(), qt.rowptr.copy(), qt.ch.copy(), qt.val.copy())
 
 
 def reconstruct(qt: QuantTensor) -> np.ndarray:

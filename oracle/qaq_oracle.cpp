@@ -330,6 +330,59 @@ void qaq_oracle_reconstruct(long T, int D, const uint8_t* bits, const float* mn,
     }
 }
 
+// ---- O9: further quantization to lower widths (Section 4.2, "Integration in text
+// generation process") ------------------------------------------------------------
+// In every generation step the widths of all cached tokens are computed again with the
+// current scores and token count; a token whose new width is lower than its current one
+// is quantized further, to the lower width.  Reading: the quantizer of O4 is nested -
+// with min and range kept, the B'-bit code of a value is its B-bit code without the low
+// B-B' bits - so "further" means code >>= (B-B') and step *= 2^(B-B'), which is what
+// quantizing the original values at B' directly would have given.  A new width that is
+// not lower leaves the token as it is (raising a width needs the unquantized copy the
+// paper keeps in CPU memory; that transfer is not part of this path).
+//
+// Widths from the stored form: the range of a token is step * 2^B (exact), so the rules
+// of O3 apply without the original values.
+void qaq_oracle_reselect_bits(long T, const uint8_t* bits, const float* step, int is_value, const float* ring,
+                              const uint8_t* nvalid, int W, float c, int bmin, int bmax, uint8_t* bits_new) {
+    std::vector<float> shat((size_t)T);
+    if (is_value) qaq_oracle_window_max(ring, nvalid, W, T, shat.data());
+    for (long t = 0; t < T; ++t) {
+        float r = std::ldexp(step[t], bits[t]);
+        int b;
+        if (!is_value) b = qaq_oracle_bits_ladder(r, c, bmin, bmax);
+        else if (std::isinf(shat[(size_t)t])) b = bmax;
+        else b = qaq_oracle_bits_ladder(r * shat[(size_t)t], c, bmin, bmax);
+        bits_new[t] = (uint8_t)b;
+    }
+}
+// One (b,h) tensor in canonical form (bits, step, off, stream) -> the same with every token
+// at width min(bits[t], max(1, bits_req[t])).  min[], the outlier lists and the code slots of
+// outliers (0) are unchanged.  Returns the new stream length, or -1 if cap is too small.
+long qaq_oracle_requantize_down(long T, int D, const uint8_t* bits, const float* step, const uint32_t* off,
+                                const uint8_t* stream, const uint8_t* bits_req, uint8_t* bits_out, float* step_out,
+                                uint32_t* off_out, uint8_t* stream_out, long cap) {
+    std::vector<uint8_t> codes((size_t)D);
+    long pos = 0;
+    for (long t = 0; t < T; ++t) {
+        int B = bits[t];
+        int want = bits_req[t] < 1 ? 1 : bits_req[t];
+        int Bn = want < B ? want : B;
+        int drop = B - Bn;
+        qaq_oracle_unpack_token(stream + off[t], D, B, codes.data());
+        for (int d = 0; d < D; ++d) codes[(size_t)d] = (uint8_t)(codes[(size_t)d] >> drop);
+        long nb = qaq_oracle_token_bytes(D, Bn);
+        if (pos + nb > cap) return -1;
+        off_out[t] = (uint32_t)pos;
+        qaq_oracle_pack_token(codes.data(), D, Bn, stream_out + pos);
+        pos += nb;
+        bits_out[t] = (uint8_t)Bn;
+        step_out[t] = std::ldexp(step[t], drop);
+    }
+    off_out[T] = (uint32_t)pos;
+    return pos;
+}
+
 // ---- O7: attention (Section 2.1, Figure 1) --------------------------------------
 // S = Softmax(scale * Q Khat^T),  X = S Vhat, on dense binary32 Khat, Vhat [T][D],
 // Q binary16 [D]; all sums in binary64; the softmax subtracts the row maximum.

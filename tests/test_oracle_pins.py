@@ -395,3 +395,70 @@ def test_batch_runner_equals_single_calls_and_threads_agree():
     assert len(set(bK.tolist())) >= 2 and len(set(bV.tolist())) >= 3
     qt = oracle.quantize(k[i], lo, hi, bK)
     assert np.array_equal(qt.stream, r1.K[i].stream) and np.array_equal(qt.val, r1.K[i].val)
+
+
+# ---- further quantization to lower widths (Section 4.2, integration in the generation process)
+def _requant_case(seed, T=40, D=64):
+    rng = np.random.default_rng(seed)
+    x = (rng.standard_normal((T, D)) * rng.lognormal(0, 0.5, (1, D))).astype(np.float16)
+    x[rng.random((T, D)) < 0.02] *= 12                       # a few entries beyond the thresholds
+    x[3] = x[3, 0]                                           # a constant token
+    xu = x.view(np.uint16)
+    lo, hi = oracle.thresholds(xu, 0.02)
+    bits = rng.integers(1, 9, T).astype(np.uint8)
+    return xu, lo, hi, bits, rng
+
+
+def test_requantize_down_equals_quantizing_the_original_at_the_lower_width():
+    # independent route to the same result: quantize the binary16 values directly at min(old, requested)
+    for seed in range(4):
+        xu, lo, hi, bits, rng = _requant_case(seed)
+        req = rng.integers(0, 10, bits.size).astype(np.uint8)            # 0 is treated as 1; 9 is above every width
+        got = oracle.requantize_down(oracle.quantize(xu, lo, hi, bits), req)
+        want_bits = np.minimum(bits, np.maximum(req, 1)).astype(np.uint8)
+        want = oracle.quantize(xu, lo, hi, want_bits)
+        assert np.array_equal(got.bits, want_bits)
+        assert np.array_equal(got.step.view(np.uint32), want.step.view(np.uint32))
+        assert np.array_equal(got.mn.view(np.uint32), want.mn.view(np.uint32))
+        assert np.array_equal(got.off, want.off) and np.array_equal(got.stream, want.stream)
+        assert np.array_equal(got.rowptr, want.rowptr) and np.array_equal(got.ch, want.ch) and np.array_equal(got.val, want.val)
+        assert (want_bits < bits).any() and (want_bits == bits).any()
+
+
+def test_requantize_down_drops_low_code_bits_and_never_raises_a_width():
+    xu, lo, hi, bits, rng = _requant_case(11)
+    q0 = oracle.quantize(xu, lo, hi, bits)
+    same = oracle.requantize_down(q0, np.full(bits.size, 8, np.uint8))   # nothing to lower
+    assert np.array_equal(same.bits, q0.bits) and np.array_equal(same.stream, q0.stream) and np.array_equal(same.step, q0.step)
+    req = np.full(bits.size, 2, np.uint8)
+    q1 = oracle.requantize_down(q0, req)
+    for t in range(q0.T):
+        B, Bn = int(q0.bits[t]), int(q1.bits[t])
+        assert Bn == min(B, 2)
+        c0 = oracle.unpack_token(q0.stream[q0.off[t]:q0.off[t + 1]], q0.D, B)
+        c1 = oracle.unpack_token(q1.stream[q1.off[t]:q1.off[t + 1]], q1.D, Bn)
+        assert np.array_equal(c1, c0 >> (B - Bn))
+        assert q1.step[t] == q0.step[t] * 2.0 ** (B - Bn)
+    # reconstruction error grows with the dropped bits but stays inside half a (new) step
+    x = xu.view(np.float16).astype(np.float64)
+    inl = (x >= lo) & (x <= hi)
+    err = np.abs(oracle.reconstruct(q1).astype(np.float64) - x)
+    assert np.all(err[inl] <= (0.5 * q1.step.astype(np.float64)[:, None] * np.ones_like(x))[inl] * (1 + 1e-3) + 1e-6)
+    assert np.all(err[~inl] == 0)                                         # outliers stay exact
+
+
+def test_reselect_from_stored_form_equals_selection_on_the_original_values():
+    rng = np.random.default_rng(3)
+    T, D, W = 48, 64, 6
+    K = (rng.standard_normal((T, D)) * 1.5).astype(np.float16).view(np.uint16)
+    V = (rng.standard_normal((T, D)) * 0.7).astype(np.float16).view(np.uint16)
+    thr = (*oracle.thresholds(K, 0.02), *oracle.thresholds(V, 0.02))
+    ring = rng.random((W, T)).astype(np.float32) * 0.05
+    nvalid = rng.integers(0, W + 1, T).astype(np.uint8)
+    cK, cV = oracle.policy(0.03, 0.035, 70.0, T)
+    bK, bV = oracle.select_bits(K, V, np.array(thr, np.float32), ring, nvalid, cK, cV, 2, 8)
+    top = np.full(T, 8, np.uint8)                                         # stored at the top width
+    qk, qv = oracle.quantize(K, thr[0], thr[1], top), oracle.quantize(V, thr[2], thr[3], top)
+    assert np.array_equal(oracle.reselect_bits(qk, False, None, None, cK, 2, 8), bK)
+    assert np.array_equal(oracle.reselect_bits(qv, True, ring, nvalid, cV, 2, 8), bV)
+    assert len(set(bK.tolist()) | set(bV.tolist())) >= 3
