@@ -409,6 +409,31 @@ def extras(qaq, calibrate, dev, peak, qn):
                      "append1_plus_decode_us": round(us_s, 1),
                      "mean_bits": [round(st.code_bytes[0] * 8 / (BH * T * D), 2), round(st.code_bytes[1] * 8 / (BH * T * D), 2)],
                      "cr_paper": round(st.cr_paper, 3)}
+        if name == "C3_layer_low_widths":
+            # the per-step lowering of widths (Section 4.2): a cache filled at mean widths (4, 3) is taken down to the
+            # widths of this point's looser budgets, in place; one call does the work, a repeat finds nothing to lower
+            _, _, pol43 = calibrate(cfg, K, V, ring, nv, thr, T, qn)
+            cache.reset()
+            qaq.qaq_quantize_append(cache, K, V, thr, policy=pol43, ring=ring, nvalid=nv)
+            qaq.qaq_requantize_down(cache, policy=pol43, ring=ring, nvalid=nv)     # warm-up: same widths, nothing changes
+            st0 = qaq.qaq_cache_stats(cache)
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            torch.cuda.synchronize()
+            ev[0].record()
+            qaq.qaq_requantize_down(cache, policy=pol, ring=ring, nvalid=nv)
+            ev[1].record()
+            qaq.qaq_requantize_down(cache, policy=pol, ring=ring, nvalid=nv)
+            ev[2].record(); torch.cuda.synchronize()
+            st1 = qaq.qaq_cache_stats(cache)
+            moved = sum(st0.code_bytes) + sum(st1.code_bytes) + BH * T * (2 * 5 + 2 + 4 * W + 1)
+            us_r = ev[0].elapsed_time(ev[1]) * 1e3
+            res["C3_layer_requantize_down"] = {
+                "from_mean_bits": [round(st0.code_bytes[x] * 8 / (BH * T * D), 2) for x in range(2)],
+                "to_mean_bits": [round(st1.code_bytes[x] * 8 / (BH * T * D), 2) for x in range(2)],
+                "requantize_us": round(us_r, 1), "bytes": int(moved), "gbs": round(moved / us_r / 1e3, 1),
+                "frac_of_hbm": round(moved / us_r / 1e3 / peak, 3),
+                "repeat_nothing_to_lower_us": round(ev[1].elapsed_time(ev[2]) * 1e3, 1),
+                "decode_after_us": round(_time_us(lambda: qaq.qaq_decode_attention(cache, q, scale, out=outb), 20), 1)}
         del cache, K, V, ring
         torch.cuda.empty_cache()
     return res

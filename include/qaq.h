@@ -137,6 +137,29 @@ qaq_status qaq_quantize_append(qaq_cache* c, const void* K_new, const void* V_ne
                                const uint8_t* nvalid, const float* thr, void* stream);
 
 /*
+ * Further quantization of the cached tokens to lower widths (Section 4.2, "Integration in
+ * text generation process": each step the widths of all existing tokens are computed again
+ * and tokens whose new width is lower are quantized further).  For every cached token and
+ * both tensors: new width = min(current width, w), where w is
+ *   - bitsK/bitsV[bh][t] (values below 1 count as 1) when both are given, else
+ *   - the width qaq_select_bits would choose now: the token's range max-min is taken from
+ *     its stored metadata, the score window and the policy scalars are the caller's current
+ *     ones (policy made for the current token count).
+ * A lowered token keeps min, max and its outliers; its codes lose their low bits
+ * (code >>= old-new, so step doubles per dropped bit), which equals quantizing the original
+ * values at the new width.  Widths are never raised (that needs the unquantized values).
+ * bitsK, bitsV: u8 [batch*heads][n_cols] or both NULL; score_ring: binary32
+ * [batch*heads][window][n_cols]; nvalid: u8 [batch*heads][n_cols]; n_cols >= cached tokens.
+ * Tiles are rewritten in place: the bytes read by qaq_decode_attention and the counters of
+ * qaq_cache_stats shrink; pool space inside closed tiles is not handed back to later appends.
+ * Device pointers; asynchronous on stream.  Errors: QAQ_ERR_INVALID_ARG (missing arrays,
+ * n_cols too small), QAQ_ERR_UNSUPPORTED_SHAPE, QAQ_ERR_CUDA; an empty cache is a no-op.
+ */
+qaq_status qaq_requantize_down(qaq_cache* c, const uint8_t* bitsK, const uint8_t* bitsV,
+                               const qaq_policy* policy, const float* score_ring, const uint8_t* nvalid,
+                               long n_cols, void* stream);
+
+/*
  * S4+S5: decode attention over the packed cache (Section 2.1, Figure 1):
  *   S = Softmax(softmax_scale * q Khat^T),  X = S Vhat,
  * Khat/Vhat = midpoint reconstruction min + (code + 1/2) * step with the stored outliers

@@ -22,6 +22,7 @@ EXPORTED = [
     "qaq_policy_from_hyper", "qaq_thresholds_workspace_bytes", "qaq_outlier_thresholds", "qaq_select_bits",
     "qaq_quantize_append", "qaq_decode_workspace_bytes", "qaq_decode_attention", "qaq_quantize_append_host",
     "qaq_decode_attention_host", "qaq_cache_stats", "qaq_cache_export", "qaq_decode_attention_static",
+    "qaq_requantize_down",
 ]
 
 
@@ -80,6 +81,8 @@ def lib():
         L.qaq_decode_attention_host.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]
         L.qaq_decode_attention_static.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]
         L.qaq_cache_stats.argtypes = [C.c_void_p, C.POINTER(Stats), C.c_void_p]
+        L.qaq_requantize_down.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(Policy), C.c_void_p, C.c_void_p,
+                                          C.c_long, C.c_void_p]
         L.qaq_cache_export.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_long, C.c_void_p, C.c_void_p, C.c_void_p, C.c_long, C.c_void_p]
         _lib = L
@@ -190,6 +193,18 @@ def qaq_quantize_append(cache: Cache, K_new, V_new, thr, *, bitsK=None, bitsV=No
     _check(lib().qaq_quantize_append(cache.handle, _ptr(K_new), _ptr(V_new), sb, sh, st, K_new.shape[2], _ptr(bitsK),
                                      _ptr(bitsV), pol, _ptr(ring), _ptr(nvalid), _ptr(thr), _stream()),
            "qaq_quantize_append")
+
+
+def qaq_requantize_down(cache: Cache, *, bitsK=None, bitsV=None, policy=None, ring=None, nvalid=None):
+    """Lower the widths of the cached tokens in place: to the given widths [BH, n_cols] where they are lower, or to
+    the widths the selection rules give now (policy for the current token count, ring [B,H,W,n_cols], nvalid)."""
+    ref = bitsK if bitsK is not None else nvalid
+    n_cols = ref.shape[-1]
+    for t in (bitsK, bitsV, ring, nvalid):
+        assert t is None or (t.is_contiguous() and t.shape[-1] == n_cols)
+    pol = C.byref(policy) if policy is not None else None
+    _check(lib().qaq_requantize_down(cache.handle, _ptr(bitsK), _ptr(bitsV), pol, _ptr(ring), _ptr(nvalid), n_cols,
+                                     _stream()), "qaq_requantize_down")
 
 
 def qaq_decode_attention(cache: Cache, q, softmax_scale, out=None, scores_out=None):

@@ -1,0 +1,104 @@
+"""GPU parity of the in-place further quantization to lower widths (Section 4.2, integration in the
+generation process) against the CPU oracle: widths, scales, byte offsets and packed codes bit for bit,
+attention over the lowered cache within the usual tolerance."""
+import math
+from types import SimpleNamespace
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2403_04643_b200 import qaq, synth
+
+from gpu_helpers import assert_attention_close, compare_export, gpu_pipeline, make_inputs, oracle_batch, u16
+
+pytestmark = pytest.mark.gpu
+
+HYPER = (0.002, 0.01, 128.0)        # mixed widths on the C2-shaped synthetic cache
+LOOSER = (0.02, 0.05, 128.0)        # larger variance budgets: lower widths
+
+
+def _decode_ref(wl, q, qk, qv):
+    qq = u16(q).reshape(wl.bh, wl.head_dim)
+    return np.stack([oracle.decode(qq[bh], qk[bh], qv[bh], 1.0 / math.sqrt(wl.head_dim))[0] for bh in range(wl.bh)])
+
+
+def test_widths_recomputed_by_the_rules_and_lowered_in_place():
+    # 1000 tokens = 15 full tiles + an open tile of 40; second window and looser budgets for the second selection
+    wl = synth.scaled(synth.CONFIGS["C2"], heads=3, tokens=1000)
+    K, V, q, ring, nv = make_inputs(wl, ragged=True)
+    T = K.shape[2]
+    polA = qaq.qaq_policy_from_hyper(*HYPER, T)
+    cfg, cache, thr, out, scores, dev = gpu_pipeline(wl, K, V, q, ring, nv, polA)
+    ref = oracle_batch(wl, K, V, q, ring, nv, *oracle.policy(*HYPER, T))
+    compare_export(cache, ref)
+
+    ring2, nv2 = synth.make_score_ring(wl, 7, ragged=True)
+    polB = qaq.qaq_policy_from_hyper(*LOOSER, T)
+    cKb, cVb = oracle.policy(*LOOSER, T)
+    qaq.qaq_requantize_down(cache, policy=polB, ring=ring2.cuda(), nvalid=nv2.cuda())
+    r2 = ring2.numpy().reshape(wl.bh, wl.window, T); n2 = nv2.numpy().reshape(wl.bh, T)
+    qk, qv = [], []
+    lowered = kept = 0
+    for bh in range(wl.bh):
+        bk = oracle.reselect_bits(ref.K[bh], False, None, None, cKb, wl.bits_min, wl.bits_max)
+        bv = oracle.reselect_bits(ref.V[bh], True, r2[bh], n2[bh], cVb, wl.bits_min, wl.bits_max)
+        qk.append(oracle.requantize_down(ref.K[bh], bk)); qv.append(oracle.requantize_down(ref.V[bh], bv))
+        for a, b in ((qk[-1], ref.K[bh]), (qv[-1], ref.V[bh])):
+            lowered += int((a.bits < b.bits).sum()); kept += int((a.bits == b.bits).sum())
+    assert lowered > 100 and kept > 100
+    compare_export(cache, SimpleNamespace(K=qk, V=qv))
+    out2 = qaq.qaq_decode_attention(cache, dev[2], 1.0 / math.sqrt(wl.head_dim))
+    assert_attention_close(out2.cpu().numpy(), _decode_ref(wl, q, qk, qv))
+    st = qaq.qaq_cache_stats(cache)
+    assert st.device_status == 0
+    assert st.code_bytes[0] == sum(int(t.off[T]) for t in qk) and st.code_bytes[1] == sum(int(t.off[T]) for t in qv)
+    # a second pass with the same inputs changes nothing
+    qaq.qaq_requantize_down(cache, policy=polB, ring=ring2.cuda(), nvalid=nv2.cuda())
+    compare_export(cache, SimpleNamespace(K=qk, V=qv))
+
+
+@pytest.mark.parametrize("D", [32, 64, 128])
+def test_given_widths_then_appends_continue_behind_the_shrunk_open_tile(D):
+    wl = synth.scaled(synth.CONFIGS["C1"], batch=2, heads=2, head_dim=D, tokens=150, seed=40 + D)
+    K, V, q, ring, nv = make_inputs(wl)
+    first, T = 100, 150                                   # 100 = one full tile + an open tile of 36
+    rng = np.random.default_rng(D)
+    b0 = rng.integers(3, 9, (2, wl.bh, T)).astype(np.uint8)       # widths at quantization time
+    req = rng.integers(0, 10, (2, wl.bh, first)).astype(np.uint8)  # requested later (0 counts as 1, 9 lowers nothing)
+    cfg = qaq.make_config(wl.batch, wl.heads, D, T, wl.bits_min, wl.bits_max, wl.window, wl.alpha)
+    Kd, Vd = K.cuda(), V.cuda()
+    thr = qaq.qaq_outlier_thresholds(cfg, Kd, Vd)
+    cache = qaq.Cache(cfg)
+    tb = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    qaq.qaq_quantize_append(cache, Kd[:, :, :first], Vd[:, :, :first], thr, bitsK=tb(b0[0][:, :first]), bitsV=tb(b0[1][:, :first]))
+    qaq.qaq_requantize_down(cache, bitsK=tb(req[0]), bitsV=tb(req[1]))
+    qaq.qaq_quantize_append(cache, Kd[:, :, first:], Vd[:, :, first:], thr, bitsK=tb(b0[0][:, first:]), bitsV=tb(b0[1][:, first:]))
+    # expected: every token quantized directly at its final width (the nesting property pinned on the CPU side)
+    final = b0.copy()
+    final[:, :, :first] = np.minimum(b0[:, :, :first], np.maximum(req, 1))
+    thr_h = thr.cpu().numpy()
+    ku, vu = u16(K).reshape(wl.bh, T, D), u16(V).reshape(wl.bh, T, D)
+    qk = [oracle.quantize(ku[bh], thr_h[bh, 0], thr_h[bh, 1], final[0, bh]) for bh in range(wl.bh)]
+    qv = [oracle.quantize(vu[bh], thr_h[bh, 2], thr_h[bh, 3], final[1, bh]) for bh in range(wl.bh)]
+    compare_export(cache, SimpleNamespace(K=qk, V=qv))
+    out = qaq.qaq_decode_attention(cache, q.cuda(), 1.0 / math.sqrt(D))
+    assert_attention_close(out.cpu().numpy(), _decode_ref(wl, q, qk, qv))
+    assert qaq.qaq_cache_stats(cache).device_status == 0
+
+
+def test_argument_errors_and_empty_cache():
+    wl = synth.scaled(synth.CONFIGS["C2"], heads=1, tokens=64)
+    cfg = qaq.make_config(1, 1, 128, 64, 2, 8, wl.window, wl.alpha)
+    cache = qaq.Cache(cfg)
+    bits = torch.full((1, 64), 4, dtype=torch.uint8, device="cuda")
+    qaq.qaq_requantize_down(cache, bitsK=bits, bitsV=bits)          # empty cache: nothing to do
+    K, V = synth.make_kv(wl)
+    thr = qaq.qaq_outlier_thresholds(cfg, K.cuda(), V.cuda())
+    qaq.qaq_quantize_append(cache, K.cuda(), V.cuda(), thr, bitsK=bits, bitsV=bits)
+    with pytest.raises(qaq.QaqError) as e:
+        qaq.qaq_requantize_down(cache, bitsK=bits[:, :32].contiguous(), bitsV=bits[:, :32].contiguous())   # fewer columns than tokens
+    assert e.value.code == 1
+    with pytest.raises(qaq.QaqError):
+        qaq.qaq_requantize_down(cache, nvalid=bits)                 # rules asked for, policy and window missing
