@@ -48,16 +48,16 @@ struct ThrArgs {
 };
 
 // rank select (0-based rank `want`) over n 16-bit keys readable through get(i); all threads of the
-// CTA (256) call it; hist is 2048 words of shared memory.  Two rounds of a radix select: the upper
+// CTA (256) call it; hist is 2048 words of shared memory.  Two passes of a radix select: the upper
 // 11 bits of the key first, then the lower 5.  binary16 data piles up in a few exponents, so a
 // histogram of the upper byte alone would send most lanes of a warp to the same handful of
-// counters; 11 bits spread them over 32 bins per octave.  In round 0 every thread sums 8 bins and a
-// CTA-wide prefix sum finds the bin holding the wanted rank; round 1 has 32 bins, one per lane of
+// counters; 11 bits spread them over 32 bins per octave.  In the first pass every thread sums 8 bins and a
+// CTA-wide prefix sum finds the bin holding the wanted rank; the second pass has 32 bins, one per lane of
 // warp 0.
 template <typename Get>
 __device__ uint32_t cta_select(Get get, uint32_t n, uint32_t want, uint32_t* hist, uint32_t* s_tmp) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // ---- round 0: upper 11 bits
+    // ---- first pass: upper 11 bits
     for (int i = threadIdx.x; i < 2048; i += blockDim.x) hist[i] = 0;
     __syncthreads();
     for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
@@ -101,7 +101,7 @@ __device__ uint32_t cta_select(Get get, uint32_t n, uint32_t want, uint32_t* his
     __syncthreads();
     const uint32_t prefix = s_tmp[0];
     const uint32_t want1 = s_tmp[1];
-    // ---- round 1: lower 5 bits of the keys in that bin
+    // ---- second pass: lower 5 bits of the keys in that bin
     if (threadIdx.x < 32) hist[threadIdx.x] = 0;
     __syncthreads();
     for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
@@ -129,7 +129,7 @@ __device__ uint32_t cta_select(Get get, uint32_t n, uint32_t want, uint32_t* his
 }
 
 // The same select for keys that sit in shared memory (16-byte aligned), read eight at a time, for
-// two ranks at once: both share the round-0 histogram and each gets 32 bins in round 1.  Every key
+// two ranks at once: both share the first-pass histogram and each gets 32 bins in the second pass.  Every key
 // counts here, NaN patterns too: as keys they sort below -inf (sign set) or above +inf, so a caller
 // whose ranks are meant among the non-NaN values adds the number of negative NaNs to them.
 // s_tmp: 4 words.
