@@ -265,6 +265,27 @@ def attention_fp16(q_u16, K_u16, V_u16, scale):
     return X, S
 
 
+def prefill_window(Q_u16, K_u16, scale):
+    """Score window after a prefill (Section 4.2, attention score prediction: the scores of the preceding n
+    queries).  Q: the last n queries [n, D], K: all T keys [T, D], binary16 patterns.  Query i (position
+    T - n + i) sees tokens 0..T-n+i; its row is the softmax over those of scale * q_i . k_t.  Rows are stored newest
+    first (row r = query n-1-r), so the rows in which token t exists are 0..nvalid[t]-1, nvalid[t] = min(n, T-t);
+    the other entries are 0.  Also returns sum_d (scale * q_d)^2 per query, in query order."""
+    Q = np.ascontiguousarray(Q_u16, dtype=np.uint16); K = np.ascontiguousarray(K_u16, dtype=np.uint16)
+    n, D = Q.shape
+    T = K.shape[0]
+    ring = np.zeros((n, T), np.float64)
+    for i in range(n):
+        vis = T - n + i + 1
+        if vis < 1:
+            continue
+        _, S = attention_fp16(Q[i], K[:vis], K[:vis], scale)
+        ring[n - 1 - i, :vis] = S
+    nvalid = np.minimum(n, T - np.arange(T)).astype(np.uint8)
+    qf = Q.view(np.float16).astype(np.float64) * scale
+    return ring, nvalid, (qf * qf).sum(axis=1)
+
+
 def decode(q_u16, qk: QuantTensor, qv: QuantTensor, scale):
     return attention_dense(q_u16, reconstruct(qk), reconstruct(qv), scale)
 

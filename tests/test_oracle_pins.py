@@ -462,3 +462,23 @@ def test_reselect_from_stored_form_equals_selection_on_the_original_values():
     assert np.array_equal(oracle.reselect_bits(qk, False, None, None, cK, 2, 8), bK)
     assert np.array_equal(oracle.reselect_bits(qv, True, ring, nvalid, cV, 2, 8), bV)
     assert len(set(bK.tolist()) | set(bV.tolist())) >= 3
+
+
+def test_prefill_window_rows_are_causal_softmax_rows_newest_first():
+    rng = np.random.default_rng(8)
+    T, n, D = 37, 5, 32
+    Q = rng.standard_normal((n, D)).astype(np.float16); K = rng.standard_normal((T, D)).astype(np.float16)
+    scale = 1.0 / math.sqrt(D)
+    ring, nvalid, qn2 = oracle.prefill_window(Q.view(np.uint16), K.view(np.uint16), scale)
+    logits = torch.from_numpy(Q.astype(np.float64)) @ torch.from_numpy(K.astype(np.float64)).T * scale   # [n, T]
+    for i in range(n):
+        vis = T - n + i + 1
+        want = torch.softmax(logits[i, :vis], dim=0).numpy()
+        row = ring[n - 1 - i]
+        assert np.allclose(row[:vis], want, rtol=1e-12, atol=1e-15) and np.all(row[vis:] == 0)
+    for t in range(T):                                   # the rows holding token t are exactly 0..nvalid[t]-1
+        assert np.all(ring[: nvalid[t], t] > 0) and np.all(ring[nvalid[t]:, t] == 0)
+    assert np.allclose(qn2, (Q.astype(np.float64) ** 2).sum(1) * scale * scale)
+    # feeds the window maximum like any other ring
+    shat = oracle.window_max(ring.astype(np.float32), nvalid)
+    assert np.allclose(shat, ring.astype(np.float32).max(axis=0))
