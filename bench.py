@@ -409,6 +409,13 @@ def extras(qaq, calibrate, dev, peak, qn):
                      "append1_plus_decode_us": round(us_s, 1),
                      "mean_bits": [round(st.code_bytes[0] * 8 / (BH * T * D), 2), round(st.code_bytes[1] * 8 / (BH * T * D), 2)],
                      "cr_paper": round(st.cr_paper, 3)}
+        if name == "C3_layer_uniform4_with_outliers":
+            # the score window after a prefill (Section 4.2): rows of the last `window` queries on the fp16 keys
+            Qw = torch.randn((BH, W, D), device=dev, dtype=torch.float32).to(torch.float16)
+            us_w = _time_us(lambda: qaq.qaq_prefill_window(cfg, Qw, K, scale), 10)
+            moved = BH * T * (2 * D + 3 * 4 * W + 1)           # K once; ring written, then read and written again
+            res["C3_layer_prefill_window"] = {"rows": W, "us": round(us_w, 1), "bytes": int(moved),
+                                              "gbs": round(moved / us_w / 1e3, 1), "frac_of_hbm": round(moved / us_w / 1e3 / peak, 3)}
         if name == "C3_layer_low_widths":
             # the per-step lowering of widths (Section 4.2): a cache filled at mean widths (4, 3) is taken down to the
             # widths of this point's looser budgets, in place; one call does the work, a repeat finds nothing to lower

@@ -117,6 +117,28 @@ qaq_status qaq_select_bits(const qaq_config* cfg, const qaq_policy* policy, cons
                            uint8_t* bitsK, uint8_t* bitsV, void* stream);
 
 /*
+ * Score window right after a prefill (Section 4.2, "Attention score prediction": the predicted
+ * score of a token is the maximum over the scores of the preceding n queries; n = cfg->window,
+ * at most 64).  From the last n queries of a prefill of n_tokens tokens and the unquantized keys:
+ *   row of query i (position n_tokens-n+i) = softmax over the tokens t <= n_tokens-n+i of
+ *   softmax_scale * q_i . k_t   (binary16 inputs, tensor-core products, binary32 sums),
+ * written newest first: score_ring[bh][r][t] with r = n-1-i, so the rows in which token t exists
+ * are 0..nvalid[t]-1, nvalid[t] = min(n, n_tokens-t); entries a query cannot see are 0.  This is
+ * the layout qaq_select_bits / qaq_quantize_append / qaq_requantize_down take.  With fewer than n
+ * tokens the queries that do not exist are ignored.
+ * Q: binary16 [batch*heads][n][head_dim], 16-byte aligned; K as in qaq_outlier_thresholds;
+ * score_ring: binary32 [batch*heads][n][n_tokens]; nvalid: u8 [batch*heads][n_tokens];
+ * qnorm2: NULL or binary32 [batch*heads][n] receiving sum_d (softmax_scale * q_d)^2 per query
+ * (the caller takes the quantile it wants for qaq_policy_from_hyper); ws:
+ * qaq_prefill_window_workspace_bytes bytes, 8-byte aligned.  Device pointers, asynchronous on
+ * stream.  Errors: QAQ_ERR_INVALID_ARG, QAQ_ERR_UNSUPPORTED_SHAPE (window > 64), QAQ_ERR_WORKSPACE.
+ */
+qaq_status qaq_prefill_window_workspace_bytes(const qaq_config* cfg, int n_tokens, size_t* host_out);
+qaq_status qaq_prefill_window(const qaq_config* cfg, const void* Q, const void* K, long stride_b, long stride_h,
+                              long stride_t, int n_tokens, float softmax_scale, float* score_ring,
+                              uint8_t* nvalid, float* qnorm2, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * S2+S3: append n_new tokens per (b,h) to the cache: outlier split (entries outside
  * [lo,hi] are kept as binary16 in a sparse side list and take code 0), uniform
  * quantization of each token at its width (Section 4.1: the range [min,max] of the

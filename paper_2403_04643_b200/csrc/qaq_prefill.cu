@@ -1,0 +1,229 @@
+// Score window after a prefill (Section 4.2 of the paper, "Attention score prediction": the
+// predicted score of a token is the maximum over the scores of the preceding n queries).  Right
+// after a prefill of T tokens those are the attention rows of its last n queries on the
+// unquantized binary16 keys:
+//   row of query i (position T-n+i):  softmax over the tokens t <= T-n+i of  scale * q_i . k_t.
+// Rows are written newest first (row r = query n-1-r), so that the rows in which token t exists
+// are 0..nvalid[t]-1 with nvalid[t] = min(n, T-t); entries of tokens a query cannot see are 0.
+//
+// This is the one dense contraction on the path ([n x D] x [D x T] per (b,h)), so the logits run
+// on the tensor cores (mma.sync m16n8k16, binary16 in, binary32 accumulate); with n <= 64 rows it is
+// bound by reading K once.  Two kernels: logits + per-chunk (max, sum of exponentials) of every
+// row; then the rows are normalised in place with the merged (max, sum).
+#include "qaq_internal.cuh"
+
+namespace {
+
+constexpr int PW_WARPS = 4;
+constexpr int PW_CHUNK = 256;          // tokens per CTA: 64 per warp, 8 at a time
+constexpr int PW_MAXQ = 64;            // rows (queries) at most
+
+struct PrefillArgs {
+    const __half* Q;     // [BH][n][D]
+    const __half* K;
+    long sb, sh, st;
+    int H, T, n;
+    float scale;
+    float* ring;         // [BH][n][T]
+    uint8_t* nvalid;     // [BH][T]
+    float* qnorm2;       // [BH][n] or null
+    float2* part;        // [BH][nchunk][n] (max, sum of exp) of the visible logits of a chunk
+    int nchunk;
+};
+
+__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// The contraction index is permuted the same way in both operands: lane c (of the four lanes that
+// share a row / a token) owns channels [c*D/4, (c+1)*D/4), read with 16-byte loads; k-step ks takes
+// words 2ks and 2ks+1 of them.
+template <int D>
+__global__ void __launch_bounds__(PW_WARPS * 32) window_logits_kernel(const PrefillArgs a) {
+    constexpr int WPL = D / 8;          // 32-bit words per lane and row
+    constexpr int KS = D / 16;          // k-steps
+    const int bh = blockIdx.y, chunk = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, c = lane & 3;
+    const int b_idx = bh / a.H, h_idx = bh % a.H;
+    const __half* Kb = a.K + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
+    const __half* Qb = a.Q + (size_t)bh * a.n * D;
+    __shared__ float2 s_part[PW_WARPS][PW_MAXQ];
+
+    if (a.qnorm2 && chunk == 0) {
+        for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
+            float s = 0.f;
+            for (int d = 0; d < D; ++d) { const float f = a.scale * __half2float(Qb[(size_t)i * D + d]); s = fmaf(f, f, s); }
+            a.qnorm2[(size_t)bh * a.n + i] = s;
+        }
+    }
+    const int t_warp = chunk * PW_CHUNK + warp * (PW_CHUNK / PW_WARPS);
+    const float NEG = __int_as_float(0xff800000);
+
+    for (int mp = 0; mp * 32 < a.n; ++mp) {            // two 16-row tiles of queries at a time
+        uint32_t afr[2][KS][4];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+            const int r0 = mp * 32 + mt * 16 + g, r1 = r0 + 8;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                const uint32_t* q0 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r0 * D + c * (D / 4)) + 2 * ks;
+                const uint32_t* q1 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r1 * D + c * (D / 4)) + 2 * ks;
+                afr[mt][ks][0] = r0 < a.n ? q0[0] : 0u;
+                afr[mt][ks][1] = r1 < a.n ? q1[0] : 0u;
+                afr[mt][ks][2] = r0 < a.n ? q0[1] : 0u;
+                afr[mt][ks][3] = r1 < a.n ? q1[1] : 0u;
+            }
+        }
+        // running (max, sum) of this lane's share of rows (mt, g) and (mt, g+8)
+        float rm[2][2], rs[2][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) { rm[mt][0] = rm[mt][1] = NEG; rs[mt][0] = rs[mt][1] = 0.f; }
+
+        for (int step = 0; step < PW_CHUNK / PW_WARPS / 8; ++step) {
+            const int t0 = t_warp + 8 * step;
+            if (t0 >= a.T) break;
+            uint32_t bw[WPL];
+            {
+                const int t = t0 + g;
+                const uint4* src = reinterpret_cast<const uint4*>(Kb + (size_t)(t < a.T ? t : 0) * a.st + c * (D / 4));
+#pragma unroll
+                for (int i = 0; i < WPL / 4; ++i) {
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (t < a.T) v = src[i];
+                    bw[4 * i] = v.x; bw[4 * i + 1] = v.y; bw[4 * i + 2] = v.z; bw[4 * i + 3] = v.w;
+                }
+            }
+            float acc[2][4];
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) mma_16816(acc[mt], afr[mt][ks], bw[2 * ks], bw[2 * ks + 1]);
+            }
+            // acc[mt][0..1]: row g, tokens t0+2c, t0+2c+1;  acc[mt][2..3]: row g+8
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int hr = 0; hr < 2; ++hr) {
+                    const int i = mp * 32 + mt * 16 + g + 8 * hr;          // query
+                    if (i >= a.n) continue;
+                    const int last = a.T - a.n + i;                         // last token the query sees
+                    float* row = a.ring + ((size_t)bh * a.n + (a.n - 1 - i)) * a.T;
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int t = t0 + 2 * c + e;
+                        if (t >= a.T) continue;
+                        const float l = a.scale * acc[mt][2 * hr + e];
+                        row[t] = l;
+                        if (t <= last) {
+                            const float mnew = fmaxf(rm[mt][hr], l);
+                            rs[mt][hr] = rs[mt][hr] * __expf(rm[mt][hr] - mnew) + __expf(l - mnew);
+                            rm[mt][hr] = mnew;
+                        }
+                    }
+                }
+        }
+        // merge the four lanes of a row, then the warps, into the chunk's partial
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int hr = 0; hr < 2; ++hr) {
+                float m = rm[mt][hr], s = rs[mt][hr];
+#pragma unroll
+                for (int o = 1; o < 4; o <<= 1) {
+                    const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, o), s2 = __shfl_xor_sync(0xFFFFFFFFu, s, o);
+                    const float mn = fmaxf(m, m2);
+                    s = (m == NEG ? 0.f : s * __expf(m - mn)) + (m2 == NEG ? 0.f : s2 * __expf(m2 - mn));
+                    m = mn;
+                }
+                const int il = mt * 16 + g + 8 * hr;                        // row inside this pair of tiles
+                if (c == 0) s_part[warp][il] = make_float2(m, s);
+            }
+        __syncthreads();
+        for (int il = threadIdx.x; il < 32; il += blockDim.x) {
+            const int i = mp * 32 + il;
+            if (i >= a.n) continue;
+            float m = NEG, s = 0.f;
+            for (int w = 0; w < PW_WARPS; ++w) {
+                const float2 p = s_part[w][il];
+                const float mn = fmaxf(m, p.x);
+                s = (m == NEG ? 0.f : s * __expf(m - mn)) + (p.x == NEG ? 0.f : p.y * __expf(p.x - mn));
+                m = mn;
+            }
+            a.part[((size_t)bh * a.nchunk + chunk) * a.n + i] = make_float2(m, s);
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void __launch_bounds__(256) window_normalize_kernel(const PrefillArgs a) {
+    const int bh = blockIdx.y, chunk = blockIdx.x;
+    __shared__ float s_m[PW_MAXQ], s_inv[PW_MAXQ];
+    const float NEG = __int_as_float(0xff800000);
+    for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
+        float m = NEG, s = 0.f;
+        for (int ch = 0; ch < a.nchunk; ++ch) {
+            const float2 p = a.part[((size_t)bh * a.nchunk + ch) * a.n + i];
+            const float mn = fmaxf(m, p.x);
+            s = (m == NEG ? 0.f : s * __expf(m - mn)) + (p.x == NEG ? 0.f : p.y * __expf(p.x - mn));
+            m = mn;
+        }
+        s_m[i] = m;
+        s_inv[i] = s > 0.f ? 1.0f / s : 0.f;
+    }
+    __syncthreads();
+    const int t_lo = chunk * PW_CHUNK;
+    const int nt = min(PW_CHUNK, a.T - t_lo);
+    for (int idx = threadIdx.x; idx < a.n * nt; idx += blockDim.x) {
+        const int r = idx / nt, t = t_lo + idx % nt;
+        const int i = a.n - 1 - r;
+        float* p = a.ring + ((size_t)bh * a.n + r) * a.T + t;
+        *p = (t <= a.T - a.n + i) ? __expf(*p - s_m[i]) * s_inv[i] : 0.f;
+    }
+    for (int k = threadIdx.x; k < nt; k += blockDim.x) {
+        const int t = t_lo + k;
+        a.nvalid[(size_t)bh * a.T + t] = (uint8_t)min(a.n, a.T - t);
+    }
+}
+
+}  // namespace
+
+extern "C" qaq_status qaq_prefill_window_workspace_bytes(const qaq_config* cfg, int n_tokens, size_t* host_out) {
+    if (!cfg || !host_out || n_tokens < 1 || cfg->batch < 1 || cfg->heads < 1 || cfg->window < 1) return QAQ_ERR_INVALID_ARG;
+    const size_t nchunk = ((size_t)n_tokens + PW_CHUNK - 1) / PW_CHUNK;
+    *host_out = (size_t)cfg->batch * cfg->heads * nchunk * (size_t)cfg->window * sizeof(float2);
+    return QAQ_OK;
+}
+
+extern "C" qaq_status qaq_prefill_window(const qaq_config* cfg, const void* Q, const void* K, long stride_b, long stride_h,
+                                         long stride_t, int n_tokens, float softmax_scale, float* score_ring,
+                                         uint8_t* nvalid, float* qnorm2, void* ws, size_t ws_bytes, void* stream) {
+    if (!cfg || !Q || !K || !score_ring || !nvalid || !ws || n_tokens < 1) return QAQ_ERR_INVALID_ARG;
+    if (!qaq_dim_ok(cfg->head_dim) || cfg->window < 1 || cfg->window > PW_MAXQ) return QAQ_ERR_UNSUPPORTED_SHAPE;
+    if (((uintptr_t)K & 15) || ((uintptr_t)Q & 15) || (stride_b & 7) || (stride_h & 7) || (stride_t & 7) ||
+        stride_t < cfg->head_dim || stride_b < 0 || stride_h < 0)
+        return QAQ_ERR_INVALID_ARG;
+    size_t need = 0;
+    qaq_prefill_window_workspace_bytes(cfg, n_tokens, &need);
+    if (ws_bytes < need || ((uintptr_t)ws & 7)) return QAQ_ERR_WORKSPACE;
+    PrefillArgs a;
+    a.Q = (const __half*)Q; a.K = (const __half*)K; a.sb = stride_b; a.sh = stride_h; a.st = stride_t;
+    a.H = cfg->heads; a.T = n_tokens; a.n = cfg->window; a.scale = softmax_scale;
+    a.ring = score_ring; a.nvalid = nvalid; a.qnorm2 = qnorm2; a.part = (float2*)ws;
+    a.nchunk = (n_tokens + PW_CHUNK - 1) / PW_CHUNK;
+    const dim3 grid((unsigned)a.nchunk, (unsigned)(cfg->batch * cfg->heads));
+    cudaStream_t s = (cudaStream_t)stream;
+    switch (cfg->head_dim) {
+        case 32: window_logits_kernel<32><<<grid, PW_WARPS * 32, 0, s>>>(a); break;
+        case 64: window_logits_kernel<64><<<grid, PW_WARPS * 32, 0, s>>>(a); break;
+        case 128: window_logits_kernel<128><<<grid, PW_WARPS * 32, 0, s>>>(a); break;
+        default: return QAQ_ERR_UNSUPPORTED_SHAPE;
+    }
+    window_normalize_kernel<<<grid, 256, 0, s>>>(a);
+    QAQ_CUDA_TRY(cudaGetLastError());
+    return QAQ_OK;
+}

@@ -22,7 +22,7 @@ EXPORTED = [
     "qaq_policy_from_hyper", "qaq_thresholds_workspace_bytes", "qaq_outlier_thresholds", "qaq_select_bits",
     "qaq_quantize_append", "qaq_decode_workspace_bytes", "qaq_decode_attention", "qaq_quantize_append_host",
     "qaq_decode_attention_host", "qaq_cache_stats", "qaq_cache_export", "qaq_decode_attention_static",
-    "qaq_requantize_down",
+    "qaq_requantize_down", "qaq_prefill_window_workspace_bytes", "qaq_prefill_window",
 ]
 
 
@@ -81,6 +81,9 @@ def lib():
         L.qaq_decode_attention_host.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]
         L.qaq_decode_attention_static.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]
         L.qaq_cache_stats.argtypes = [C.c_void_p, C.POINTER(Stats), C.c_void_p]
+        L.qaq_prefill_window_workspace_bytes.argtypes = [C.POINTER(Config), C.c_int, C.POINTER(C.c_size_t)]
+        L.qaq_prefill_window.argtypes = [C.POINTER(Config), C.c_void_p, C.c_void_p, C.c_long, C.c_long, C.c_long, C.c_int,
+                                         C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.qaq_requantize_down.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(Policy), C.c_void_p, C.c_void_p,
                                           C.c_long, C.c_void_p]
         L.qaq_cache_export.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -193,6 +196,23 @@ def qaq_quantize_append(cache: Cache, K_new, V_new, thr, *, bitsK=None, bitsV=No
     _check(lib().qaq_quantize_append(cache.handle, _ptr(K_new), _ptr(V_new), sb, sh, st, K_new.shape[2], _ptr(bitsK),
                                      _ptr(bitsV), pol, _ptr(ring), _ptr(nvalid), _ptr(thr), _stream()),
            "qaq_quantize_append")
+
+
+def qaq_prefill_window(cfg: Config, Q, K, softmax_scale, want_qnorm2=False):
+    """Score window after a prefill: Q [B*H, window, D] (the last `window` queries), K [B,H,T,D], both fp16 on the
+    device.  Returns (ring [B,H,window,T] fp32, nvalid [B,H,T] u8[, qnorm2 [B*H, window]])."""
+    sb, sh, st = _strides(K)
+    BH, T, n = cfg.batch * cfg.heads, K.shape[2], cfg.window
+    assert Q.dtype == torch.float16 and Q.is_contiguous() and Q.numel() == BH * n * cfg.head_dim
+    ring = torch.empty((cfg.batch, cfg.heads, n, T), dtype=torch.float32, device=K.device)
+    nvalid = torch.empty((cfg.batch, cfg.heads, T), dtype=torch.uint8, device=K.device)
+    qn = torch.empty((BH, n), dtype=torch.float32, device=K.device) if want_qnorm2 else None
+    nb = C.c_size_t()
+    _check(lib().qaq_prefill_window_workspace_bytes(C.byref(cfg), T, C.byref(nb)), "qaq_prefill_window_workspace_bytes")
+    ws = torch.empty(max(nb.value, 8), dtype=torch.uint8, device=K.device)
+    _check(lib().qaq_prefill_window(C.byref(cfg), _ptr(Q), _ptr(K), sb, sh, st, T, float(softmax_scale), _ptr(ring),
+                                    _ptr(nvalid), _ptr(qn), _ptr(ws), ws.numel(), _stream()), "qaq_prefill_window")
+    return (ring, nvalid, qn) if want_qnorm2 else (ring, nvalid)
 
 
 def qaq_requantize_down(cache: Cache, *, bitsK=None, bitsV=None, policy=None, ring=None, nvalid=None):
