@@ -133,8 +133,8 @@ __device__ __forceinline__ uint32_t pool_take(uint32_t* pool, uint32_t amount, u
 
 // One CTA = one tile of 64 tokens of one (b,h); P = D/32 lanes own a token, each lane 32
 // consecutive channels (64 bytes) of K and of V, kept in registers across all phases.
-// Order of work (barriers in brackets): loads, attention window, outlier masks and ranges
-// [0] widths [A] warp 0 scans the tile and takes pool space with four atomics in flight at once
+// Order of work (barriers in brackets): loads, attention window, outlier masks and ranges,
+// widths [A] warp 0 scans the tile and takes pool space with four atomics in flight at once
 // while every warp computes its codes [B] planes into a shared-memory image of the tile
 // [C] the image goes out with 16-byte stores; outlier entries and per-token metadata follow.
 template <int D, bool SELECT_ONLY>
@@ -153,8 +153,6 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
     const bool valid = slot >= s_lo && slot < s_hi;
     const int tn = tile * QAQ_TILE + slot - a.t_old;  // index among the new tokens
 
-    __shared__ float s_part[P][QAQ_TILE];
-    __shared__ uint8_t s_nv[QAQ_TILE];
     __shared__ uint32_t s_len[2][QAQ_TILE];   // bytes, then exclusive byte offsets
     __shared__ uint32_t s_cnt[2][QAQ_TILE];   // outlier counts, then exclusive offsets
     __shared__ uint32_t s_tot[2], s_base[2], s_obase[2], s_olimit[2];
@@ -182,23 +180,18 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
         }
     }
 
-    // ---- attention window; P threads share the rows of one token
+    // ---- attention window: the P lanes of a token take its rows p, p+P, ... and combine by shuffles
+    float shat = __int_as_float(0xff800000);
+    int nv_tok = 0;
     {
-        const int g = tid / QAQ_TILE, tok = tid % QAQ_TILE;
-        float m = __int_as_float(0xff800000);
-        int nv = 0;
-        if (!given && tok >= s_lo && tok < s_hi) {
-            const int t2 = tile * QAQ_TILE + tok - a.t_old;
-            nv = a.nvalid[(size_t)bh * a.n_new + t2];
-            nv = nv < a.W ? nv : a.W;
-            const float* r = a.ring + (size_t)bh * a.W * a.n_new + t2;
-            for (int i = g; i < nv; i += P) m = fmaxf(m, r[(size_t)i * a.n_new]);
+        if (!given && valid) {
+            nv_tok = a.nvalid[(size_t)bh * a.n_new + tn];
+            nv_tok = nv_tok < a.W ? nv_tok : a.W;
+            const float* r = a.ring + (size_t)bh * a.W * a.n_new + tn;
+            for (int i = p; i < nv_tok; i += P) shat = fmaxf(shat, r[(size_t)i * a.n_new]);
         }
-        s_part[g][tok] = m;
-        if (g == 0) {
-            s_nv[tok] = (uint8_t)nv;
-            s_len[0][tok] = 0; s_len[1][tok] = 0; s_cnt[0][tok] = 0; s_cnt[1][tok] = 0;
-        }
+#pragma unroll
+        for (int o = 1; o < P; o <<= 1) shat = fmaxf(shat, __shfl_xor_sync(0xFFFFFFFFu, shat, o));
     }
 
     // ---- outlier masks and range of the rest (register work, needs nothing from shared memory)
@@ -222,7 +215,6 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
         for (int o = 1; o < P; o <<= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
         mnf[x] = mn; mxf[x] = mx; cntx[x] = cnt;
     }
-    __syncthreads();   // [0] window partials visible
 
     // ---- widths
     int Bx[2];
@@ -237,17 +229,14 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
             if (x == 0) {
                 B = ladder(r, a.cK, a.bmin, a.bmax);
             } else {
-                float sh = __int_as_float(0xff800000);
-#pragma unroll
-                for (int g = 0; g < P; ++g) sh = fmaxf(sh, s_part[g][slot]);
-                B = (s_nv[slot] == 0) ? a.bmax : ladder(__fmul_rn(r, sh), a.cV, a.bmin, a.bmax);
+                B = (nv_tok == 0) ? a.bmax : ladder(__fmul_rn(r, shat), a.cV, a.bmin, a.bmax);
             }
         }
         Bx[x] = valid ? B : 0;
-        if (valid && p == 0) {
-            s_len[x][slot] = (uint32_t)(D * B / 8);
-            s_cnt[x][slot] = cntx[x];
-            if (SELECT_ONLY) (x ? a.out_bitsV : a.out_bitsK)[(size_t)bh * a.n_new + tn] = (uint8_t)B;
+        if (p == 0) {                                   // every slot of the tile is written: empty ones count nothing
+            s_len[x][slot] = valid ? (uint32_t)(D * B / 8) : 0u;
+            s_cnt[x][slot] = valid ? cntx[x] : 0u;
+            if (SELECT_ONLY && valid) (x ? a.out_bitsV : a.out_bitsK)[(size_t)bh * a.n_new + tn] = (uint8_t)B;
         }
     }
     if (SELECT_ONLY) return;
