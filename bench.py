@@ -160,6 +160,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch the timed steps on the stream instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -233,13 +234,31 @@ def main():
     for _ in range(args.warmup):
         step()
     barrier()
-    timers = {"thr": ([], []), "quant": ([], []), "dec": ([], [])}
+    # the launches of one step (32 layers x reset + 6 kernels) are captured once into a CUDA graph and replayed
+    run_step, launch_mode = step, "stream"
+    if not args.no_graph:
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            graph.replay()
+            torch.cuda.synchronize()
+            run_step, launch_mode = graph.replay, "cuda graph"
+        except Exception as exc:      # capture refused: plain stream launches
+            sys.stderr.write(f"bench: graph capture failed ({exc}); launching on the stream\n")
+            torch.cuda.synchronize()
+    barrier()
     e0 = ev()
     for _ in range(args.steps):
-        step(timers)
+        run_step()
     e1 = ev()
     barrier()
     clocks = sampler.stop()
+    # per-stage times from a separate pass with an event pair around every stage (kept out of the timed steps)
+    timers = {"thr": ([], []), "quant": ([], []), "dec": ([], [])}
+    for _ in range(min(args.steps, 3)):
+        step(timers)
+    torch.cuda.synchronize()
     ms_total, _ = qdist.aggregate(e0.elapsed_time(e1), 1.0, dev)     # slowest rank
     ms_step = ms_total / args.steps
     stage_ms = {k: sum(a.elapsed_time(b) for a, b in zip(*v)) / len(v[0]) for k, v in timers.items()}
@@ -263,7 +282,7 @@ def main():
                                                                      round(st.code_bytes[1] * 8 / (BH * T * D), 3)],
                    "cr_paper": round(st.cr_paper, 3), "cr_total": round(st.cr_total, 3),
                    "l2": "each layer's inputs (>0.5 GB) and packed cache exceed L2; no flush needed",
-                   "per_rank": "own batch, no collective"},
+                   "per_rank": "own batch, no collective", "launch": launch_mode},
         "stages": {
             "thresholds": {"ms_per_layer": round(stage_ms["thr"], 4), "gbs": round(thr_gbs, 1), "frac_of_hbm": round(thr_gbs / peak, 3)},
             "quantize": {"ms_per_layer": round(stage_ms["quant"], 4), "gbs": round(quant_gbs, 1), "frac_of_hbm": round(quant_gbs / peak, 3),
