@@ -182,6 +182,27 @@ qaq_status qaq_requantize_down(qaq_cache* c, const uint8_t* bitsK, const uint8_t
                                long n_cols, void* stream);
 
 /*
+ * Re-quantization in both directions (Section 4.2, "Integration in text generation process":
+ * tokens whose new width is lower are quantized further; "for those otherwise, we take the
+ * unquantized KV cache from CPU memory and re-quantize it to the required bits").
+ * K_full, V_full: the unquantized binary16 values of the cached tokens, [batch][heads][>=tokens]
+ * [head_dim] with element strides as in qaq_outlier_thresholds, in any memory the GPU can read:
+ * device memory, or pinned host memory that is mapped into the device's address space (then only
+ * the rows of the raised tokens cross the bus).  Pageable host memory is refused.  Both NULL:
+ * exactly qaq_requantize_down.  thr: the thresholds the tokens were appended with.
+ * New widths as in qaq_requantize_down (given, clamped to 1..8, or by the rules), but taken as
+ * they are: a raised token keeps its min, max and outliers and gets the codes an append at the
+ * new width would have produced, so after the call the cache equals one filled at the new widths.
+ * A closed tile that grows is moved to the end of its (b,h) pool and its old bytes stay unused
+ * until qaq_cache_reset; if the pool has no room left the tile is left as it was and
+ * qaq_cache_stats().device_status reports QAQ_ERR_CAPACITY.
+ */
+qaq_status qaq_requantize(qaq_cache* c, const void* K_full, const void* V_full, long stride_b, long stride_h,
+                          long stride_t, const float* thr, const uint8_t* bitsK, const uint8_t* bitsV,
+                          const qaq_policy* policy, const float* score_ring, const uint8_t* nvalid, long n_cols,
+                          void* stream);
+
+/*
  * S4+S5: decode attention over the packed cache (Section 2.1, Figure 1):
  *   S = Softmax(softmax_scale * q Khat^T),  X = S Vhat,
  * Khat/Vhat = midpoint reconstruction min + (code + 1/2) * step with the stored outliers

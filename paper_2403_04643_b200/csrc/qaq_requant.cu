@@ -1,18 +1,24 @@
-// Further quantization of cached tokens to lower widths (Section 4.2 of the paper,
-// "Integration in text generation process"): in every generation step the widths of all
-// cached tokens are computed again; a token whose new width is lower than its current one is
-// quantized further.  The quantizer is nested (min and range kept, the B'-bit code is the
-// B-bit code without its low B-B' bits), so this needs nothing but the packed cache itself:
-//   range = max - min from the token's metadata  ->  new width by the rules of Section 4.1
-//   code >>= (B - B'),  planes rebuilt for B',  the tile rewritten in place (it only shrinks).
-// Widths are never raised here (that needs the unquantized copy the paper keeps in CPU memory).
+// Re-quantization of cached tokens (Section 4.2 of the paper, "Integration in text generation
+// process"): in every generation step the widths of all cached tokens are computed again.
+//   lower width:  the token is quantized further.  The quantizer is nested (min and range kept,
+//                 the B'-bit code is the B-bit code without its low B-B' bits), so this needs
+//                 nothing but the packed cache:  code >>= (B - B').
+//   higher width: the paper takes the unquantized values from a copy kept in CPU memory and
+//                 quantizes them again.  Here the caller passes that copy (any memory the GPU can
+//                 read, e.g. mapped pinned host memory: only the rows of the raised tokens are
+//                 touched); min, max and the outliers of the token stay what they were, the codes
+//                 are computed as at append time.  Without a copy, widths are only lowered.
+// The new widths come from the caller or from the rules of Section 4.1 applied to the stored
+// range (max - min of the token's metadata) with the current score window and policy scalars.
 //
 // One CTA = one tile (QAQ_TILE tokens) of one (b,h), both tensors; head_dim/32 lanes own a
 // token, each lane the codes of 32 consecutive channels, one byte per code in 8 registers.
 // All of a tile's old bytes are in registers before the first new byte is written (the new
-// planes are built in a shared-memory image of the tile first), so rewriting in place is safe.
-// Pool space freed inside closed tiles is not handed back; an open (last, partly filled) tile
-// gives its bytes back to the pool so that later appends continue right behind it.
+// planes are built in a shared-memory image of the tile first), so a tile that does not grow is
+// rewritten in place.  A closed tile that grows takes a new place at the end of its pool (the
+// old bytes stay unused); the open (last, partly filled) tile is handled in a launch of its own
+// after the closed ones and is kept - or made again - the last thing in its pool, so that later
+// appends continue right behind it.
 #include "qaq_internal.cuh"
 
 namespace {
@@ -30,6 +36,13 @@ struct RequantArgs {
     int W;
     float cK, cV;
     int bmin, bmax;
+    // raising widths: the unquantized values [B,H,T,D] (element strides), the thresholds, the tile to start at
+    const __half* Ks;
+    const __half* Vs;
+    long sb, sh, st;
+    const float* thr;        // [BH][4]
+    int first_tile;
+    int* status;
 };
 
 // B = min{b in [bmin,bmax] : v <= c * 2^b}, bmax if none (c * 2^b is an exact scaling)
@@ -138,12 +151,53 @@ __device__ __forceinline__ void write_planes(uint8_t* tok, int B, int p, const u
     }
 }
 
-template <int D>
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+// binary32 (x - c) with x a binary16 value: one rounding
+__device__ __forceinline__ float sub_f32_f16(unsigned short x, float c) {
+    float d;
+    asm("sub.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
+    return d;
+}
+// Codes of one lane's 32 channels computed from the unquantized row, as at append time:
+// code = min(2^B - 1, floor((x - min) * (1/step))) in binary32, 0 for an outlier (outside [lo, hi]).
+__device__ __forceinline__ void fresh_codes(const __half* row, float lo, float hi, float mn, float mx, int B, uint32_t (&creg)[8]) {
+    const __half2 lo2 = __half2half2(__float2half_ru(lo)), hi2 = __half2half2(__float2half_rd(hi));
+    const float step = __fmul_rn(__fsub_rn(mx, mn), __int_as_float((127 - B) << 23));
+    const float inv = step > 0.f ? __fdiv_rn(1.0f, step) : 0.f;
+    const float topf = step > 0.f ? (float)((1 << B) - 1) : 0.f;
+#pragma unroll
+    for (int q4 = 0; q4 < 4; ++q4) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(row + 8 * q4);
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        uint32_t f[8];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const __half2 x = *reinterpret_cast<const __half2*>(&w[k]);
+            const uint32_t m = __hge2_mask(x, lo2) & __hle2_mask(x, hi2);       // all-ones halves: inside [lo, hi]
+            const uint32_t v = (w[k] & m) | (0xFC00FC00u & ~m);                    // outliers become -inf: code 0
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const unsigned short h = e ? (unsigned short)(v >> 16) : (unsigned short)(v & 0xFFFF);
+                float t = __fmul_rn(sub_f32_f16(h, mn), inv);
+                t = fminf(t, topf);
+                f[2 * k + e] = __float_as_uint(__fadd_rd(t, 8388608.0f));          // 2^23 + floor(t): the code is the low byte
+            }
+        }
+        creg[2 * q4] = prmt(prmt(f[0], f[1], 0x0040u), prmt(f[2], f[3], 0x0040u), 0x5410u);
+        creg[2 * q4 + 1] = prmt(prmt(f[4], f[5], 0x0040u), prmt(f[6], f[7], 0x0040u), 0x5410u);
+    }
+}
+
+template <int D, bool UP>
 __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
     constexpr int P = D / 32;
     constexpr int ALIGN = D / 8 >= 16 ? 16 : D / 8;
     constexpr int NT = 2 * D;
-    const int tile = blockIdx.x, bh = blockIdx.y;
+    const int tile = a.first_tile + blockIdx.x, bh = blockIdx.y;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slot = tid / P, p = tid % P;
     const int tok = tile * QAQ_TILE + slot;
@@ -153,7 +207,8 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
     __shared__ float s_part[P][QAQ_TILE];
     __shared__ uint8_t s_nv[QAQ_TILE];
     __shared__ uint32_t s_old[2][QAQ_TILE], s_new[2][QAQ_TILE];   // byte lengths, then exclusive offsets in the tile
-    __shared__ uint32_t s_tot[2];                                  // new bytes of the tile
+    __shared__ uint32_t s_tot[2], s_off[2];                        // new bytes of the tile, where they go in the pool
+    __shared__ int s_skip[2];
     __shared__ __align__(16) uint8_t s_img[2][QAQ_TILE * D];
 
     // ---- attention window of the tile's tokens (value rule); P threads share a token's rows
@@ -174,21 +229,21 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
     // ---- current widths and ranges
     const size_t mt = (size_t)bh * a.tmax_pad + tok;
     int Bo[2] = {0, 0};
-    float rng[2] = {0.f, 0.f};
+    float rng[2] = {0.f, 0.f}, mnf[2] = {0.f, 0.f}, mxf[2] = {0.f, 0.f};
     if (valid) {
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
             const TensorStore& ts = x ? a.v : a.k;
             Bo[x] = ts.bits[mt];
             const uint32_t mm = ts.mnmx[mt];
-            const float mn = __half2float(__ushort_as_half((unsigned short)(mm & 0xFFFF)));
-            const float mx = __half2float(__ushort_as_half((unsigned short)(mm >> 16)));
-            rng[x] = __fsub_rn(mx, mn);
+            mnf[x] = __half2float(__ushort_as_half((unsigned short)(mm & 0xFFFF)));
+            mxf[x] = __half2float(__ushort_as_half((unsigned short)(mm >> 16)));
+            rng[x] = __fsub_rn(mxf[x], mnf[x]);
         }
     }
     __syncthreads();   // window partials visible
 
-    // ---- new widths: the rule's (or the caller's) width where it is lower, else the current one
+    // ---- new widths: the rule's (or the caller's) width; without the unquantized copy only where it is lower
     int Bn[2];
     bool changed[2];
 #pragma unroll
@@ -197,7 +252,7 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
         if (valid) {
             if (given) {
                 B = (x ? a.bitsV : a.bitsK)[(size_t)bh * a.ncols + tok];
-                B = B < 1 ? 1 : B;
+                B = B < 1 ? 1 : (B > 8 ? 8 : B);
             } else if (x == 0) {
                 B = ladder(rng[0], a.cK, a.bmin, a.bmax);
             } else {
@@ -207,12 +262,24 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
                 B = (s_nv[slot] == 0) ? a.bmax : ladder(__fmul_rn(rng[1], sh), a.cV, a.bmin, a.bmax);
             }
         }
-        Bn[x] = B < Bo[x] ? B : Bo[x];
+        Bn[x] = !valid ? 0 : ((UP || B < Bo[x]) ? B : Bo[x]);
         if (p == 0) {
             s_old[x][slot] = (uint32_t)(D * Bo[x] / 8);
             s_new[x][slot] = (uint32_t)(D * Bn[x] / 8);
         }
         changed[x] = __syncthreads_or(Bn[x] != Bo[x]) != 0;   // also makes the lengths visible
+    }
+    // An open tile has to be the last thing in its pool.  If closed tiles of this (b,h) have just been moved
+    // behind it, it moves to the end as well, whether its own tokens change or not.
+    bool relocate[2] = {false, false};
+    if (UP && tile == a.T / QAQ_TILE && (a.T % QAQ_TILE) != 0) {
+        const size_t ti0 = (size_t)bh * a.ntiles + tile;
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            const TensorStore& ts = x ? a.v : a.k;
+            relocate[x] = ts.tile_off[ti0] + ts.tile_nbytes[ti0] != ts.pool_end[bh];
+            changed[x] = changed[x] || relocate[x];
+        }
     }
     if (!changed[0] && !changed[1]) return;
 
@@ -232,10 +299,36 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
             const uint32_t tn1 = __shfl_sync(0xFFFFFFFFu, in1, 31);
             s_old[x][lane] = io0 - o0; s_old[x][lane + 32] = to0 + io1 - o1;
             s_new[x][lane] = in0 - n0; s_new[x][lane + 32] = tn0 + in1 - n1;
-            if (lane == 0) s_tot[x] = tn0 + tn1;
+            if (lane == 0) {
+                // where the new tile goes: in place unless it grows
+                const TensorStore& ts = x ? a.v : a.k;
+                const size_t ti0 = (size_t)bh * a.ntiles + tile;
+                const uint32_t nb = tn0 + tn1, off = ts.tile_off[ti0], old_nb = ts.tile_nbytes[ti0];
+                uint32_t noff = off;
+                int skip = 0;
+                if (UP && changed[x] && (nb > old_nb || relocate[x])) {
+                    const bool open = tile == a.T / QAQ_TILE && (a.T % QAQ_TILE) != 0;
+                    if (open && off + old_nb == ts.pool_end[bh]) {
+                        // still the last thing in its pool: it grows where it is
+                        if ((size_t)off + nb + 16 > a.pool_bytes) skip = 1;
+                        else ts.pool_end[bh] = off + nb;
+                    } else {
+                        // closed tiles take a rounded amount; an open tile the exact one, which makes it the last again
+                        const uint32_t take = open ? nb : ((nb + 15u) & ~15u);
+                        noff = atomicAdd(&ts.pool_end[bh], take);
+                        if ((size_t)noff + take + 16 > a.pool_bytes) skip = 1;
+                    }
+                    if (skip) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
+                }
+                s_tot[x] = nb; s_off[x] = noff; s_skip[x] = skip;
+            }
         }
     }
     __syncthreads();
+    if (UP) {   // no room in the pool: that tensor's tile stays as it is
+        if (s_skip[0]) changed[0] = false;
+        if (s_skip[1]) changed[1] = false;
+    }
 
     // ---- old planes -> codes -> low bits dropped -> new planes in the shared-memory image
     const size_t ti = (size_t)bh * a.ntiles + tile;
@@ -245,12 +338,19 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
         const TensorStore& ts = x ? a.v : a.k;
         uint32_t creg[8];
         if (valid) {
-            const uint8_t* src = ts.codes + (size_t)bh * a.pool_bytes + ts.tile_off[ti] + s_old[x][slot];
-            read_planes<D, ALIGN>(src, Bo[x], p, creg);
-            const int drop = Bo[x] - Bn[x];
-            const uint32_t keep = 0x01010101u * (0xFFu >> drop);
+            if (UP && Bn[x] > Bo[x]) {
+                // raised: codes from the unquantized row, with the token's stored min / max and the thresholds
+                const __half* row = (x ? a.Vs : a.Ks) + (size_t)(bh / a.H) * a.sb + (size_t)(bh % a.H) * a.sh +
+                                    (size_t)tok * a.st + 32 * p;
+                fresh_codes(row, a.thr[(size_t)bh * 4 + 2 * x], a.thr[(size_t)bh * 4 + 2 * x + 1], mnf[x], mxf[x], Bn[x], creg);
+            } else {
+                const uint8_t* src = ts.codes + (size_t)bh * a.pool_bytes + ts.tile_off[ti] + s_old[x][slot];
+                read_planes<D, ALIGN>(src, Bo[x], p, creg);
+                const int drop = Bo[x] - Bn[x];
+                const uint32_t keep = 0x01010101u * (0xFFu >> drop);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) creg[j] = (creg[j] >> drop) & keep;
+                for (int j = 0; j < 8; ++j) creg[j] = (creg[j] >> drop) & keep;
+            }
             write_planes<D, ALIGN>(s_img[x] + s_new[x][slot], Bn[x], p, creg);
         }
     }
@@ -261,7 +361,7 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
     for (int x = 0; x < 2; ++x) {
         if (!changed[x]) continue;
         const TensorStore& ts = x ? a.v : a.k;
-        const uint32_t off = ts.tile_off[ti];
+        const uint32_t off = s_off[x];
         uint8_t* dst = ts.codes + (size_t)bh * a.pool_bytes + off;
         const uint32_t nb = s_tot[x];
         for (uint32_t o = tid * ALIGN; o < nb; o += NT * ALIGN) {
@@ -271,21 +371,49 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
         }
         if (valid && p == 0) ts.bits[mt] = (uint8_t)Bn[x];
         if (tid == 0) {
+            // an open tile that is still the last thing in its pool gives back what it no longer needs:
+            // appends continue right behind its bytes
+            const uint32_t old_off = ts.tile_off[ti], old_nb = ts.tile_nbytes[ti];
+            if (tile == a.T / QAQ_TILE && (a.T % QAQ_TILE) != 0 && off == old_off && nb < old_nb &&
+                old_off + old_nb == ts.pool_end[bh])
+                ts.pool_end[bh] = off + nb;
+            ts.tile_off[ti] = off;
             ts.tile_nbytes[ti] = nb;
-            // an open tile is the last thing in its pool: appends continue right behind its bytes
-            if (tile == a.T / QAQ_TILE && (a.T % QAQ_TILE) != 0) ts.pool_end[bh] = off + nb;
         }
     }
 }
 
+template <bool UP>
+qaq_status launch_requant(int D, dim3 grid, const RequantArgs& a, cudaStream_t s) {
+    switch (D) {
+        case 32: requant_kernel<32, UP><<<grid, 64, 0, s>>>(a); break;
+        case 64: requant_kernel<64, UP><<<grid, 128, 0, s>>>(a); break;
+        case 128: requant_kernel<128, UP><<<grid, 256, 0, s>>>(a); break;
+        default: return QAQ_ERR_UNSUPPORTED_SHAPE;
+    }
+    QAQ_CUDA_TRY(cudaGetLastError());
+    return QAQ_OK;
+}
+
+// a pointer the GPU can read: device memory, managed memory or mapped (pinned) host memory
+const void* device_view(const void* p) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    if (at.type == cudaMemoryTypeUnregistered) return nullptr;   // pageable host memory
+    return at.devicePointer;
+}
+
 }  // namespace
 
-extern "C" qaq_status qaq_requantize_down(qaq_cache* c, const uint8_t* bitsK, const uint8_t* bitsV,
-                                          const qaq_policy* policy, const float* score_ring, const uint8_t* nvalid,
-                                          long n_cols, void* stream) {
+extern "C" qaq_status qaq_requantize(qaq_cache* c, const void* K_full, const void* V_full, long stride_b, long stride_h,
+                                     long stride_t, const float* thr, const uint8_t* bitsK, const uint8_t* bitsV,
+                                     const qaq_policy* policy, const float* score_ring, const uint8_t* nvalid,
+                                     long n_cols, void* stream) {
     if (!c) return QAQ_ERR_INVALID_ARG;
     if ((bitsK == nullptr) != (bitsV == nullptr)) return QAQ_ERR_INVALID_ARG;
     if (!bitsK && (!policy || !score_ring || !nvalid)) return QAQ_ERR_INVALID_ARG;
+    if ((K_full == nullptr) != (V_full == nullptr)) return QAQ_ERR_INVALID_ARG;
+    const bool up = K_full != nullptr;
     if (c->tokens == 0) return QAQ_OK;
     if (n_cols < c->tokens) return QAQ_ERR_INVALID_ARG;
     RequantArgs a{};
@@ -294,14 +422,36 @@ extern "C" qaq_status qaq_requantize_down(qaq_cache* c, const uint8_t* bitsK, co
     a.bitsK = bitsK; a.bitsV = bitsV; a.ring = score_ring; a.nvalid = nvalid; a.W = c->cfg.window;
     a.cK = policy ? policy->cK : 0.f; a.cV = policy ? policy->cV : 0.f;
     a.bmin = c->cfg.bits_min; a.bmax = c->cfg.bits_max;
-    const dim3 grid((unsigned)((c->tokens + QAQ_TILE - 1) / QAQ_TILE), (unsigned)c->BH);
+    a.status = c->d_status;
     cudaStream_t s = (cudaStream_t)stream;
-    switch (c->cfg.head_dim) {
-        case 32: requant_kernel<32><<<grid, 64, 0, s>>>(a); break;
-        case 64: requant_kernel<64><<<grid, 128, 0, s>>>(a); break;
-        case 128: requant_kernel<128><<<grid, 256, 0, s>>>(a); break;
-        default: return QAQ_ERR_UNSUPPORTED_SHAPE;
+    const int D = c->cfg.head_dim;
+    const int ntile = (int)((c->tokens + QAQ_TILE - 1) / QAQ_TILE);
+    if (!up) {
+        a.first_tile = 0;
+        return launch_requant<false>(D, dim3((unsigned)ntile, (unsigned)c->BH), a, s);
     }
-    QAQ_CUDA_TRY(cudaGetLastError());
-    return QAQ_OK;
+    if (!thr) return QAQ_ERR_INVALID_ARG;
+    if (stride_t < D || (stride_b & 7) || (stride_h & 7) || (stride_t & 7) || stride_b < 0 || stride_h < 0) return QAQ_ERR_INVALID_ARG;
+    a.Ks = (const __half*)device_view(K_full); a.Vs = (const __half*)device_view(V_full);
+    if (!a.Ks || !a.Vs || ((uintptr_t)a.Ks & 15) || ((uintptr_t)a.Vs & 15)) return QAQ_ERR_INVALID_ARG;
+    a.sb = stride_b; a.sh = stride_h; a.st = stride_t; a.thr = thr;
+    // closed tiles first (a tile that grows moves to the end of its pool), then the open tile, which has to be
+    // the last thing in its pool when this call is over
+    const int closed = (int)(c->tokens / QAQ_TILE);
+    qaq_status st = QAQ_OK;
+    if (closed > 0) {
+        a.first_tile = 0;
+        if ((st = launch_requant<true>(D, dim3((unsigned)closed, (unsigned)c->BH), a, s)) != QAQ_OK) return st;
+    }
+    if (closed < ntile) {
+        a.first_tile = closed;
+        st = launch_requant<true>(D, dim3(1, (unsigned)c->BH), a, s);
+    }
+    return st;
+}
+
+extern "C" qaq_status qaq_requantize_down(qaq_cache* c, const uint8_t* bitsK, const uint8_t* bitsV,
+                                          const qaq_policy* policy, const float* score_ring, const uint8_t* nvalid,
+                                          long n_cols, void* stream) {
+    return qaq_requantize(c, nullptr, nullptr, 0, 0, 0, nullptr, bitsK, bitsV, policy, score_ring, nvalid, n_cols, stream);
 }

@@ -22,7 +22,7 @@ EXPORTED = [
     "qaq_policy_from_hyper", "qaq_thresholds_workspace_bytes", "qaq_outlier_thresholds", "qaq_select_bits",
     "qaq_quantize_append", "qaq_decode_workspace_bytes", "qaq_decode_attention", "qaq_quantize_append_host",
     "qaq_decode_attention_host", "qaq_cache_stats", "qaq_cache_export", "qaq_decode_attention_static",
-    "qaq_requantize_down", "qaq_prefill_window_workspace_bytes", "qaq_prefill_window",
+    "qaq_requantize_down", "qaq_requantize", "qaq_prefill_window_workspace_bytes", "qaq_prefill_window",
 ]
 
 
@@ -84,6 +84,8 @@ def lib():
         L.qaq_prefill_window_workspace_bytes.argtypes = [C.POINTER(Config), C.c_int, C.POINTER(C.c_size_t)]
         L.qaq_prefill_window.argtypes = [C.POINTER(Config), C.c_void_p, C.c_void_p, C.c_long, C.c_long, C.c_long, C.c_int,
                                          C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qaq_requantize.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_long, C.c_long, C.c_long, C.c_void_p, C.c_void_p,
+                                     C.c_void_p, C.POINTER(Policy), C.c_void_p, C.c_void_p, C.c_long, C.c_void_p]
         L.qaq_requantize_down.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(Policy), C.c_void_p, C.c_void_p,
                                           C.c_long, C.c_void_p]
         L.qaq_cache_export.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -225,6 +227,20 @@ def qaq_requantize_down(cache: Cache, *, bitsK=None, bitsV=None, policy=None, ri
     pol = C.byref(policy) if policy is not None else None
     _check(lib().qaq_requantize_down(cache.handle, _ptr(bitsK), _ptr(bitsV), pol, _ptr(ring), _ptr(nvalid), n_cols,
                                      _stream()), "qaq_requantize_down")
+
+
+def qaq_requantize(cache: Cache, K_full, V_full, thr, *, bitsK=None, bitsV=None, policy=None, ring=None, nvalid=None):
+    """Bring every cached token to its new width, lower or higher.  K_full/V_full: the unquantized fp16 values
+    [B,H,>=tokens,D] on the device or in pinned (mapped) host memory; the rest as in qaq_requantize_down."""
+    sb, sh, st = _strides(K_full)
+    assert _strides(V_full) == (sb, sh, st)
+    ref = bitsK if bitsK is not None else nvalid
+    n_cols = ref.shape[-1]
+    for t in (bitsK, bitsV, ring, nvalid):
+        assert t is None or (t.is_contiguous() and t.shape[-1] == n_cols)
+    pol = C.byref(policy) if policy is not None else None
+    _check(lib().qaq_requantize(cache.handle, _ptr(K_full), _ptr(V_full), sb, sh, st, _ptr(thr), _ptr(bitsK), _ptr(bitsV), pol,
+                                _ptr(ring), _ptr(nvalid), n_cols, _stream()), "qaq_requantize")
 
 
 def qaq_decode_attention(cache: Cache, q, softmax_scale, out=None, scores_out=None):

@@ -102,3 +102,107 @@ def test_argument_errors_and_empty_cache():
     assert e.value.code == 1
     with pytest.raises(qaq.QaqError):
         qaq.qaq_requantize_down(cache, nvalid=bits)                 # rules asked for, policy and window missing
+
+
+def _quantized(wl, K, V, thr_h, bits, T):
+    ku, vu = u16(K).reshape(wl.bh, -1, wl.head_dim)[:, :T], u16(V).reshape(wl.bh, -1, wl.head_dim)[:, :T]
+    qk = [oracle.quantize(ku[bh], thr_h[bh, 0], thr_h[bh, 1], bits[0, bh, :T]) for bh in range(wl.bh)]
+    qv = [oracle.quantize(vu[bh], thr_h[bh, 2], thr_h[bh, 3], bits[1, bh, :T]) for bh in range(wl.bh)]
+    return qk, qv
+
+
+@pytest.mark.parametrize("D,shadow", [(32, "device"), (64, "device"), (128, "device"), (128, "pinned")])
+def test_both_directions_leave_the_cache_as_if_filled_at_the_new_widths(D, shadow):
+    # widths go up and down at random, twice, with appends in between: tiles that grow move to the end of their
+    # pool, the open tile stays the last thing in it.  Expected: direct quantization at the final widths.
+    wl = synth.scaled(synth.CONFIGS["C1"], batch=2, heads=2, head_dim=D, tokens=300, seed=90 + D)
+    K, V, q, ring, nv = make_inputs(wl)
+    T0, T1, T2 = 150, 180, 300                            # 150 = two closed tiles + an open one of 22
+    rng = np.random.default_rng(D + 1)
+    bits = rng.integers(1, 9, (2, wl.bh, T2)).astype(np.uint8)
+    # token capacity three times what is appended: tiles that grow leave their old bytes unused in the pool
+    cfg = qaq.make_config(wl.batch, wl.heads, D, 3 * T2, wl.bits_min, wl.bits_max, wl.window, wl.alpha)
+    Kd, Vd = K.cuda(), V.cuda()
+    Ks, Vs = (Kd, Vd) if shadow == "device" else (K.pin_memory(), V.pin_memory())
+    thr = qaq.qaq_outlier_thresholds(cfg, Kd, Vd)
+    thr_h = thr.cpu().numpy()
+    cache = qaq.Cache(cfg)
+    tb = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    scale = 1.0 / math.sqrt(D)
+
+    def append(lo, hi):
+        qaq.qaq_quantize_append(cache, Kd[:, :, lo:hi], Vd[:, :, lo:hi], thr, bitsK=tb(bits[0][:, lo:hi]), bitsV=tb(bits[1][:, lo:hi]))
+
+    def requantize(T):
+        new = rng.integers(1, 9, (2, wl.bh, T)).astype(np.uint8)
+        try:
+            qaq.qaq_requantize(cache, Ks, Vs, thr, bitsK=tb(new[0]), bitsV=tb(new[1]))
+        except qaq.QaqError as e:
+            if shadow == "pinned" and e.code == 1:
+                pytest.skip("pinned host memory is not mapped into the device's address space here")
+            raise
+        bits[:, :, :T] = new
+
+    def check(T):
+        qk, qv = _quantized(wl, K, V, thr_h, bits, T)
+        compare_export(cache, SimpleNamespace(K=qk, V=qv))
+        out = qaq.qaq_decode_attention(cache, q.cuda(), scale)
+        qq = u16(q).reshape(wl.bh, D)
+        ref = np.stack([oracle.decode(qq[bh], qk[bh], qv[bh], scale)[0] for bh in range(wl.bh)])
+        assert_attention_close(out.cpu().numpy(), ref)
+        assert qaq.qaq_cache_stats(cache).device_status == 0
+
+    append(0, T0); requantize(T0); check(T0)
+    append(T0, T1); check(T1)                             # continues behind the (moved or resized) open tile
+    requantize(T1); check(T1)
+    append(T1, T2); requantize(T2); check(T2)
+
+
+def test_widths_by_the_rules_raise_and_lower():
+    wl = synth.scaled(synth.CONFIGS["C2"], heads=2, tokens=500)
+    K, V, q, ring, nv = make_inputs(wl)
+    T = K.shape[2]
+    polA = qaq.qaq_policy_from_hyper(*LOOSER, T)          # filled at low widths
+    cfg, cache, thr, out, scores, dev = gpu_pipeline(wl, K, V, q, ring, nv, polA, max_tokens=2 * T)   # room for tiles that move
+    ring2, nv2 = synth.make_score_ring(wl, 5)
+    polB = qaq.qaq_policy_from_hyper(*HYPER, T)           # tighter budgets: most widths go up
+    qaq.qaq_requantize(cache, dev[0], dev[1], thr, policy=polB, ring=ring2.cuda(), nvalid=nv2.cuda())
+    ref = oracle_batch(wl, K, V, q, ring2, nv2, *oracle.policy(*HYPER, T), thr=thr.cpu().numpy())
+    assert qaq.qaq_cache_stats(cache).device_status == 0
+    compare_export(cache, ref)                            # as if selected and quantized with the second window and policy
+    out2 = qaq.qaq_decode_attention(cache, dev[2], 1.0 / math.sqrt(wl.head_dim))
+    assert_attention_close(out2.cpu().numpy(), ref.X)
+    first = oracle_batch(wl, K, V, q, ring, nv, *oracle.policy(*LOOSER, T), thr=thr.cpu().numpy())
+    up = sum(int((a.bits > b.bits).sum()) for a, b in zip(ref.K + ref.V, first.K + first.V))
+    down = sum(int((a.bits < b.bits).sum()) for a, b in zip(ref.K + ref.V, first.K + first.V))
+    assert up > 200 and qaq.qaq_cache_stats(cache).device_status == 0, (up, down)
+
+
+def test_pageable_host_memory_is_refused():
+    wl = synth.scaled(synth.CONFIGS["C2"], heads=1, tokens=64)
+    K, V = synth.make_kv(wl)
+    cfg = qaq.make_config(1, 1, 128, 64, 2, 8, wl.window, wl.alpha)
+    cache = qaq.Cache(cfg)
+    bits = torch.full((1, 64), 4, dtype=torch.uint8, device="cuda")
+    thr = qaq.qaq_outlier_thresholds(cfg, K.cuda(), V.cuda())
+    qaq.qaq_quantize_append(cache, K.cuda(), V.cuda(), thr, bitsK=bits, bitsV=bits)
+    with pytest.raises(qaq.QaqError) as e:
+        qaq.qaq_requantize(cache, K, V, thr, bitsK=bits, bitsV=bits)    # plain CPU tensors: the GPU cannot read them
+    assert e.value.code == 1
+
+
+def test_a_full_pool_is_reported_and_every_tile_stays_consistent():
+    # token capacity exactly what is cached: tiles that grow find no room at the end of the pool sooner or later.
+    # Those tiles stay as they were; whatever width a token ends up with, its codes are the ones for that width.
+    wl = synth.scaled(synth.CONFIGS["C2"], heads=2, tokens=500)
+    K, V, q, ring, nv = make_inputs(wl)
+    T = K.shape[2]
+    cfg, cache, thr, out, scores, dev = gpu_pipeline(wl, K, V, q, ring, nv, qaq.qaq_policy_from_hyper(*LOOSER, T))
+    ring2, nv2 = synth.make_score_ring(wl, 5)
+    qaq.qaq_requantize(cache, dev[0], dev[1], thr, policy=qaq.qaq_policy_from_hyper(*HYPER, T), ring=ring2.cuda(), nvalid=nv2.cuda())
+    assert qaq.qaq_cache_stats(cache).device_status == 3
+    got = np.stack([qaq.qaq_cache_export(cache, x)["bits"].cpu().numpy() for x in range(2)])
+    qk, qv = _quantized(wl, K, V, thr.cpu().numpy(), got, T)
+    compare_export(cache, SimpleNamespace(K=qk, V=qv))
+    out2 = qaq.qaq_decode_attention(cache, dev[2], 1.0 / math.sqrt(wl.head_dim))
+    assert_attention_close(out2.cpu().numpy(), _decode_ref(wl, q, qk, qv))
