@@ -481,6 +481,25 @@ def extras(qaq, calibrate, dev, peak, qn):
                 "frac_of_hbm": round(moved / us_r / 1e3 / peak, 3),
                 "repeat_nothing_to_lower_us": round(ev[1].elapsed_time(ev[2]) * 1e3, 1),
                 "decode_after_us": round(_time_us(lambda: qaq.qaq_decode_attention(cache, q, scale, out=outb), 20), 1)}
+            # and back up to (4, 3) from the unquantized copy: in device memory, then in pinned host memory that the
+            # kernel reads through the bus (only the rows of raised tokens)
+            big = qaq.make_config(wl.batch, wl.heads, D, 2 * T, wl.bits_min, wl.bits_max, W, wl.alpha)   # room for tiles that move
+            up = {}
+            for where in ("device", "pinned_host"):
+                c2 = qaq.Cache(big)
+                qaq.qaq_quantize_append(c2, K, V, thr, policy=pol, ring=ring, nvalid=nv)
+                Ks, Vs = (K, V) if where == "device" else (K.cpu().pin_memory(), V.cpu().pin_memory())
+                torch.cuda.synchronize()
+                e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+                e[0].record()
+                qaq.qaq_requantize(c2, Ks, Vs, thr, policy=pol43, ring=ring, nvalid=nv)
+                e[1].record(); torch.cuda.synchronize()
+                stu = qaq.qaq_cache_stats(c2)
+                up[where + "_us"] = round(e[0].elapsed_time(e[1]) * 1e3, 1)
+                up["to_mean_bits"] = [round(stu.code_bytes[x] * 8 / (BH * T * D), 2) for x in range(2)]
+                up["device_status"] = int(stu.device_status)
+                del c2, Ks, Vs
+            res["C3_layer_requantize_up"] = up
         del cache, K, V, ring
         torch.cuda.empty_cache()
     return res
