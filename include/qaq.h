@@ -75,6 +75,10 @@ qaq_status qaq_cache_reset(qaq_cache* c, void* stream);
 /* Tokens currently cached per (b,h) (host counter). */
 long qaq_cache_tokens(const qaq_cache* c);
 
+/* Name of the CUDA error behind the most recent QAQ_ERR_CUDA returned in this process
+ * ("cudaSuccess" if there was none).  Host function. */
+const char* qaq_last_cuda_error(void);
+
 /*
  * Bit-width rule scalars from the paper's hyper-parameters (Section 4.1):
  *   key bound    sigma2(K_t) <= log(T^3/(T-1) * sigmaS_max^2 + 1) / qnorm2
@@ -274,6 +278,19 @@ qaq_status qaq_cache_stats(const qaq_cache* c, qaq_stats* host_out, void* stream
 qaq_status qaq_cache_export(const qaq_cache* c, int tensor, uint8_t* bits, float* mn, float* step,
                             uint32_t* off, uint8_t* codes, long codes_stride, uint32_t* rowptr,
                             uint8_t* ch, void* val, long outl_stride, void* stream);
+
+/*
+ * Housekeeping for caches whose widths are raised (no counterpart in the paper, which keeps its
+ * cache in framework tensors).  qaq_requantize places a tile that grows at the end of its (b,h)
+ * pool and leaves the old bytes unused; qaq_cache_compact moves the tiles of every pool down
+ * until they are contiguous again (order in memory kept, open tile last), so that the space can
+ * be appended to.  Contents, widths and outlier lists are unchanged; only tile offsets move.
+ * At most 4096 tiles (262144 tokens) per (b,h), else QAQ_ERR_UNSUPPORTED_SHAPE.  Asynchronous
+ * on stream.  qaq_cache_pool_use reports the largest pool fill over all (b,h), in bytes, for
+ * K (host_used[0]) and V (host_used[1]), and the pool capacity per (b,h); it synchronises stream.
+ */
+qaq_status qaq_cache_compact(qaq_cache* c, void* stream);
+qaq_status qaq_cache_pool_use(const qaq_cache* c, long* host_used, long* host_capacity, void* stream);
 
 #ifdef __cplusplus
 }

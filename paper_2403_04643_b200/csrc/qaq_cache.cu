@@ -128,6 +128,10 @@ extern "C" qaq_status qaq_cache_reset(qaq_cache* c, void* stream) {
     return QAQ_OK;
 }
 
+int g_qaq_last_cuda_error = 0;
+
+extern "C" const char* qaq_last_cuda_error(void) { return cudaGetErrorName((cudaError_t)g_qaq_last_cuda_error); }
+
 extern "C" long qaq_cache_tokens(const qaq_cache* c) { return c ? c->tokens : -1; }
 
 extern "C" qaq_status qaq_policy_from_hyper(double sigmaS_max, double sigmaX_max, double qnorm2, long T,

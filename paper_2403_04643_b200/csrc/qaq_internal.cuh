@@ -45,10 +45,13 @@ struct qaq_cache {
     size_t stage_bytes[8];
 };
 
+// the CUDA error behind the most recent QAQ_ERR_CUDA of this process (qaq_last_cuda_error)
+extern int g_qaq_last_cuda_error;
+
 #define QAQ_CUDA_TRY(expr)                                  \
     do {                                                    \
         cudaError_t _e = (expr);                            \
-        if (_e != cudaSuccess) { (void)cudaGetLastError(); return QAQ_ERR_CUDA; } \
+        if (_e != cudaSuccess) { g_qaq_last_cuda_error = (int)_e; (void)cudaGetLastError(); return QAQ_ERR_CUDA; } \
     } while (0)
 
 static inline bool qaq_dim_ok(int D) { return D == 32 || D == 64 || D == 128; }

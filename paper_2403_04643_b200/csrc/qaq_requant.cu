@@ -312,10 +312,16 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
                         // still the last thing in its pool: it grows where it is
                         if ((size_t)off + nb + 16 > a.pool_bytes) skip = 1;
                         else ts.pool_end[bh] = off + nb;
+                    } else if (open) {
+                        // behind everything else, 16-byte aligned, and exactly as long as its bytes: the last thing
+                        // in the pool again (this launch has one CTA per (b,h), nobody else touches the pool)
+                        noff = (ts.pool_end[bh] + 15u) & ~15u;
+                        if ((size_t)noff + nb + 16 > a.pool_bytes) skip = 1;
+                        else ts.pool_end[bh] = noff + nb;
                     } else {
-                        // closed tiles take a rounded amount; an open tile the exact one, which makes it the last again
-                        const uint32_t take = open ? nb : ((nb + 15u) & ~15u);
-                        noff = atomicAdd(&ts.pool_end[bh], take);
+                        // the end of the pool need not be aligned while a tile is open: take 16 bytes more and align
+                        const uint32_t take = ((nb + 15u) & ~15u) + 16u;
+                        noff = (atomicAdd(&ts.pool_end[bh], take) + 15u) & ~15u;
                         if ((size_t)noff + take + 16 > a.pool_bytes) skip = 1;
                     }
                     if (skip) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
@@ -454,4 +460,106 @@ extern "C" qaq_status qaq_requantize_down(qaq_cache* c, const uint8_t* bitsK, co
                                           const qaq_policy* policy, const float* score_ring, const uint8_t* nvalid,
                                           long n_cols, void* stream) {
     return qaq_requantize(c, nullptr, nullptr, 0, 0, 0, nullptr, bitsK, bitsV, policy, score_ring, nvalid, n_cols, stream);
+}
+
+// ---------------------------------------------------------------------------------------
+// Compaction of the code pools.  Tiles that grew in qaq_requantize were placed anew at the end
+// of their pool and left their old bytes behind; this closes the gaps again: the tiles of a
+// (b,h) pool are moved down, in the order in which they lie in memory, until they are
+// contiguous (16-byte aligned each), the open tile last.  One CTA per (b,h) and tensor works
+// through its tiles one after the other; a tile is copied forward in 4 KB pieces, every piece
+// read completely before it is written, so that overlapping source and destination are safe.
+namespace {
+
+constexpr int COMPACT_MAX_TILES = 4096;
+
+struct CompactArgs {
+    TensorStore t[2];
+    size_t pool_bytes;
+    int ntiles, T;
+};
+
+__global__ void __launch_bounds__(256) compact_kernel(const CompactArgs a) {
+    const int bh = blockIdx.x;
+    const TensorStore& ts = a.t[blockIdx.y];
+    __shared__ unsigned long long s_key[COMPACT_MAX_TILES];   // current offset << 32 | tile index
+    const int nt = (a.T + QAQ_TILE - 1) / QAQ_TILE;
+    int n2 = 1;
+    while (n2 < nt) n2 <<= 1;
+    const size_t row = (size_t)bh * a.ntiles;
+    for (int i = threadIdx.x; i < n2; i += blockDim.x)
+        s_key[i] = i < nt ? ((unsigned long long)ts.tile_off[row + i] << 32) | (unsigned)i : ~0ull;
+    __syncthreads();
+    // bitonic sort by current offset
+    for (int k = 2; k <= n2; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = threadIdx.x; i < n2; i += blockDim.x) {
+                const int l = i ^ j;
+                if (l > i) {
+                    const unsigned long long x = s_key[i], y = s_key[l];
+                    const bool up = (i & k) == 0;
+                    if ((x > y) == up) { s_key[i] = y; s_key[l] = x; }
+                }
+            }
+            __syncthreads();
+        }
+    uint8_t* pool = ts.codes + (size_t)bh * a.pool_bytes;
+    uint32_t dst = 0;
+    for (int s = 0; s < nt; ++s) {
+        const uint32_t src = (uint32_t)(s_key[s] >> 32);
+        const int tile = (int)(s_key[s] & 0xFFFFFFFFu);
+        const uint32_t n = ts.tile_nbytes[row + tile];
+        const uint32_t n16 = (n + 15u) & ~15u;
+        if (src != dst) {                                  // dst < src: tiles before this one only moved down
+            for (uint32_t o = 0; o < n16; o += 256 * 16) {
+                const uint32_t b = o + threadIdx.x * 16;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (b < n16) v = *reinterpret_cast<const uint4*>(pool + src + b);
+                __syncthreads();
+                if (b < n16) *reinterpret_cast<uint4*>(pool + dst + b) = v;
+            }
+            if (threadIdx.x == 0) ts.tile_off[row + tile] = dst;
+        }
+        // closed tiles own a 16-byte rounded amount; the open tile, which is the last one, its exact bytes
+        const bool open = tile == a.T / QAQ_TILE && (a.T % QAQ_TILE) != 0;
+        dst += open ? n : n16;
+        __syncthreads();                                   // the next tile's source may be this tile's old place
+    }
+    if (threadIdx.x == 0) ts.pool_end[bh] = dst;
+}
+
+__global__ void pool_use_kernel(TensorStore tk, TensorStore tv, int BH, unsigned int* out) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < BH; i += gridDim.x * blockDim.x) {
+        atomicMax(&out[0], tk.pool_end[i]);
+        atomicMax(&out[1], tv.pool_end[i]);
+    }
+}
+
+}  // namespace
+
+extern "C" qaq_status qaq_cache_compact(qaq_cache* c, void* stream) {
+    if (!c) return QAQ_ERR_INVALID_ARG;
+    if (c->tokens == 0) return QAQ_OK;
+    const long nt = (c->tokens + QAQ_TILE - 1) / QAQ_TILE;
+    if (nt > COMPACT_MAX_TILES) return QAQ_ERR_UNSUPPORTED_SHAPE;
+    CompactArgs a;
+    a.t[0] = c->t[0]; a.t[1] = c->t[1]; a.pool_bytes = c->pool_bytes; a.ntiles = c->ntiles; a.T = (int)c->tokens;
+    compact_kernel<<<dim3((unsigned)c->BH, 2), 256, 0, (cudaStream_t)stream>>>(a);
+    QAQ_CUDA_TRY(cudaGetLastError());
+    return QAQ_OK;
+}
+
+extern "C" qaq_status qaq_cache_pool_use(const qaq_cache* c, long* host_used, long* host_capacity, void* stream) {
+    if (!c || !host_used) return QAQ_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    unsigned int* d = (unsigned int*)c->d_status + 2;      // two spare words behind the status word
+    QAQ_CUDA_TRY(cudaMemsetAsync(d, 0, 8, s));
+    pool_use_kernel<<<32, 256, 0, s>>>(c->t[0], c->t[1], c->BH, d);
+    QAQ_CUDA_TRY(cudaGetLastError());
+    unsigned int h[2] = {0, 0};
+    QAQ_CUDA_TRY(cudaMemcpyAsync(h, d, 8, cudaMemcpyDeviceToHost, s));
+    QAQ_CUDA_TRY(cudaStreamSynchronize(s));
+    host_used[0] = (long)h[0]; host_used[1] = (long)h[1];
+    if (host_capacity) *host_capacity = (long)c->pool_bytes;
+    return QAQ_OK;
 }

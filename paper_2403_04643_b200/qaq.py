@@ -18,18 +18,19 @@ _lib = None
 QAQ_OK = 0
 TILE_TOKENS = 64
 EXPORTED = [
-    "qaq_status_string", "qaq_cache_create", "qaq_cache_destroy", "qaq_cache_reset", "qaq_cache_tokens",
+    "qaq_status_string", "qaq_last_cuda_error", "qaq_cache_create", "qaq_cache_destroy", "qaq_cache_reset", "qaq_cache_tokens",
     "qaq_policy_from_hyper", "qaq_thresholds_workspace_bytes", "qaq_outlier_thresholds", "qaq_select_bits",
     "qaq_quantize_append", "qaq_decode_workspace_bytes", "qaq_decode_attention", "qaq_quantize_append_host",
     "qaq_decode_attention_host", "qaq_cache_stats", "qaq_cache_export", "qaq_decode_attention_static",
-    "qaq_requantize_down", "qaq_requantize", "qaq_prefill_window_workspace_bytes", "qaq_prefill_window",
+    "qaq_requantize_down", "qaq_requantize", "qaq_cache_compact", "qaq_cache_pool_use", "qaq_prefill_window_workspace_bytes", "qaq_prefill_window",
 ]
 
 
 class QaqError(RuntimeError):
     def __init__(self, code, where):
         self.code = int(code)
-        super().__init__(f"{where}: {status_string(code)} ({int(code)})")
+        detail = f" [{lib().qaq_last_cuda_error().decode()}]" if int(code) == 4 else ""
+        super().__init__(f"{where}: {status_string(code)} ({int(code)}){detail}")
 
 
 class Config(C.Structure):
@@ -57,6 +58,8 @@ def lib():
                                "(there is no CPU or PyTorch fallback)")
         L = C.CDLL(_LIB_PATH)
         L.qaq_status_string.restype = C.c_char_p
+        L.qaq_last_cuda_error.restype = C.c_char_p
+        L.qaq_last_cuda_error.argtypes = []
         L.qaq_status_string.argtypes = [C.c_int]
         L.qaq_cache_tokens.restype = C.c_long
         L.qaq_cache_tokens.argtypes = [C.c_void_p]
@@ -84,6 +87,8 @@ def lib():
         L.qaq_prefill_window_workspace_bytes.argtypes = [C.POINTER(Config), C.c_int, C.POINTER(C.c_size_t)]
         L.qaq_prefill_window.argtypes = [C.POINTER(Config), C.c_void_p, C.c_void_p, C.c_long, C.c_long, C.c_long, C.c_int,
                                          C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qaq_cache_compact.argtypes = [C.c_void_p, C.c_void_p]
+        L.qaq_cache_pool_use.argtypes = [C.c_void_p, C.POINTER(C.c_long), C.POINTER(C.c_long), C.c_void_p]
         L.qaq_requantize.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_long, C.c_long, C.c_long, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.POINTER(Policy), C.c_void_p, C.c_void_p, C.c_long, C.c_void_p]
         L.qaq_requantize_down.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(Policy), C.c_void_p, C.c_void_p,
@@ -241,6 +246,19 @@ def qaq_requantize(cache: Cache, K_full, V_full, thr, *, bitsK=None, bitsV=None,
     pol = C.byref(policy) if policy is not None else None
     _check(lib().qaq_requantize(cache.handle, _ptr(K_full), _ptr(V_full), sb, sh, st, _ptr(thr), _ptr(bitsK), _ptr(bitsV), pol,
                                 _ptr(ring), _ptr(nvalid), n_cols, _stream()), "qaq_requantize")
+
+
+def qaq_cache_compact(cache: Cache):
+    """Close the gaps that moved tiles left in the code pools."""
+    _check(lib().qaq_cache_compact(cache.handle, _stream()), "qaq_cache_compact")
+
+
+def qaq_cache_pool_use(cache: Cache):
+    """(largest K pool fill, largest V pool fill, pool capacity), bytes per (b,h)."""
+    used = (C.c_long * 2)()
+    cap = C.c_long()
+    _check(lib().qaq_cache_pool_use(cache.handle, used, C.byref(cap), _stream()), "qaq_cache_pool_use")
+    return int(used[0]), int(used[1]), int(cap.value)
 
 
 def qaq_decode_attention(cache: Cache, q, softmax_scale, out=None, scores_out=None):

@@ -156,6 +156,16 @@ def test_both_directions_leave_the_cache_as_if_filled_at_the_new_widths(D, shado
     append(T0, T1); check(T1)                             # continues behind the (moved or resized) open tile
     requantize(T1); check(T1)
     append(T1, T2); requantize(T2); check(T2)
+    # the moves left gaps in the pools; compaction closes them without changing what the cache holds
+    before = qaq.qaq_cache_pool_use(cache)
+    qaq.qaq_cache_compact(cache)
+    after = qaq.qaq_cache_pool_use(cache)
+    check(T2)
+    assert after[0] < before[0] and after[1] < before[1] and after[2] == before[2]
+    per_bh = [max(sum((int(t.off[i + 64 if i + 64 < T2 else T2]) - int(t.off[i]) + 15) // 16 * 16 for i in range(0, T2, 64))
+                  for t in ts) for ts in _quantized(wl, K, V, thr_h, bits, T2)]
+    assert after[0] <= per_bh[0] and after[1] <= per_bh[1]          # nothing but the tiles, 16-byte aligned each
+    requantize(T2); check(T2)                                       # and the cache goes on working
 
 
 def test_widths_by_the_rules_raise_and_lower():
