@@ -216,3 +216,32 @@ def test_a_full_pool_is_reported_and_every_tile_stays_consistent():
     compare_export(cache, SimpleNamespace(K=qk, V=qv))
     out2 = qaq.qaq_decode_attention(cache, dev[2], 1.0 / math.sqrt(wl.head_dim))
     assert_attention_close(out2.cpu().numpy(), _decode_ref(wl, q, qk, qv))
+
+
+def test_compaction_of_a_pool_with_many_moved_tiles():
+    # 5000 tokens = 78 closed tiles + an open one; raising the widths moves most tiles, compaction brings the pool
+    # back to the size of its contents and later appends and decodes work on it
+    wl = synth.scaled(synth.CONFIGS["C2"], heads=2, tokens=5100)
+    K, V, q, ring, nv = make_inputs(wl)
+    T, D = 5000, wl.head_dim
+    rng = np.random.default_rng(17)
+    bits = rng.integers(1, 5, (2, wl.bh, 5100)).astype(np.uint8)
+    cfg = qaq.make_config(wl.batch, wl.heads, D, 3 * 5100, wl.bits_min, wl.bits_max, wl.window, wl.alpha)
+    Kd, Vd = K.cuda(), V.cuda()
+    thr = qaq.qaq_outlier_thresholds(cfg, Kd, Vd)
+    cache = qaq.Cache(cfg)
+    tb = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    qaq.qaq_quantize_append(cache, Kd[:, :, :T], Vd[:, :, :T], thr, bitsK=tb(bits[0][:, :T]), bitsV=tb(bits[1][:, :T]))
+    filled = qaq.qaq_cache_pool_use(cache)
+    bits[:, :, :T] = rng.integers(3, 9, (2, wl.bh, T)).astype(np.uint8)
+    qaq.qaq_requantize(cache, Kd, Vd, thr, bitsK=tb(bits[0][:, :T]), bitsV=tb(bits[1][:, :T]))
+    moved = qaq.qaq_cache_pool_use(cache)
+    qaq.qaq_cache_compact(cache)
+    packed = qaq.qaq_cache_pool_use(cache)
+    assert moved[0] > 1.5 * filled[0] and packed[0] < 0.8 * moved[0] and packed[1] < 0.8 * moved[1]
+    qaq.qaq_quantize_append(cache, Kd[:, :, T:], Vd[:, :, T:], thr, bitsK=tb(bits[0][:, T:]), bitsV=tb(bits[1][:, T:]))
+    qk, qv = _quantized(wl, K, V, thr.cpu().numpy(), bits, 5100)
+    compare_export(cache, SimpleNamespace(K=qk, V=qv))
+    out = qaq.qaq_decode_attention(cache, q.cuda(), 1.0 / math.sqrt(D))
+    assert_attention_close(out.cpu().numpy(), _decode_ref(wl, q, qk, qv))
+    assert qaq.qaq_cache_stats(cache).device_status == 0
