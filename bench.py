@@ -160,6 +160,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--extras", default="", help="run only the extra points whose name starts with this")
     ap.add_argument("--streams", type=int, default=2, help="streams the independent layers of a step are spread over")
     ap.add_argument("--no-graph", action="store_true", help="launch the timed steps on the stream instead of replaying a CUDA graph")
     args = ap.parse_args()
@@ -353,7 +354,7 @@ def main():
     # ---- the other 7B-shaped configurations, for context (rank 0, one GPU): one layer at batch 1 (launch-latency
     # regime) and the long-context cache (values of tokens beyond the prefill stay at 8 bits: no score seen yet)
     if rank == 0 and world == 1 and not args.no_extras:
-        out["extras"] = extras(qaq, calibrate, dev, peak, hyper_qn)
+        out["extras"] = extras(qaq, calibrate, dev, peak, hyper_qn, args.extras)
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(wl, (sS, sX, hyper_qn))
@@ -378,7 +379,7 @@ def _time_us(fn, reps):
     return a.elapsed_time(b) * 1e3 / reps
 
 
-def extras(qaq, calibrate, dev, peak, qn):
+def extras(qaq, calibrate, dev, peak, qn, only=""):
     res = {}
     c3 = synth.scaled(synth.CONFIGS["C3"], layers=1)
     # (name, workload, tokens, prefill, target mean widths (K, V) or None, constant width or None)
@@ -389,6 +390,8 @@ def extras(qaq, calibrate, dev, peak, qn):
               # the comparison codec of Section 5.2: one width for every token, outliers kept apart as before
               ("C3_layer_uniform4_with_outliers", c3, c3.tokens, c3.tokens, None, 4))
     for name, wl, T, prefill, targets, uniform in points:
+        if only and not name.startswith(only):
+            continue
         D, BH, W = wl.head_dim, wl.bh, wl.window
         wlx = synth.scaled(wl, tokens=T, grow_to=0)
         K, V = synth.make_kv(wlx, 0, device=dev)

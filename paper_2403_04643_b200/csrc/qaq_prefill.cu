@@ -82,6 +82,7 @@ __global__ void __launch_bounds__(PW_WARPS * 32) window_logits_kernel(const Pref
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) { rm[mt][0] = rm[mt][1] = NEG; rs[mt][0] = rs[mt][1] = 0.f; }
 
+#pragma unroll 2
         for (int step = 0; step < PW_CHUNK / PW_WARPS / 8; ++step) {
             const int t0 = t_warp + 8 * step;
             if (t0 >= a.T) break;
@@ -178,14 +179,14 @@ __global__ void __launch_bounds__(256) window_normalize_kernel(const PrefillArgs
     __syncthreads();
     const int t_lo = chunk * PW_CHUNK;
     const int nt = min(PW_CHUNK, a.T - t_lo);
-    for (int idx = threadIdx.x; idx < a.n * nt; idx += blockDim.x) {
-        const int r = idx / nt, t = t_lo + idx % nt;
-        const int i = a.n - 1 - r;
-        float* p = a.ring + ((size_t)bh * a.n + r) * a.T + t;
-        *p = (t <= a.T - a.n + i) ? __expf(*p - s_m[i]) * s_inv[i] : 0.f;
-    }
-    for (int k = threadIdx.x; k < nt; k += blockDim.x) {
+    for (int k = threadIdx.x; k < nt; k += blockDim.x) {      // a thread takes a token through all rows
         const int t = t_lo + k;
+        float* p = a.ring + (size_t)bh * a.n * a.T + t;
+#pragma unroll 4
+        for (int r = 0; r < a.n; ++r) {
+            const int i = a.n - 1 - r;
+            p[(size_t)r * a.T] = (t <= a.T - a.n + i) ? __expf(p[(size_t)r * a.T] - s_m[i]) * s_inv[i] : 0.f;
+        }
         a.nvalid[(size_t)bh * a.T + t] = (uint8_t)min(a.n, a.T - t);
     }
 }

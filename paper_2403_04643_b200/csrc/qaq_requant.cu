@@ -46,11 +46,19 @@ struct RequantArgs {
 };
 
 // B = min{b in [bmin,bmax] : v <= c * 2^b}, bmax if none (c * 2^b is an exact scaling)
+// For positive normal v and c the answer is read off the exponents: with v = mv * 2^ev, c = mc * 2^ec
+// (mv, mc in [1,2)) the smallest b is ev - ec if mv <= mc, else ev - ec + 1.
 __device__ __forceinline__ int ladder(float v, float c, int bmin, int bmax) {
     if (!(c > 0.f)) return bmax;
-    for (int b = bmin; b <= bmax; ++b)
-        if (v <= __fmul_rn(c, (float)(1 << b))) return b;
-    return bmax;
+    if (v <= __fmul_rn(c, (float)(1 << bmin))) return bmin;
+    const int vb = __float_as_int(v), cb = __float_as_int(c);
+    if (cb < 0x00800000 || vb < 0x00800000) {  // subnormal operand: plain ladder
+        for (int b = bmin; b <= bmax; ++b)
+            if (v <= __fmul_rn(c, (float)(1 << b))) return b;
+        return bmax;
+    }
+    const int b = (vb >> 23) - (cb >> 23) + (((vb & 0x7FFFFF) > (cb & 0x7FFFFF)) ? 1 : 0);
+    return b < bmin ? bmin : (b > bmax ? bmax : b);
 }
 
 // NW words from / to an address that is ALIGN-byte aligned (ALIGN in {4, 8, 16})
