@@ -115,12 +115,13 @@ __device__ __forceinline__ int plane_dot(const uint32_t (&words)[8], const uint3
     return (ah[0] + ah[1]) * 256 + (al[0] + al[1]);
 }
 
-// acc[r][i] += b * (f - 2^(W-1)) for the lane's 32 channels of a w-bit plane, b = bm[m] * 2^(W*m).
+// acc[r][i] += b * (f - 2^(W-1)) for the lane's 32 channels of a w-bit plane.
 // Fields are taken two at a time (the same bit positions of the two 16-bit halves of a word) by
-// OR-ing them into the mantissa of binary16 1024: 1024 + f * 2^(W*m); subtracting 1024 +
-// 2^(W-1) * 2^(W*m) is exact and centres the code.  The products go into binary32 accumulators.
+// OR-ing them into the mantissa of a binary16 power of two whose last mantissa bit weighs
+// 2^-(W*m) for field slot m: 2^(10-Wm) + f, exactly; subtracting 2^(10-Wm) + 2^(W-1) is exact and
+// centres the code, so every slot uses the same weight.  The products go into binary32 accumulators.
 template <int W>
-__device__ __forceinline__ void plane_axpy(const uint32_t (&words)[8], const unsigned short (&bm)[8 / W], float (&acc)[8][4]) {
+__device__ __forceinline__ void plane_axpy(const uint32_t (&words)[8], unsigned short b, float (&acc)[8][4]) {
     constexpr int PER = 8 / W;
 #pragma unroll
     for (int j = 0; j < W; ++j) {
@@ -129,16 +130,17 @@ __device__ __forceinline__ void plane_axpy(const uint32_t (&words)[8], const uns
 #pragma unroll
         for (int m = 0; m < PER; ++m) {
             const uint32_t mask = (((1u << W) - 1u) << (W * m)) * 0x00010001u;
-            const uint32_t cen = (0x6400u + (1u << (W - 1 + W * m))) * 0x00010001u;   // binary16 of 1024 + 2^(W-1+Wm), twice
+            const uint32_t magic = (0x6400u - ((uint32_t)(W * m) << 10)) * 0x00010001u;        // binary16 2^(10-Wm), twice
+            const uint32_t cen = magic + (1u << (W - 1 + W * m)) * 0x00010001u;              // ... + 2^(W-1)
             const __half2 c2 = *reinterpret_cast<const __half2*>(&cen);
-            uint32_t xe = lop3_and_or(ev, mask, 0x64006400u), xo = lop3_and_or(od, mask, 0x64006400u);
+            uint32_t xe = lop3_and_or(ev, mask, magic), xo = lop3_and_or(od, mask, magic);
             const __half2 ye = __hsub2(*reinterpret_cast<__half2*>(&xe), c2);
             const __half2 yo = __hsub2(*reinterpret_cast<__half2*>(&xo), c2);
             const int r = PER * j + m;
-            fma_f32_f16(acc[r][0], __half_as_ushort(__low2half(ye)), bm[m]);
-            fma_f32_f16(acc[r][2], __half_as_ushort(__high2half(ye)), bm[m]);
-            fma_f32_f16(acc[r][1], __half_as_ushort(__low2half(yo)), bm[m]);
-            fma_f32_f16(acc[r][3], __half_as_ushort(__high2half(yo)), bm[m]);
+            fma_f32_f16(acc[r][0], __half_as_ushort(__low2half(ye)), b);
+            fma_f32_f16(acc[r][2], __half_as_ushort(__high2half(ye)), b);
+            fma_f32_f16(acc[r][1], __half_as_ushort(__low2half(yo)), b);
+            fma_f32_f16(acc[r][3], __half_as_ushort(__high2half(yo)), b);
         }
     }
 }
@@ -198,19 +200,15 @@ __device__ __forceinline__ void k_items(WarpScratch<D>& ws, int first, int n, co
 
 template <int D, int W, int ALIGN>
 __device__ __forceinline__ void v_items(WarpScratch<D>& ws, int first, int n, float (&acc)[8][4], int part, int sub) {
-    constexpr int P = D / 32, IPW = 32 / P, PER = 8 / W;
+    constexpr int P = D / 32, IPW = 32 / P;
 #pragma unroll 1
     for (int i0 = sub; i0 < n; i0 += IPW) {
         uint32_t w0[8];
         const uint32_t de = ws.item[1][first + i0];
         load_words<W, ALIGN>(ws.bufV + (de & 0xFFFFu) + part * 4 * W, w0);
-        // weight of field slot m: p_t * step_t * 2^g * 2^shift / 2^(W*m), in binary16
+        // weight of the piece: p_t * step_t * 2^g * 2^shift, in binary16
         const float wt = ws.wv[de >> 24] * __int_as_float((127 + ((de >> 16) & 7)) << 23);
-        unsigned short bm[PER];
-        const __half b0 = __float2half_rn(wt);
-#pragma unroll
-        for (int m = 0; m < PER; ++m) bm[m] = __half_as_ushort(__hmul(b0, __ushort_as_half((unsigned short)((15 - W * m) << 10))));
-        plane_axpy<W>(w0, bm, acc);
+        plane_axpy<W>(w0, __half_as_ushort(__float2half_rn(wt)), acc);
     }
 }
 
