@@ -35,6 +35,18 @@ def oracle_batch(wl, K, V, q, ring, nv, cK, cV, thr=None, bitsK=None, bitsV=None
                             out_cap=max(1024, T * D // 2))
 
 
+def oracle_thresholds(wl, K, V, thr_gpu, bh_sel=None, tokens=None):
+    """Thresholds computed by the oracle for the chosen (b,h); the device's must equal them bit for bit.  Returns
+    the oracle's values (what the oracle is fed with afterwards never comes from the device)."""
+    T = K.shape[2] if tokens is None else tokens
+    ku = u16(K).reshape(wl.bh, K.shape[2], wl.head_dim)[:, :T]; vu = u16(V).reshape(wl.bh, V.shape[2], wl.head_dim)[:, :T]
+    rows = range(wl.bh) if bh_sel is None else bh_sel
+    out = np.array([[*oracle.thresholds(ku[bh], wl.alpha), *oracle.thresholds(vu[bh], wl.alpha)] for bh in rows], dtype=np.float32)
+    got = thr_gpu.detach().cpu().numpy()[list(rows)]
+    assert np.array_equal(got, out), "thresholds differ from the oracle's order statistics"
+    return out
+
+
 def compare_export(cache, ref, bh_sel=None):
     """Bit-exact comparison of the canonical arrays of both tensors with the oracle's."""
     for x, refs in ((0, ref.K), (1, ref.V)):

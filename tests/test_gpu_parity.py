@@ -112,7 +112,7 @@ def test_appends_equal_bulk_quantization():
     Tp = cache.tokens
     wlp = synth.scaled(wl, tokens=Tp)
     refp = oracle_batch(wlp, K[:, :, :Tp], V[:, :, :Tp], q, ring[:, :, :, :Tp].contiguous(), nv[:, :, :Tp].contiguous(),
-                        pol.cK, pol.cV, thr=thr.cpu().numpy())
+                        pol.cK, pol.cV, thr=ref.thr)              # the oracle's own thresholds of the full sequence, frozen
     out = qaq.qaq_decode_attention(cache, qd, 1 / math.sqrt(128))
     assert_attention_close(out.cpu().numpy(), refp.X)
 

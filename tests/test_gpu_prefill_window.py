@@ -9,7 +9,7 @@ import torch
 import oracle
 from paper_2403_04643_b200 import qaq, synth
 
-from gpu_helpers import u16
+from gpu_helpers import oracle_thresholds, u16
 
 pytestmark = pytest.mark.gpu
 
@@ -54,7 +54,7 @@ def test_window_feeds_the_width_selection_like_any_ring():
     bK, bV = qaq.qaq_select_bits(cfg, pol, Kd, Vd, ring, nvalid, thr)
     cK, cV = oracle.policy(*hyper, T)
     ku, vu, qu = u16(K).reshape(wl.bh, T, D), u16(V).reshape(wl.bh, T, D), u16(Q)
-    thr_h = thr.cpu().numpy()
+    thr_h = oracle_thresholds(wl, K, V, thr)
     agree = total = 0
     for bh in range(wl.bh):
         r, nv, _ = oracle.prefill_window(qu[bh], ku[bh], scale)

@@ -11,7 +11,7 @@ import torch
 import oracle
 from paper_2403_04643_b200 import qaq, synth
 
-from gpu_helpers import assert_attention_close, compare_export, gpu_pipeline, make_inputs, oracle_batch, u16
+from gpu_helpers import assert_attention_close, compare_export, gpu_pipeline, make_inputs, oracle_batch, oracle_thresholds, u16
 
 pytestmark = pytest.mark.gpu
 
@@ -78,7 +78,7 @@ def test_given_widths_then_appends_continue_behind_the_shrunk_open_tile(D):
     # expected: every token quantized directly at its final width (the nesting property pinned on the CPU side)
     final = b0.copy()
     final[:, :, :first] = np.minimum(b0[:, :, :first], np.maximum(req, 1))
-    thr_h = thr.cpu().numpy()
+    thr_h = oracle_thresholds(wl, K, V, thr)
     ku, vu = u16(K).reshape(wl.bh, T, D), u16(V).reshape(wl.bh, T, D)
     qk = [oracle.quantize(ku[bh], thr_h[bh, 0], thr_h[bh, 1], final[0, bh]) for bh in range(wl.bh)]
     qv = [oracle.quantize(vu[bh], thr_h[bh, 2], thr_h[bh, 3], final[1, bh]) for bh in range(wl.bh)]
@@ -125,7 +125,7 @@ def test_both_directions_leave_the_cache_as_if_filled_at_the_new_widths(D, shado
     Kd, Vd = K.cuda(), V.cuda()
     Ks, Vs = (Kd, Vd) if shadow == "device" else (K.pin_memory(), V.pin_memory())
     thr = qaq.qaq_outlier_thresholds(cfg, Kd, Vd)
-    thr_h = thr.cpu().numpy()
+    thr_h = oracle_thresholds(wl, K, V, thr)
     cache = qaq.Cache(cfg)
     tb = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
     scale = 1.0 / math.sqrt(D)
@@ -177,12 +177,13 @@ def test_widths_by_the_rules_raise_and_lower():
     ring2, nv2 = synth.make_score_ring(wl, 5)
     polB = qaq.qaq_policy_from_hyper(*HYPER, T)           # tighter budgets: most widths go up
     qaq.qaq_requantize(cache, dev[0], dev[1], thr, policy=polB, ring=ring2.cuda(), nvalid=nv2.cuda())
-    ref = oracle_batch(wl, K, V, q, ring2, nv2, *oracle.policy(*HYPER, T), thr=thr.cpu().numpy())
+    thr_h = oracle_thresholds(wl, K, V, thr)
+    ref = oracle_batch(wl, K, V, q, ring2, nv2, *oracle.policy(*HYPER, T), thr=thr_h)
     assert qaq.qaq_cache_stats(cache).device_status == 0
     compare_export(cache, ref)                            # as if selected and quantized with the second window and policy
     out2 = qaq.qaq_decode_attention(cache, dev[2], 1.0 / math.sqrt(wl.head_dim))
     assert_attention_close(out2.cpu().numpy(), ref.X)
-    first = oracle_batch(wl, K, V, q, ring, nv, *oracle.policy(*LOOSER, T), thr=thr.cpu().numpy())
+    first = oracle_batch(wl, K, V, q, ring, nv, *oracle.policy(*LOOSER, T), thr=thr_h)
     up = sum(int((a.bits > b.bits).sum()) for a, b in zip(ref.K + ref.V, first.K + first.V))
     down = sum(int((a.bits < b.bits).sum()) for a, b in zip(ref.K + ref.V, first.K + first.V))
     assert up > 200 and qaq.qaq_cache_stats(cache).device_status == 0, (up, down)
@@ -212,7 +213,7 @@ def test_a_full_pool_is_reported_and_every_tile_stays_consistent():
     qaq.qaq_requantize(cache, dev[0], dev[1], thr, policy=qaq.qaq_policy_from_hyper(*HYPER, T), ring=ring2.cuda(), nvalid=nv2.cuda())
     assert qaq.qaq_cache_stats(cache).device_status == 3
     got = np.stack([qaq.qaq_cache_export(cache, x)["bits"].cpu().numpy() for x in range(2)])
-    qk, qv = _quantized(wl, K, V, thr.cpu().numpy(), got, T)
+    qk, qv = _quantized(wl, K, V, oracle_thresholds(wl, K, V, thr), got, T)
     compare_export(cache, SimpleNamespace(K=qk, V=qv))
     out2 = qaq.qaq_decode_attention(cache, dev[2], 1.0 / math.sqrt(wl.head_dim))
     assert_attention_close(out2.cpu().numpy(), _decode_ref(wl, q, qk, qv))
@@ -240,7 +241,7 @@ def test_compaction_of_a_pool_with_many_moved_tiles():
     packed = qaq.qaq_cache_pool_use(cache)
     assert moved[0] > 1.5 * filled[0] and packed[0] < 0.8 * moved[0] and packed[1] < 0.8 * moved[1]
     qaq.qaq_quantize_append(cache, Kd[:, :, T:], Vd[:, :, T:], thr, bitsK=tb(bits[0][:, T:]), bitsV=tb(bits[1][:, T:]))
-    qk, qv = _quantized(wl, K, V, thr.cpu().numpy(), bits, 5100)
+    qk, qv = _quantized(wl, K, V, oracle_thresholds(wl, K, V, thr), bits, 5100)
     compare_export(cache, SimpleNamespace(K=qk, V=qv))
     out = qaq.qaq_decode_attention(cache, q.cuda(), 1.0 / math.sqrt(D))
     assert_attention_close(out.cpu().numpy(), _decode_ref(wl, q, qk, qv))
