@@ -35,6 +35,21 @@ from paper_2403_04643_b200 import synth  # noqa: E402
 # only valid for that shape and for the kernels as they were when the capture was taken.
 NCU_TRAFFIC = {("C3", "quant"): 672.9e6 + 128.4e6, ("C3", "decode"): 140.7e6 + 0.3e6}
 
+# Warp instructions per launch from the same captures (smsp__inst_executed.sum), for the secondary ceiling: the
+# kernels are limited by instruction issue, whose peak is 148 SMs x 4 schedulers x 1 instruction per clock.
+NCU_WARP_INSTR = {("C3", "quant"): 197.9e6, ("C3", "decode"): 64.6e6, ("C3_low", "decode"): 59.7e6}
+ISSUE_SLOTS_PER_CLOCK = 148 * 4
+
+
+def issue_roofline(key, seconds, sm_mhz):
+    n = NCU_WARP_INSTR.get(key)
+    if not n or not seconds or not sm_mhz:
+        return None
+    peak = ISSUE_SLOTS_PER_CLOCK * sm_mhz * 1e6
+    return {"bound": "alu", "warp_instr_per_launch": n, "achieved": round(n / seconds / 1e9, 1), "peak": round(peak / 1e9, 1),
+            "unit": "G warp-instr/s", "frac": round(n / seconds / peak, 3)}
+
+
 METRIC = "QAQ quantize GB/s + packed decode-attn tokens/s, % of B200 HBM peak"
 QNORM2 = 1.16   # stand-in for the upper-10% quantile of sum_d (q_d / sqrt(D))^2 of N(0,1) queries
 
@@ -319,6 +334,8 @@ def main():
         "roofline_decode": {"kernel": "decode_kernel (+ merge)", "bound": "hbm", "achieved": round(dec_gbs, 1), "peak": peak,
                             "unit": "GB/s", "frac": round(dec_gbs / peak, 3), "traffic": NCU_TRAFFIC.get((args.workload, "decode")), "peak_kind": peak_kind,
                             "bytes_per_launch": ab["decode"]},
+        "roofline_issue": {"quant_kernel": issue_roofline((args.workload, "quant"), stage_ms["quant"] * 1e-3, clocks.get("sm_mhz")),
+                           "decode_kernel": issue_roofline((args.workload, "decode"), stage_ms["dec"] * 1e-3, clocks.get("sm_mhz"))},
         "gpu_launches": args.steps * L * 6,
         "clocks": clocks,
     }
@@ -354,7 +371,7 @@ def main():
     # ---- the other 7B-shaped configurations, for context (rank 0, one GPU): one layer at batch 1 (launch-latency
     # regime) and the long-context cache (values of tokens beyond the prefill stay at 8 bits: no score seen yet)
     if rank == 0 and world == 1 and not args.no_extras:
-        out["extras"] = extras(qaq, calibrate, dev, peak, hyper_qn, args.extras)
+        out["extras"] = extras(qaq, calibrate, dev, peak, hyper_qn, args.extras, clocks.get("sm_mhz"))
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(wl, (sS, sX, hyper_qn))
@@ -379,7 +396,7 @@ def _time_us(fn, reps):
     return a.elapsed_time(b) * 1e3 / reps
 
 
-def extras(qaq, calibrate, dev, peak, qn, only=""):
+def extras(qaq, calibrate, dev, peak, qn, only="", sm_mhz=None):
     res = {}
     c3 = synth.scaled(synth.CONFIGS["C3"], layers=1)
     # (name, workload, tokens, prefill, target mean widths (K, V) or None, constant width or None)
@@ -452,6 +469,8 @@ def extras(qaq, calibrate, dev, peak, qn, only=""):
                      "append1_plus_decode_us": round(us_s, 1),
                      "mean_bits": [round(st.code_bytes[0] * 8 / (BH * T * D), 2), round(st.code_bytes[1] * 8 / (BH * T * D), 2)],
                      "cr_paper": round(st.cr_paper, 3)}
+        if name == "C3_layer_low_widths":      # fewer bytes, the same instructions: the issue ceiling is the one that binds
+            res[name]["decode_issue"] = issue_roofline(("C3_low", "decode"), us_d * 1e-6, sm_mhz)
         if name == "C3_layer_uniform4_with_outliers":
             # the score window after a prefill (Section 4.2): rows of the last `window` queries on the fp16 keys
             Qw = torch.randn((BH, W, D), device=dev, dtype=torch.float32).to(torch.float16)
