@@ -527,14 +527,14 @@ def extras(qaq, calibrate, dev, peak, qn, only="", sm_mhz=None):
     return res
 
 
-def cpu_baseline(wl, hyper, budget_s=20.0):
+def cpu_baseline(wl, hyper, budget_s=15.0):
     cores = os.cpu_count() or 1
     n_bh = min(wl.bh, 16 * cores)
     run = oracle_sample(wl, hyper, n_bh, cores, "cpu")
     dt, r = run()
     reps = 1
     total = dt
-    while total + dt < budget_s and reps < 4:
+    while total + dt < budget_s and reps < 12:
         d2, r = run()
         total += d2
         reps += 1
