@@ -137,8 +137,11 @@ __device__ __forceinline__ uint32_t pool_take(uint32_t* pool, uint32_t amount, u
 // widths [A] warp 0 scans the tile and takes pool space with four atomics in flight at once
 // while every warp computes its codes [B] planes into a shared-memory image of the tile
 // [C] the image goes out with 16-byte stores; outlier entries and per-token metadata follow.
-template <int D, bool SELECT_ONLY>
-__global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const QuantArgs a) {
+// XSEL: -1 = keys and values in one CTA; 0 / 1 = this launch handles only the keys / only the values of a tile
+// (half the registers and shared memory per CTA, so more tiles are in flight per SM).
+template <int D, bool SELECT_ONLY, int XSEL>
+__global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 128 ? 5 : 6)) quant_kernel(const QuantArgs a) {
+    constexpr int X0 = XSEL < 0 ? 0 : XSEL, X1 = XSEL < 0 ? 2 : XSEL + 1;
     constexpr int P = D / 32;            // lanes per token
     constexpr int ALIGN = D / 8 >= 16 ? 16 : D / 8;  // alignment of a token's bytes inside a tile
     constexpr int NT = 2 * D;            // threads
@@ -157,7 +160,7 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
     __shared__ uint32_t s_cnt[2][QAQ_TILE];   // outlier counts, then exclusive offsets
     __shared__ uint32_t s_tot[2], s_base[2], s_obase[2], s_olimit[2];
     __shared__ int s_skip;
-    __shared__ __align__(16) uint8_t s_img[SELECT_ONLY ? 1 : 2][SELECT_ONLY ? 16 : QAQ_TILE * D];  // packed tile, K and V
+    __shared__ __align__(16) uint8_t s_img[SELECT_ONLY ? 1 : X1 - X0][SELECT_ONLY ? 16 : QAQ_TILE * D];  // packed tile (K and V)
 
     const float* thr = a.thr + (size_t)bh * 4;
     const bool given = a.bitsK != nullptr;
@@ -172,8 +175,8 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
         for (int i = 0; i < 4; ++i) {
             uint4 x = make_uint4(0, 0, 0, 0), y = make_uint4(0, 0, 0, 0);
             if (valid) {
-                x = *reinterpret_cast<const uint4*>(Kr + 8 * i);
-                y = *reinterpret_cast<const uint4*>(Vr + 8 * i);
+                if (XSEL != 1) x = *reinterpret_cast<const uint4*>(Kr + 8 * i);
+                if (XSEL != 0) y = *reinterpret_cast<const uint4*>(Vr + 8 * i);
             }
             vk[4 * i] = x.x; vk[4 * i + 1] = x.y; vk[4 * i + 2] = x.z; vk[4 * i + 3] = x.w;
             vv[4 * i] = y.x; vv[4 * i + 1] = y.y; vv[4 * i + 2] = y.z; vv[4 * i + 3] = y.w;
@@ -184,7 +187,7 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
     float shat = __int_as_float(0xff800000);
     int nv_tok = 0;
     {
-        if (!given && valid) {
+        if (XSEL != 0 && !given && valid) {
             nv_tok = a.nvalid[(size_t)bh * a.n_new + tn];
             nv_tok = nv_tok < a.W ? nv_tok : a.W;
             const float* r = a.ring + (size_t)bh * a.W * a.n_new + tn;
@@ -198,7 +201,7 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
     uint32_t inl[2], cntx[2];
     float mnf[2], mxf[2];
 #pragma unroll
-    for (int x = 0; x < 2; ++x) {
+    for (int x = X0; x < X1; ++x) {
         // thresholds as binary16 bounds that decide exactly like the binary32 ones on binary16 data
         const __half lo = __float2half_ru(thr[2 * x]), hi = __float2half_rd(thr[2 * x + 1]);
         __half2 mn2, mx2;
@@ -219,7 +222,7 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
     // ---- widths
     int Bx[2];
 #pragma unroll
-    for (int x = 0; x < 2; ++x) {
+    for (int x = X0; x < X1; ++x) {
         int B;
         if (given) {
             B = valid ? (x ? a.bitsV : a.bitsK)[(size_t)bh * a.n_new + tn] : 0;
@@ -248,7 +251,7 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
     if (warp == 0) {
         uint32_t amount[2][2];   // [tensor][0: bytes, 1: outliers]
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
+        for (int x = X0; x < X1; ++x) {
             uint32_t l0 = s_len[x][lane], l1 = s_len[x][lane + 32];
             uint32_t c0 = s_cnt[x][lane], c1 = s_cnt[x][lane + 32];
             uint32_t il0 = l0, il1 = l1, ic0 = c0, ic1 = c1;
@@ -265,10 +268,10 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
             amount[x][0] = tot0 + tot1; amount[x][1] = ctot0 + ctot1;
             if (lane == 0) s_tot[x] = amount[x][0];
         }
-        if (lane < 4) {
+        if (lane >= 2 * X0 && lane < 2 * X1) {
             const int x = lane >> 1, pool = lane & 1;
             const TensorStore& ts = x ? a.v : a.k;
-            my_amount = amount[x][pool];
+            my_amount = x ? amount[1][pool] : amount[0][pool];
             my_base = pool_take(pool ? &ts.opool_end[bh] : &ts.pool_end[bh], my_amount, pool ? 3u : 15u, whole, closes);
         }
     }
@@ -276,7 +279,7 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
     // ---- codes (every warp; needs only registers): channels 4j..4j+3 in the byte lanes of creg[j]
     uint32_t cregs[2][8];
 #pragma unroll
-    for (int x = 0; x < 2; ++x) {
+    for (int x = X0; x < X1; ++x) {
         const uint32_t (&v)[16] = x ? vv : vk;
         const int B = Bx[x];
         const float mn = mnf[x];
@@ -302,10 +305,10 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
 
     // ---- planes into the shared-memory image of the tile
 #pragma unroll
-    for (int x = 0; x < 2; ++x) {
+    for (int x = X0; x < X1; ++x) {
         const uint32_t (&creg)[8] = cregs[x];
         const int B = Bx[x];
-        uint8_t* tok = s_img[x] + s_len[x][slot & (QAQ_TILE - 1)];
+        uint8_t* tok = s_img[x - X0] + s_len[x][slot & (QAQ_TILE - 1)];
         if (B & 8) {
             store_words<ALIGN>(tok + p * 32, creg, 8);
         }
@@ -337,11 +340,11 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
         }
     }
     // ---- allocation results (the atomics were issued before the codes were computed)
-    if (warp == 0 && lane < 4) {
+    if (warp == 0 && lane >= 2 * X0 && lane < 2 * X1) {
         const int x = lane >> 1, pool = lane & 1;
         const TensorStore& ts = x ? a.v : a.k;
         const size_t ti = (size_t)bh * a.ntiles + tile;
-        if (lane == 0) s_skip = 0;
+        if (lane == 2 * X0) s_skip = 0;
         if (pool == 0) {
             if ((size_t)my_base + my_amount + 16 > a.pool_bytes) { atomicMax(a.status, (int)QAQ_ERR_CAPACITY); s_skip = 1; }
             if (starts) { ts.tile_off[ti] = my_base; ts.tile_nbytes[ti] = my_amount; }
@@ -362,14 +365,14 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
 
     // ---- the image goes out with vector stores; outlier list; per-token metadata
 #pragma unroll
-    for (int x = 0; x < 2; ++x) {
+    for (int x = X0; x < X1; ++x) {
         const TensorStore& ts = x ? a.v : a.k;
         uint8_t* dst = ts.codes + (size_t)bh * a.pool_bytes + s_base[x];
         const uint32_t nb = s_tot[x];
         for (uint32_t o = tid * ALIGN; o < nb; o += NT * ALIGN) {
-            if (ALIGN == 16) *reinterpret_cast<uint4*>(dst + o) = *reinterpret_cast<const uint4*>(s_img[x] + o);
-            else if (ALIGN == 8) *reinterpret_cast<uint2*>(dst + o) = *reinterpret_cast<const uint2*>(s_img[x] + o);
-            else *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(s_img[x] + o);
+            if (ALIGN == 16) *reinterpret_cast<uint4*>(dst + o) = *reinterpret_cast<const uint4*>(s_img[x - X0] + o);
+            else if (ALIGN == 8) *reinterpret_cast<uint2*>(dst + o) = *reinterpret_cast<const uint2*>(s_img[x - X0] + o);
+            else *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(s_img[x - X0] + o);
         }
         // outliers in (token, channel) order: entries of lanes p' < p come first
         uint32_t ob = valid ? ~inl[x] : 0u;
@@ -405,14 +408,27 @@ __global__ void __launch_bounds__(2 * D, D == 128 ? 3 : 4) quant_kernel(const Qu
     }
 }
 
-template <bool SELECT_ONLY>
-qaq_status launch(int D, dim3 grid, const QuantArgs& a, cudaStream_t s) {
+template <bool SELECT_ONLY, int XSEL>
+qaq_status launch_x(int D, dim3 grid, const QuantArgs& a, cudaStream_t s) {
     switch (D) {
-        case 32: quant_kernel<32, SELECT_ONLY><<<grid, 64, 0, s>>>(a); break;
-        case 64: quant_kernel<64, SELECT_ONLY><<<grid, 128, 0, s>>>(a); break;
-        case 128: quant_kernel<128, SELECT_ONLY><<<grid, 256, 0, s>>>(a); break;
+        case 32: quant_kernel<32, SELECT_ONLY, XSEL><<<grid, 64, 0, s>>>(a); break;
+        case 64: quant_kernel<64, SELECT_ONLY, XSEL><<<grid, 128, 0, s>>>(a); break;
+        case 128: quant_kernel<128, SELECT_ONLY, XSEL><<<grid, 256, 0, s>>>(a); break;
         default: return QAQ_ERR_UNSUPPORTED_SHAPE;
     }
+    return QAQ_OK;
+}
+
+template <bool SELECT_ONLY>
+qaq_status launch(int D, dim3 grid, const QuantArgs& a, cudaStream_t s) {
+    qaq_status st;
+    if (SELECT_ONLY || grid.x * grid.y < 4096) {
+        st = launch_x<SELECT_ONLY, -1>(D, grid, a, s);
+    } else {   // large launches: keys and values of a tile in separate CTAs
+        st = launch_x<SELECT_ONLY, 0>(D, grid, a, s);
+        if (st == QAQ_OK) st = launch_x<SELECT_ONLY, 1>(D, grid, a, s);
+    }
+    if (st != QAQ_OK) return st;
     QAQ_CUDA_TRY(cudaGetLastError());
     return QAQ_OK;
 }
