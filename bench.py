@@ -336,7 +336,7 @@ def main():
                             "bytes_per_launch": ab["decode"]},
         "roofline_issue": {"quant_kernel": issue_roofline((args.workload, "quant"), stage_ms["quant"] * 1e-3, clocks.get("sm_mhz")),
                            "decode_kernel": issue_roofline((args.workload, "decode"), stage_ms["dec"] * 1e-3, clocks.get("sm_mhz"))},
-        "gpu_launches": args.steps * L * 6,
+        "gpu_launches": args.steps * L * 7,   # thresholds 3 (sample, scan, select), quantize 2 (keys, values), decode 2 (+ merge)
         "clocks": clocks,
     }
 
