@@ -270,7 +270,7 @@ def main():
     for _ in range(args.warmup):
         step()
     barrier()
-    # the launches of one step (32 layers x reset + 6 kernels) are captured once into a CUDA graph and replayed
+    # the launches of one step (per layer: reset + 7 kernels) are captured once into a CUDA graph and replayed
     run_step, launch_mode = step, "stream"
     if not args.no_graph:
         try:
