@@ -154,10 +154,11 @@ struct WarpScratch {
     alignas(16) uint8_t bufK[UNIT * D + 16];
     alignas(16) uint8_t bufV[UNIT * D + 16];
     float stepK[UNIT];
-    float midK[UNIT];           // min + step/2
-    float midV[UNIT];
-    float ocorr[UNIT];          // sum over a token's key outliers of q_ch * (x - mid)
-    float p[UNIT];
+    // per token of the whole tile (both halves): the tile's outlier lists are gone through once
+    float midK[2 * UNIT];       // min + step/2
+    float midV[2 * UNIT];
+    float ocorr[2 * UNIT];      // sum over a token's key outliers of q_ch * (x - mid)
+    float p[2 * UNIT];          // attention weights, kept at the current scale of the running sums
     float wv[UNIT];             // p_t * step_t * 2^g of the value side
     float vout[D];              // value-outlier corrections
     int dot[UNIT];
@@ -356,7 +357,6 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
         const uint32_t ooV = __shfl_sync(0xFFFFFFFFu, cur.tb, 6), ocV = __shfl_sync(0xFFFFFFFFu, cur.tb, 7);
         const bool has_next = tile + DEC_WARPS < tile_hi;
         uint32_t n0K = 0, n0V = 0;   // first-half bytes of the next tile
-        uint32_t resumeK = 0, resumeV = 0;   // where half 1 resumes in the tile's outlier lists
 
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
@@ -364,7 +364,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
             const bool valid = t < a.T;
             // ---- per-token scalars, byte offsets inside the half tile, item lists
             int ncls[2][4];
-            float rngV = 0.f;
+            float rngV = 0.f, cstV = 0.f;
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
                 const int B = valid ? (int)((cur.bits4 >> (16 * x + 8 * half)) & 0xFF) : 0;
@@ -376,16 +376,29 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
                 const float st = __fmul_rn(rng, __int_as_float((127 - B) << 23));
                 const float mid = fmaf(0.5f, st, mn);
                 if (x == 0) {
-                    ws.stepK[lane] = st; ws.midK[lane] = valid ? mid : 0.f;
-                    ws.dot[lane] = 0; ws.ocorr[lane] = 0.f;
+                    ws.stepK[lane] = st;
+                    ws.dot[lane] = 0;
+                    if (half == 0) {
+                        ws.midK[lane] = valid ? mid : 0.f;
+                        ws.ocorr[lane] = 0.f;
+                        // the lane's token of the second half: its mid is needed already, because all key outliers of
+                        // the tile are gone through in this half
+                        const bool valid2 = t + UNIT < a.T;
+                        const int B2 = valid2 ? (int)((cur.bits4 >> 8) & 0xFF) : 0;
+                        const float mn2 = __half2float(__ushort_as_half((unsigned short)(cur.mm[1] & 0xFFFF)));
+                        const float mx2 = __half2float(__ushort_as_half((unsigned short)(cur.mm[1] >> 16)));
+                        const float st2 = __fmul_rn(valid2 ? __fsub_rn(mx2, mn2) : 0.f, __int_as_float((127 - B2) << 23));
+                        ws.midK[UNIT + lane] = valid2 ? fmaf(0.5f, st2, mn2) : 0.f;
+                        ws.ocorr[UNIT + lane] = 0.f;
+                    }
                 } else {
                     // centred planes: piece w contributes a constant step * 2^((B & (2w-1)) - 1)
                     float cst = 0.5f;
 #pragma unroll
                     for (int w = 8; w >= 1; w >>= 1)
                         if (B & w) cst += __int_as_float((127 + (B & (2 * w - 1)) - 1) << 23);
-                    ws.midV[lane] = valid ? mid : 0.f;                     // value of a zero code slot (outliers)
-                    ws.p[lane] = valid ? fmaf(cst, st, mn) : 0.f;           // constant part, picked up below
+                    ws.midV[UNIT * half + lane] = valid ? mid : 0.f;       // value of a zero code slot (outliers)
+                    cstV = valid ? fmaf(cst, st, mn) : 0.f;                 // constant part, picked up below
                     ws.wv[lane] = st;                                       // step for now, weight after the softmax
                     rngV = rng;
                 }
@@ -435,23 +448,20 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
                 k_items<D, 4, ALIGN>(ws, first, ncls[0][1], qh, ql, part, sub); first += ncls[0][1];
                 k_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, first, ncls[0][2], qh, ql, part, sub); first += ncls[0][2];
                 k_items<D, 1, 4>(ws, first, ncls[0][3], qh, ql, part, sub);
-                // the tile's outlier entries are sorted by token: half 0 stops at the first batch that lies
-                // entirely in tokens >= 32, half 1 resumes there
-                const uint32_t* og = a.k.outl + (size_t)bh * a.ocap + ooK;
-                uint32_t e0 = half ? resumeK : 0u;
+                // all key outliers of the tile, once, while its first half is worked on
+                if (half == 0) {
+                    const uint32_t* og = a.k.outl + (size_t)bh * a.ocap + ooK;
 #pragma unroll 1
-                for (; e0 < ocK; e0 += 32) {
-                    const uint32_t e = e0 + lane;
-                    const uint32_t v = e < ocK ? (e < (uint32_t)OSTAGE ? ws.outl[0][e] : __ldg(og + e)) : 0xFF000000u;
-                    const int tok = v >> 24, ch = (v >> 16) & 0xFF;
-                    if (half == 0 && __all_sync(0xFFFFFFFFu, tok >= UNIT)) break;
-                    if (e < ocK && (tok >> 5) == half) {
-                        const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
-                        atomicAdd(&ws.ocorr[tok & 31], sm.qf[ch] * (val - ws.midK[tok & 31]));
+                    for (uint32_t e0 = 0; e0 < ocK; e0 += 32) {
+                        const uint32_t e = e0 + lane;
+                        if (e < ocK) {
+                            const uint32_t v = e < (uint32_t)OSTAGE ? ws.outl[0][e] : __ldg(og + e);
+                            const int tok = v >> 24, ch = (v >> 16) & 0xFF;
+                            const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
+                            atomicAdd(&ws.ocorr[tok], sm.qf[ch] * (val - ws.midK[tok]));
+                        }
                     }
-                    if (half == 0 && __any_sync(0xFFFFFFFFu, tok >= UNIT)) break;   // this batch straddles the halves
                 }
-                if (half == 0) resumeK = e0 < ocK ? e0 : ocK;
             }
             __syncwarp();
             // ---- the key buffer is free: start the copy of the next unit's keys
@@ -468,7 +478,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
             {
                 float lg = __int_as_float(0xff800000);
                 if (valid) {
-                    const float qk = fmaf(qscale * ws.stepK[lane], (float)ws.dot[lane], fmaf(ws.midK[lane], qsum, ws.ocorr[lane]));
+                    const float qk = fmaf(qscale * ws.stepK[lane], (float)ws.dot[lane], fmaf(ws.midK[UNIT * half + lane], qsum, ws.ocorr[UNIT * half + lane]));
                     lg = a.scale * qk;
                     if (a.scores) a.scores[(size_t)bh * a.T + t] = lg;
                 }
@@ -485,6 +495,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
                         for (int i = 0; i < 4; ++i) acc[r][i] *= alpha;
                     c_run *= alpha;
                     for (int d = lane; d < D; d += 32) ws.vout[d] *= alpha;
+                    if (half == 1) ws.p[lane] *= alpha;       // the first half's weights follow the new scale
                 }
                 float p = __expf(lg - m_new);                // 0 for slots beyond T
                 float sx = p;
@@ -496,7 +507,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
                 const float wr = __fsub_rn(big, __fsub_rn(big, wfull));
                 if (wfull > 0.f) p *= __fdividef(wr, wfull);
                 ws.wv[lane] = wr;
-                c_run = fmaf(p, ws.p[lane], c_run);           // ws.p held the token's constant part
+                c_run = fmaf(p, cstV, c_run);
                 float s = p;
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) {
@@ -505,8 +516,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
                 }
                 l_run = l_run * alpha + s;
                 lx_run = lx_run * alpha + sx;
-                __syncwarp();
-                ws.p[lane] = p;
+                ws.p[UNIT * half + lane] = p;
             }
             cp_async_wait<1>();     // this half's values have landed
             __syncwarp();
@@ -518,21 +528,20 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
                 v_items<D, 4, ALIGN>(ws, first, ncls[1][1], acc, part, sub); first += ncls[1][1];
                 v_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, first, ncls[1][2], acc, part, sub); first += ncls[1][2];
                 v_items<D, 1, 4>(ws, first, ncls[1][3], acc, part, sub);
-                const uint32_t* og = a.v.outl + (size_t)bh * a.ocap + ooV;
-                uint32_t e0 = half ? resumeV : 0u;
+                // all value outliers of the tile, once, when the weights of both halves are known
+                if (half == 1) {
+                    const uint32_t* og = a.v.outl + (size_t)bh * a.ocap + ooV;
 #pragma unroll 1
-                for (; e0 < ocV; e0 += 32) {
-                    const uint32_t e = e0 + lane;
-                    const uint32_t v = e < ocV ? (e < (uint32_t)OSTAGE ? ws.outl[1][e] : __ldg(og + e)) : 0xFF000000u;
-                    const int tok = v >> 24, ch = (v >> 16) & 0xFF;
-                    if (half == 0 && __all_sync(0xFFFFFFFFu, tok >= UNIT)) break;
-                    if (e < ocV && (tok >> 5) == half) {
-                        const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
-                        atomicAdd(&ws.vout[ch], ws.p[tok & 31] * (val - ws.midV[tok & 31]));
+                    for (uint32_t e0 = 0; e0 < ocV; e0 += 32) {
+                        const uint32_t e = e0 + lane;
+                        if (e < ocV) {
+                            const uint32_t v = e < (uint32_t)OSTAGE ? ws.outl[1][e] : __ldg(og + e);
+                            const int tok = v >> 24, ch = (v >> 16) & 0xFF;
+                            const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
+                            atomicAdd(&ws.vout[ch], ws.p[tok] * (val - ws.midV[tok]));
+                        }
                     }
-                    if (half == 0 && __any_sync(0xFFFFFFFFu, tok >= UNIT)) break;
                 }
-                if (half == 0) resumeV = e0 < ocV ? e0 : ocV;
             }
             __syncwarp();
             // ---- the value buffer is free: start the copy of the next unit's values
