@@ -33,11 +33,11 @@ from paper_2403_04643_b200 import synth  # noqa: E402
 
 # DRAM bytes (read + write) per launch from an ncu capture of the C3 layer shape (profiles/kernels_C3_layer.md);
 # only valid for that shape and for the kernels as they were when the capture was taken.
-NCU_TRAFFIC = {("C3", "quant"): 672.8e6 + 114.6e6, ("C3", "decode"): 140.7e6 + 0.3e6}   # quant: K launch + V launch
+NCU_TRAFFIC = {("C3", "quant"): 672.8e6 + 114.6e6, ("C3", "decode"): 140.8e6 + 1.0e6}   # quant: K launch + V launch
 
 # Warp instructions per launch from the same captures (smsp__inst_executed.sum), for the secondary ceiling: the
 # kernels are limited by instruction issue, whose peak is 148 SMs x 4 schedulers x 1 instruction per clock.
-NCU_WARP_INSTR = {("C3", "quant"): 100.0e6 + 119.1e6, ("C3", "decode"): 64.6e6, ("C3_low", "decode"): 59.7e6}
+NCU_WARP_INSTR = {("C3", "quant"): 100.0e6 + 119.1e6, ("C3", "decode"): 62.0e6, ("C3_low", "decode"): 56.9e6}
 ISSUE_SLOTS_PER_CLOCK = 148 * 4
 
 
