@@ -57,7 +57,7 @@ def compare_export(cache, ref, bh_sel=None):
             r = refs[j]
             T = r.T
             assert np.array_equal(g["bits"][bh], r.bits), f"bits tensor {x} bh {bh}"
-            assert np.array_equal(g["mn"][bh].view(np.uint32), r.mn.view(np.uint32)) or np.array_equal(g["mn"][bh], r.mn)
+            assert np.array_equal(g["mn"][bh].view(np.uint32), r.mn.view(np.uint32)), f"min tensor {x} bh {bh}"
             assert np.array_equal(g["step"][bh], r.step), f"step tensor {x} bh {bh}"
             assert np.array_equal(g["off"][bh].astype(np.uint32), r.off), f"off tensor {x} bh {bh}"
             nb = int(r.off[T])

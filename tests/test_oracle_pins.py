@@ -209,6 +209,43 @@ def test_thresholds_are_order_statistics():
     assert (lo, hi) == (0.0, 5.0)
 
 
+def test_thresholds_leave_nans_of_both_signs_out_of_the_population():
+    # Section 4.2 "Outliers": the quantile is taken over the values of the tensor; a NaN has no rank, so the
+    # population is the non-NaN values and k = floor(alpha * N / 2) counts only them.
+    rng = np.random.default_rng(17)
+    x = rng.standard_normal(40 * 64).astype(np.float16)
+    u = x.view(np.uint16).copy()
+    nan_pos = rng.choice(u.size, 300, replace=False)
+    u[nan_pos[:150]] = 0x7E00 | rng.integers(0, 0x1FF, 150).astype(np.uint16)   # +NaN, several payloads
+    u[nan_pos[150:]] = 0xFE00 | rng.integers(0, 0x1FF, 150).astype(np.uint16)   # -NaN
+    xf = u.view(np.float16).astype(np.float32)
+    good = np.sort(xf[~np.isnan(xf)])               # numpy's sort of the values that have a rank
+    N = good.size
+    assert N == u.size - 300
+    for alpha in (0.0, 0.01, 0.05, 0.3):
+        lo, hi = oracle.thresholds(u, alpha)
+        k = int(math.floor(alpha * N / 2))
+        assert lo == good[k] and hi == good[N - 1 - k]
+        assert int(np.sum((good < lo) | (good > hi))) <= alpha * N
+    # a tiny case where counting the NaNs in N would move the rank
+    tiny = np.array([1, 2, 3, 4, 5, 6, 7, 8, 9, 10], np.float16).view(np.uint16).copy()
+    with_nan = np.concatenate([tiny, np.array([0x7E00, 0xFE00, 0x7FFF, 0xFFFF], np.uint16)])
+    # alpha = 0.4: N = 10 -> k = 2 -> (3, 8); counting the NaNs (N = 14) would give k = 2.8 -> 2 as well,
+    # alpha = 0.6: N = 10 -> k = 3 -> (4, 7); with N = 14, k = 4 -> (5, 6): this one tells them apart
+    assert oracle.thresholds(with_nan, 0.4) == (3.0, 8.0)
+    assert oracle.thresholds(with_nan, 0.6) == (4.0, 7.0)
+    # NaNs must not sort to either end either: the extremes at alpha = 0 are the finite ones
+    assert oracle.thresholds(with_nan, 0.0) == (1.0, 10.0)
+    # nothing but NaNs: no population, thresholds (0, 0)
+    assert oracle.thresholds(np.array([0x7E00, 0xFE01, 0x7FFF], np.uint16), 0.01) == (0.0, 0.0)
+    # alpha at a tie: the k-th values are repeated, equal values are not outliers, so the count stays <= alpha N
+    t = np.array([-2.0] * 5 + [0.0] * 10 + [2.0] * 5, np.float16).view(np.uint16)
+    lo, hi = oracle.thresholds(np.concatenate([t, np.array([0xFE00], np.uint16)]), 0.5)   # k = 5: first of the zeros
+    assert (lo, hi) == (0.0, 0.0)
+    lo, hi = oracle.thresholds(np.concatenate([t, np.array([0x7E00], np.uint16)]), 0.4)   # k = 4: inside the tie at -2 / 2
+    assert (lo, hi) == (-2.0, 2.0)
+
+
 def test_planted_outliers_are_split_off_and_kept_exactly():
     wl = synth.scaled(synth.CONFIGS["C2"], heads=2, tokens=256)
     K, _ = synth.make_kv(wl)
