@@ -3,6 +3,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include "qaq_codec.cuh"
 #include "qaq_internal.cuh"
 
 extern "C" const char* qaq_status_string(qaq_status s) {
@@ -42,8 +43,9 @@ extern "C" qaq_status qaq_cache_create(const qaq_config* cfg, qaq_cache** out) {
     c->tmax_pad = (int)align_up((size_t)cfg->max_tokens, QAQ_TILE);
     c->ntiles = c->tmax_pad / QAQ_TILE;
     const int D = cfg->head_dim;
-    // worst case: every token at 8 bits, plus alignment padding per tile and a read-ahead margin
-    c->pool_bytes = align_up((size_t)c->tmax_pad * D + 16 * (size_t)c->ntiles + 256, 256);
+    // worst case per tile: every token at 8 bits or the largest padding of the value groups, plus alignment
+    // padding per tile and a read-ahead margin
+    c->pool_bytes = align_up((size_t)c->ntiles * (size_t)qaqc::v_tile_bytes_max(D) + 16 * (size_t)c->ntiles + 256, 256);
     if (c->pool_bytes >= ((size_t)1 << 32)) { free(c); return QAQ_ERR_UNSUPPORTED_SHAPE; }
     long ocap = cfg->max_outliers_per_bh;
     if (ocap <= 0) {
@@ -154,13 +156,14 @@ struct StatsDev {
     unsigned long long hist[2][9];
     unsigned long long code_bytes[2];
     unsigned long long outliers[2];
+    unsigned long long stored_bytes[2];   // bytes the tiles occupy (values: with the padding of their groups)
 };
 
 __global__ void stats_kernel(TensorStore tk, TensorStore tv, int T, int tmax_pad, int ntiles, int D, StatsDev* out) {
     __shared__ unsigned long long sh[2][9];
-    __shared__ unsigned long long so[2];
+    __shared__ unsigned long long so[2], sb[2];
     if (threadIdx.x < 18) ((unsigned long long*)sh)[threadIdx.x] = 0;
-    if (threadIdx.x < 2) so[threadIdx.x] = 0;
+    if (threadIdx.x < 2) { so[threadIdx.x] = 0; sb[threadIdx.x] = 0; }
     __syncthreads();
     const int bh = blockIdx.x;
     for (int x = 0; x < 2; ++x) {
@@ -170,7 +173,10 @@ __global__ void stats_kernel(TensorStore tk, TensorStore tv, int T, int tmax_pad
             atomicAdd(&sh[x][b > 8 ? 8 : b], 1ULL);
         }
         int nt = (T + QAQ_TILE - 1) / QAQ_TILE;
-        for (int i = threadIdx.x; i < nt; i += blockDim.x) atomicAdd(&so[x], (unsigned long long)ts.tile_ocnt[(size_t)bh * ntiles + i]);
+        for (int i = threadIdx.x; i < nt; i += blockDim.x) {
+            atomicAdd(&so[x], (unsigned long long)ts.tile_ocnt[(size_t)bh * ntiles + i]);
+            atomicAdd(&sb[x], (unsigned long long)ts.tile_nbytes[(size_t)bh * ntiles + i]);
+        }
     }
     __syncthreads();
     if (threadIdx.x < 18) {
@@ -178,7 +184,10 @@ __global__ void stats_kernel(TensorStore tk, TensorStore tv, int T, int tmax_pad
         atomicAdd(&out->hist[x][b], sh[x][b]);
         atomicAdd(&out->code_bytes[x], sh[x][b] * (unsigned long long)(D * b / 8));
     }
-    if (threadIdx.x < 2) atomicAdd(&out->outliers[threadIdx.x], so[threadIdx.x]);
+    if (threadIdx.x < 2) {
+        atomicAdd(&out->outliers[threadIdx.x], so[threadIdx.x]);
+        atomicAdd(&out->stored_bytes[threadIdx.x], sb[threadIdx.x]);
+    }
 }
 
 static qaq_status ensure_stage(qaq_cache* c, int slot, size_t bytes) {
@@ -215,7 +224,7 @@ extern "C" qaq_status qaq_cache_stats(const qaq_cache* cc, qaq_stats* host_out, 
         host_out->outliers[x] = (long)h.outliers[x];
         for (int b = 0; b < 9; ++b) host_out->hist[x][b] = (long)h.hist[x][b];
         bits_total += 8.0 * (double)h.code_bytes[x] + 16.0 * (double)h.outliers[x];
-        resident += (long)h.code_bytes[x] + 4 * (long)h.outliers[x] + BH * T * 5 + BH * nt * 16;
+        resident += (long)h.stored_bytes[x] + 4 * (long)h.outliers[x] + BH * T * 5 + BH * nt * 16;
     }
     host_out->resident_bytes = resident;
     double orig_bits = 16.0 * 2.0 * (double)BH * (double)T * (double)D;
@@ -273,37 +282,88 @@ __global__ void export_scan_kernel(uint32_t* a, int T) {
     }
 }
 
-__global__ void export_gather_kernel(TensorStore ts, int T, int tmax_pad, int ntiles, int D, size_t pool_bytes, uint32_t ocap,
+// one canonical byte of a token: byte y of its string (the planes of its pieces, widest first; inside the plane of
+// a w-bit piece channel d = 32p + 4j + i sits in word p*w + j*w/8 at bit 8i + w*(j mod 8/w)), put together from the
+// pieces as the tile stores them
+template <bool IS_V>
+__device__ uint32_t canonical_byte(const uint8_t* tile, const qaqc::TileMasks& tm, const uint32_t (&base)[5], int D, int slot,
+                                   int B, uint32_t y) {
+    for (int c = 0; c < 4; ++c) {
+        const int w = 8 >> c;
+        if (!(B & w)) continue;
+        const uint32_t plen = (uint32_t)D * w / 8;
+        if (y >= plen) { y -= plen; continue; }
+        const int per = 8 / w, cw = y >> 2, i = y & 3, p = cw / w, rr = cw % w;
+        const int r = qaqc::rank_in(tm, c, slot);
+        uint32_t v = 0;
+        for (int mm = 0; mm < per; ++mm) v |= qaqc::piece_at<IS_V>(tile, base, D, c, r, 32 * p + 4 * (rr * per + mm) + i) << (w * mm);
+        return v;
+    }
+    return 0;
+}
+
+__global__ void export_gather_kernel(TensorStore ts, int is_v, int T, int tmax_pad, int ntiles, int D, size_t pool_bytes, uint32_t ocap,
                                      uint8_t* bits, float* mn, float* step, const uint32_t* off, uint8_t* codes,
                                      long codes_stride, const uint32_t* rowptr, uint8_t* ch, __half* val, long outl_stride) {
     const int bh = blockIdx.y, tile = blockIdx.x;
     __shared__ uint32_t s_in[QAQ_TILE + 1];
+    __shared__ uint8_t s_b[QAQ_TILE];
+    __shared__ unsigned int s_m[4][2];
     const int t0 = tile * QAQ_TILE;
+    if (threadIdx.x < QAQ_TILE) {
+        const int t = t0 + threadIdx.x;
+        int B = t < T ? ts.bits[(size_t)bh * tmax_pad + t] : 0;
+        B = B > 8 ? 8 : B;
+        s_b[threadIdx.x] = (uint8_t)B;
+        for (int c = 0; c < 4; ++c) {
+            const unsigned int bal = __ballot_sync(0xFFFFFFFFu, (B & (8 >> c)) != 0);
+            if ((threadIdx.x & 31) == 0) s_m[c][threadIdx.x >> 5] = bal;
+        }
+    }
+    __syncthreads();
     if (threadIdx.x == 0) {
         uint32_t acc = 0;
         for (int k = 0; k < QAQ_TILE; ++k) {
             s_in[k] = acc;
-            int t = t0 + k;
-            acc += t < T ? (uint32_t)D * ts.bits[(size_t)bh * tmax_pad + t] / 8 : 0;
+            acc += (uint32_t)D * s_b[k] / 8;
         }
         s_in[QAQ_TILE] = acc;
     }
     __syncthreads();
     if (threadIdx.x < QAQ_TILE && t0 + (int)threadIdx.x < T) {
         const int t = t0 + threadIdx.x;
-        const int B = ts.bits[(size_t)bh * tmax_pad + t];
+        const int B = s_b[threadIdx.x];
         const uint32_t mm = ts.mnmx[(size_t)bh * tmax_pad + t];
         const float fmn = __half2float(__ushort_as_half((unsigned short)(mm & 0xFFFF)));
         const float fmx = __half2float(__ushort_as_half((unsigned short)(mm >> 16)));
         if (bits) bits[(size_t)bh * T + t] = (uint8_t)B;
         if (mn) mn[(size_t)bh * T + t] = fmn;
-        if (step) step[(size_t)bh * T + t] = __fmul_rn(__fsub_rn(fmx, fmn), __int_as_float((127 - B) << 23));
+        if (step) step[(size_t)bh * T + t] = qaqc::step_of(fmn, fmx, B);
     }
     if (codes && off) {
         const uint8_t* src = ts.codes + (size_t)bh * pool_bytes + ts.tile_off[(size_t)bh * ntiles + tile];
-        const uint32_t nbytes = s_in[QAQ_TILE];
         uint8_t* dst = codes + (size_t)bh * codes_stride + off[(size_t)bh * (T + 1) + t0];
-        for (uint32_t i = threadIdx.x; i < nbytes; i += blockDim.x) dst[i] = src[i];
+        qaqc::TileMasks tm;
+        for (int c = 0; c < 4; ++c) tm.m[c] = (unsigned long long)s_m[c][0] | ((unsigned long long)s_m[c][1] << 32);
+        int n[4];
+        for (int c = 0; c < 4; ++c) n[c] = __popcll(tm.m[c]);
+        uint32_t base[5];
+        {   // section offsets for any head_dim (the templates of the codec header fix it at compile time)
+            uint32_t o = 0;
+            for (int c = 0; c < 4; ++c) {
+                const int w = 8 >> c;
+                base[c] = o;
+                o += is_v ? (uint32_t)((n[c] + 3) >> 2) * (uint32_t)(D * w / 2) : (uint32_t)n[c] * (uint32_t)(D * w / 8);
+            }
+            base[4] = o;
+        }
+        for (int k0 = 0; k0 < QAQ_TILE; k0 += 4) {
+            const int k = k0 + (threadIdx.x >> 6);
+            const uint32_t len = s_in[k + 1] - s_in[k];
+            for (uint32_t y = threadIdx.x & 63; y < len; y += 64)
+                dst[s_in[k] + y] = (uint8_t)(is_v ? canonical_byte<true>(src, tm, base, D, k, s_b[k], y)
+                                                  : canonical_byte<false>(src, tm, base, D, k, s_b[k], y));
+        }
     }
     if (rowptr && (ch || val)) {
         const uint32_t n = ts.tile_ocnt[(size_t)bh * ntiles + tile];
@@ -341,7 +401,7 @@ extern "C" qaq_status qaq_cache_export(const qaq_cache* c, int tensor, uint8_t* 
         export_ocount_kernel<<<grid, 128, 0, s>>>(ts, T, c->ntiles, c->ocap, rowptr);
         export_scan_kernel<<<c->BH, 256, 0, s>>>(rowptr, T);
     }
-    export_gather_kernel<<<grid, 256, 0, s>>>(ts, T, c->tmax_pad, c->ntiles, c->cfg.head_dim, c->pool_bytes, c->ocap, bits, mn,
+    export_gather_kernel<<<grid, 256, 0, s>>>(ts, tensor, T, c->tmax_pad, c->ntiles, c->cfg.head_dim, c->pool_bytes, c->ocap, bits, mn,
                                               step, off, codes, codes_stride, rowptr, ch, (__half*)val, outl_stride);
     QAQ_CUDA_TRY(cudaGetLastError());
     return QAQ_OK;

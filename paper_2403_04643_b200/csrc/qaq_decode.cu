@@ -17,16 +17,28 @@
 // One CTA = one run of consecutive tiles of the flattened (b,h, tile) sequence (runs of equal
 // length, so every SM gets the same amount of work); each warp works through whole tiles
 // (QAQ_TILE tokens) on its own, with its own running max / sum / accumulators and no CTA
-// barrier in the tile loop; warps are merged once at the end.  A (token, plane) pair is one
-// work item, handled by head_dim/32 lanes that read their words of the plane straight from
-// global memory (every packed byte is read once, by one lane); items are grouped by plane
-// width so that the lanes of a warp run the same extraction code.
+// barrier in the tile loop; warps are merged once at the end.  A tile is stored as sections of
+// equal-width pieces (qaq_codec.cuh), so every inner loop runs one extraction routine over the
+// items of one section, and a token finds its items by its rank among the tokens that have a
+// piece of that width (ballots over the widths; no lists are built).
+//
+// X = S Vhat runs on integer dot products as well: the value pieces of four tokens share a word
+// (one per byte lane), the per-token weights p_t * step_t * 2^shift become 24-bit fixed point
+// with one scale per tile (three dp4a per word and field), and the integer sums of a tile are
+// added to binary32 accumulators once per tile.  The rounded weight of a token is also what the
+// softmax denominator and the constant part of its values use, so numerator and denominator see
+// the same slightly perturbed probability.
+//
+// Outlier corrections are summed in fixed point with integer atomics (scale from the largest
+// term of the tile), so that the result does not depend on the order in which lanes arrive.
+#include "qaq_codec.cuh"
 #include "qaq_internal.cuh"
 
 namespace {
 
 constexpr int DEC_WARPS = 4;
 constexpr int DEC_THREADS = DEC_WARPS * 32;
+constexpr int DEC_CTAS_PER_SM = 2;   // what the per-warp staging buffers of head_dim 128 leave room for
 
 struct DecArgs {
     TensorStore k, v;
@@ -54,15 +66,6 @@ __device__ __forceinline__ int dp4a_uu(uint32_t a, uint32_t b, int c) {  // unsi
     return d;
 }
 
-__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t c) {  // (a & b) | c
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-// acc += a * b with a, b binary16 and acc binary32 (one rounding)
-__device__ __forceinline__ void fma_f32_f16(float& acc, unsigned short a, unsigned short b) {
-    asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc) : "h"(a), "h"(b));
-}
 template <int BYTES>
 __device__ __forceinline__ void cp_async(void* smem, const void* gmem) {
     const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
@@ -73,27 +76,6 @@ __device__ __forceinline__ void cp_async(void* smem, const void* gmem) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
-
-// W words (4*W bytes) of a plane; the address is ALIGN-byte aligned
-template <int W, int ALIGN>
-__device__ __forceinline__ void load_words(const uint8_t* __restrict__ p, uint32_t (&w)[8]) {
-    if (ALIGN == 16 && W % 4 == 0) {
-#pragma unroll
-        for (int i = 0; i < W; i += 4) {
-            const uint4 v = *reinterpret_cast<const uint4*>(p + 4 * i);
-            w[i] = v.x; w[i + 1] = v.y; w[i + 2] = v.z; w[i + 3] = v.w;
-        }
-    } else if (ALIGN >= 8 && W % 2 == 0) {
-#pragma unroll
-        for (int i = 0; i < W; i += 2) {
-            const uint2 v = *reinterpret_cast<const uint2*>(p + 4 * i);
-            w[i] = v.x; w[i + 1] = v.y;
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < W; ++i) w[i] = *reinterpret_cast<const uint32_t*>(p + 4 * i);
-    }
-}
 
 // integer dot product of one lane's 32 channels of a w-bit plane with q (hi/lo bytes)
 template <int W>
@@ -115,56 +97,40 @@ __device__ __forceinline__ int plane_dot(const uint32_t (&words)[8], const uint3
     return (ah[0] + ah[1]) * 256 + (al[0] + al[1]);
 }
 
-// acc[r][i] += b * (f - 2^(W-1)) for the lane's 32 channels of a w-bit plane.
-// Fields are taken two at a time (the same bit positions of the two 16-bit halves of a word) by
-// OR-ing them into the mantissa of a binary16 power of two whose last mantissa bit weighs
-// 2^-(W*m) for field slot m: 2^(10-Wm) + f, exactly; subtracting 2^(10-Wm) + 2^(W-1) is exact and
-// centres the code, so every slot uses the same weight.  The products go into binary32 accumulators.
+// weighted sums of one lane's 8 channels over the four tokens of a value group:
+// acc[cl] += sum_i weight_i * piece_i(channel cl); wt.x / wt.y / wt.z hold the high / middle / low bytes of the four
+// 24-bit weights
 template <int W>
-__device__ __forceinline__ void plane_axpy(const uint32_t (&words)[8], unsigned short b, float (&acc)[8][4]) {
+__device__ __forceinline__ void group_axpy(const uint32_t (&words)[8], const uint4 wt, int (&ahi)[8], int (&amd)[8], int (&alo)[8]) {
     constexpr int PER = 8 / W;
+    constexpr uint32_t MASK = 0x01010101u * ((1u << W) - 1u);
 #pragma unroll
-    for (int j = 0; j < W; ++j) {
-        const uint32_t ev = words[j];          // byte lanes 0 and 2 in the low bytes of the halves
-        const uint32_t od = words[j] >> 8;     // byte lanes 1 and 3
+    for (int k = 0; k < W; ++k) {
 #pragma unroll
         for (int m = 0; m < PER; ++m) {
-            const uint32_t mask = (((1u << W) - 1u) << (W * m)) * 0x00010001u;
-            const uint32_t magic = (0x6400u - ((uint32_t)(W * m) << 10)) * 0x00010001u;        // binary16 2^(10-Wm), twice
-            const uint32_t cen = magic + (1u << (W - 1 + W * m)) * 0x00010001u;              // ... + 2^(W-1)
-            const __half2 c2 = *reinterpret_cast<const __half2*>(&cen);
-            uint32_t xe = lop3_and_or(ev, mask, magic), xo = lop3_and_or(od, mask, magic);
-            const __half2 ye = __hsub2(*reinterpret_cast<__half2*>(&xe), c2);
-            const __half2 yo = __hsub2(*reinterpret_cast<__half2*>(&xo), c2);
-            const int r = PER * j + m;
-            fma_f32_f16(acc[r][0], __half_as_ushort(__low2half(ye)), b);
-            fma_f32_f16(acc[r][2], __half_as_ushort(__high2half(ye)), b);
-            fma_f32_f16(acc[r][1], __half_as_ushort(__low2half(yo)), b);
-            fma_f32_f16(acc[r][3], __half_as_ushort(__high2half(yo)), b);
+            const uint32_t f = (words[k] >> (W * m)) & MASK;
+            ahi[PER * k + m] = dp4a_uu(f, wt.x, ahi[PER * k + m]);
+            amd[PER * k + m] = dp4a_uu(f, wt.y, amd[PER * k + m]);
+            alo[PER * k + m] = dp4a_uu(f, wt.z, alo[PER * k + m]);
         }
     }
 }
 
-constexpr int UNIT = QAQ_TILE / 2;   // tokens a warp handles at a time (half a tile)
 constexpr int OSTAGE = 192;          // outlier entries per tile and tensor staged in shared memory
 
-// per-warp scratch for the half tile a warp is working on
+// per-warp scratch for the tile a warp is working on
 template <int D>
 struct WarpScratch {
-    alignas(16) uint8_t bufK[UNIT * D + 16];
-    alignas(16) uint8_t bufV[UNIT * D + 16];
-    float stepK[UNIT];
-    // per token of the whole tile (both halves): the tile's outlier lists are gone through once
-    float midK[2 * UNIT];       // min + step/2
-    float midV[2 * UNIT];
-    float ocorr[2 * UNIT];      // sum over a token's key outliers of q_ch * (x - mid)
-    float p[2 * UNIT];          // attention weights, kept at the current scale of the running sums
-    float wv[UNIT];             // p_t * step_t * 2^g of the value side
+    alignas(16) uint8_t bufK[QAQ_TILE * D + 16];
+    alignas(16) uint8_t bufV[(qaqc::v_tile_bytes_max(D) + 15) / 16 * 16 + 16];
+    int dotw[4][QAQ_TILE];                    // integer q . piece per section and rank
+    alignas(16) uint32_t wts[4][QAQ_TILE / 4][4];  // per section and value group: high, middle, low bytes of the four weights
+    float midK[QAQ_TILE];       // min + step/2
+    float midV[QAQ_TILE];
+    float p[QAQ_TILE];          // attention weights of the tile's tokens at the current scale of the running sums
+    int iocorr[2][QAQ_TILE];    // fixed-point sums (high, low part) of the key-outlier corrections per token
+    int ivout[2][D];            // ... of the value-outlier corrections per channel (zero between tiles)
     float vout[D];              // value-outlier corrections
-    int dot[UNIT];
-    // work items grouped by plane width (8, 4, 2, 1):
-    //   byte offset of the plane inside the half tile | shift of the piece << 16 | token << 24
-    uint32_t item[2][3 * UNIT];
     alignas(16) uint32_t outl[2][OSTAGE];   // the tile's outlier entries (K, V); longer lists continue in global memory
 };
 
@@ -178,55 +144,93 @@ struct DecSmem {
     float qscale, qsum;
 };
 
-template <int D, int W, int ALIGN>
-__device__ __forceinline__ void k_items(WarpScratch<D>& ws, int first, int n, const uint32_t (&qh)[8],
-                                        const uint32_t (&ql)[8], int part, int sub) {
+// q . piece for the items of one key section: P = D/32 lanes per item, each 32 channels
+template <int D, int W>
+__device__ __forceinline__ void k_section(const uint8_t* sec, int n, int* dots, const uint32_t (&qh)[8], const uint32_t (&ql)[8],
+                                          int part, int sub) {
     constexpr int P = D / 32, IPW = 32 / P;
 #pragma unroll 1
     for (int i0 = 0; i0 < n; i0 += IPW) {
-        uint32_t w0[8];
-        const int ia = i0 + sub;
-        const bool va = ia < n;
-        const uint32_t de = va ? ws.item[0][first + ia] : 0u;
+        const int r = i0 + sub;
         int da = 0;
-        if (va) {
-            load_words<W, ALIGN>(ws.bufK + (de & 0xFFFFu) + part * 4 * W, w0);
+        if (r < n) {
+            uint32_t w0[8];
+            qaqc::load_words<W>(sec + r * (D * W / 8) + part * 4 * W, w0);
             da = plane_dot<W>(w0, qh, ql);
         }
 #pragma unroll
         for (int o = 1; o < P; o <<= 1) da += __shfl_xor_sync(0xFFFFFFFFu, da, o);
-        if (va && part == 0) atomicAdd(&ws.dot[de >> 24], da << ((de >> 16) & 7));
+        if (r < n && part == 0) dots[r] = da;
     }
 }
 
-template <int D, int W, int ALIGN>
-__device__ __forceinline__ void v_items(WarpScratch<D>& ws, int first, int n, float (&acc)[8][4], int part, int sub) {
-    constexpr int P = D / 32, IPW = 32 / P;
+// weighted accumulation over the groups of one value section: LPG = D/8 lanes per group, each 8 channels
+template <int D, int W>
+__device__ __forceinline__ void v_section(const uint8_t* sec, int ngroups, const uint32_t (*wts)[4], int (&ahi)[8], int (&amd)[8],
+                                          int (&alo)[8], int h, int grp) {
+    constexpr int LPG = D / 8, GPW = 32 / LPG;
 #pragma unroll 1
-    for (int i0 = sub; i0 < n; i0 += IPW) {
+    for (int g = grp; g < ngroups; g += GPW) {
         uint32_t w0[8];
-        const uint32_t de = ws.item[1][first + i0];
-        load_words<W, ALIGN>(ws.bufV + (de & 0xFFFFu) + part * 4 * W, w0);
-        // weight of the piece: p_t * step_t * 2^g * 2^shift, in binary16
-        const float wt = ws.wv[de >> 24] * __int_as_float((127 + ((de >> 16) & 7)) << 23);
-        plane_axpy<W>(w0, __half_as_ushort(__float2half_rn(wt)), acc);
+        qaqc::load_words<W>(sec + g * (D * W / 2) + h * 4 * W, w0);
+        const uint4 wt = *reinterpret_cast<const uint4*>(wts[g]);
+        group_axpy<W>(w0, wt, ahi, amd, alo);
     }
+}
+
+// Sum of per-entry corrections into integer cells, independent of the order in which lanes arrive: the terms of a
+// tile's outlier list are brought to fixed point with one scale for the tile (from the largest term) and added with
+// integer atomics.  A term is split into a high part (units of 2^eu, below 2^24 of them) and the exact remainder in
+// units of 2^(eu-20), so a cell keeps about 44 bits below the largest term of the tile whatever the other cells hold.
+// term(e) gives the cell and the binary32 term of entry e; cells[0][.] / cells[1][.] take the high / low parts.
+// Returns the weight of one high unit (0: nothing was added).
+constexpr float OUTL_LO = 1048576.0f;     // 2^20 low units per high unit
+template <int NCELL, typename F>
+__device__ __forceinline__ float outlier_sums(uint32_t count, int lane, int (*cells)[NCELL], F term) {
+    float mx = 0.f;
+#pragma unroll 1
+    for (uint32_t e = lane; e < count; e += 32) {
+        int cell; float t;
+        term(e, cell, t);
+        mx = fmaxf(mx, fabsf(t));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    if (!(mx > 0.f) || !(mx < 3.0e38f)) return 0.f;        // nothing to add (or not finite: left out)
+    // largest term below 2^24 units, so that the up to 128 terms of a cell stay inside 32 bits
+    const int ex = (__float_as_int(mx) >> 23) & 0xFF;       // mx < 2^(ex-126)
+    const int eu = max(-100, min(100, ex - 126 - 24));      // one unit = 2^eu
+    const float inv = __int_as_float((127 - eu) << 23), unit = __int_as_float((127 + eu) << 23);
+#pragma unroll 1
+    for (uint32_t e = lane; e < count; e += 32) {
+        int cell; float t;
+        term(e, cell, t);
+        const float hi = rintf(t * inv);
+        const float rem = fmaf(-hi, unit, t);               // exact: |rem| <= unit / 2
+        atomicAdd(&cells[0][cell], (int)hi);
+        atomicAdd(&cells[1][cell], __float2int_rn(rem * inv * OUTL_LO));
+    }
+    return unit;
 }
 
 // One CTA = one run of consecutive tiles, which meets one or two (b,h): the body below runs once
 // per (b,h) segment and leaves one partial per segment.  Every warp works through whole tiles on its
-// own, half a tile (32 tokens) at a time: own running max / sum / accumulators, own staging
-// buffers, no CTA barrier in the loop; the warps are merged once at the end.  The packed bytes
-// of the next half tile are copied to shared memory with cp.async while the current one is being
-// processed: the keys during the value phase, the values during the key phase.
+// own: own running max / sum / accumulators, own staging buffers, no CTA barrier in the loop; the
+// warps are merged once at the end.  The packed bytes of the next tile are copied to shared memory
+// with cp.async while the current one is being processed: the keys during the value phase, the
+// values during the key phase.  Lane l looks after tokens l and l + 32 of the tile (logit, softmax
+// weight, fixed-point value weight); the section loops spread the items over the lanes.
 template <int D>
-__global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a) {
-    constexpr int P = D / 32;        // lanes per item
-    constexpr int ALIGN = D / 8 >= 16 ? 16 : D / 8;
+__global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(const DecArgs a) {
+    constexpr int P = D / 32;        // lanes per key item
+    constexpr int LPG = D / 8;       // lanes per value group
+    constexpr int HALF = QAQ_TILE / 2;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DecSmem<D>& sm = *reinterpret_cast<DecSmem<D>*>(smem_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int part = lane % P, sub = lane / P;
+    const int vh = lane % LPG, vgrp = lane / LPG;
+    const unsigned lt = (1u << lane) - 1u;
     WarpScratch<D>& ws = sm.ws[warp];
 
 #pragma unroll 1
@@ -255,7 +259,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
         qs += __shfl_xor_sync(0xFFFFFFFFu, qs, o);
     }
     if (lane == 0) { sm.red[warp] = qmax; sm.red2[warp] = qs; }
-    for (int d = lane; d < D; d += 32) ws.vout[d] = 0.f;
+    for (int d = lane; d < D; d += 32) { ws.vout[d] = 0.f; ws.ivout[0][d] = 0; ws.ivout[1][d] = 0; }
     __syncthreads();
     if (tid == 0) {
         float m = 0.f, s = 0.f;
@@ -280,16 +284,11 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
         qh[r] = h; ql[r] = l;
     }
 
-    float acc[8][4];
+    float X[8];                 // this lane's 8 channels (8*vh ..), summed over the groups this lane has handled
 #pragma unroll
-    for (int r = 0; r < 8; ++r)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc[r][i] = 0.f;
+    for (int i = 0; i < 8; ++i) X[i] = 0.f;
     float m_run = __int_as_float(0xff800000), l_run = 0.f, lx_run = 0.f;   // lx: sum of the unperturbed p
-    float c_run = 0.f;       // per-lane part of sum_t p_t * (constant part of the token's values)
-    // The binary16 weights of the value side carry a common power-of-two factor 2^g so that the
-    // largest possible weight (range/2) sits near 2^12; g only ever decreases.
-    int g_run = 24;
+    float c_run = 0.f;       // per-lane part of sum_t p_t * (min_t + step_t/2) of the values
 
     const size_t trow = (size_t)bh * a.ntiles_max;
     const size_t mrow = (size_t)bh * a.tmax_pad;
@@ -315,263 +314,237 @@ __global__ void __launch_bounds__(DEC_THREADS, 4) decode_kernel(const DecArgs a)
         }
         return m;
     };
-    // bytes of the first half (tokens 0..31) of a tile, per tensor (slots beyond T have width 0)
-    auto first_half_bytes = [&](const Meta& m, uint32_t& hK, uint32_t& hV) {
-        uint32_t k = (m.bits4 & 0xFF) * (D / 8), v = ((m.bits4 >> 16) & 0xFF) * (D / 8);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            k += __shfl_xor_sync(0xFFFFFFFFu, k, o);
-            v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-        }
-        hK = k; hV = v;
-    };
-    auto stage = [&](uint8_t* dst, const uint8_t* src, uint32_t nbytes) {
+    // a tile's bytes (rounded up to 16, never more than the buffer holds) and its outlier entries
+    auto stage = [&](uint8_t* dst, const uint8_t* pool, uint32_t off, uint32_t nbytes, uint32_t cap) {
+        nbytes = (min(nbytes, cap) + 15u) & ~15u;
+        if ((size_t)off + nbytes > a.pool_bytes) nbytes = 0;      // a table entry that points outside the pool is not followed
 #pragma unroll 1
-        for (uint32_t o = lane * ALIGN; o < nbytes; o += 32 * ALIGN) cp_async<ALIGN>(dst + o, src + o);
+        for (uint32_t o = lane * 16; o < nbytes; o += 32 * 16) cp_async<16>(dst + o, pool + off + o);
     };
-
     auto stage_outl = [&](int x, uint32_t first, uint32_t count) {   // entries are 4 bytes, lists start 16-byte aligned
         const uint32_t* src = (x ? a.v.outl : a.k.outl) + (size_t)bh * a.ocap + first;
         const uint32_t n16 = ((count < (uint32_t)OSTAGE ? count : (uint32_t)OSTAGE) + 3u) >> 2;
+        if ((size_t)first + 4 * n16 > a.ocap) return;
 #pragma unroll 1
         for (uint32_t o = lane; o < n16; o += 32) cp_async<16>(&ws.outl[x][4 * o], src + 4 * o);
+    };
+    auto stage_K = [&](const Meta& m) {
+        stage(ws.bufK, poolK, __shfl_sync(0xFFFFFFFFu, m.tb, 0), __shfl_sync(0xFFFFFFFFu, m.tb, 1), QAQ_TILE * D);
+        stage_outl(0, __shfl_sync(0xFFFFFFFFu, m.tb, 2), __shfl_sync(0xFFFFFFFFu, m.tb, 3));
+        cp_async_commit();
+    };
+    auto stage_V = [&](const Meta& m) {
+        stage(ws.bufV, poolV, __shfl_sync(0xFFFFFFFFu, m.tb, 4), __shfl_sync(0xFFFFFFFFu, m.tb, 5), (uint32_t)sizeof(ws.bufV) - 16u);
+        stage_outl(1, __shfl_sync(0xFFFFFFFFu, m.tb, 6), __shfl_sync(0xFFFFFFFFu, m.tb, 7));
+        cp_async_commit();
     };
     int tile = tile_lo + warp;
     Meta cur = fetch_meta(tile);
     Meta nxt = fetch_meta(tile + DEC_WARPS);
-    uint32_t h0K = 0, h0V = 0;
-    first_half_bytes(cur, h0K, h0V);
-    if (tile < tile_hi) {
-        stage(ws.bufK, poolK + __shfl_sync(0xFFFFFFFFu, cur.tb, 0), h0K);
-        stage_outl(0, __shfl_sync(0xFFFFFFFFu, cur.tb, 2), __shfl_sync(0xFFFFFFFFu, cur.tb, 3));
-        cp_async_commit();
-        stage(ws.bufV, poolV + __shfl_sync(0xFFFFFFFFu, cur.tb, 4), h0V);
-        stage_outl(1, __shfl_sync(0xFFFFFFFFu, cur.tb, 6), __shfl_sync(0xFFFFFFFFu, cur.tb, 7));
-        cp_async_commit();
-    }
+    if (tile < tile_hi) { stage_K(cur); stage_V(cur); }
 
     for (; tile < tile_hi; tile += DEC_WARPS) {
-        const uint32_t offK = __shfl_sync(0xFFFFFFFFu, cur.tb, 0), totK = __shfl_sync(0xFFFFFFFFu, cur.tb, 1);
         const uint32_t ooK = __shfl_sync(0xFFFFFFFFu, cur.tb, 2), ocK = __shfl_sync(0xFFFFFFFFu, cur.tb, 3);
-        const uint32_t offV = __shfl_sync(0xFFFFFFFFu, cur.tb, 4), totV = __shfl_sync(0xFFFFFFFFu, cur.tb, 5);
         const uint32_t ooV = __shfl_sync(0xFFFFFFFFu, cur.tb, 6), ocV = __shfl_sync(0xFFFFFFFFu, cur.tb, 7);
         const bool has_next = tile + DEC_WARPS < tile_hi;
-        uint32_t n0K = 0, n0V = 0;   // first-half bytes of the next tile
+        const int t0 = tile * QAQ_TILE + lane;              // this lane's tokens: t0 and t0 + 32
+        const bool val0 = t0 < a.T, val1 = t0 + HALF < a.T;
 
-#pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-            const int t = tile * QAQ_TILE + UNIT * half + lane;   // this lane's token
-            const bool valid = t < a.T;
-            // ---- per-token scalars, byte offsets inside the half tile, item lists
-            int ncls[2][4];
-            float rngV = 0.f, cstV = 0.f;
+        // ---- widths, ranks of this lane's tokens in the sections, section sizes
+        int B[2][2];          // [tensor][token]
+        uint32_t rk[2][2];    // rank in section c in byte c
+        int n[2][4];
 #pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                const int B = valid ? (int)((cur.bits4 >> (16 * x + 8 * half)) & 0xFF) : 0;
-                const uint32_t len = (uint32_t)(D * B / 8);
-                const uint32_t mmw = half ? cur.mm[2 * x + 1] : cur.mm[2 * x];
-                const float mn = __half2float(__ushort_as_half((unsigned short)(mmw & 0xFFFF)));
-                const float mx = __half2float(__ushort_as_half((unsigned short)(mmw >> 16)));
-                const float rng = valid ? __fsub_rn(mx, mn) : 0.f;
-                const float st = __fmul_rn(rng, __int_as_float((127 - B) << 23));
-                const float mid = fmaf(0.5f, st, mn);
-                if (x == 0) {
-                    ws.stepK[lane] = st;
-                    ws.dot[lane] = 0;
-                    if (half == 0) {
-                        ws.midK[lane] = valid ? mid : 0.f;
-                        ws.ocorr[lane] = 0.f;
-                        // the lane's token of the second half: its mid is needed already, because all key outliers of
-                        // the tile are gone through in this half
-                        const bool valid2 = t + UNIT < a.T;
-                        const int B2 = valid2 ? (int)((cur.bits4 >> 8) & 0xFF) : 0;
-                        const float mn2 = __half2float(__ushort_as_half((unsigned short)(cur.mm[1] & 0xFFFF)));
-                        const float mx2 = __half2float(__ushort_as_half((unsigned short)(cur.mm[1] >> 16)));
-                        const float st2 = __fmul_rn(valid2 ? __fsub_rn(mx2, mn2) : 0.f, __int_as_float((127 - B2) << 23));
-                        ws.midK[UNIT + lane] = valid2 ? fmaf(0.5f, st2, mn2) : 0.f;
-                        ws.ocorr[UNIT + lane] = 0.f;
-                    }
-                } else {
-                    // centred planes: piece w contributes a constant step * 2^((B & (2w-1)) - 1)
-                    float cst = 0.5f;
+        for (int x = 0; x < 2; ++x) {
+            B[x][0] = val0 ? min(8, (int)((cur.bits4 >> (16 * x)) & 0xFF)) : 0;
+            B[x][1] = val1 ? min(8, (int)((cur.bits4 >> (16 * x + 8)) & 0xFF)) : 0;
+            rk[x][0] = rk[x][1] = 0;
 #pragma unroll
-                    for (int w = 8; w >= 1; w >>= 1)
-                        if (B & w) cst += __int_as_float((127 + (B & (2 * w - 1)) - 1) << 23);
-                    ws.midV[UNIT * half + lane] = valid ? mid : 0.f;       // value of a zero code slot (outliers)
-                    cstV = valid ? fmaf(cst, st, mn) : 0.f;                 // constant part, picked up below
-                    ws.wv[lane] = st;                                       // step for now, weight after the softmax
-                    rngV = rng;
-                }
-                uint32_t inc = len;
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-                    if (lane >= d) inc += u;
-                }
-                const uint32_t toff = inc - len;
-                int base = 0;
-                const unsigned lt = (1u << lane) - 1u;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int w = 8 >> c;
-                    const unsigned bal = __ballot_sync(0xFFFFFFFFu, (B & w) != 0);
-                    if (B & w) {
-                        const uint32_t plane = toff + (uint32_t)((B & ~(2 * w - 1)) * (D / 8));
-                        ws.item[x][base + __popc(bal & lt)] = plane | ((uint32_t)(B & (w - 1)) << 16) | ((uint32_t)lane << 24);
-                    }
-                    ncls[x][c] = __popc(bal);
-                    base += ncls[x][c];
-                }
+            for (int c = 0; c < 4; ++c) {
+                const unsigned b0 = __ballot_sync(0xFFFFFFFFu, (B[x][0] & (8 >> c)) != 0);
+                const unsigned b1 = __ballot_sync(0xFFFFFFFFu, (B[x][1] & (8 >> c)) != 0);
+                const int n0 = __popc(b0);
+                n[x][c] = n0 + __popc(b1);
+                rk[x][0] |= (uint32_t)__popc(b0 & lt) << (8 * c);
+                rk[x][1] |= (uint32_t)(n0 + __popc(b1 & lt)) << (8 * c);
             }
-            // common exponent of the value weights
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) rngV = fmaxf(rngV, __shfl_xor_sync(0xFFFFFFFFu, rngV, o));
-            {
-                const int e = rngV > 0.f ? ((__float_as_int(rngV) >> 23) & 0xFF) - 127 : -12;
-                const int g = 12 - e;
-                if (g < g_run) {
-                    const float f = __int_as_float((127 + g - g_run) << 23);
-#pragma unroll
-                    for (int r = 0; r < 8; ++r)
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) acc[r][i] *= f;
-                    g_run = g;
-                }
-            }
-            cp_async_wait<1>();     // this half's keys have landed (its values may still be in flight)
-            __syncwarp();
-
-            // ---- K: integer dot products per (token, plane), outlier corrections
-            {
-                int first = 0;
-                k_items<D, 8, ALIGN>(ws, first, ncls[0][0], qh, ql, part, sub); first += ncls[0][0];
-                k_items<D, 4, ALIGN>(ws, first, ncls[0][1], qh, ql, part, sub); first += ncls[0][1];
-                k_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, first, ncls[0][2], qh, ql, part, sub); first += ncls[0][2];
-                k_items<D, 1, 4>(ws, first, ncls[0][3], qh, ql, part, sub);
-                // all key outliers of the tile, once, while its first half is worked on
-                if (half == 0) {
-                    const uint32_t* og = a.k.outl + (size_t)bh * a.ocap + ooK;
-#pragma unroll 1
-                    for (uint32_t e0 = 0; e0 < ocK; e0 += 32) {
-                        const uint32_t e = e0 + lane;
-                        if (e < ocK) {
-                            const uint32_t v = e < (uint32_t)OSTAGE ? ws.outl[0][e] : __ldg(og + e);
-                            const int tok = v >> 24, ch = (v >> 16) & 0xFF;
-                            const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
-                            atomicAdd(&ws.ocorr[tok], sm.qf[ch] * (val - ws.midK[tok]));
-                        }
-                    }
-                }
-            }
-            __syncwarp();
-            // ---- the key buffer is free: start the copy of the next unit's keys
-            if (half == 0) {
-                stage(ws.bufK, poolK + offK + h0K, totK - h0K);
-            } else if (has_next) {
-                first_half_bytes(nxt, n0K, n0V);
-                stage(ws.bufK, poolK + __shfl_sync(0xFFFFFFFFu, nxt.tb, 0), n0K);
-                stage_outl(0, __shfl_sync(0xFFFFFFFFu, nxt.tb, 2), __shfl_sync(0xFFFFFFFFu, nxt.tb, 3));
-            }
-            cp_async_commit();
-
-            // ---- logit of this lane's token; running max / sum; weights
-            {
-                float lg = __int_as_float(0xff800000);
-                if (valid) {
-                    const float qk = fmaf(qscale * ws.stepK[lane], (float)ws.dot[lane], fmaf(ws.midK[UNIT * half + lane], qsum, ws.ocorr[UNIT * half + lane]));
-                    lg = a.scale * qk;
-                    if (a.scores) a.scores[(size_t)bh * a.T + t] = lg;
-                }
-                float m = lg;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-                const float m_new = fmaxf(m_run, m);
-                const float alpha = __expf(m_run - m_new);   // 0 on the first unit (m_run = -inf)
-                m_run = m_new;
-                if (alpha != 1.0f) {
-#pragma unroll
-                    for (int r = 0; r < 8; ++r)
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) acc[r][i] *= alpha;
-                    c_run *= alpha;
-                    for (int d = lane; d < D; d += 32) ws.vout[d] *= alpha;
-                    if (half == 1) ws.p[lane] *= alpha;       // the first half's weights follow the new scale
-                }
-                float p = __expf(lg - m_new);                // 0 for slots beyond T
-                float sx = p;
-                // The value weight p * step * 2^g is used in binary16.  It is rounded to 11 significant
-                // bits here, once, and p is adjusted by the same factor, so that the planes, the constant
-                // part and the softmax denominator all see the same (slightly perturbed) probability.
-                const float wfull = p * ws.wv[lane] * __int_as_float((127 + g_run) << 23);
-                const float big = __fmul_rn(wfull, 8193.0f);  // 2^13 + 1: splits off the upper 11 bits (no contraction)
-                const float wr = __fsub_rn(big, __fsub_rn(big, wfull));
-                if (wfull > 0.f) p *= __fdividef(wr, wfull);
-                ws.wv[lane] = wr;
-                c_run = fmaf(p, cstV, c_run);
-                float s = p;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-                    sx += __shfl_xor_sync(0xFFFFFFFFu, sx, o);
-                }
-                l_run = l_run * alpha + s;
-                lx_run = lx_run * alpha + sx;
-                ws.p[UNIT * half + lane] = p;
-            }
-            cp_async_wait<1>();     // this half's values have landed
-            __syncwarp();
-
-            // ---- V: weighted accumulation of centred codes, outlier corrections
-            {
-                int first = 0;
-                v_items<D, 8, ALIGN>(ws, first, ncls[1][0], acc, part, sub); first += ncls[1][0];
-                v_items<D, 4, ALIGN>(ws, first, ncls[1][1], acc, part, sub); first += ncls[1][1];
-                v_items<D, 2, (ALIGN > 8 ? 8 : ALIGN)>(ws, first, ncls[1][2], acc, part, sub); first += ncls[1][2];
-                v_items<D, 1, 4>(ws, first, ncls[1][3], acc, part, sub);
-                // all value outliers of the tile, once, when the weights of both halves are known
-                if (half == 1) {
-                    const uint32_t* og = a.v.outl + (size_t)bh * a.ocap + ooV;
-#pragma unroll 1
-                    for (uint32_t e0 = 0; e0 < ocV; e0 += 32) {
-                        const uint32_t e = e0 + lane;
-                        if (e < ocV) {
-                            const uint32_t v = e < (uint32_t)OSTAGE ? ws.outl[1][e] : __ldg(og + e);
-                            const int tok = v >> 24, ch = (v >> 16) & 0xFF;
-                            const float val = __half2float(__ushort_as_half((unsigned short)(v & 0xFFFF)));
-                            atomicAdd(&ws.vout[ch], ws.p[tok] * (val - ws.midV[tok]));
-                        }
-                    }
-                }
-            }
-            __syncwarp();
-            // ---- the value buffer is free: start the copy of the next unit's values
-            if (half == 0) stage(ws.bufV, poolV + offV + h0V, totV - h0V);
-            else if (has_next) {
-                stage(ws.bufV, poolV + __shfl_sync(0xFFFFFFFFu, nxt.tb, 4), n0V);
-                stage_outl(1, __shfl_sync(0xFFFFFFFFu, nxt.tb, 6), __shfl_sync(0xFFFFFFFFu, nxt.tb, 7));
-            }
-            cp_async_commit();
         }
+        uint32_t kb[5], vb[5];
+        qaqc::section_bases<D, false>(n[0], kb);
+        qaqc::section_bases<D, true>(n[1], vb);
+
+        // ---- per-token scalars
+        float stepK[2], stepV[2], midV[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const bool v = j ? val1 : val0;
+            const uint32_t mk = cur.mm[j], mv = cur.mm[2 + j];
+            const float kmn = __half2float(__ushort_as_half((unsigned short)(mk & 0xFFFF)));
+            const float kmx = __half2float(__ushort_as_half((unsigned short)(mk >> 16)));
+            const float vmn = __half2float(__ushort_as_half((unsigned short)(mv & 0xFFFF)));
+            const float vmx = __half2float(__ushort_as_half((unsigned short)(mv >> 16)));
+            stepK[j] = v ? qaqc::step_of(kmn, kmx, B[0][j]) : 0.f;
+            stepV[j] = v ? qaqc::step_of(vmn, vmx, B[1][j]) : 0.f;
+            ws.midK[lane + HALF * j] = v ? fmaf(0.5f, stepK[j], kmn) : 0.f;
+            midV[j] = v ? fmaf(0.5f, stepV[j], vmn) : 0.f;
+            ws.midV[lane + HALF * j] = midV[j];
+            ws.iocorr[0][lane + HALF * j] = 0;
+            ws.iocorr[1][lane + HALF * j] = 0;
+        }
+        cp_async_wait<1>();     // this tile's keys have landed (its values may still be in flight)
+        __syncwarp();
+
+        // ---- K: integer dot products per section
+        k_section<D, 8>(ws.bufK + kb[0], n[0][0], ws.dotw[0], qh, ql, part, sub);
+        k_section<D, 4>(ws.bufK + kb[1], n[0][1], ws.dotw[1], qh, ql, part, sub);
+        k_section<D, 2>(ws.bufK + kb[2], n[0][2], ws.dotw[2], qh, ql, part, sub);
+        k_section<D, 1>(ws.bufK + kb[3], n[0][3], ws.dotw[3], qh, ql, part, sub);
+        // key outliers: q_ch * (x - mid) per token
+        const uint32_t* ogK = a.k.outl + (size_t)bh * a.ocap + ooK;
+        const float ounit = outlier_sums(ocK, lane, ws.iocorr, [&](uint32_t e, int& cell, float& t) {
+            const uint32_t v = e < (uint32_t)OSTAGE ? ws.outl[0][e] : __ldg(ogK + e);
+            cell = (v >> 24) & (QAQ_TILE - 1);
+            t = sm.qf[(v >> 16) & (D - 1)] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midK[cell]);
+        });
+        __syncwarp();
+        // ---- the key buffer is free: start the copy of the next tile's keys
+        if (has_next) stage_K(nxt); else cp_async_commit();
+
+        // ---- logits of this lane's tokens; running max / sum
+        float lg[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            int dot = 0;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int w = 8 >> c;
+                if (B[0][j] & w) dot += ws.dotw[c][(rk[0][j] >> (8 * c)) & 0xFF] << (B[0][j] & (w - 1));
+            }
+            lg[j] = __int_as_float(0xff800000);
+            if (j ? val1 : val0) {
+                const int tk = lane + HALF * j;
+                const float qk = fmaf(qscale * stepK[j], (float)dot, fmaf(ws.midK[tk], qsum, ounit * fmaf((float)ws.iocorr[1][tk], 1.0f / OUTL_LO, (float)ws.iocorr[0][tk])));
+                lg[j] = a.scale * qk;
+                if (a.scores) a.scores[(size_t)bh * a.T + t0 + HALF * j] = lg[j];
+            }
+        }
+        float m = fmaxf(lg[0], lg[1]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+        const float m_new = fmaxf(m_run, m);
+        const float alpha = __expf(m_run - m_new);   // 0 on the first tile (m_run = -inf)
+        m_run = m_new;
+        if (alpha != 1.0f) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) X[i] *= alpha;
+            c_run *= alpha;
+            for (int d = lane; d < D; d += 32) ws.vout[d] *= alpha;
+        }
+        // ---- value weights p * step * 2^shift as 24-bit fixed point with one scale for the tile (a token's step
+        //      falls with its width, so next to a 2-bit token an 8-bit token of the same p has a weight 64 times
+        //      smaller: 16 bits would leave it about 10).  The weight of the
+        //      token's lowest piece is rounded once; the other pieces use exact multiples of it, and p is replaced
+        //      by what the rounded weight stands for, so that the pieces, the constant part and the softmax
+        //      denominator all see the same (slightly perturbed) probability.
+        float pe[2], wf[2];
+        int top[2];
+        float wmax = 0.f;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            pe[j] = __expf(lg[j] - m_new);           // 0 for slots beyond T
+            wf[j] = pe[j] * stepV[j];
+            const int Bv = B[1][j];
+            top[j] = Bv ? Bv - (1 << (31 - __clz(Bv))) : 0;      // shift of the widest piece
+            wmax = fmaxf(wmax, wf[j] * __int_as_float((127 + top[j]) << 23));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) wmax = fmaxf(wmax, __shfl_xor_sync(0xFFFFFFFFu, wmax, o));
+        // wmax < 2^(ex-126): one unit = 2^(ex-126-24) keeps every shifted weight below 2^24
+        const int wex = (__float_as_int(wmax) >> 23) & 0xFF;
+        const bool wok = wex > 24 && wex < 255;                    // zero, tiny or non-finite weights: the pieces add nothing
+        const float wunit = wok ? __int_as_float((wex - 23) << 23) : 0.f;
+        const float winv = wok ? __int_as_float((254 - (wex - 23)) << 23) : 0.f;
+        float s = 0.f, sx = 0.f;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int Bv = B[1][j];
+            uint32_t iw = (uint32_t)__float2int_rn(wf[j] * winv);
+            iw = min(iw, 0xFFFFFFu >> top[j]);
+            float p = pe[j];
+            if (stepV[j] > 0.f && wok) p = __fdividef((float)iw * wunit, stepV[j]);
+            uint8_t* wb = reinterpret_cast<uint8_t*>(ws.wts);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int w = 8 >> c;
+                if (Bv & w) {
+                    const uint32_t r = (rk[1][j] >> (8 * c)) & 0xFF, wt = iw << (Bv & (w - 1));
+                    uint8_t* g = wb + c * (QAQ_TILE / 4) * 16 + (r >> 2) * 16 + (r & 3);
+                    g[0] = (uint8_t)(wt >> 16);
+                    g[4] = (uint8_t)(wt >> 8);
+                    g[8] = (uint8_t)wt;
+                }
+            }
+            c_run = fmaf(p, midV[j], c_run);
+            s += p; sx += pe[j];
+            ws.p[lane + HALF * j] = p;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+            sx += __shfl_xor_sync(0xFFFFFFFFu, sx, o);
+        }
+        l_run = l_run * alpha + s;
+        lx_run = lx_run * alpha + sx;
+        cp_async_wait<1>();     // this tile's values have landed
+        __syncwarp();
+
+        // ---- V: integer weighted sums per section, added to the binary32 accumulators once per tile
+        if (wok) {
+            int ahi[8], amd[8], alo[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { ahi[i] = 0; amd[i] = 0; alo[i] = 0; }
+            v_section<D, 8>(ws.bufV + vb[0], (n[1][0] + 3) >> 2, ws.wts[0], ahi, amd, alo, vh, vgrp);
+            v_section<D, 4>(ws.bufV + vb[1], (n[1][1] + 3) >> 2, ws.wts[1], ahi, amd, alo, vh, vgrp);
+            v_section<D, 2>(ws.bufV + vb[2], (n[1][2] + 3) >> 2, ws.wts[2], ahi, amd, alo, vh, vgrp);
+            v_section<D, 1>(ws.bufV + vb[3], (n[1][3] + 3) >> 2, ws.wts[3], ahi, amd, alo, vh, vgrp);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                X[i] = fmaf(fmaf((float)ahi[i], 65536.0f, (float)(amd[i] * 256 + alo[i])), wunit, X[i]);
+        }
+        // value outliers: p_t * (v - mid) per channel
+        const uint32_t* ogV = a.v.outl + (size_t)bh * a.ocap + ooV;
+        const float vunit = outlier_sums(ocV, lane, ws.ivout, [&](uint32_t e, int& cell, float& t) {
+            const uint32_t v = e < (uint32_t)OSTAGE ? ws.outl[1][e] : __ldg(ogV + e);
+            const int tok = (v >> 24) & (QAQ_TILE - 1);
+            cell = (v >> 16) & (D - 1);
+            t = ws.p[tok] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midV[tok]);
+        });
+        __syncwarp();
+        if (vunit != 0.f) {
+            for (int d = lane; d < D; d += 32) {
+                ws.vout[d] = fmaf(fmaf((float)ws.ivout[1][d], 1.0f / OUTL_LO, (float)ws.ivout[0][d]), vunit, ws.vout[d]);
+                ws.ivout[0][d] = 0; ws.ivout[1][d] = 0;
+            }
+        }
+        __syncwarp();
+        // ---- the value buffer is free: start the copy of the next tile's values
+        if (has_next) stage_V(nxt); else cp_async_commit();
         cur = nxt;
-        h0K = n0K; h0V = n0V;
         nxt = fetch_meta(tile + 2 * DEC_WARPS);
     }
     cp_async_wait<0>();
 
-    // ---- warp result: lanes with the same part hold partial sums of the same channels
+    // ---- warp result: lanes with the same vh hold partial sums of the same channels
     float cs = c_run;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) cs += __shfl_xor_sync(0xFFFFFFFFu, cs, o);
-    const float unscale = __int_as_float((127 - g_run) << 23);
 #pragma unroll
-    for (int r = 0; r < 8; ++r)
+    for (int i = 0; i < 8; ++i) {
+        float v = X[i];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float v = acc[r][i];
-#pragma unroll
-            for (int o = P; o < 32; o <<= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-            if (sub == 0) sm.macc[warp][32 * part + 4 * r + i] = fmaf(v, unscale, ws.vout[32 * part + 4 * r + i] + cs);
-        }
+        for (int o = LPG; o < 32; o <<= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        if (vgrp == 0) sm.macc[warp][8 * vh + i] = v + ws.vout[8 * vh + i] + cs;
+    }
     if (lane == 0) { sm.mm[warp] = m_run; sm.ml[warp] = l_run; sm.mlx[warp] = lx_run; }
     __syncthreads();
     // ---- merge the warps (log-sum-exp) into this segment's partial
@@ -636,7 +609,7 @@ __global__ void scores_kernel(float* scores, const float* ml, int T) {
 // The flattened sequence of BH * ntiles tiles is cut into runs of `run` consecutive tiles, one CTA
 // each: enough CTAs to fill every SM (148 SMs, 4 resident CTAs each) evenly, at least one tile per
 // warp where there are that many, and never more than one (b,h) boundary inside a run.
-constexpr int DEC_SLOTS = 148 * 4;
+constexpr int DEC_SLOTS = 148 * DEC_CTAS_PER_SM;
 struct DecPlan { int run, ncta; };
 DecPlan plan_decode(int BH, int ntiles) {
     const long long total = (long long)BH * ntiles;

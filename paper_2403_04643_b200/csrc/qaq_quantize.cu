@@ -6,10 +6,14 @@
 //   phase 0  attention-window maximum of the score rows (Section 4.2)
 //   phase 1  outlier masks and min/max of the non-outliers in binary16 pair arithmetic
 //            (exact: the inputs are binary16), width from the exponents (Section 4.1)
-//   phase 2  warp 0: exclusive scans of byte lengths and outlier counts over the tile,
-//            space taken from the (b,h) pools by atomicAdd
-//   phase 3  codes (binary32: one sub, one mul, round down), planes built lane-locally,
-//            vector stores; outlier entries placed by popc ranks
+//   phase 2  warp 0: which slots have a piece of each width (ballots), section sizes of the tile,
+//            exclusive scan of the outlier counts, space taken from the (b,h) pools by atomicAdd
+//   phase 3  codes (binary32: one sub, one mul, round down), pieces written into a shared-memory
+//            image of the tile in the section layout of qaq_codec.cuh, vector stores; outlier
+//            entries placed by popc ranks
+// A tile that is continued (an append behind a partly filled tile) is built anew: the codes of
+// its old tokens are read back from the pool, the image of old and new tokens replaces it.
+#include "qaq_codec.cuh"
 #include "qaq_internal.cuh"
 
 namespace {
@@ -40,22 +44,7 @@ struct QuantArgs {
     uint8_t* out_bitsV;
 };
 
-// B = min{b in [bmin,bmax] : v <= c * 2^b}, bmax if none; c * 2^b is an exact power-of-two
-// scaling.  For positive normal v and c the answer is read off the exponents: with
-// v = mv * 2^ev, c = mc * 2^ec (mv, mc in [1,2)) the smallest b is ev - ec if mv <= mc,
-// else ev - ec + 1.
-__device__ __forceinline__ int ladder(float v, float c, int bmin, int bmax) {
-    if (!(c > 0.f)) return bmax;
-    if (v <= __fmul_rn(c, (float)(1 << bmin))) return bmin;
-    const int vb = __float_as_int(v), cb = __float_as_int(c);
-    if (cb < 0x00800000 || vb < 0x00800000) {  // subnormal operand: plain ladder
-        for (int b = bmin; b <= bmax; ++b)
-            if (v <= __fmul_rn(c, (float)(1 << b))) return b;
-        return bmax;
-    }
-    int b = (vb >> 23) - (cb >> 23) + (((vb & 0x7FFFFF) > (cb & 0x7FFFFF)) ? 1 : 0);
-    return b < bmin ? bmin : (b > bmax ? bmax : b);
-}
+using qaqc::ladder;
 
 __device__ __forceinline__ uint32_t lop3_sel(uint32_t a, uint32_t m, uint32_t c) {  // (a & m) | (c & ~m)
     uint32_t d;
@@ -67,20 +56,8 @@ __device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t
     asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
 }
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
 __device__ __forceinline__ __half2 as_h2(uint32_t x) { return *reinterpret_cast<__half2*>(&x); }
 __device__ __forceinline__ uint32_t as_u32(__half2 x) { return *reinterpret_cast<uint32_t*>(&x); }
-// binary32 (x - c) with x a binary16 value: one rounding, same as widening x exactly and subtracting
-__device__ __forceinline__ float sub_f32_f16(unsigned short x, float c) {
-    float d;
-    asm("sub.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
-    return d;
-}
-
 // One lane's 32 channels of one token and tensor: outlier masks, masked min / max.
 //   v[k] holds channels 2k, 2k+1 (binary16 pairs).  On return every outlier entry of v has
 //   been replaced by -inf: in the code computation that yields code byte 0 without a mask
@@ -103,29 +80,22 @@ __device__ __forceinline__ void analyze32(uint32_t (&v)[16], __half2 lo2, __half
     mx2 = as_h2(mxacc);
 }
 
-template <int BYTES>
-__device__ __forceinline__ void store_words(uint8_t* dst, const uint32_t* w, int nwords) {
-    // nwords * 4 bytes to dst, which is BYTES-aligned (BYTES in {4, 8, 16})
-    if (BYTES == 16 && nwords % 4 == 0) {
-        for (int i = 0; i < nwords; i += 4) *reinterpret_cast<uint4*>(dst + 4 * i) = make_uint4(w[i], w[i + 1], w[i + 2], w[i + 3]);
-    } else if (BYTES >= 8 && nwords % 2 == 0) {
-        for (int i = 0; i < nwords; i += 2) *reinterpret_cast<uint2*>(dst + 4 * i) = make_uint2(w[i], w[i + 1]);
-    } else {
-        for (int i = 0; i < nwords; ++i) *reinterpret_cast<uint32_t*>(dst + 4 * i) = w[i];
-    }
-}
-
 // space from a (b,h) pool: `whole` tiles take a rounded-up amount in one atomic; a tile that is
-// being continued takes the exact amount and is padded to the unit when it closes
-__device__ __forceinline__ uint32_t pool_take(uint32_t* pool, uint32_t amount, uint32_t unit_mask, bool whole, bool closes) {
+// being continued takes the exact amount and is padded to the unit when it closes.  `taken` is
+// what the pool end moved by (to be given back if the space turns out not to fit).
+__device__ __forceinline__ uint32_t pool_take(uint32_t* pool, uint32_t amount, uint32_t unit_mask, bool whole, bool closes,
+                                              uint32_t& taken) {
     uint32_t base;
     if (whole) {
-        base = atomicAdd(pool, (amount + unit_mask) & ~unit_mask);
+        taken = (amount + unit_mask) & ~unit_mask;
+        base = atomicAdd(pool, taken);
     } else {
         base = atomicAdd(pool, amount);
+        taken = amount;
         if (closes) {
             const uint32_t pad = (0u - (base + amount)) & unit_mask;
             if (pad) atomicAdd(pool, pad);
+            taken += pad;
         }
     }
     return base;
@@ -134,17 +104,19 @@ __device__ __forceinline__ uint32_t pool_take(uint32_t* pool, uint32_t amount, u
 // One CTA = one tile of 64 tokens of one (b,h); P = D/32 lanes own a token, each lane 32
 // consecutive channels (64 bytes) of K and of V, kept in registers across all phases.
 // Order of work (barriers in brackets): loads, attention window, outlier masks and ranges,
-// widths [A] warp 0 scans the tile and takes pool space with four atomics in flight at once
-// while every warp computes its codes [B] planes into a shared-memory image of the tile
-// [C] the image goes out with 16-byte stores; outlier entries and per-token metadata follow.
+// widths [A] warp 0 finds the section sizes of the tile, scans the outlier counts and takes pool
+// space with four atomics in flight at once while every warp computes its codes [B] pieces into a
+// shared-memory image of the tile [C] the image goes out with 16-byte stores; outlier entries and
+// per-token metadata follow.  Slots below the first new token of a continued tile hold the tile's
+// old tokens: their widths come from the metadata, their codes from the tile as it is stored.
 // XSEL: -1 = keys and values in one CTA; 0 / 1 = this launch handles only the keys / only the values of a tile
 // (half the registers and shared memory per CTA, so more tiles are in flight per SM).
 template <int D, bool SELECT_ONLY, int XSEL>
 __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 128 ? 5 : 6)) quant_kernel(const QuantArgs a) {
     constexpr int X0 = XSEL < 0 ? 0 : XSEL, X1 = XSEL < 0 ? 2 : XSEL + 1;
     constexpr int P = D / 32;            // lanes per token
-    constexpr int ALIGN = D / 8 >= 16 ? 16 : D / 8;  // alignment of a token's bytes inside a tile
     constexpr int NT = 2 * D;            // threads
+    constexpr int IMG = qaqc::v_tile_bytes_max(D);
     const int bh = blockIdx.y;
     const int tile = a.first_tile + blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -153,17 +125,21 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
     const int abs_lo = max(tile * QAQ_TILE, a.t_old + a.tok_lo);
     const int abs_hi = min((tile + 1) * QAQ_TILE, a.t_old + a.tok_hi);
     const int s_lo = abs_lo - tile * QAQ_TILE, s_hi = abs_hi - tile * QAQ_TILE;
-    const bool valid = slot >= s_lo && slot < s_hi;
-    const int tn = tile * QAQ_TILE + slot - a.t_old;  // index among the new tokens
+    const bool valid = slot >= s_lo && slot < s_hi;       // a new token
+    const bool old = !SELECT_ONLY && slot < s_lo;         // a token the tile already holds
+    const int tn = tile * QAQ_TILE + slot - a.t_old;      // index among the new tokens
 
-    __shared__ uint32_t s_len[2][QAQ_TILE];   // bytes, then exclusive byte offsets
-    __shared__ uint32_t s_cnt[2][QAQ_TILE];   // outlier counts, then exclusive offsets
+    __shared__ uint8_t s_bits[2][QAQ_TILE];   // widths of the tile's slots (0: empty)
+    __shared__ uint32_t s_cnt[2][QAQ_TILE];   // outlier counts of the new tokens, then exclusive offsets
+    __shared__ qaqc::TileMasks s_tm[2];
     __shared__ uint32_t s_tot[2], s_base[2], s_obase[2], s_olimit[2];
     __shared__ int s_skip;
-    __shared__ __align__(16) uint8_t s_img[SELECT_ONLY ? 1 : X1 - X0][SELECT_ONLY ? 16 : QAQ_TILE * D];  // packed tile (K and V)
+    __shared__ __align__(16) uint8_t s_img[SELECT_ONLY ? 1 : X1 - X0][SELECT_ONLY ? 16 : IMG];  // the tile as it will be stored
 
     const float* thr = a.thr + (size_t)bh * 4;
     const bool given = a.bitsK != nullptr;
+    const size_t ti = (size_t)bh * a.ntiles + tile;
+    const size_t mt = (size_t)bh * a.tmax_pad + (size_t)tile * QAQ_TILE + slot;
 
     // ---- loads first (independent of everything else)
     const int b_idx = bh / a.H, h_idx = bh % a.H;
@@ -181,6 +157,11 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
             vk[4 * i] = x.x; vk[4 * i + 1] = x.y; vk[4 * i + 2] = x.z; vk[4 * i + 3] = x.w;
             vv[4 * i] = y.x; vv[4 * i + 1] = y.y; vv[4 * i + 2] = y.z; vv[4 * i + 3] = y.w;
         }
+    }
+    // the padding of the value groups has to read as zero
+    if (!SELECT_ONLY && XSEL != 0) {
+        uint4* z = reinterpret_cast<uint4*>(s_img[X1 - X0 - 1]);
+        for (int o = tid; o < IMG / 16; o += NT) z[o] = make_uint4(0, 0, 0, 0);
     }
 
     // ---- attention window: the P lanes of a token take its rows p, p+P, ... and combine by shuffles
@@ -236,131 +217,128 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
             }
         }
         Bx[x] = valid ? B : 0;
+        if (old) {
+            const int bo = (x ? a.v : a.k).bits[mt];
+            Bx[x] = bo > 8 ? 8 : bo;
+        }
         if (p == 0) {                                   // every slot of the tile is written: empty ones count nothing
-            s_len[x][slot] = valid ? (uint32_t)(D * B / 8) : 0u;
+            s_bits[x][slot] = (uint8_t)Bx[x];
             s_cnt[x][slot] = valid ? cntx[x] : 0u;
             if (SELECT_ONLY && valid) (x ? a.out_bitsV : a.out_bitsK)[(size_t)bh * a.n_new + tn] = (uint8_t)B;
         }
     }
     if (SELECT_ONLY) return;
-    __syncthreads();   // [A] byte lengths and outlier counts visible
+    __syncthreads();   // [A] widths and outlier counts visible
 
-    // ---- warp 0: scans over the tile; lanes 0..3 each take space from one pool (four atomics in flight)
+    // ---- warp 0: section masks of the tile, scan of the outlier counts; lanes 0..3 each take space from one
+    //      pool (four atomics in flight)
     const bool starts = (s_lo == 0), closes = (s_hi == QAQ_TILE), whole = starts && closes;
-    uint32_t my_base = 0, my_amount = 0;
+    uint32_t my_base = 0, my_amount = 0, my_taken = 0;
     if (warp == 0) {
         uint32_t amount[2][2];   // [tensor][0: bytes, 1: outliers]
 #pragma unroll
         for (int x = X0; x < X1; ++x) {
-            uint32_t l0 = s_len[x][lane], l1 = s_len[x][lane + 32];
-            uint32_t c0 = s_cnt[x][lane], c1 = s_cnt[x][lane + 32];
-            uint32_t il0 = l0, il1 = l1, ic0 = c0, ic1 = c1;
+            const uint32_t b0 = s_bits[x][lane], b1 = s_bits[x][lane + 32];
+            qaqc::TileMasks tm;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                tm.m[c] = (unsigned long long)__ballot_sync(0xFFFFFFFFu, (b0 & (8u >> c)) != 0) |
+                          ((unsigned long long)__ballot_sync(0xFFFFFFFFu, (b1 & (8u >> c)) != 0) << 32);
+            uint32_t base[5];
+            if (x == 0) qaqc::section_bases<D, false>(tm, base); else qaqc::section_bases<D, true>(tm, base);
+            const uint32_t c0 = s_cnt[x][lane], c1 = s_cnt[x][lane + 32];
+            uint32_t ic0 = c0, ic1 = c1;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
-                uint32_t t0 = __shfl_up_sync(0xFFFFFFFFu, il0, d), t1 = __shfl_up_sync(0xFFFFFFFFu, il1, d);
-                uint32_t u0 = __shfl_up_sync(0xFFFFFFFFu, ic0, d), u1 = __shfl_up_sync(0xFFFFFFFFu, ic1, d);
-                if (lane >= d) { il0 += t0; il1 += t1; ic0 += u0; ic1 += u1; }
+                const uint32_t u0 = __shfl_up_sync(0xFFFFFFFFu, ic0, d), u1 = __shfl_up_sync(0xFFFFFFFFu, ic1, d);
+                if (lane >= d) { ic0 += u0; ic1 += u1; }
             }
-            const uint32_t tot0 = __shfl_sync(0xFFFFFFFFu, il0, 31), tot1 = __shfl_sync(0xFFFFFFFFu, il1, 31);
             const uint32_t ctot0 = __shfl_sync(0xFFFFFFFFu, ic0, 31), ctot1 = __shfl_sync(0xFFFFFFFFu, ic1, 31);
-            s_len[x][lane] = il0 - l0; s_len[x][lane + 32] = tot0 + il1 - l1;
             s_cnt[x][lane] = ic0 - c0; s_cnt[x][lane + 32] = ctot0 + ic1 - c1;
-            amount[x][0] = tot0 + tot1; amount[x][1] = ctot0 + ctot1;
-            if (lane == 0) s_tot[x] = amount[x][0];
+            // a continued tile stays where it is and takes only what it grows by behind its end
+            const uint32_t old_nb = starts ? 0u : (x ? a.v : a.k).tile_nbytes[ti];
+            amount[x][0] = base[4] - old_nb; amount[x][1] = ctot0 + ctot1;
+            if (lane == 0) { s_tm[x] = tm; s_tot[x] = base[4]; }
         }
         if (lane >= 2 * X0 && lane < 2 * X1) {
             const int x = lane >> 1, pool = lane & 1;
             const TensorStore& ts = x ? a.v : a.k;
             my_amount = x ? amount[1][pool] : amount[0][pool];
-            my_base = pool_take(pool ? &ts.opool_end[bh] : &ts.pool_end[bh], my_amount, pool ? 3u : 15u, whole, closes);
+            my_base = pool_take(pool ? &ts.opool_end[bh] : &ts.pool_end[bh], my_amount, pool ? 3u : 15u, whole, closes, my_taken);
         }
     }
 
-    // ---- codes (every warp; needs only registers): channels 4j..4j+3 in the byte lanes of creg[j]
+    // ---- codes of the new tokens (every warp; needs only registers): channels 4j..4j+3 in the byte lanes of creg[j]
     uint32_t cregs[2][8];
 #pragma unroll
-    for (int x = X0; x < X1; ++x) {
-        const uint32_t (&v)[16] = x ? vv : vk;
-        const int B = Bx[x];
-        const float mn = mnf[x];
-        const float step = __fmul_rn(__fsub_rn(mxf[x], mn), __int_as_float((127 - B) << 23));
-        const float inv = step > 0.f ? __fdiv_rn(1.0f, step) : 0.f;
-        // zero step (constant token): every code is 0, and -inf * 0 = NaN must not clamp to the top code
-        const float topf = step > 0.f ? (float)((1 << B) - 1) : 0.f;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            uint32_t f[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t pair = v[2 * j + (i >> 1)];
-                const unsigned short h = (i & 1) ? (unsigned short)(pair >> 16) : (unsigned short)(pair & 0xFFFF);
-                float t = __fmul_rn(sub_f32_f16(h, mn), inv);            // -inf for an outlier
-                t = fminf(t, topf);
-                f[i] = __float_as_uint(__fadd_rd(t, 8388608.0f));   // 2^23 + floor(t): the code is the low byte (0 for -inf)
-            }
-            cregs[x][j] = prmt(prmt(f[0], f[1], 0x0040u), prmt(f[2], f[3], 0x0040u), 0x5410u);
-        }
-    }
-    __syncthreads();   // [B] offsets inside the tile visible
+    for (int x = X0; x < X1; ++x) qaqc::codes32(x ? vv : vk, mnf[x], mxf[x], Bx[x], cregs[x]);
+    __syncthreads();   // [B] section masks visible
 
-    // ---- planes into the shared-memory image of the tile
+    // ---- old tokens of a continued tile: their codes from the tile as it is stored (read before anything is written)
+    if (!starts) {
+#pragma unroll
+        for (int x = X0; x < X1; ++x) {
+            if (!old) continue;
+            const TensorStore& ts = x ? a.v : a.k;
+            const uint8_t* src = ts.codes + (size_t)bh * a.pool_bytes + ts.tile_off[ti];
+            qaqc::TileMasks om;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) om.m[c] = s_tm[x].m[c] & ((1ull << s_lo) - 1ull);
+            uint32_t ob[5];
+            if (x == 0) { qaqc::section_bases<D, false>(om, ob); qaqc::read_pieces<D, false>(src, om, ob, slot, Bx[x], p, cregs[x]); }
+            else        { qaqc::section_bases<D, true>(om, ob);  qaqc::read_pieces<D, true>(src, om, ob, slot, Bx[x], p, cregs[x]); }
+        }
+    }
+    // ---- pieces into the shared-memory image of the tile
 #pragma unroll
     for (int x = X0; x < X1; ++x) {
-        const uint32_t (&creg)[8] = cregs[x];
-        const int B = Bx[x];
-        uint8_t* tok = s_img[x - X0] + s_len[x][slot & (QAQ_TILE - 1)];
-        if (B & 8) {
-            store_words<ALIGN>(tok + p * 32, creg, 8);
-        }
-        if (B & 4) {
-            const int sh = B & 3;
-            uint32_t w[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                w[j] = ((creg[2 * j] >> sh) & 0x0F0F0F0Fu) | (((creg[2 * j + 1] >> sh) & 0x0F0F0F0Fu) << 4);
-            store_words<ALIGN>(tok + (B & 8) * (D / 8) + p * 16, w, 4);
-        }
-        if (B & 2) {
-            const int sh = B & 1;
-            uint32_t w[2];
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                uint32_t acc = 0;
-#pragma unroll
-                for (int m = 0; m < 4; ++m) acc |= ((creg[4 * j + m] >> sh) & 0x03030303u) << (2 * m);
-                w[j] = acc;
+        if (!(valid || old)) continue;
+        const qaqc::TileMasks tm = s_tm[x];
+        uint32_t base[5];
+        if (x == 0) { qaqc::section_bases<D, false>(tm, base); qaqc::write_pieces<D, false>(s_img[x - X0], tm, base, slot, Bx[x], p, cregs[x]); }
+        else        { qaqc::section_bases<D, true>(tm, base);  qaqc::write_pieces<D, true>(s_img[x - X0], tm, base, slot, Bx[x], p, cregs[x]); }
+    }
+    // ---- allocation results (the atomics were issued before the codes were computed).  A pool without room:
+    //      the space is given back, nothing about the tile is published and the CTA stops; the device status
+    //      reports the lost tokens.
+    if (warp == 0) {
+        bool fail = false;
+        if (lane >= 2 * X0 && lane < 2 * X1) {
+            const int x = lane >> 1, pool = lane & 1;
+            const TensorStore& ts = x ? a.v : a.k;
+            if (pool == 0) {
+                const uint32_t off = starts ? my_base : ts.tile_off[ti];
+                fail = (size_t)my_base + my_taken + 16 > a.pool_bytes || (size_t)off + s_tot[x] + 16 > a.pool_bytes;
+                s_base[x] = off;
+            } else {
+                const uint32_t room = my_base + 8 < a.ocap ? a.ocap - 8 - my_base : 0;  // 8 entries of read-ahead margin
+                const uint32_t stored = my_amount < room ? my_amount : room;
+                if (stored < my_amount) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
+                s_obase[x] = my_base;
+                s_olimit[x] = my_base + stored;
             }
-            store_words<(ALIGN > 8 ? 8 : ALIGN)>(tok + (B & 12) * (D / 8) + p * 8, w, 2);
         }
-        if (B & 1) {
-            uint32_t acc = 0;
-#pragma unroll
-            for (int m = 0; m < 8; ++m) acc |= (creg[m] & 0x01010101u) << m;
-            *reinterpret_cast<uint32_t*>(tok + (B & 14) * (D / 8) + p * 4) = acc;
+        const bool any_fail = __any_sync(0xFFFFFFFFu, fail);
+        if (lane >= 2 * X0 && lane < 2 * X1) {
+            const int x = lane >> 1, pool = lane & 1;
+            const TensorStore& ts = x ? a.v : a.k;
+            if (any_fail) {
+                if (my_taken) atomicSub(pool ? &ts.opool_end[bh] : &ts.pool_end[bh], my_taken);
+            } else if (pool == 0) {
+                if (starts) ts.tile_off[ti] = my_base;
+                ts.tile_nbytes[ti] = s_tot[x];
+            } else {
+                const uint32_t stored = s_olimit[x] - s_obase[x];
+                if (starts) { ts.tile_ooff[ti] = my_base; ts.tile_ocnt[ti] = stored; }
+                else ts.tile_ocnt[ti] += stored;
+            }
         }
-    }
-    // ---- allocation results (the atomics were issued before the codes were computed)
-    if (warp == 0 && lane >= 2 * X0 && lane < 2 * X1) {
-        const int x = lane >> 1, pool = lane & 1;
-        const TensorStore& ts = x ? a.v : a.k;
-        const size_t ti = (size_t)bh * a.ntiles + tile;
-        if (lane == 2 * X0) s_skip = 0;
-        if (pool == 0) {
-            if ((size_t)my_base + my_amount + 16 > a.pool_bytes) { atomicMax(a.status, (int)QAQ_ERR_CAPACITY); s_skip = 1; }
-            if (starts) { ts.tile_off[ti] = my_base; ts.tile_nbytes[ti] = my_amount; }
-            else ts.tile_nbytes[ti] += my_amount;
-            s_base[x] = my_base;
-        } else {
-            const uint32_t room = my_base + 8 < a.ocap ? a.ocap - 8 - my_base : 0;  // 8 entries of read-ahead margin
-            const uint32_t stored = my_amount < room ? my_amount : room;
-            if (stored < my_amount) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
-            if (starts) { ts.tile_ooff[ti] = my_base; ts.tile_ocnt[ti] = stored; }
-            else ts.tile_ocnt[ti] += stored;
-            s_obase[x] = my_base;
-            s_olimit[x] = my_base + stored;
+        if (lane == 0) {
+            s_skip = any_fail ? 1 : 0;
+            if (any_fail) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
         }
     }
-    __syncthreads();   // [C] image complete, pool positions known
+    __syncthreads();   // [C] image complete, pool positions known, every old byte of the tile has been read
     if (s_skip) return;
 
     // ---- the image goes out with vector stores; outlier list; per-token metadata
@@ -368,12 +346,9 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
     for (int x = X0; x < X1; ++x) {
         const TensorStore& ts = x ? a.v : a.k;
         uint8_t* dst = ts.codes + (size_t)bh * a.pool_bytes + s_base[x];
-        const uint32_t nb = s_tot[x];
-        for (uint32_t o = tid * ALIGN; o < nb; o += NT * ALIGN) {
-            if (ALIGN == 16) *reinterpret_cast<uint4*>(dst + o) = *reinterpret_cast<const uint4*>(s_img[x - X0] + o);
-            else if (ALIGN == 8) *reinterpret_cast<uint2*>(dst + o) = *reinterpret_cast<const uint2*>(s_img[x - X0] + o);
-            else *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(s_img[x - X0] + o);
-        }
+        const uint32_t nb = (s_tot[x] + 15u) & ~15u;     // tiles start 16-byte aligned and own a rounded amount
+        for (uint32_t o = tid * 16; o < nb; o += NT * 16)
+            *reinterpret_cast<uint4*>(dst + o) = *reinterpret_cast<const uint4*>(s_img[x - X0] + o);
         // outliers in (token, channel) order: entries of lanes p' < p come first
         uint32_t ob = valid ? ~inl[x] : 0u;
         const uint32_t mine = (uint32_t)__popc(ob);
@@ -401,12 +376,12 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
             }
         }
         if (valid && p == 0) {
-            const size_t t = (size_t)bh * a.tmax_pad + (size_t)tile * QAQ_TILE + slot;
-            ts.bits[t] = (uint8_t)Bx[x];
-            ts.mnmx[t] = (uint32_t)__half_as_ushort(__float2half_rn(mnf[x])) | ((uint32_t)__half_as_ushort(__float2half_rn(mxf[x])) << 16);
+            ts.bits[mt] = (uint8_t)Bx[x];
+            ts.mnmx[mt] = (uint32_t)__half_as_ushort(__float2half_rn(mnf[x])) | ((uint32_t)__half_as_ushort(__float2half_rn(mxf[x])) << 16);
         }
     }
 }
+
 
 template <bool SELECT_ONLY, int XSEL>
 qaq_status launch_x(int D, dim3 grid, const QuantArgs& a, cudaStream_t s) {

@@ -19,6 +19,7 @@
 // old bytes stay unused); the open (last, partly filled) tile is handled in a launch of its own
 // after the closed ones and is kept - or made again - the last thing in its pool, so that later
 // appends continue right behind it.
+#include "qaq_codec.cuh"
 #include "qaq_internal.cuh"
 
 namespace {
@@ -45,166 +46,29 @@ struct RequantArgs {
     int* status;
 };
 
-// B = min{b in [bmin,bmax] : v <= c * 2^b}, bmax if none (c * 2^b is an exact scaling)
-// For positive normal v and c the answer is read off the exponents: with v = mv * 2^ev, c = mc * 2^ec
-// (mv, mc in [1,2)) the smallest b is ev - ec if mv <= mc, else ev - ec + 1.
-__device__ __forceinline__ int ladder(float v, float c, int bmin, int bmax) {
-    if (!(c > 0.f)) return bmax;
-    if (v <= __fmul_rn(c, (float)(1 << bmin))) return bmin;
-    const int vb = __float_as_int(v), cb = __float_as_int(c);
-    if (cb < 0x00800000 || vb < 0x00800000) {  // subnormal operand: plain ladder
-        for (int b = bmin; b <= bmax; ++b)
-            if (v <= __fmul_rn(c, (float)(1 << b))) return b;
-        return bmax;
-    }
-    const int b = (vb >> 23) - (cb >> 23) + (((vb & 0x7FFFFF) > (cb & 0x7FFFFF)) ? 1 : 0);
-    return b < bmin ? bmin : (b > bmax ? bmax : b);
-}
+using qaqc::ladder;
 
-// NW words from / to an address that is ALIGN-byte aligned (ALIGN in {4, 8, 16})
-template <int NW, int ALIGN>
-__device__ __forceinline__ void load_words(const uint8_t* __restrict__ p, uint32_t* w) {
-    if (ALIGN == 16 && NW % 4 == 0) {
-#pragma unroll
-        for (int i = 0; i < NW; i += 4) {
-            const uint4 v = *reinterpret_cast<const uint4*>(p + 4 * i);
-            w[i] = v.x; w[i + 1] = v.y; w[i + 2] = v.z; w[i + 3] = v.w;
-        }
-    } else if (ALIGN >= 8 && NW % 2 == 0) {
-#pragma unroll
-        for (int i = 0; i < NW; i += 2) {
-            const uint2 v = *reinterpret_cast<const uint2*>(p + 4 * i);
-            w[i] = v.x; w[i + 1] = v.y;
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < NW; ++i) w[i] = *reinterpret_cast<const uint32_t*>(p + 4 * i);
-    }
-}
-template <int NW, int ALIGN>
-__device__ __forceinline__ void store_words(uint8_t* p, const uint32_t* w) {
-    if (ALIGN == 16 && NW % 4 == 0) {
-#pragma unroll
-        for (int i = 0; i < NW; i += 4) *reinterpret_cast<uint4*>(p + 4 * i) = make_uint4(w[i], w[i + 1], w[i + 2], w[i + 3]);
-    } else if (ALIGN >= 8 && NW % 2 == 0) {
-#pragma unroll
-        for (int i = 0; i < NW; i += 2) *reinterpret_cast<uint2*>(p + 4 * i) = make_uint2(w[i], w[i + 1]);
-    } else {
-#pragma unroll
-        for (int i = 0; i < NW; ++i) *reinterpret_cast<uint32_t*>(p + 4 * i) = w[i];
-    }
-}
-
-// A token's bytes are the planes of the power-of-two pieces of its width, widest first, each
-// holding the next lower bits of the codes; a lane's 32 channels of a w-bit plane are w words at
-// plane + p * 4w.  creg[j] holds the codes of channels 4j..4j+3, one per byte.
-template <int D, int ALIGN>
-__device__ __forceinline__ void read_planes(const uint8_t* tok, int B, int p, uint32_t (&creg)[8]) {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) creg[j] = 0;
-    if (B & 8) load_words<8, ALIGN>(tok + p * 32, creg);
-    if (B & 4) {
-        const int sh = B & 3;
-        uint32_t w[4];
-        load_words<4, ALIGN>(tok + (B & 8) * (D / 8) + p * 16, w);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            creg[2 * j] |= (w[j] & 0x0F0F0F0Fu) << sh;
-            creg[2 * j + 1] |= ((w[j] >> 4) & 0x0F0F0F0Fu) << sh;
-        }
-    }
-    if (B & 2) {
-        const int sh = B & 1;
-        uint32_t w[2];
-        load_words<2, (ALIGN > 8 ? 8 : ALIGN)>(tok + (B & 12) * (D / 8) + p * 8, w);
-#pragma unroll
-        for (int j = 0; j < 2; ++j)
-#pragma unroll
-            for (int m = 0; m < 4; ++m) creg[4 * j + m] |= ((w[j] >> (2 * m)) & 0x03030303u) << sh;
-    }
-    if (B & 1) {
-        const uint32_t w = *reinterpret_cast<const uint32_t*>(tok + (B & 14) * (D / 8) + p * 4);
-#pragma unroll
-        for (int m = 0; m < 8; ++m) creg[m] |= (w >> m) & 0x01010101u;
-    }
-}
-template <int D, int ALIGN>
-__device__ __forceinline__ void write_planes(uint8_t* tok, int B, int p, const uint32_t (&creg)[8]) {
-    if (B & 8) store_words<8, ALIGN>(tok + p * 32, creg);
-    if (B & 4) {
-        const int sh = B & 3;
-        uint32_t w[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            w[j] = ((creg[2 * j] >> sh) & 0x0F0F0F0Fu) | (((creg[2 * j + 1] >> sh) & 0x0F0F0F0Fu) << 4);
-        store_words<4, ALIGN>(tok + (B & 8) * (D / 8) + p * 16, w);
-    }
-    if (B & 2) {
-        const int sh = B & 1;
-        uint32_t w[2];
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            uint32_t acc = 0;
-#pragma unroll
-            for (int m = 0; m < 4; ++m) acc |= ((creg[4 * j + m] >> sh) & 0x03030303u) << (2 * m);
-            w[j] = acc;
-        }
-        store_words<2, (ALIGN > 8 ? 8 : ALIGN)>(tok + (B & 12) * (D / 8) + p * 8, w);
-    }
-    if (B & 1) {
-        uint32_t acc = 0;
-#pragma unroll
-        for (int m = 0; m < 8; ++m) acc |= (creg[m] & 0x01010101u) << m;
-        *reinterpret_cast<uint32_t*>(tok + (B & 14) * (D / 8) + p * 4) = acc;
-    }
-}
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
-// binary32 (x - c) with x a binary16 value: one rounding
-__device__ __forceinline__ float sub_f32_f16(unsigned short x, float c) {
-    float d;
-    asm("sub.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
-    return d;
-}
 // Codes of one lane's 32 channels computed from the unquantized row, as at append time:
 // code = min(2^B - 1, floor((x - min) * (1/step))) in binary32, 0 for an outlier (outside [lo, hi]).
 __device__ __forceinline__ void fresh_codes(const __half* row, float lo, float hi, float mn, float mx, int B, uint32_t (&creg)[8]) {
-    const __half2 lo2 = __half2half2(__float2half_ru(lo)), hi2 = __half2half2(__float2half_rd(hi));
-    const float step = __fmul_rn(__fsub_rn(mx, mn), __int_as_float((127 - B) << 23));
-    const float inv = step > 0.f ? __fdiv_rn(1.0f, step) : 0.f;
-    const float topf = step > 0.f ? (float)((1 << B) - 1) : 0.f;
+    uint32_t v[16];
 #pragma unroll
     for (int q4 = 0; q4 < 4; ++q4) {
         const uint4 raw = *reinterpret_cast<const uint4*>(row + 8 * q4);
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-        uint32_t f[8];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const __half2 x = *reinterpret_cast<const __half2*>(&w[k]);
-            const uint32_t m = __hge2_mask(x, lo2) & __hle2_mask(x, hi2);       // all-ones halves: inside [lo, hi]
-            const uint32_t v = (w[k] & m) | (0xFC00FC00u & ~m);                    // outliers become -inf: code 0
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const unsigned short h = e ? (unsigned short)(v >> 16) : (unsigned short)(v & 0xFFFF);
-                float t = __fmul_rn(sub_f32_f16(h, mn), inv);
-                t = fminf(t, topf);
-                f[2 * k + e] = __float_as_uint(__fadd_rd(t, 8388608.0f));          // 2^23 + floor(t): the code is the low byte
-            }
-        }
-        creg[2 * q4] = prmt(prmt(f[0], f[1], 0x0040u), prmt(f[2], f[3], 0x0040u), 0x5410u);
-        creg[2 * q4 + 1] = prmt(prmt(f[4], f[5], 0x0040u), prmt(f[6], f[7], 0x0040u), 0x5410u);
+        v[4 * q4] = raw.x; v[4 * q4 + 1] = raw.y; v[4 * q4 + 2] = raw.z; v[4 * q4 + 3] = raw.w;
     }
+    qaqc::mask_outliers32(v, __half2half2(__float2half_ru(lo)), __half2half2(__float2half_rd(hi)));
+    qaqc::codes32(v, mn, mx, B, creg);
 }
 
+// UP: widths may be raised (the unquantized copy is there).  Either way a tile whose bytes grow - raised widths,
+// or lowered ones that need more padding of the value groups than before - takes a new place at the end of its
+// pool; closed tiles are handled by one launch, the open tile by a launch of its own after it.
 template <int D, bool UP>
 __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
     constexpr int P = D / 32;
-    constexpr int ALIGN = D / 8 >= 16 ? 16 : D / 8;
     constexpr int NT = 2 * D;
+    constexpr int IMG = qaqc::v_tile_bytes_max(D);
     const int tile = a.first_tile + blockIdx.x, bh = blockIdx.y;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slot = tid / P, p = tid % P;
@@ -214,10 +78,14 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
 
     __shared__ float s_part[P][QAQ_TILE];
     __shared__ uint8_t s_nv[QAQ_TILE];
-    __shared__ uint32_t s_old[2][QAQ_TILE], s_new[2][QAQ_TILE];   // byte lengths, then exclusive offsets in the tile
+    __shared__ uint8_t s_bo[2][QAQ_TILE], s_bn[2][QAQ_TILE];      // widths before and after
+    __shared__ qaqc::TileMasks s_tmo[2], s_tmn[2];
     __shared__ uint32_t s_tot[2], s_off[2];                        // new bytes of the tile, where they go in the pool
     __shared__ int s_skip[2];
-    __shared__ __align__(16) uint8_t s_img[2][QAQ_TILE * D];
+    __shared__ __align__(16) uint8_t s_img[2][IMG];
+
+    // the padding of the value groups has to read as zero
+    for (int o = tid; o < IMG / 16; o += NT) reinterpret_cast<uint4*>(s_img[1])[o] = make_uint4(0, 0, 0, 0);
 
     // ---- attention window of the tile's tokens (value rule); P threads share a token's rows
     {
@@ -243,6 +111,7 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
         for (int x = 0; x < 2; ++x) {
             const TensorStore& ts = x ? a.v : a.k;
             Bo[x] = ts.bits[mt];
+            Bo[x] = Bo[x] > 8 ? 8 : Bo[x];
             const uint32_t mm = ts.mnmx[mt];
             mnf[x] = __half2float(__ushort_as_half((unsigned short)(mm & 0xFFFF)));
             mxf[x] = __half2float(__ushort_as_half((unsigned short)(mm >> 16)));
@@ -272,15 +141,16 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
         }
         Bn[x] = !valid ? 0 : ((UP || B < Bo[x]) ? B : Bo[x]);
         if (p == 0) {
-            s_old[x][slot] = (uint32_t)(D * Bo[x] / 8);
-            s_new[x][slot] = (uint32_t)(D * Bn[x] / 8);
+            s_bo[x][slot] = (uint8_t)Bo[x];
+            s_bn[x][slot] = (uint8_t)Bn[x];
         }
-        changed[x] = __syncthreads_or(Bn[x] != Bo[x]) != 0;   // also makes the lengths visible
+        changed[x] = __syncthreads_or(Bn[x] != Bo[x]) != 0;   // also makes the widths visible
     }
     // An open tile has to be the last thing in its pool.  If closed tiles of this (b,h) have just been moved
     // behind it, it moves to the end as well, whether its own tokens change or not.
+    const bool open = tile == a.T / QAQ_TILE && (a.T % QAQ_TILE) != 0;
     bool relocate[2] = {false, false};
-    if (UP && tile == a.T / QAQ_TILE && (a.T % QAQ_TILE) != 0) {
+    if (open) {
         const size_t ti0 = (size_t)bh * a.ntiles + tile;
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
@@ -291,31 +161,31 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
     }
     if (!changed[0] && !changed[1]) return;
 
-    // ---- warp 0: exclusive offsets of the tokens inside the tile, before and after
+    // ---- warp 0: which slots have a piece of each width, before and after; size and place of the new tile
     if (warp == 0) {
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
-            uint32_t o0 = s_old[x][lane], o1 = s_old[x][lane + 32], n0 = s_new[x][lane], n1 = s_new[x][lane + 32];
-            uint32_t io0 = o0, io1 = o1, in0 = n0, in1 = n1;
+            const uint32_t o0 = s_bo[x][lane], o1 = s_bo[x][lane + 32], n0 = s_bn[x][lane], n1 = s_bn[x][lane + 32];
+            qaqc::TileMasks mo, mn_;
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t a0 = __shfl_up_sync(0xFFFFFFFFu, io0, d), a1 = __shfl_up_sync(0xFFFFFFFFu, io1, d);
-                const uint32_t b0 = __shfl_up_sync(0xFFFFFFFFu, in0, d), b1 = __shfl_up_sync(0xFFFFFFFFu, in1, d);
-                if (lane >= d) { io0 += a0; io1 += a1; in0 += b0; in1 += b1; }
+            for (int c = 0; c < 4; ++c) {
+                mo.m[c] = (unsigned long long)__ballot_sync(0xFFFFFFFFu, (o0 & (8u >> c)) != 0) |
+                          ((unsigned long long)__ballot_sync(0xFFFFFFFFu, (o1 & (8u >> c)) != 0) << 32);
+                mn_.m[c] = (unsigned long long)__ballot_sync(0xFFFFFFFFu, (n0 & (8u >> c)) != 0) |
+                           ((unsigned long long)__ballot_sync(0xFFFFFFFFu, (n1 & (8u >> c)) != 0) << 32);
             }
-            const uint32_t to0 = __shfl_sync(0xFFFFFFFFu, io0, 31), tn0 = __shfl_sync(0xFFFFFFFFu, in0, 31);
-            const uint32_t tn1 = __shfl_sync(0xFFFFFFFFu, in1, 31);
-            s_old[x][lane] = io0 - o0; s_old[x][lane + 32] = to0 + io1 - o1;
-            s_new[x][lane] = in0 - n0; s_new[x][lane + 32] = tn0 + in1 - n1;
             if (lane == 0) {
+                s_tmo[x] = mo; s_tmn[x] = mn_;
+                uint32_t nbase[5];
+                if (x == 0) qaqc::section_bases<D, false>(mn_, nbase); else qaqc::section_bases<D, true>(mn_, nbase);
                 // where the new tile goes: in place unless it grows
                 const TensorStore& ts = x ? a.v : a.k;
                 const size_t ti0 = (size_t)bh * a.ntiles + tile;
-                const uint32_t nb = tn0 + tn1, off = ts.tile_off[ti0], old_nb = ts.tile_nbytes[ti0];
+                const uint32_t nb = nbase[4], off = ts.tile_off[ti0], old_nb = ts.tile_nbytes[ti0];
+                const uint32_t old_own = open ? old_nb : ((old_nb + 15u) & ~15u);   // closed tiles own a rounded amount
                 uint32_t noff = off;
                 int skip = 0;
-                if (UP && changed[x] && (nb > old_nb || relocate[x])) {
-                    const bool open = tile == a.T / QAQ_TILE && (a.T % QAQ_TILE) != 0;
+                if (changed[x] && (nb > old_own || relocate[x])) {
                     if (open && off + old_nb == ts.pool_end[bh]) {
                         // still the last thing in its pool: it grows where it is
                         if ((size_t)off + nb + 16 > a.pool_bytes) skip = 1;
@@ -327,10 +197,12 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
                         if ((size_t)noff + nb + 16 > a.pool_bytes) skip = 1;
                         else ts.pool_end[bh] = noff + nb;
                     } else {
-                        // the end of the pool need not be aligned while a tile is open: take 16 bytes more and align
+                        // the end of the pool need not be aligned while a tile is open: take 16 bytes more and align;
+                        // space that does not fit is given back
                         const uint32_t take = ((nb + 15u) & ~15u) + 16u;
-                        noff = (atomicAdd(&ts.pool_end[bh], take) + 15u) & ~15u;
-                        if ((size_t)noff + take + 16 > a.pool_bytes) skip = 1;
+                        const uint32_t at = atomicAdd(&ts.pool_end[bh], take);
+                        noff = (at + 15u) & ~15u;
+                        if ((size_t)at + take + 16 > a.pool_bytes) { skip = 1; atomicSub(&ts.pool_end[bh], take); }
                     }
                     if (skip) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
                 }
@@ -339,12 +211,11 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
         }
     }
     __syncthreads();
-    if (UP) {   // no room in the pool: that tensor's tile stays as it is
-        if (s_skip[0]) changed[0] = false;
-        if (s_skip[1]) changed[1] = false;
-    }
+    // no room in the pool: that tensor's tile stays as it is
+    if (s_skip[0]) changed[0] = false;
+    if (s_skip[1]) changed[1] = false;
 
-    // ---- old planes -> codes -> low bits dropped -> new planes in the shared-memory image
+    // ---- old pieces -> codes -> low bits dropped -> new pieces in the shared-memory image
     const size_t ti = (size_t)bh * a.ntiles + tile;
 #pragma unroll
     for (int x = 0; x < 2; ++x) {
@@ -358,14 +229,20 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
                                     (size_t)tok * a.st + 32 * p;
                 fresh_codes(row, a.thr[(size_t)bh * 4 + 2 * x], a.thr[(size_t)bh * 4 + 2 * x + 1], mnf[x], mxf[x], Bn[x], creg);
             } else {
-                const uint8_t* src = ts.codes + (size_t)bh * a.pool_bytes + ts.tile_off[ti] + s_old[x][slot];
-                read_planes<D, ALIGN>(src, Bo[x], p, creg);
+                const uint8_t* src = ts.codes + (size_t)bh * a.pool_bytes + ts.tile_off[ti];
+                const qaqc::TileMasks mo = s_tmo[x];
+                uint32_t ob[5];
+                if (x == 0) { qaqc::section_bases<D, false>(mo, ob); qaqc::read_pieces<D, false>(src, mo, ob, slot, Bo[x], p, creg); }
+                else        { qaqc::section_bases<D, true>(mo, ob);  qaqc::read_pieces<D, true>(src, mo, ob, slot, Bo[x], p, creg); }
                 const int drop = Bo[x] - Bn[x];
                 const uint32_t keep = 0x01010101u * (0xFFu >> drop);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) creg[j] = (creg[j] >> drop) & keep;
             }
-            write_planes<D, ALIGN>(s_img[x] + s_new[x][slot], Bn[x], p, creg);
+            const qaqc::TileMasks mn_ = s_tmn[x];
+            uint32_t nbs[5];
+            if (x == 0) { qaqc::section_bases<D, false>(mn_, nbs); qaqc::write_pieces<D, false>(s_img[0], mn_, nbs, slot, Bn[x], p, creg); }
+            else        { qaqc::section_bases<D, true>(mn_, nbs);  qaqc::write_pieces<D, true>(s_img[1], mn_, nbs, slot, Bn[x], p, creg); }
         }
     }
     __syncthreads();   // every old byte of the tile has been read, the image is complete
@@ -377,20 +254,15 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
         const TensorStore& ts = x ? a.v : a.k;
         const uint32_t off = s_off[x];
         uint8_t* dst = ts.codes + (size_t)bh * a.pool_bytes + off;
-        const uint32_t nb = s_tot[x];
-        for (uint32_t o = tid * ALIGN; o < nb; o += NT * ALIGN) {
-            if (ALIGN == 16) *reinterpret_cast<uint4*>(dst + o) = *reinterpret_cast<const uint4*>(s_img[x] + o);
-            else if (ALIGN == 8) *reinterpret_cast<uint2*>(dst + o) = *reinterpret_cast<const uint2*>(s_img[x] + o);
-            else *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(s_img[x] + o);
-        }
+        const uint32_t nb = s_tot[x], nb16 = (nb + 15u) & ~15u;
+        for (uint32_t o = tid * 16; o < nb16; o += NT * 16)
+            *reinterpret_cast<uint4*>(dst + o) = *reinterpret_cast<const uint4*>(s_img[x] + o);
         if (valid && p == 0) ts.bits[mt] = (uint8_t)Bn[x];
         if (tid == 0) {
             // an open tile that is still the last thing in its pool gives back what it no longer needs:
             // appends continue right behind its bytes
             const uint32_t old_off = ts.tile_off[ti], old_nb = ts.tile_nbytes[ti];
-            if (tile == a.T / QAQ_TILE && (a.T % QAQ_TILE) != 0 && off == old_off && nb < old_nb &&
-                old_off + old_nb == ts.pool_end[bh])
-                ts.pool_end[bh] = off + nb;
+            if (open && off == old_off && nb < old_nb && old_off + old_nb == ts.pool_end[bh]) ts.pool_end[bh] = off + nb;
             ts.tile_off[ti] = off;
             ts.tile_nbytes[ti] = nb;
         }
@@ -440,26 +312,26 @@ extern "C" qaq_status qaq_requantize(qaq_cache* c, const void* K_full, const voi
     cudaStream_t s = (cudaStream_t)stream;
     const int D = c->cfg.head_dim;
     const int ntile = (int)((c->tokens + QAQ_TILE - 1) / QAQ_TILE);
-    if (!up) {
-        a.first_tile = 0;
-        return launch_requant<false>(D, dim3((unsigned)ntile, (unsigned)c->BH), a, s);
+    if (up) {
+        if (!thr) return QAQ_ERR_INVALID_ARG;
+        if (stride_t < D || (stride_b & 7) || (stride_h & 7) || (stride_t & 7) || stride_b < 0 || stride_h < 0) return QAQ_ERR_INVALID_ARG;
+        a.Ks = (const __half*)device_view(K_full); a.Vs = (const __half*)device_view(V_full);
+        if (!a.Ks || !a.Vs || ((uintptr_t)a.Ks & 15) || ((uintptr_t)a.Vs & 15)) return QAQ_ERR_INVALID_ARG;
+        a.sb = stride_b; a.sh = stride_h; a.st = stride_t; a.thr = thr;
     }
-    if (!thr) return QAQ_ERR_INVALID_ARG;
-    if (stride_t < D || (stride_b & 7) || (stride_h & 7) || (stride_t & 7) || stride_b < 0 || stride_h < 0) return QAQ_ERR_INVALID_ARG;
-    a.Ks = (const __half*)device_view(K_full); a.Vs = (const __half*)device_view(V_full);
-    if (!a.Ks || !a.Vs || ((uintptr_t)a.Ks & 15) || ((uintptr_t)a.Vs & 15)) return QAQ_ERR_INVALID_ARG;
-    a.sb = stride_b; a.sh = stride_h; a.st = stride_t; a.thr = thr;
     // closed tiles first (a tile that grows moves to the end of its pool), then the open tile, which has to be
     // the last thing in its pool when this call is over
     const int closed = (int)(c->tokens / QAQ_TILE);
     qaq_status st = QAQ_OK;
     if (closed > 0) {
         a.first_tile = 0;
-        if ((st = launch_requant<true>(D, dim3((unsigned)closed, (unsigned)c->BH), a, s)) != QAQ_OK) return st;
+        const dim3 grid((unsigned)closed, (unsigned)c->BH);
+        if ((st = up ? launch_requant<true>(D, grid, a, s) : launch_requant<false>(D, grid, a, s)) != QAQ_OK) return st;
     }
     if (closed < ntile) {
         a.first_tile = closed;
-        st = launch_requant<true>(D, dim3(1, (unsigned)c->BH), a, s);
+        const dim3 grid(1, (unsigned)c->BH);
+        st = up ? launch_requant<true>(D, grid, a, s) : launch_requant<false>(D, grid, a, s);
     }
     return st;
 }
