@@ -349,7 +349,7 @@ __global__ void export_gather_kernel(TensorStore ts, int is_v, int T, int tmax_p
         for (int c = 0; c < 4; ++c) n[c] = __popcll(tm.m[c]);
         uint32_t base[5];
         {   // section offsets for any head_dim (the templates of the codec header fix it at compile time)
-            uint32_t o = 0;
+            uint32_t o = qaqc::QAQ_TILE_HDR;
             for (int c = 0; c < 4; ++c) {
                 const int w = 8 >> c;
                 base[c] = o;

@@ -17,11 +17,16 @@
 //            byte-replicated mask a word has one field per byte lane: the operand of dp4a against four channels
 //            of the query).
 //   values:  items are stored in groups of four (the last group of a section is padded with zero bytes):
-//            group g = items 4g..4g+3, head_dim*w/2 bytes; channels 8h..8h+7 are the w words at byte 4*w*h of
-//            the group; in word k, byte lane i belongs to item 4g+i and bit field m (bits w*m .. w*m+w-1) of that
-//            byte is channel 8h + k*(8/w) + m  (one field per byte lane = four tokens of one channel: the operand
-//            of dp4a against four per-token weights).
-// A tile therefore takes sum_t head_dim*B_t/8 bytes for keys and that plus the group padding for values.
+//            group G = items 4G..4G+3, head_dim*w/2 bytes, made of 32-bit words whose byte lane i belongs to item
+//            4G+i and whose bit field m (bits w*m .. w*m+w-1 of every byte) is one channel, so that a masked word is
+//            four tokens of one channel, one per byte: the A operand of the integer tensor-core instruction
+//            mma.m16n8k32 with rows = channels and k = tokens.  Channel c = 16*mb + 8*s + g has register index
+//            R = g*(head_dim/8) + 2*mb + s and sits in word R / (8/w), field R % (8/w): the registers that the MMA
+//            lane with group id g needs for all 16-channel row blocks mb are consecutive, one vector load.
+// The sections are preceded by a header of QAQ_TILE_HDR bytes: the four 64-bit masks "slot t has a piece of width
+// 8, 4, 2, 1" (widths, ranks and section sizes of a tile can be read off them without the per-token metadata).
+// A tile therefore takes the header plus sum_t head_dim*B_t/8 bytes for keys, and that plus the group padding for
+// values.
 #pragma once
 #include <cuda_fp16.h>
 #include <stdint.h>
@@ -97,21 +102,23 @@ __device__ __forceinline__ void mask_outliers32(uint32_t (&v)[16], __half2 lo2, 
 }
 
 // ------------------------------------------------------------------------------------------ tile layout
+constexpr int QAQ_TILE_HDR = 32;
+
 // Which slots of a tile have a piece of width 8 >> c (c = 0..3): one 64-bit mask per width.
 struct TileMasks {
     unsigned long long m[4];
 };
 
-// largest tile: 64 tokens at 8 bits plus the worst padding of the value groups (three items in each of the four
+// largest tile: the header, 64 tokens at 8 bits plus the worst padding of the value groups (three items in each of the four
 // sections), rounded up to a multiple of 16 so that images of tiles can sit back to back in shared memory
 __host__ __device__ constexpr int v_tile_bytes_max(int D) {
-    return (QAQ_TILE_TOKENS * D + 3 * (D * 15 / 8) + 15) / 16 * 16;
+    return (QAQ_TILE_HDR + QAQ_TILE_TOKENS * D + 3 * (D * 15 / 8) + 15) / 16 * 16;
 }
 
 // Byte offsets of the four sections inside a tile (base[4] = bytes of the tile).
 template <int D, bool IS_V>
 __device__ __forceinline__ void section_bases(const int (&n)[4], uint32_t (&base)[5]) {
-    uint32_t o = 0;
+    uint32_t o = QAQ_TILE_HDR;
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         const int w = 8 >> c;
@@ -126,6 +133,10 @@ __device__ __forceinline__ void section_bases(const TileMasks& tm, uint32_t (&ba
 #pragma unroll
     for (int c = 0; c < 4; ++c) n[c] = __popcll(tm.m[c]);
     section_bases<D, IS_V>(n, base);
+}
+// the header of a tile image (16-byte aligned, shared or global memory)
+__device__ __forceinline__ void write_header(uint8_t* img, const TileMasks& tm, int c) {
+    reinterpret_cast<unsigned long long*>(img)[c] = tm.m[c];
 }
 __device__ __forceinline__ int rank_in(const TileMasks& tm, int c, int slot) {
     return __popcll(tm.m[c] & ((1ull << slot) - 1ull));
@@ -192,46 +203,61 @@ __device__ __forceinline__ void write_pieces(uint8_t* img, const TileMasks& tm, 
             *reinterpret_cast<uint32_t*>(img + base[3] + rank_in(tm, 3, slot) * (D / 8) + p * 4) = acc;
         }
     } else {
-        // values: byte lane (rank & 3) of the words of group rank >> 2; this thread covers the 8-channel blocks 4p..4p+3
+        // values: byte lane (rank & 3) of the words of group rank >> 2.  Channel 32p + 4j + b has g = 4(j&1) + b and
+        // register R = g*NRV + 4p + (j>>1): for every g this thread holds four consecutive registers.
+        constexpr int NRV = D / 8;
         if (B & 8) {
             const int r = rank_in(tm, 0, slot);
-            uint8_t* g = img + base[0] + (r >> 2) * (D * 4) + (r & 3) + p * 128;
+            uint8_t* grp = img + base[0] + (r >> 2) * (D * 4) + (r & 3);
 #pragma unroll
-            for (int hh = 0; hh < 4; ++hh)
+            for (int g = 0; g < 8; ++g)
 #pragma unroll
-                for (int k = 0; k < 8; ++k) g[hh * 32 + 4 * k] = (uint8_t)(creg[2 * hh + (k >> 2)] >> (8 * (k & 3)));
+                for (int q = 0; q < 4; ++q)
+                    grp[4 * (g * NRV + 4 * p + q)] = (uint8_t)(creg[(g >> 2) + 2 * q] >> (8 * (g & 3)));
         }
         if (B & 4) {
             const int sh = B & 3, r = rank_in(tm, 1, slot);
-            uint8_t* g = img + base[1] + (r >> 2) * (D * 2) + (r & 3) + p * 64;
+            uint8_t* grp = img + base[1] + (r >> 2) * (D * 2) + (r & 3);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint32_t x = (creg[j] >> sh) & 0x0F0F0F0Fu;
-                const uint32_t y = x | (x >> 4);     // byte 0: channels 4j, 4j+1; byte 2: channels 4j+2, 4j+3
-                const int hh = j >> 1, k = 2 * (j & 1);
-                g[hh * 16 + 4 * k] = (uint8_t)y;
-                g[hh * 16 + 4 * (k + 1)] = (uint8_t)(y >> 16);
-            }
+            for (int g = 0; g < 8; ++g)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t f0 = (creg[(g >> 2) + 4 * h] >> (8 * (g & 3) + sh)) & 15u;
+                    const uint32_t f1 = (creg[(g >> 2) + 4 * h + 2] >> (8 * (g & 3) + sh)) & 15u;
+                    grp[4 * ((g * NRV + 4 * p) / 2 + h)] = (uint8_t)(f0 | (f1 << 4));
+                }
         }
         if (B & 2) {
             const int sh = B & 1, r = rank_in(tm, 2, slot);
-            uint8_t* g = img + base[2] + (r >> 2) * D + (r & 3) + p * 32;
+            uint8_t* grp = img + base[2] + (r >> 2) * D + (r & 3);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint32_t x = (creg[j] >> sh) & 0x03030303u;
-                const uint32_t z = x | (x >> 6);
-                const uint32_t t = z | (z >> 12);    // byte 0: the four 2-bit pieces of channels 4j..4j+3
-                g[(j >> 1) * 8 + 4 * (j & 1)] = (uint8_t)t;
+            for (int g = 0; g < 8; ++g) {
+                uint32_t v = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) v |= ((creg[(g >> 2) + 2 * q] >> (8 * (g & 3) + sh)) & 3u) << (2 * q);
+                grp[4 * ((g * NRV + 4 * p) / 4)] = (uint8_t)v;
             }
         }
         if (B & 1) {
             const int r = rank_in(tm, 3, slot);
-            uint8_t* g = img + base[3] + (r >> 2) * (D / 2) + (r & 3) + p * 16;
+            uint8_t* grp = img + base[3] + (r >> 2) * (D / 2);
+            uint32_t nib[8];
 #pragma unroll
-            for (int hh = 0; hh < 4; ++hh) {
-                const uint32_t n0 = (((creg[2 * hh] & 0x01010101u) * 0x01020408u) >> 24) & 15u;
-                const uint32_t n1 = (((creg[2 * hh + 1] & 0x01010101u) * 0x01020408u) >> 24) & 15u;
-                g[hh * 4] = (uint8_t)(n0 | (n1 << 4));
+            for (int g = 0; g < 8; ++g) {
+                uint32_t v = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) v |= ((creg[(g >> 2) + 2 * q] >> (8 * (g & 3))) & 1u) << q;
+                nib[g] = v;
+            }
+            if (D == 32) {       // registers 4g .. 4g+3: two g share a byte, both held by this thread
+#pragma unroll
+                for (int g = 0; g < 8; g += 2) grp[4 * (g / 2) + (r & 3)] = (uint8_t)(nib[g] | (nib[g + 1] << 4));
+            } else {             // a byte is shared with the neighbouring thread of the token: OR into the (zeroed) image
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    const int Rb = g * NRV + 4 * p;
+                    atomicOr(reinterpret_cast<uint32_t*>(grp + 4 * (Rb / 8)), nib[g] << (8 * (r & 3) + (Rb & 7)));
+                }
             }
         }
     }
@@ -270,42 +296,47 @@ __device__ __forceinline__ void read_pieces(const uint8_t* img, const TileMasks&
             for (int m = 0; m < 8; ++m) creg[m] |= (w >> m) & 0x01010101u;
         }
     } else {
+        constexpr int NRV = D / 8;
         if (B & 8) {
             const int r = rank_in(tm, 0, slot);
-            const uint8_t* g = img + base[0] + (r >> 2) * (D * 4) + (r & 3) + p * 128;
+            const uint8_t* grp = img + base[0] + (r >> 2) * (D * 4) + (r & 3);
 #pragma unroll
-            for (int hh = 0; hh < 4; ++hh)
+            for (int g = 0; g < 8; ++g)
 #pragma unroll
-                for (int k = 0; k < 8; ++k) creg[2 * hh + (k >> 2)] |= (uint32_t)g[hh * 32 + 4 * k] << (8 * (k & 3));
+                for (int q = 0; q < 4; ++q)
+                    creg[(g >> 2) + 2 * q] |= (uint32_t)grp[4 * (g * NRV + 4 * p + q)] << (8 * (g & 3));
         }
         if (B & 4) {
             const int sh = B & 3, r = rank_in(tm, 1, slot);
-            const uint8_t* g = img + base[1] + (r >> 2) * (D * 2) + (r & 3) + p * 64;
+            const uint8_t* grp = img + base[1] + (r >> 2) * (D * 2) + (r & 3);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint32_t b0 = g[(j >> 1) * 16 + 8 * (j & 1)], b1 = g[(j >> 1) * 16 + 8 * (j & 1) + 4];
-                const uint32_t x = (b0 & 15u) | ((b0 >> 4) << 8) | ((b1 & 15u) << 16) | ((b1 >> 4) << 24);
-                creg[j] |= x << sh;
-            }
+            for (int g = 0; g < 8; ++g)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t b = grp[4 * ((g * NRV + 4 * p) / 2 + h)];
+                    creg[(g >> 2) + 4 * h] |= ((b & 15u) << sh) << (8 * (g & 3));
+                    creg[(g >> 2) + 4 * h + 2] |= ((b >> 4) << sh) << (8 * (g & 3));
+                }
         }
         if (B & 2) {
             const int sh = B & 1, r = rank_in(tm, 2, slot);
-            const uint8_t* g = img + base[2] + (r >> 2) * D + (r & 3) + p * 32;
+            const uint8_t* grp = img + base[2] + (r >> 2) * D + (r & 3);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint32_t b = g[(j >> 1) * 8 + 4 * (j & 1)];
-                const uint32_t u = b | (b << 12);
-                creg[j] |= ((u | (u << 6)) & 0x03030303u) << sh;
+            for (int g = 0; g < 8; ++g) {
+                const uint32_t b = grp[4 * ((g * NRV + 4 * p) / 4)];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) creg[(g >> 2) + 2 * q] |= (((b >> (2 * q)) & 3u) << sh) << (8 * (g & 3));
             }
         }
         if (B & 1) {
             const int r = rank_in(tm, 3, slot);
-            const uint8_t* g = img + base[3] + (r >> 2) * (D / 2) + (r & 3) + p * 16;
+            const uint8_t* grp = img + base[3] + (r >> 2) * (D / 2) + (r & 3);
 #pragma unroll
-            for (int hh = 0; hh < 4; ++hh) {
-                const uint32_t b = g[hh * 4];
-                creg[2 * hh] |= ((b & 15u) * 0x00204081u) & 0x01010101u;
-                creg[2 * hh + 1] |= ((b >> 4) * 0x00204081u) & 0x01010101u;
+            for (int g = 0; g < 8; ++g) {
+                const int Rb = g * NRV + 4 * p;
+                const uint32_t b = (uint32_t)grp[4 * (Rb / 8)] >> (Rb & 7);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) creg[(g >> 2) + 2 * q] |= ((b >> q) & 1u) << (8 * (g & 3));
             }
         }
     }
@@ -321,9 +352,9 @@ __device__ __forceinline__ uint32_t piece_at(const uint8_t* tile, const uint32_t
         const uint32_t word = *reinterpret_cast<const uint32_t*>(item + 4 * (p * w + j * w / 8));
         return (word >> (8 * i + w * (j & (per - 1)))) & ((1u << w) - 1u);
     } else {
-        const uint8_t* g = tile + base[c] + (size_t)(r >> 2) * (D * w / 2);
-        const int h = d >> 3, cl = d & 7, k = cl / per, m = cl & (per - 1);
-        return ((uint32_t)g[h * 4 * w + 4 * k + (r & 3)] >> (w * m)) & ((1u << w) - 1u);
+        const uint8_t* grp = tile + base[c] + (size_t)(r >> 2) * (D * w / 2);
+        const int R = (d & 7) * (D / 8) + 2 * (d >> 4) + ((d >> 3) & 1);
+        return ((uint32_t)grp[4 * (R / per) + (r & 3)] >> (w * (R & (per - 1)))) & ((1u << w) - 1u);
     }
 }
 

@@ -9,28 +9,32 @@
 // and a token's outliers add  q_ch * (x - (min_t + step_t/2))  resp.  p_t * (v - ...)
 // because their code slot holds 0.
 //
-// q.K runs on integer dot products (dp4a): q is converted per (b,h) to 16-bit fixed point
-// q_d ~ qscale * (256 * hi_d + lo_d), hi signed / lo unsigned bytes, so that every plane
-// word of codes (already one field per byte lane after a mask) feeds two dp4a.  The sums
-// are exact integers; the fixed-point error of q is below 2^-16 of max|q|.
+// Both sums over codes run on the integer tensor-core instruction mma.sync.m16n8k32 (u8 x s8 -> s32).  A plane
+// word of the cache, after one shift and a byte-replicated mask, holds one w-bit field per byte lane, which is
+// exactly an A-operand register of that instruction (four consecutive k), so a decode step - a GEMV, whose cost
+// here is taking bit fields apart, not multiplying - spends one instruction per 512 code-times-weight products
+// instead of one per four.  The exact integer sums make the result independent of any accumulation order.
+//   q.K:  rows = 16 tokens of a section, k = channels; B = q in 16-bit fixed point per (b,h), split into two
+//         signed byte digits that sit in columns 0 and 1 (q_d ~ qscale * (256 * hi_d + lo_d)).
+//   S.V:  rows = 16 channels, k = 32 tokens of a section (the value pieces of four tokens share a word, one per
+//         byte lane); B = the per-token weights p_t * step_t * 2^shift in 23-bit fixed point with one scale per
+//         tile, three signed byte digits in columns 0..2.  The integer sums of a tile are added to binary32
+//         accumulators once per tile.  The rounded weight of a token is also what the softmax denominator and the
+//         constant part of its values use, so numerator and denominator see the same slightly perturbed probability.
 //
-// One CTA = one run of consecutive tiles of the flattened (b,h, tile) sequence (runs of equal
-// length, so every SM gets the same amount of work); each warp works through whole tiles
-// (QAQ_TILE tokens) on its own, with its own running max / sum / accumulators and no CTA
-// barrier in the tile loop; warps are merged once at the end.  A tile is stored as sections of
-// equal-width pieces (qaq_codec.cuh), so every inner loop runs one extraction routine over the
-// items of one section, and a token finds its items by its rank among the tokens that have a
-// piece of that width (ballots over the widths; no lists are built).
+// One CTA = one run of consecutive tiles of the flattened (b,h, tile) sequence (runs of equal length, so every SM
+// gets the same amount of work); each warp works through whole tiles (QAQ_TILE tokens) on its own, with its own
+// running max / sum / accumulators and no CTA barrier in the tile loop; warps are merged once at the end.  A tile
+// is stored as sections of equal-width pieces behind a header of four masks (qaq_codec.cuh), so every inner loop
+// runs one extraction routine over the items of one section, and a token finds its items by its rank among the
+// tokens that have a piece of that width (population counts on the masks; no lists are built, the per-token
+// widths are not read).  The packed bytes of the next tile are copied to a per-warp shared-memory buffer with
+// cp.async while the current one is worked on: the keys during the value phase (at the front of the buffer), the
+// values during the key phase (at its back).  The buffer is sized for typical tiles; a tile that does not fit
+// beside its neighbour is read in place from global memory by the same loops.
 //
-// X = S Vhat runs on integer dot products as well: the value pieces of four tokens share a word
-// (one per byte lane), the per-token weights p_t * step_t * 2^shift become 24-bit fixed point
-// with one scale per tile (three dp4a per word and field), and the integer sums of a tile are
-// added to binary32 accumulators once per tile.  The rounded weight of a token is also what the
-// softmax denominator and the constant part of its values use, so numerator and denominator see
-// the same slightly perturbed probability.
-//
-// Outlier corrections are summed in fixed point with integer atomics (scale from the largest
-// term of the tile), so that the result does not depend on the order in which lanes arrive.
+// Outlier corrections are summed in fixed point with 32-bit integer atomics in shared memory (a high and a low
+// part with fixed scales), so the result does not depend on the order in which lanes arrive.
 #include "qaq_codec.cuh"
 #include "qaq_internal.cuh"
 
@@ -38,7 +42,7 @@ namespace {
 
 constexpr int DEC_WARPS = 4;
 constexpr int DEC_THREADS = DEC_WARPS * 32;
-constexpr int DEC_CTAS_PER_SM = 2;   // what the per-warp staging buffers of head_dim 128 leave room for
+constexpr int DEC_CTAS_PER_SM = 4;
 
 struct DecArgs {
     TensorStore k, v;
@@ -55,83 +59,57 @@ struct DecArgs {
     float* scores;     // [BH][T] or null
 };
 
-__device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {  // unsigned bytes x signed bytes
-    int d;
-    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-__device__ __forceinline__ int dp4a_uu(uint32_t a, uint32_t b, int c) {  // unsigned x unsigned
-    int d;
-    asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
+// D(16x8, s32) += A(16x32, u8, row) * B(32x8, s8, col).  Lane = 4*g + t holds
+//   a0: row g, k 4t..4t+3   a1: row g+8, k 4t..4t+3   a2: row g, k 16+4t..   a3: row g+8, k 16+4t..   (one k per byte)
+//   b0: k 4t..4t+3, column g   b1: k 16+4t.., column g
+//   d0, d1: row g, columns 2t, 2t+1   d2, d3: row g+8, columns 2t, 2t+1
+__device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 template <int BYTES>
 __device__ __forceinline__ void cp_async(void* smem, const void* gmem) {
     const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
-    if (BYTES == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem));
-    else if (BYTES == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(s), "l"(gmem));
-    else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(s), "l"(gmem));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem));
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
-// integer dot product of one lane's 32 channels of a w-bit plane with q (hi/lo bytes)
-template <int W>
-__device__ __forceinline__ int plane_dot(const uint32_t (&words)[8], const uint32_t (&qh)[8], const uint32_t (&ql)[8]) {
+// NREG operand registers (one W-bit field per byte lane) with register indices R0 .. R0+NREG-1 of a key plane or
+// of a value group (staged in shared memory, or in place in global memory): register R sits in word R / (8/W) at bit W * (R % (8/W)) of every byte.  Nothing is read
+// when !ok (the registers are zero).
+template <int W, int NREG>
+__device__ __forceinline__ void fetch_regs(const uint8_t* base, int R0, bool ok, uint32_t (&reg)[NREG]) {
     constexpr int PER = 8 / W;
+    constexpr int NW = NREG >= PER ? NREG / PER : 1;
     constexpr uint32_t MASK = 0x01010101u * ((1u << W) - 1u);
-    int ah[2] = {0, 0}, al[2] = {0, 0};
+    uint32_t w[NW];
 #pragma unroll
-    for (int j = 0; j < W; ++j) {
-        const uint32_t wd = words[j];
+    for (int i = 0; i < NW; ++i) w[i] = 0;
+    if (ok) qaqc::load_words<NW>(base + 4 * (R0 / PER), w);
+    const int f0 = NREG >= PER ? 0 : W * (R0 % PER);     // only a word shared by several lanes starts inside it
 #pragma unroll
-        for (int m = 0; m < PER; ++m) {
-            const uint32_t f = (wd >> (W * m)) & MASK;
-            const int r = PER * j + m;
-            ah[r & 1] = dp4a_us(f, qh[r], ah[r & 1]);
-            al[r & 1] = dp4a_uu(f, ql[r], al[r & 1]);
-        }
-    }
-    return (ah[0] + ah[1]) * 256 + (al[0] + al[1]);
-}
-
-// weighted sums of one lane's 8 channels over the four tokens of a value group:
-// acc[cl] += sum_i weight_i * piece_i(channel cl); wt.x / wt.y / wt.z hold the high / middle / low bytes of the four
-// 24-bit weights
-template <int W>
-__device__ __forceinline__ void group_axpy(const uint32_t (&words)[8], const uint4 wt, int (&ahi)[8], int (&amd)[8], int (&alo)[8]) {
-    constexpr int PER = 8 / W;
-    constexpr uint32_t MASK = 0x01010101u * ((1u << W) - 1u);
-#pragma unroll
-    for (int k = 0; k < W; ++k) {
-#pragma unroll
-        for (int m = 0; m < PER; ++m) {
-            const uint32_t f = (words[k] >> (W * m)) & MASK;
-            ahi[PER * k + m] = dp4a_uu(f, wt.x, ahi[PER * k + m]);
-            amd[PER * k + m] = dp4a_uu(f, wt.y, amd[PER * k + m]);
-            alo[PER * k + m] = dp4a_uu(f, wt.z, alo[PER * k + m]);
-        }
+    for (int r = 0; r < NREG; ++r) {
+        if (W == 8) reg[r] = w[r];
+        else reg[r] = (w[r / PER] >> (W * (r % PER) + f0)) & MASK;
     }
 }
-
-constexpr int OSTAGE = 192;          // outlier entries per tile and tensor staged in shared memory
 
 // per-warp scratch for the tile a warp is working on
 template <int D>
 struct WarpScratch {
-    alignas(16) uint8_t bufK[QAQ_TILE * D + 16];
-    alignas(16) uint8_t bufV[(qaqc::v_tile_bytes_max(D) + 15) / 16 * 16 + 16];
+    static constexpr int STAGE = 72 * D;      // bytes of the staging buffer (9 KB at head_dim 128: four CTAs per SM)
+    alignas(16) uint8_t buf[STAGE];           // keys of a tile from the front, values from the back
     int dotw[4][QAQ_TILE];                    // integer q . piece per section and rank
-    alignas(16) uint32_t wts[4][QAQ_TILE / 4][4];  // per section and value group: high, middle, low bytes of the four weights
+    alignas(16) uint32_t wts[4][QAQ_TILE / 4][4];  // per section and value group: the three byte digits of the four weights
     float midK[QAQ_TILE];       // min + step/2
     float midV[QAQ_TILE];
     float p[QAQ_TILE];          // attention weights of the tile's tokens at the current scale of the running sums
-    int iocorr[2][QAQ_TILE];    // fixed-point sums (high, low part) of the key-outlier corrections per token
-    int ivout[2][D];            // ... of the value-outlier corrections per channel (zero between tiles)
-    float vout[D];              // value-outlier corrections
-    alignas(16) uint32_t outl[2][OSTAGE];   // the tile's outlier entries (K, V); longer lists continue in global memory
+    int kcorr[2][QAQ_TILE];     // fixed-point sums (high, low part) of the key-outlier corrections per token (zero between tiles)
+    int vcorr[2][D];            // ... of the value-outlier corrections per channel (zero between tiles)
 };
 
 template <int D>
@@ -144,92 +122,74 @@ struct DecSmem {
     float qscale, qsum;
 };
 
-// q . piece for the items of one key section: P = D/32 lanes per item, each 32 channels
+// q . piece for the items of one key section: 16 items per instruction row block, lane 4g+t holds the channels
+// 4*(t*NR + r) + i (r < NR = D/16) of items g and g+8
 template <int D, int W>
-__device__ __forceinline__ void k_section(const uint8_t* sec, int n, int* dots, const uint32_t (&qh)[8], const uint32_t (&ql)[8],
-                                          int part, int sub) {
-    constexpr int P = D / 32, IPW = 32 / P;
+__device__ __forceinline__ void k_section(const uint8_t* sec, int n, int* dots, const uint32_t (&qb)[D / 16], int g, int t) {
+    constexpr int NR = D / 16, ITEM = D * W / 8;
 #pragma unroll 1
-    for (int i0 = 0; i0 < n; i0 += IPW) {
-        const int r = i0 + sub;
-        int da = 0;
-        if (r < n) {
-            uint32_t w0[8];
-            qaqc::load_words<W>(sec + r * (D * W / 8) + part * 4 * W, w0);
-            da = plane_dot<W>(w0, qh, ql);
+    for (int i0 = 0; i0 < n; i0 += 16) {
+        const int r0 = i0 + g, r1 = r0 + 8;
+        uint32_t x0[NR], x1[NR];
+        fetch_regs<W, NR>(sec + r0 * ITEM, t * NR, r0 < n, x0);
+        fetch_regs<W, NR>(sec + r1 * ITEM, t * NR, r1 < n, x1);
+        int d[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int m = 0; m < NR / 2; ++m) mma_u8s8(d, x0[2 * m], x1[2 * m], x0[2 * m + 1], x1[2 * m + 1], qb[2 * m], qb[2 * m + 1]);
+        if (t == 0) {          // columns 0 and 1: the high and the low digit of q
+            if (r0 < n) dots[r0] = d[0] * 256 + d[1];
+            if (r1 < n) dots[r1] = d[2] * 256 + d[3];
         }
-#pragma unroll
-        for (int o = 1; o < P; o <<= 1) da += __shfl_xor_sync(0xFFFFFFFFu, da, o);
-        if (r < n && part == 0) dots[r] = da;
     }
 }
 
-// weighted accumulation over the groups of one value section: LPG = D/8 lanes per group, each 8 channels
+// weighted sums over the groups of one value section: 8 groups (32 tokens) per instruction, lane 4g+t holds the
+// channels 16*mb + 8*s + g of groups t and t+4
 template <int D, int W>
-__device__ __forceinline__ void v_section(const uint8_t* sec, int ngroups, const uint32_t (*wts)[4], int (&ahi)[8], int (&amd)[8],
-                                          int (&alo)[8], int h, int grp) {
-    constexpr int LPG = D / 8, GPW = 32 / LPG;
+__device__ __forceinline__ void v_section(const uint8_t* sec, int ngroups, const uint32_t (*wts)[4], int (&acc)[D / 16][4], int g, int t) {
+    constexpr int NRV = D / 8, GB = D * W / 2;
 #pragma unroll 1
-    for (int g = grp; g < ngroups; g += GPW) {
-        uint32_t w0[8];
-        qaqc::load_words<W>(sec + g * (D * W / 2) + h * 4 * W, w0);
-        const uint4 wt = *reinterpret_cast<const uint4*>(wts[g]);
-        group_axpy<W>(w0, wt, ahi, amd, alo);
+    for (int g0 = 0; g0 < ngroups; g0 += 8) {
+        const int ga = g0 + t, gb = ga + 4;
+        uint32_t xa[NRV], xb[NRV];
+        fetch_regs<W, NRV>(sec + ga * GB, g * NRV, ga < ngroups, xa);
+        fetch_regs<W, NRV>(sec + gb * GB, g * NRV, gb < ngroups, xb);
+        const uint32_t b0 = (g < 3 && ga < ngroups) ? wts[ga][g] : 0u;
+        const uint32_t b1 = (g < 3 && gb < ngroups) ? wts[gb][g] : 0u;
+#pragma unroll
+        for (int mb = 0; mb < D / 16; ++mb) mma_u8s8(acc[mb], xa[2 * mb], xa[2 * mb + 1], xb[2 * mb], xb[2 * mb + 1], b0, b1);
     }
 }
 
-// Sum of per-entry corrections into integer cells, independent of the order in which lanes arrive: the terms of a
-// tile's outlier list are brought to fixed point with one scale for the tile (from the largest term) and added with
-// integer atomics.  A term is split into a high part (units of 2^eu, below 2^24 of them) and the exact remainder in
-// units of 2^(eu-20), so a cell keeps about 44 bits below the largest term of the tile whatever the other cells hold.
-// term(e) gives the cell and the binary32 term of entry e; cells[0][.] / cells[1][.] take the high / low parts.
-// Returns the weight of one high unit (0: nothing was added).
-constexpr float OUTL_LO = 1048576.0f;     // 2^20 low units per high unit
-template <int NCELL, typename F>
-__device__ __forceinline__ float outlier_sums(uint32_t count, int lane, int (*cells)[NCELL], F term) {
-    float mx = 0.f;
-#pragma unroll 1
-    for (uint32_t e = lane; e < count; e += 32) {
-        int cell; float t;
-        term(e, cell, t);
-        mx = fmaxf(mx, fabsf(t));
+// Fixed-point form of an outlier term for integer atomics: a high part in units of 2^-4 and the exact remainder
+// in units of 2^-28.  Terms of 2^18 or more (and non-finite ones) are left out, so that 128 of them stay inside
+// 32 bits in both parts.
+constexpr float OC_LIMIT = 262144.0f;
+__device__ __forceinline__ void outlier_add(int* hi_cell, int* lo_cell, float tm) {
+    if (fabsf(tm) < OC_LIMIT) {
+        const float hi = rintf(tm * 16.0f);
+        const float rem = fmaf(hi, -0.0625f, tm);              // exact, |rem| <= 2^-5
+        atomicAdd(hi_cell, (int)hi);
+        atomicAdd(lo_cell, __float2int_rn(rem * 268435456.0f));
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-    if (!(mx > 0.f) || !(mx < 3.0e38f)) return 0.f;        // nothing to add (or not finite: left out)
-    // largest term below 2^24 units, so that the up to 128 terms of a cell stay inside 32 bits
-    const int ex = (__float_as_int(mx) >> 23) & 0xFF;       // mx < 2^(ex-126)
-    const int eu = max(-100, min(100, ex - 126 - 24));      // one unit = 2^eu
-    const float inv = __int_as_float((127 - eu) << 23), unit = __int_as_float((127 + eu) << 23);
-#pragma unroll 1
-    for (uint32_t e = lane; e < count; e += 32) {
-        int cell; float t;
-        term(e, cell, t);
-        const float hi = rintf(t * inv);
-        const float rem = fmaf(-hi, unit, t);               // exact: |rem| <= unit / 2
-        atomicAdd(&cells[0][cell], (int)hi);
-        atomicAdd(&cells[1][cell], __float2int_rn(rem * inv * OUTL_LO));
-    }
-    return unit;
 }
+__device__ __forceinline__ float outlier_sum(int hi, int lo) { return fmaf((float)lo, 1.0f / 268435456.0f, (float)hi * 0.0625f); }
 
 // One CTA = one run of consecutive tiles, which meets one or two (b,h): the body below runs once
 // per (b,h) segment and leaves one partial per segment.  Every warp works through whole tiles on its
-// own: own running max / sum / accumulators, own staging buffers, no CTA barrier in the loop; the
-// warps are merged once at the end.  The packed bytes of the next tile are copied to shared memory
-// with cp.async while the current one is being processed: the keys during the value phase, the
-// values during the key phase.  Lane l looks after tokens l and l + 32 of the tile (logit, softmax
-// weight, fixed-point value weight); the section loops spread the items over the lanes.
+// own: own running max / sum / accumulators, own staging buffer, no CTA barrier in the loop; the
+// warps are merged once at the end.  Lane l looks after tokens l and l + 32 of the tile (logit, softmax
+// weight, fixed-point value weight); in the section loops lane 4g+t is lane (g, t) of the tensor-core fragments.
 template <int D>
 __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(const DecArgs a) {
-    constexpr int P = D / 32;        // lanes per key item
-    constexpr int LPG = D / 8;       // lanes per value group
+    constexpr int NR = D / 16;       // key operand registers per lane and item
+    constexpr int MB = D / 16;       // 16-channel row blocks of the value side
     constexpr int HALF = QAQ_TILE / 2;
+    constexpr uint32_t STAGE = WarpScratch<D>::STAGE;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DecSmem<D>& sm = *reinterpret_cast<DecSmem<D>*>(smem_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int part = lane % P, sub = lane / P;
-    const int vh = lane % LPG, vgrp = lane / LPG;
+    const int fg = lane >> 2, ft = lane & 3;
     const unsigned lt = (1u << lane) - 1u;
     WarpScratch<D>& ws = sm.ws[warp];
 
@@ -245,7 +205,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
     const int tile_lo = max(flat_lo, bh * ntiles) - bh * ntiles, tile_hi = min(flat_hi, (bh + 1) * ntiles) - bh * ntiles;
     if (tile_lo >= tile_hi) continue;   // the same for every thread of the CTA
 
-    // ---- q: float copy, fixed-point bytes per lane
+    // ---- q: float copy, fixed-point byte digits per lane
     float qmax = 0.f, qs = 0.f;
     for (int d = tid; d < D; d += DEC_THREADS) {
         const float f = __half2float(a.q[(size_t)bh * D + d]);
@@ -259,156 +219,171 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         qs += __shfl_xor_sync(0xFFFFFFFFu, qs, o);
     }
     if (lane == 0) { sm.red[warp] = qmax; sm.red2[warp] = qs; }
-    for (int d = lane; d < D; d += 32) { ws.vout[d] = 0.f; ws.ivout[0][d] = 0; ws.ivout[1][d] = 0; }
+    for (int d = lane; d < D; d += 32) { ws.vcorr[0][d] = 0; ws.vcorr[1][d] = 0; }
+    for (int i = lane; i < QAQ_TILE; i += 32) { ws.kcorr[0][i] = 0; ws.kcorr[1][i] = 0; }
     __syncthreads();
     if (tid == 0) {
         float m = 0.f, s = 0.f;
         for (int w = 0; w < DEC_WARPS; ++w) { m = fmaxf(m, sm.red[w]); s += sm.red2[w]; }
-        sm.qscale = m / 32767.0f;
+        sm.qscale = m / 32639.0f;        // |q| <= 32639 units: both byte digits of 256 * hi + lo stay signed bytes
         sm.qsum = s;
     }
     __syncthreads();
     const float qscale = sm.qscale, qsum = sm.qsum;
     const float qinv = qscale > 0.f ? 1.0f / qscale : 0.f;
-    uint32_t qh[8], ql[8];
+    uint32_t qb[NR];             // column fg of the B operand: the high (fg = 0) or low (fg = 1) digit, zero otherwise
 #pragma unroll
-    for (int r = 0; r < 8; ++r) {
-        uint32_t h = 0, l = 0;
+    for (int r = 0; r < NR; ++r) {
+        uint32_t v = 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            int qi = __float2int_rn(sm.qf[32 * part + 4 * r + i] * qinv);
-            qi = max(-32767, min(32767, qi));
-            h |= (uint32_t)((qi >> 8) & 0xFF) << (8 * i);
-            l |= (uint32_t)(qi & 0xFF) << (8 * i);
+            int qi = __float2int_rn(sm.qf[4 * (ft * NR + r) + i] * qinv);
+            qi = max(-32639, min(32639, qi));
+            const int dg = fg == 0 ? ((qi + 128) >> 8) : qi;     // 256 * hi + lo with lo in [-128, 127]
+            v |= (uint32_t)(dg & 0xFF) << (8 * i);
         }
-        qh[r] = h; ql[r] = l;
+        qb[r] = fg < 2 ? v : 0u;
     }
 
-    float X[8];                 // this lane's 8 channels (8*vh ..), summed over the groups this lane has handled
+    float X[MB][2];             // channels 16*mb + 8*s + fg: this lane's share of the digit columns (summed over ft at the end)
 #pragma unroll
-    for (int i = 0; i < 8; ++i) X[i] = 0.f;
+    for (int mb = 0; mb < MB; ++mb) { X[mb][0] = 0.f; X[mb][1] = 0.f; }
+    // what the accumulator columns of this lane stand for: lane ft = 0 holds the digits 2^16 and 2^8, ft = 1 the units
+    const float dig0 = ft == 0 ? 65536.0f : (ft == 1 ? 1.0f : 0.f), dig1 = ft == 0 ? 256.0f : 0.f;
     float m_run = __int_as_float(0xff800000), l_run = 0.f, lx_run = 0.f;   // lx: sum of the unperturbed p
     float c_run = 0.f;       // per-lane part of sum_t p_t * (min_t + step_t/2) of the values
+    float vout[(D + 31) / 32];   // value-outlier corrections of channels lane, lane + 32, ...
+#pragma unroll
+    for (int k = 0; k < (D + 31) / 32; ++k) vout[k] = 0.f;
 
     const size_t trow = (size_t)bh * a.ntiles_max;
     const size_t mrow = (size_t)bh * a.tmax_pad;
     const uint8_t* poolK = a.k.codes + (size_t)bh * a.pool_bytes;
     const uint8_t* poolV = a.v.codes + (size_t)bh * a.pool_bytes;
+    const uint32_t* ogK = a.k.outl + (size_t)bh * a.ocap;
+    const uint32_t* ogV = a.v.outl + (size_t)bh * a.ocap;
 
-    // ---- tile metadata in registers: table words in lanes 0..7, widths and min/max of tokens lane, lane+32
-    struct Meta { uint32_t tb, bits4, mm[4]; };
+    // ---- tile metadata in registers: table words in lanes 0..7 (offset and length of the bytes, first entry and
+    //      length of the outlier list; keys in lanes 0..3, values in 4..7), min/max of tokens lane, lane+32.
+    //      Table entries that point outside the pool or the list are not followed (length 0).
+    struct Meta { uint32_t tb, mm[4]; };
     auto fetch_meta = [&](int tile) {
         Meta m;
-        m.tb = 0; m.bits4 = 0; m.mm[0] = m.mm[1] = m.mm[2] = m.mm[3] = 0;
+        m.tb = 0; m.mm[0] = m.mm[1] = m.mm[2] = m.mm[3] = 0;
         if (tile < tile_hi) {
+            uint32_t first = 0, len = 0;
             if (lane < 8) {
                 const TensorStore& ts = (lane >= 4) ? a.v : a.k;
                 const size_t ti = trow + tile;
-                const int f = lane & 3;
-                m.tb = f == 0 ? ts.tile_off[ti] : f == 1 ? ts.tile_nbytes[ti] : f == 2 ? ts.tile_ooff[ti] : ts.tile_ocnt[ti];
+                if (lane & 2) { first = ts.tile_ooff[ti]; len = ts.tile_ocnt[ti]; if ((size_t)first + len > a.ocap) len = 0; }
+                else {
+                    first = ts.tile_off[ti]; len = ts.tile_nbytes[ti];
+                    if ((first & 15u) || len < (uint32_t)qaqc::QAQ_TILE_HDR || (size_t)first + ((len + 15u) & ~15u) > a.pool_bytes) len = 0;
+                }
+                m.tb = (lane & 1) ? len : first;
             }
             const size_t t0 = mrow + (size_t)tile * QAQ_TILE + lane;
-            m.bits4 = (uint32_t)a.k.bits[t0] | ((uint32_t)a.k.bits[t0 + 32] << 8) | ((uint32_t)a.v.bits[t0] << 16) |
-                      ((uint32_t)a.v.bits[t0 + 32] << 24);
             m.mm[0] = a.k.mnmx[t0]; m.mm[1] = a.k.mnmx[t0 + 32]; m.mm[2] = a.v.mnmx[t0]; m.mm[3] = a.v.mnmx[t0 + 32];
         }
         return m;
     };
-    // a tile's bytes (rounded up to 16, never more than the buffer holds) and its outlier entries
-    auto stage = [&](uint8_t* dst, const uint8_t* pool, uint32_t off, uint32_t nbytes, uint32_t cap) {
-        nbytes = (min(nbytes, cap) + 15u) & ~15u;
-        if ((size_t)off + nbytes > a.pool_bytes) nbytes = 0;      // a table entry that points outside the pool is not followed
+    // copies nb bytes (a multiple of 16) of a tile to the staging buffer
+    auto stage = [&](uint8_t* dst, const uint8_t* src, uint32_t nb) {
 #pragma unroll 1
-        for (uint32_t o = lane * 16; o < nbytes; o += 32 * 16) cp_async<16>(dst + o, pool + off + o);
-    };
-    auto stage_outl = [&](int x, uint32_t first, uint32_t count) {   // entries are 4 bytes, lists start 16-byte aligned
-        const uint32_t* src = (x ? a.v.outl : a.k.outl) + (size_t)bh * a.ocap + first;
-        const uint32_t n16 = ((count < (uint32_t)OSTAGE ? count : (uint32_t)OSTAGE) + 3u) >> 2;
-        if ((size_t)first + 4 * n16 > a.ocap) return;
-#pragma unroll 1
-        for (uint32_t o = lane; o < n16; o += 32) cp_async<16>(&ws.outl[x][4 * o], src + 4 * o);
-    };
-    auto stage_K = [&](const Meta& m) {
-        stage(ws.bufK, poolK, __shfl_sync(0xFFFFFFFFu, m.tb, 0), __shfl_sync(0xFFFFFFFFu, m.tb, 1), QAQ_TILE * D);
-        stage_outl(0, __shfl_sync(0xFFFFFFFFu, m.tb, 2), __shfl_sync(0xFFFFFFFFu, m.tb, 3));
-        cp_async_commit();
-    };
-    auto stage_V = [&](const Meta& m) {
-        stage(ws.bufV, poolV, __shfl_sync(0xFFFFFFFFu, m.tb, 4), __shfl_sync(0xFFFFFFFFu, m.tb, 5), (uint32_t)sizeof(ws.bufV) - 16u);
-        stage_outl(1, __shfl_sync(0xFFFFFFFFu, m.tb, 6), __shfl_sync(0xFFFFFFFFu, m.tb, 7));
-        cp_async_commit();
+        for (uint32_t o = lane * 16; o < nb; o += 32 * 16) cp_async<16>(dst + o, src + o);
     };
     int tile = tile_lo + warp;
     Meta cur = fetch_meta(tile);
     Meta nxt = fetch_meta(tile + DEC_WARPS);
-    if (tile < tile_hi) { stage_K(cur); stage_V(cur); }
+    // what is staged: bytes (rounded up to 16) of the current keys / values in the buffer, 0 = read in place
+    uint32_t stK = 0, stV = 0;
+    if (tile < tile_hi) {
+        const uint32_t nbK = (__shfl_sync(0xFFFFFFFFu, cur.tb, 1) + 15u) & ~15u, nbV = (__shfl_sync(0xFFFFFFFFu, cur.tb, 5) + 15u) & ~15u;
+        if (nbK <= STAGE) { stK = nbK; stage(ws.buf, poolK + __shfl_sync(0xFFFFFFFFu, cur.tb, 0), nbK); }
+        cp_async_commit();
+        if (stK + nbV <= STAGE) { stV = nbV; stage(ws.buf + STAGE - nbV, poolV + __shfl_sync(0xFFFFFFFFu, cur.tb, 4), nbV); }
+        cp_async_commit();
+    }
 
     for (; tile < tile_hi; tile += DEC_WARPS) {
+        const uint32_t offK = __shfl_sync(0xFFFFFFFFu, cur.tb, 0), nbK = __shfl_sync(0xFFFFFFFFu, cur.tb, 1);
         const uint32_t ooK = __shfl_sync(0xFFFFFFFFu, cur.tb, 2), ocK = __shfl_sync(0xFFFFFFFFu, cur.tb, 3);
+        const uint32_t offV = __shfl_sync(0xFFFFFFFFu, cur.tb, 4), nbV = __shfl_sync(0xFFFFFFFFu, cur.tb, 5);
         const uint32_t ooV = __shfl_sync(0xFFFFFFFFu, cur.tb, 6), ocV = __shfl_sync(0xFFFFFFFFu, cur.tb, 7);
         const bool has_next = tile + DEC_WARPS < tile_hi;
         const int t0 = tile * QAQ_TILE + lane;              // this lane's tokens: t0 and t0 + 32
         const bool val0 = t0 < a.T, val1 = t0 + HALF < a.T;
-
-        // ---- widths, ranks of this lane's tokens in the sections, section sizes
-        int B[2][2];          // [tensor][token]
-        uint32_t rk[2][2];    // rank in section c in byte c
-        int n[2][4];
+        const uint8_t* tK = stK ? ws.buf : poolK + offK;
+        const uint8_t* tV = stV ? ws.buf + STAGE - stV : poolV + offV;
+        // the first outlier entries of the tile (used after the section loops)
+        uint32_t eK[2], eV[2];
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
-            B[x][0] = val0 ? min(8, (int)((cur.bits4 >> (16 * x)) & 0xFF)) : 0;
-            B[x][1] = val1 ? min(8, (int)((cur.bits4 >> (16 * x + 8)) & 0xFF)) : 0;
-            rk[x][0] = rk[x][1] = 0;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const unsigned b0 = __ballot_sync(0xFFFFFFFFu, (B[x][0] & (8 >> c)) != 0);
-                const unsigned b1 = __ballot_sync(0xFFFFFFFFu, (B[x][1] & (8 >> c)) != 0);
-                const int n0 = __popc(b0);
-                n[x][c] = n0 + __popc(b1);
-                rk[x][0] |= (uint32_t)__popc(b0 & lt) << (8 * c);
-                rk[x][1] |= (uint32_t)(n0 + __popc(b1 & lt)) << (8 * c);
-            }
-        }
-        uint32_t kb[5], vb[5];
-        qaqc::section_bases<D, false>(n[0], kb);
-        qaqc::section_bases<D, true>(n[1], vb);
-
-        // ---- per-token scalars
-        float stepK[2], stepV[2], midV[2];
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const bool v = j ? val1 : val0;
-            const uint32_t mk = cur.mm[j], mv = cur.mm[2 + j];
-            const float kmn = __half2float(__ushort_as_half((unsigned short)(mk & 0xFFFF)));
-            const float kmx = __half2float(__ushort_as_half((unsigned short)(mk >> 16)));
-            const float vmn = __half2float(__ushort_as_half((unsigned short)(mv & 0xFFFF)));
-            const float vmx = __half2float(__ushort_as_half((unsigned short)(mv >> 16)));
-            stepK[j] = v ? qaqc::step_of(kmn, kmx, B[0][j]) : 0.f;
-            stepV[j] = v ? qaqc::step_of(vmn, vmx, B[1][j]) : 0.f;
-            ws.midK[lane + HALF * j] = v ? fmaf(0.5f, stepK[j], kmn) : 0.f;
-            midV[j] = v ? fmaf(0.5f, stepV[j], vmn) : 0.f;
-            ws.midV[lane + HALF * j] = midV[j];
-            ws.iocorr[0][lane + HALF * j] = 0;
-            ws.iocorr[1][lane + HALF * j] = 0;
+        for (int k = 0; k < 2; ++k) {
+            eK[k] = lane + 32 * k < ocK ? __ldg(ogK + ooK + lane + 32 * k) : 0u;
+            eV[k] = lane + 32 * k < ocV ? __ldg(ogV + ooV + lane + 32 * k) : 0u;
         }
         cp_async_wait<1>();     // this tile's keys have landed (its values may still be in flight)
         __syncwarp();
 
-        // ---- K: integer dot products per section
-        k_section<D, 8>(ws.bufK + kb[0], n[0][0], ws.dotw[0], qh, ql, part, sub);
-        k_section<D, 4>(ws.bufK + kb[1], n[0][1], ws.dotw[1], qh, ql, part, sub);
-        k_section<D, 2>(ws.bufK + kb[2], n[0][2], ws.dotw[2], qh, ql, part, sub);
-        k_section<D, 1>(ws.bufK + kb[3], n[0][3], ws.dotw[3], qh, ql, part, sub);
-        // key outliers: q_ch * (x - mid) per token
-        const uint32_t* ogK = a.k.outl + (size_t)bh * a.ocap + ooK;
-        const float ounit = outlier_sums(ocK, lane, ws.iocorr, [&](uint32_t e, int& cell, float& t) {
-            const uint32_t v = e < (uint32_t)OSTAGE ? ws.outl[0][e] : __ldg(ogK + e);
-            cell = (v >> 24) & (QAQ_TILE - 1);
-            t = sm.qf[(v >> 16) & (D - 1)] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midK[cell]);
-        });
+        // ---- keys: widths, ranks of this lane's tokens in the sections, section sizes (from the tile's header)
+        int B[2][2];          // [tensor][token]
+        uint32_t rk[2][2];    // rank in section c in byte c
+        int n[2][4];
+        B[0][0] = B[0][1] = B[1][0] = B[1][1] = 0;
+        rk[0][0] = rk[0][1] = rk[1][0] = rk[1][1] = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint2 mk = nbK ? *reinterpret_cast<const uint2*>(tK + 8 * c) : make_uint2(0u, 0u);
+            if ((mk.x >> lane) & 1u) B[0][0] |= 8 >> c;
+            if ((mk.y >> lane) & 1u) B[0][1] |= 8 >> c;
+            const int n0 = __popc(mk.x);
+            n[0][c] = n0 + __popc(mk.y);
+            rk[0][0] |= (uint32_t)__popc(mk.x & lt) << (8 * c);
+            rk[0][1] |= (uint32_t)(n0 + __popc(mk.y & lt)) << (8 * c);
+        }
+        if (!val0) B[0][0] = 0;
+        if (!val1) B[0][1] = 0;
+        uint32_t kb[5];
+        qaqc::section_bases<D, false>(n[0], kb);
+        // a tile that does not hold the sections its masks ask for is not read: its tokens then count with their
+        // constant parts only
+        const bool okK = kb[4] <= nbK;
+        if (!okK) { n[0][0] = n[0][1] = n[0][2] = n[0][3] = 0; }
+
+        // ---- per-token scalars of the keys
+        float stepK[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const bool v = j ? val1 : val0;
+            const uint32_t mk = cur.mm[j];
+            const float kmn = __half2float(__ushort_as_half((unsigned short)(mk & 0xFFFF)));
+            const float kmx = __half2float(__ushort_as_half((unsigned short)(mk >> 16)));
+            stepK[j] = v ? qaqc::step_of(kmn, kmx, B[0][j]) : 0.f;
+            ws.midK[lane + HALF * j] = v ? fmaf(0.5f, stepK[j], kmn) : 0.f;
+        }
         __syncwarp();
-        // ---- the key buffer is free: start the copy of the next tile's keys
-        if (has_next) stage_K(nxt); else cp_async_commit();
+
+        // ---- K: integer dot products per section
+        k_section<D, 8>(tK + kb[0], n[0][0], ws.dotw[0], qb, fg, ft);
+        k_section<D, 4>(tK + kb[1], n[0][1], ws.dotw[1], qb, fg, ft);
+        k_section<D, 2>(tK + kb[2], n[0][2], ws.dotw[2], qb, fg, ft);
+        k_section<D, 1>(tK + kb[3], n[0][3], ws.dotw[3], qb, fg, ft);
+        // key outliers: q_ch * (x - mid) per token
+#pragma unroll 1
+        for (uint32_t e = lane; e < ocK; e += 32) {
+            const uint32_t v = e < 64 ? (e < 32 ? eK[0] : eK[1]) : __ldg(ogK + ooK + e);
+            const int tok = (v >> 24) & (QAQ_TILE - 1);
+            const float tm = sm.qf[(v >> 16) & (D - 1)] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midK[tok]);
+            outlier_add(&ws.kcorr[0][tok], &ws.kcorr[1][tok], tm);
+        }
+        __syncwarp();
+        // ---- the front of the buffer is free: start the copy of the next tile's keys (beside this tile's values)
+        uint32_t stKn = 0;
+        if (has_next) {
+            const uint32_t nb = (__shfl_sync(0xFFFFFFFFu, nxt.tb, 1) + 15u) & ~15u;
+            if (nb + stV <= STAGE) { stKn = nb; stage(ws.buf, poolK + __shfl_sync(0xFFFFFFFFu, nxt.tb, 0), nb); }
+        }
+        cp_async_commit();
 
         // ---- logits of this lane's tokens; running max / sum
         float lg[2];
@@ -418,12 +393,14 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int w = 8 >> c;
-                if (B[0][j] & w) dot += ws.dotw[c][(rk[0][j] >> (8 * c)) & 0xFF] << (B[0][j] & (w - 1));
+                if ((B[0][j] & w) && okK) dot += ws.dotw[c][(rk[0][j] >> (8 * c)) & 0xFF] << (B[0][j] & (w - 1));
             }
             lg[j] = __int_as_float(0xff800000);
+            const int tk = lane + HALF * j;
+            const int kh = ws.kcorr[0][tk], kl = ws.kcorr[1][tk];
+            if (kh | kl) { ws.kcorr[0][tk] = 0; ws.kcorr[1][tk] = 0; }
             if (j ? val1 : val0) {
-                const int tk = lane + HALF * j;
-                const float qk = fmaf(qscale * stepK[j], (float)dot, fmaf(ws.midK[tk], qsum, ounit * fmaf((float)ws.iocorr[1][tk], 1.0f / OUTL_LO, (float)ws.iocorr[0][tk])));
+                const float qk = fmaf(qscale * stepK[j], (float)dot, fmaf(ws.midK[tk], qsum, outlier_sum(kh, kl)));
                 lg[j] = a.scale * qk;
                 if (a.scores) a.scores[(size_t)bh * a.T + t0 + HALF * j] = lg[j];
             }
@@ -436,16 +413,48 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         m_run = m_new;
         if (alpha != 1.0f) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) X[i] *= alpha;
+            for (int mb = 0; mb < MB; ++mb) { X[mb][0] *= alpha; X[mb][1] *= alpha; }
             c_run *= alpha;
-            for (int d = lane; d < D; d += 32) ws.vout[d] *= alpha;
+#pragma unroll
+            for (int k = 0; k < (D + 31) / 32; ++k) vout[k] *= alpha;
         }
-        // ---- value weights p * step * 2^shift as 24-bit fixed point with one scale for the tile (a token's step
+        cp_async_wait<1>();     // this tile's values have landed
+        __syncwarp();
+
+        // ---- values: widths, ranks, section sizes; per-token scalars
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint2 mv = nbV ? *reinterpret_cast<const uint2*>(tV + 8 * c) : make_uint2(0u, 0u);
+            if ((mv.x >> lane) & 1u) B[1][0] |= 8 >> c;
+            if ((mv.y >> lane) & 1u) B[1][1] |= 8 >> c;
+            const int n0 = __popc(mv.x);
+            n[1][c] = n0 + __popc(mv.y);
+            rk[1][0] |= (uint32_t)__popc(mv.x & lt) << (8 * c);
+            rk[1][1] |= (uint32_t)(n0 + __popc(mv.y & lt)) << (8 * c);
+        }
+        if (!val0) B[1][0] = 0;
+        if (!val1) B[1][1] = 0;
+        uint32_t vb[5];
+        qaqc::section_bases<D, true>(n[1], vb);
+        const bool okV = vb[4] <= nbV;
+        if (!okV) { n[1][0] = n[1][1] = n[1][2] = n[1][3] = 0; }
+        float stepV[2], midV[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const bool v = j ? val1 : val0;
+            const uint32_t mv = cur.mm[2 + j];
+            const float vmn = __half2float(__ushort_as_half((unsigned short)(mv & 0xFFFF)));
+            const float vmx = __half2float(__ushort_as_half((unsigned short)(mv >> 16)));
+            stepV[j] = v ? qaqc::step_of(vmn, vmx, B[1][j]) : 0.f;
+            midV[j] = v ? fmaf(0.5f, stepV[j], vmn) : 0.f;
+            ws.midV[lane + HALF * j] = midV[j];
+        }
+        // ---- value weights p * step * 2^shift as 22-bit fixed point with one scale for the tile (a token's step
         //      falls with its width, so next to a 2-bit token an 8-bit token of the same p has a weight 64 times
-        //      smaller: 16 bits would leave it about 10).  The weight of the
-        //      token's lowest piece is rounded once; the other pieces use exact multiples of it, and p is replaced
-        //      by what the rounded weight stands for, so that the pieces, the constant part and the softmax
-        //      denominator all see the same (slightly perturbed) probability.
+        //      smaller: 16 bits would leave it about 10).  The weight of the token's lowest piece is rounded once;
+        //      the other pieces use exact multiples of it, and p is replaced by what the rounded weight stands for,
+        //      so that the pieces, the constant part and the softmax denominator all see the same (slightly
+        //      perturbed) probability.
         float pe[2], wf[2];
         int top[2];
         float wmax = 0.f;
@@ -459,29 +468,31 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) wmax = fmaxf(wmax, __shfl_xor_sync(0xFFFFFFFFu, wmax, o));
-        // wmax < 2^(ex-126): one unit = 2^(ex-126-24) keeps every shifted weight below 2^24
+        // wmax < 2^(ex-126): one unit = 2^(ex-126-22) keeps every shifted weight at or below 2^22
         const int wex = (__float_as_int(wmax) >> 23) & 0xFF;
-        const bool wok = wex > 24 && wex < 255;                    // zero, tiny or non-finite weights: the pieces add nothing
-        const float wunit = wok ? __int_as_float((wex - 23) << 23) : 0.f;
-        const float winv = wok ? __int_as_float((254 - (wex - 23)) << 23) : 0.f;
+        const bool wok = wex > 24 && wex < 255 && okV;             // zero, tiny or non-finite weights: the pieces add nothing
+        const float wunit = wok ? __int_as_float((wex - 21) << 23) : 0.f;
+        const float winv = wok ? __int_as_float((254 - (wex - 21)) << 23) : 0.f;
         float s = 0.f, sx = 0.f;
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
             const int Bv = B[1][j];
             uint32_t iw = (uint32_t)__float2int_rn(wf[j] * winv);
-            iw = min(iw, 0xFFFFFFu >> top[j]);
+            iw = min(iw, 0x7F0000u >> top[j]);       // the three balanced byte digits of a shifted weight stay signed bytes
             float p = pe[j];
             if (stepV[j] > 0.f && wok) p = __fdividef((float)iw * wunit, stepV[j]);
-            uint8_t* wb = reinterpret_cast<uint8_t*>(ws.wts);
+            uint8_t* wbytes = reinterpret_cast<uint8_t*>(ws.wts);
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int w = 8 >> c;
                 if (Bv & w) {
                     const uint32_t r = (rk[1][j] >> (8 * c)) & 0xFF, wt = iw << (Bv & (w - 1));
-                    uint8_t* g = wb + c * (QAQ_TILE / 4) * 16 + (r >> 2) * 16 + (r & 3);
-                    g[0] = (uint8_t)(wt >> 16);
-                    g[4] = (uint8_t)(wt >> 8);
-                    g[8] = (uint8_t)wt;
+                    // wt = 65536 * d2 + 256 * d1 + d0 with d1, d0 in [-128, 127]
+                    const uint32_t r1 = (wt + 128u) >> 8, r2 = (r1 + 128u) >> 8;
+                    uint8_t* gp = wbytes + c * (QAQ_TILE / 4) * 16 + (r >> 2) * 16 + (r & 3);
+                    gp[0] = (uint8_t)r2;
+                    gp[4] = (uint8_t)r1;
+                    gp[8] = (uint8_t)wt;
                 }
             }
             c_run = fmaf(p, midV[j], c_run);
@@ -495,56 +506,74 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         }
         l_run = l_run * alpha + s;
         lx_run = lx_run * alpha + sx;
-        cp_async_wait<1>();     // this tile's values have landed
         __syncwarp();
 
         // ---- V: integer weighted sums per section, added to the binary32 accumulators once per tile
         if (wok) {
-            int ahi[8], amd[8], alo[8];
+            int acc[MB][4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) { ahi[i] = 0; amd[i] = 0; alo[i] = 0; }
-            v_section<D, 8>(ws.bufV + vb[0], (n[1][0] + 3) >> 2, ws.wts[0], ahi, amd, alo, vh, vgrp);
-            v_section<D, 4>(ws.bufV + vb[1], (n[1][1] + 3) >> 2, ws.wts[1], ahi, amd, alo, vh, vgrp);
-            v_section<D, 2>(ws.bufV + vb[2], (n[1][2] + 3) >> 2, ws.wts[2], ahi, amd, alo, vh, vgrp);
-            v_section<D, 1>(ws.bufV + vb[3], (n[1][3] + 3) >> 2, ws.wts[3], ahi, amd, alo, vh, vgrp);
+            for (int mb = 0; mb < MB; ++mb) { acc[mb][0] = 0; acc[mb][1] = 0; acc[mb][2] = 0; acc[mb][3] = 0; }
+            v_section<D, 8>(tV + vb[0], (n[1][0] + 3) >> 2, ws.wts[0], acc, fg, ft);
+            v_section<D, 4>(tV + vb[1], (n[1][1] + 3) >> 2, ws.wts[1], acc, fg, ft);
+            v_section<D, 2>(tV + vb[2], (n[1][2] + 3) >> 2, ws.wts[2], acc, fg, ft);
+            v_section<D, 1>(tV + vb[3], (n[1][3] + 3) >> 2, ws.wts[3], acc, fg, ft);
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-                X[i] = fmaf(fmaf((float)ahi[i], 65536.0f, (float)(amd[i] * 256 + alo[i])), wunit, X[i]);
+            for (int mb = 0; mb < MB; ++mb) {
+                X[mb][0] = fmaf(fmaf((float)acc[mb][0], dig0, (float)acc[mb][1] * dig1), wunit, X[mb][0]);
+                X[mb][1] = fmaf(fmaf((float)acc[mb][2], dig0, (float)acc[mb][3] * dig1), wunit, X[mb][1]);
+            }
         }
         // value outliers: p_t * (v - mid) per channel
-        const uint32_t* ogV = a.v.outl + (size_t)bh * a.ocap + ooV;
-        const float vunit = outlier_sums(ocV, lane, ws.ivout, [&](uint32_t e, int& cell, float& t) {
-            const uint32_t v = e < (uint32_t)OSTAGE ? ws.outl[1][e] : __ldg(ogV + e);
-            const int tok = (v >> 24) & (QAQ_TILE - 1);
-            cell = (v >> 16) & (D - 1);
-            t = ws.p[tok] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midV[tok]);
-        });
+#pragma unroll 1
+        for (uint32_t e = lane; e < ocV; e += 32) {
+            const uint32_t v = e < 64 ? (e < 32 ? eV[0] : eV[1]) : __ldg(ogV + ooV + e);
+            const int tok = (v >> 24) & (QAQ_TILE - 1), ch = (v >> 16) & (D - 1);
+            const float tm = ws.p[tok] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midV[tok]);
+            outlier_add(&ws.vcorr[0][ch], &ws.vcorr[1][ch], tm);
+        }
         __syncwarp();
-        if (vunit != 0.f) {
-            for (int d = lane; d < D; d += 32) {
-                ws.vout[d] = fmaf(fmaf((float)ws.ivout[1][d], 1.0f / OUTL_LO, (float)ws.ivout[0][d]), vunit, ws.vout[d]);
-                ws.ivout[0][d] = 0; ws.ivout[1][d] = 0;
+        if (ocV) {
+#pragma unroll
+            for (int k = 0; k < (D + 31) / 32; ++k) {
+                const int d = lane + 32 * k;
+                if (d < D) {
+                    const int h = ws.vcorr[0][d], l = ws.vcorr[1][d];
+                    if (h | l) { vout[k] += outlier_sum(h, l); ws.vcorr[0][d] = 0; ws.vcorr[1][d] = 0; }
+                }
             }
         }
         __syncwarp();
-        // ---- the value buffer is free: start the copy of the next tile's values
-        if (has_next) stage_V(nxt); else cp_async_commit();
+        // ---- the back of the buffer is free: start the copy of the next tile's values (beside its keys)
+        uint32_t stVn = 0;
+        if (has_next) {
+            const uint32_t nb = (__shfl_sync(0xFFFFFFFFu, nxt.tb, 5) + 15u) & ~15u;
+            if (nb + stKn <= STAGE) { stVn = nb; stage(ws.buf + STAGE - nb, poolV + __shfl_sync(0xFFFFFFFFu, nxt.tb, 4), nb); }
+        }
+        cp_async_commit();
+        stK = stKn; stV = stVn;
         cur = nxt;
         nxt = fetch_meta(tile + 2 * DEC_WARPS);
     }
     cp_async_wait<0>();
 
-    // ---- warp result: lanes with the same vh hold partial sums of the same channels
+    // ---- warp result: the four lanes ft of a group hold the digit columns of the same channels
     float cs = c_run;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) cs += __shfl_xor_sync(0xFFFFFFFFu, cs, o);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        float v = X[i];
+    for (int k = 0; k < (D + 31) / 32; ++k)
+        if (lane + 32 * k < D) sm.macc[warp][lane + 32 * k] = vout[k] + cs;
+    __syncwarp();
 #pragma unroll
-        for (int o = LPG; o < 32; o <<= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-        if (vgrp == 0) sm.macc[warp][8 * vh + i] = v + ws.vout[8 * vh + i] + cs;
-    }
+    for (int mb = 0; mb < MB; ++mb)
+#pragma unroll
+        for (int s2 = 0; s2 < 2; ++s2) {
+            float v = X[mb][s2];
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+            const int ch = 16 * mb + 8 * s2 + fg;
+            if (ft == 0) sm.macc[warp][ch] += v;
+        }
     if (lane == 0) { sm.mm[warp] = m_run; sm.ml[warp] = l_run; sm.mlx[warp] = lx_run; }
     __syncthreads();
     // ---- merge the warps (log-sum-exp) into this segment's partial

@@ -289,9 +289,10 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
             else        { qaqc::section_bases<D, true>(om, ob);  qaqc::read_pieces<D, true>(src, om, ob, slot, Bx[x], p, cregs[x]); }
         }
     }
-    // ---- pieces into the shared-memory image of the tile
+    // ---- header and pieces into the shared-memory image of the tile
 #pragma unroll
     for (int x = X0; x < X1; ++x) {
+        if (tid < 4) qaqc::write_header(s_img[x - X0], s_tm[x], tid);
         if (!(valid || old)) continue;
         const qaqc::TileMasks tm = s_tm[x];
         uint32_t base[5];

@@ -221,6 +221,7 @@ __global__ void __launch_bounds__(2 * D) requant_kernel(const RequantArgs a) {
     for (int x = 0; x < 2; ++x) {
         if (!changed[x]) continue;
         const TensorStore& ts = x ? a.v : a.k;
+        if (tid < 4) qaqc::write_header(s_img[x], s_tmn[x], tid);
         uint32_t creg[8];
         if (valid) {
             if (UP && Bn[x] > Bo[x]) {

@@ -162,12 +162,13 @@ def test_both_directions_leave_the_cache_as_if_filled_at_the_new_widths(D, shado
     after = qaq.qaq_cache_pool_use(cache)
     check(T2)
     assert after[0] < before[0] and after[1] < before[1] and after[2] == before[2]
-    # nothing but the tiles, 16-byte aligned each.  A tile of keys takes the bytes of its tokens; a tile of values stores
-    # the pieces of each width (8, 4, 2, 1) in groups of four tokens, the last group of a width padded.
+    # nothing but the tiles, 16-byte aligned each.  A tile has a 32-byte header (which slots have a piece of each width);
+    # a tile of keys then takes the bytes of its tokens; a tile of values stores the pieces of each width (8, 4, 2, 1)
+    # in groups of four tokens, the last group of a width padded.
     def tile_bytes(b, is_v):
         if not is_v:
-            return int(b.astype(np.int64).sum()) * D // 8
-        return sum(-(-int(np.count_nonzero(b & w)) // 4) * 4 * D * w // 8 for w in (8, 4, 2, 1))
+            return 32 + int(b.astype(np.int64).sum()) * D // 8
+        return 32 + sum(-(-int(np.count_nonzero(b & w)) // 4) * 4 * D * w // 8 for w in (8, 4, 2, 1))
     per_bh = [max(sum((tile_bytes(bits[x][bh, i:min(i + 64, T2)], x == 1) + 15) // 16 * 16 for i in range(0, T2, 64))
                   for bh in range(wl.bh)) for x in range(2)]
     assert after[0] <= per_bh[0] and after[1] <= per_bh[1]
