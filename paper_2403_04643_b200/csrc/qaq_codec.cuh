@@ -20,9 +20,10 @@
 //            group G = items 4G..4G+3, head_dim*w/2 bytes, made of 32-bit words whose byte lane i belongs to item
 //            4G+i and whose bit field m (bits w*m .. w*m+w-1 of every byte) is one channel, so that a masked word is
 //            four tokens of one channel, one per byte: the A operand of the integer tensor-core instruction
-//            mma.m16n8k32 with rows = channels and k = tokens.  Channel c = 16*mb + 8*s + g has register index
-//            R = g*(head_dim/8) + 2*mb + s and sits in word R / (8/w), field R % (8/w): the registers that the MMA
-//            lane with group id g needs for all 16-channel row blocks mb are consecutive, one vector load.
+//            mma.m16n8k32 with rows = channels and k = tokens.  Channel c sits in word c / (8/w), field
+//            c % (8/w): seen per token, a group interleaves byte by byte the four tokens' rows of packed fields
+//            (consecutive channels, lowest bits first).  The MMA lane with group id g takes the head_dim/8
+//            channels from g*head_dim/8 on as its rows, one vector load per group.
 // The sections are preceded by a header of QAQ_TILE_HDR bytes: the four 64-bit masks "slot t has a piece of width
 // 8, 4, 2, 1" (widths, ranks and section sizes of a tile can be read off them without the per-token metadata).
 // A tile therefore takes the header plus sum_t head_dim*B_t/8 bytes for keys, and that plus the group padding for
@@ -203,61 +204,44 @@ __device__ __forceinline__ void write_pieces(uint8_t* img, const TileMasks& tm, 
             *reinterpret_cast<uint32_t*>(img + base[3] + rank_in(tm, 3, slot) * (D / 8) + p * 4) = acc;
         }
     } else {
-        // values: byte lane (rank & 3) of the words of group rank >> 2.  Channel 32p + 4j + b has g = 4(j&1) + b and
-        // register R = g*NRV + 4p + (j>>1): for every g this thread holds four consecutive registers.
-        constexpr int NRV = D / 8;
+        // values: byte lane (rank & 3) of the words of group rank >> 2; channel 32p + 4j + b is byte b of creg[j]
         if (B & 8) {
             const int r = rank_in(tm, 0, slot);
             uint8_t* grp = img + base[0] + (r >> 2) * (D * 4) + (r & 3);
 #pragma unroll
-            for (int g = 0; g < 8; ++g)
+            for (int j = 0; j < 8; ++j)
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    grp[4 * (g * NRV + 4 * p + q)] = (uint8_t)(creg[(g >> 2) + 2 * q] >> (8 * (g & 3)));
+                for (int b = 0; b < 4; ++b) grp[4 * (32 * p + 4 * j + b)] = (uint8_t)(creg[j] >> (8 * b));
         }
         if (B & 4) {
             const int sh = B & 3, r = rank_in(tm, 1, slot);
             uint8_t* grp = img + base[1] + (r >> 2) * (D * 2) + (r & 3);
 #pragma unroll
-            for (int g = 0; g < 8; ++g)
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint32_t f0 = (creg[(g >> 2) + 4 * h] >> (8 * (g & 3) + sh)) & 15u;
-                    const uint32_t f1 = (creg[(g >> 2) + 4 * h + 2] >> (8 * (g & 3) + sh)) & 15u;
-                    grp[4 * ((g * NRV + 4 * p) / 2 + h)] = (uint8_t)(f0 | (f1 << 4));
-                }
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t x = (creg[j] >> sh) & 0x0F0F0F0Fu;
+                const uint32_t y = x | (x >> 4);     // byte 0: channels 4j, 4j+1; byte 2: channels 4j+2, 4j+3
+                grp[4 * (16 * p + 2 * j)] = (uint8_t)y;
+                grp[4 * (16 * p + 2 * j + 1)] = (uint8_t)(y >> 16);
+            }
         }
         if (B & 2) {
             const int sh = B & 1, r = rank_in(tm, 2, slot);
             uint8_t* grp = img + base[2] + (r >> 2) * D + (r & 3);
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                uint32_t v = 0;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) v |= ((creg[(g >> 2) + 2 * q] >> (8 * (g & 3) + sh)) & 3u) << (2 * q);
-                grp[4 * ((g * NRV + 4 * p) / 4)] = (uint8_t)v;
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t x = (creg[j] >> sh) & 0x03030303u;
+                const uint32_t z = x | (x >> 6);
+                grp[4 * (8 * p + j)] = (uint8_t)(z | (z >> 12));    // the four 2-bit fields of channels 4j..4j+3
             }
         }
         if (B & 1) {
             const int r = rank_in(tm, 3, slot);
-            uint8_t* grp = img + base[3] + (r >> 2) * (D / 2);
-            uint32_t nib[8];
+            uint8_t* grp = img + base[3] + (r >> 2) * (D / 2) + (r & 3);
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                uint32_t v = 0;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) v |= ((creg[(g >> 2) + 2 * q] >> (8 * (g & 3))) & 1u) << q;
-                nib[g] = v;
-            }
-            if (D == 32) {       // registers 4g .. 4g+3: two g share a byte, both held by this thread
-#pragma unroll
-                for (int g = 0; g < 8; g += 2) grp[4 * (g / 2) + (r & 3)] = (uint8_t)(nib[g] | (nib[g + 1] << 4));
-            } else {             // a byte is shared with the neighbouring thread of the token: OR into the (zeroed) image
-#pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                    const int Rb = g * NRV + 4 * p;
-                    atomicOr(reinterpret_cast<uint32_t*>(grp + 4 * (Rb / 8)), nib[g] << (8 * (r & 3) + (Rb & 7)));
-                }
+            for (int j = 0; j < 8; j += 2) {
+                const uint32_t n0 = (((creg[j] & 0x01010101u) * 0x01020408u) >> 24) & 15u;
+                const uint32_t n1 = (((creg[j + 1] & 0x01010101u) * 0x01020408u) >> 24) & 15u;
+                grp[4 * (4 * p + j / 2)] = (uint8_t)(n0 | (n1 << 4));
             }
         }
     }
@@ -296,50 +280,111 @@ __device__ __forceinline__ void read_pieces(const uint8_t* img, const TileMasks&
             for (int m = 0; m < 8; ++m) creg[m] |= (w >> m) & 0x01010101u;
         }
     } else {
-        constexpr int NRV = D / 8;
         if (B & 8) {
             const int r = rank_in(tm, 0, slot);
             const uint8_t* grp = img + base[0] + (r >> 2) * (D * 4) + (r & 3);
 #pragma unroll
-            for (int g = 0; g < 8; ++g)
+            for (int j = 0; j < 8; ++j)
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    creg[(g >> 2) + 2 * q] |= (uint32_t)grp[4 * (g * NRV + 4 * p + q)] << (8 * (g & 3));
+                for (int b = 0; b < 4; ++b) creg[j] |= (uint32_t)grp[4 * (32 * p + 4 * j + b)] << (8 * b);
         }
         if (B & 4) {
             const int sh = B & 3, r = rank_in(tm, 1, slot);
             const uint8_t* grp = img + base[1] + (r >> 2) * (D * 2) + (r & 3);
 #pragma unroll
-            for (int g = 0; g < 8; ++g)
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint32_t b = grp[4 * ((g * NRV + 4 * p) / 2 + h)];
-                    creg[(g >> 2) + 4 * h] |= ((b & 15u) << sh) << (8 * (g & 3));
-                    creg[(g >> 2) + 4 * h + 2] |= ((b >> 4) << sh) << (8 * (g & 3));
-                }
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t b0 = grp[4 * (16 * p + 2 * j)], b1 = grp[4 * (16 * p + 2 * j + 1)];
+                const uint32_t x = (b0 & 15u) | ((b0 >> 4) << 8) | ((b1 & 15u) << 16) | ((b1 >> 4) << 24);
+                creg[j] |= x << sh;
+            }
         }
         if (B & 2) {
             const int sh = B & 1, r = rank_in(tm, 2, slot);
             const uint8_t* grp = img + base[2] + (r >> 2) * D + (r & 3);
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                const uint32_t b = grp[4 * ((g * NRV + 4 * p) / 4)];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) creg[(g >> 2) + 2 * q] |= (((b >> (2 * q)) & 3u) << sh) << (8 * (g & 3));
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t b = grp[4 * (8 * p + j)];
+                const uint32_t u = b | (b << 12);
+                creg[j] |= ((u | (u << 6)) & 0x03030303u) << sh;
             }
         }
         if (B & 1) {
             const int r = rank_in(tm, 3, slot);
             const uint8_t* grp = img + base[3] + (r >> 2) * (D / 2) + (r & 3);
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                const int Rb = g * NRV + 4 * p;
-                const uint32_t b = (uint32_t)grp[4 * (Rb / 8)] >> (Rb & 7);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) creg[(g >> 2) + 2 * q] |= ((b >> q) & 1u) << (8 * (g & 3));
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t b = ((uint32_t)grp[4 * (4 * p + j / 2)] >> (4 * (j & 1))) & 15u;
+                creg[j] |= (b * 0x00204081u) & 0x01010101u;
             }
         }
     }
+}
+
+// ------------------------------------------------------------------------------------------ values, fast writer
+// The quantizer builds the values of a tile in two steps so that it never stores single bytes of a word that four
+// tokens share.  Step 1 (write_planes_v): every token writes its row of packed w-bit fields (consecutive channels,
+// lowest bits first) on its own with vector stores: the item of rank r of section c takes the quarter (r & 3) of
+// its group.  Step 2 (group_unit_v): 16 bytes of the final layout, words 4u .. 4u+3 of a group, are the 4x4 byte
+// transpose of word u of the group's four rows.
+template <int D>
+__device__ __forceinline__ void write_planes_v(uint8_t* img, const TileMasks& tm, const uint32_t (&base)[5], int slot, int B,
+                                               int p, const uint32_t (&creg)[8]) {
+    if (B & 8) {
+        const int r = rank_in(tm, 0, slot);
+        store_words<8>(img + base[0] + (r >> 2) * (D * 4) + (r & 3) * D + 32 * p, creg);
+    }
+    if (B & 4) {
+        const int sh = B & 3, r = rank_in(tm, 1, slot);
+        uint32_t y[8], w[4];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t x = (creg[j] >> sh) & 0x0F0F0F0Fu;
+            y[j] = x | (x >> 4);                     // byte 0: channels 4j, 4j+1; byte 2: channels 4j+2, 4j+3
+        }
+#pragma unroll
+        for (int m = 0; m < 4; ++m) w[m] = prmt(y[2 * m], y[2 * m + 1], 0x6420u);
+        store_words<4>(img + base[1] + (r >> 2) * (D * 2) + (r & 3) * (D / 2) + 16 * p, w);
+    }
+    if (B & 2) {
+        const int sh = B & 1, r = rank_in(tm, 2, slot);
+        uint32_t w[2] = {0, 0};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t x = (creg[j] >> sh) & 0x03030303u;
+            const uint32_t z = x | (x >> 6);
+            w[j >> 2] |= ((z | (z >> 12)) & 0xFFu) << (8 * (j & 3));
+        }
+        store_words<2>(img + base[2] + (r >> 2) * D + (r & 3) * (D / 4) + 8 * p, w);
+    }
+    if (B & 1) {
+        const int r = rank_in(tm, 3, slot);
+        uint32_t w = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) w |= ((((creg[j] & 0x01010101u) * 0x01020408u) >> 24) & 15u) << (4 * j);
+        *reinterpret_cast<uint32_t*>(img + base[3] + (r >> 2) * (D / 2) + (r & 3) * (D / 8) + 4 * p) = w;
+    }
+}
+
+// 16 bytes at offset o (a multiple of 16, QAQ_TILE_HDR <= o < base[4]) of the final layout of a values tile, from
+// the rows that write_planes_v left in the image
+template <int D, int C>
+__device__ __forceinline__ uint4 group_unit_c(const uint8_t* img, uint32_t sec, uint32_t rel) {
+    constexpr int W = 8 >> C, GB = D * W / 2;
+    const uint32_t G = rel / GB, u = (rel % GB) >> 4;
+    const uint8_t* grp = img + sec + G * GB + 4 * u;
+    uint32_t in[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) in[i] = *reinterpret_cast<const uint32_t*>(grp + i * (GB / 4));
+    const uint32_t t0 = prmt(in[0], in[1], 0x5140u), t1 = prmt(in[2], in[3], 0x5140u);
+    const uint32_t t2 = prmt(in[0], in[1], 0x7362u), t3 = prmt(in[2], in[3], 0x7362u);
+    return make_uint4(prmt(t0, t1, 0x5410u), prmt(t0, t1, 0x7632u), prmt(t2, t3, 0x5410u), prmt(t2, t3, 0x7632u));
+}
+template <int D>
+__device__ __forceinline__ uint4 group_unit_v(const uint8_t* img, const uint32_t (&base)[5], uint32_t o) {
+    if (o >= base[3]) return group_unit_c<D, 3>(img, base[3], o - base[3]);
+    if (o >= base[2]) return group_unit_c<D, 2>(img, base[2], o - base[2]);
+    if (o >= base[1]) return group_unit_c<D, 1>(img, base[1], o - base[1]);
+    return group_unit_c<D, 0>(img, base[0], o - base[0]);
 }
 
 // The w-bit piece (w = 8 >> c) of channel d of the item of rank r in section c (for the canonical export).
@@ -353,8 +398,7 @@ __device__ __forceinline__ uint32_t piece_at(const uint8_t* tile, const uint32_t
         return (word >> (8 * i + w * (j & (per - 1)))) & ((1u << w) - 1u);
     } else {
         const uint8_t* grp = tile + base[c] + (size_t)(r >> 2) * (D * w / 2);
-        const int R = (d & 7) * (D / 8) + 2 * (d >> 4) + ((d >> 3) & 1);
-        return ((uint32_t)grp[4 * (R / per) + (r & 3)] >> (w * (R & (per - 1)))) & ((1u << w) - 1u);
+        return ((uint32_t)grp[4 * (d / per) + (r & 3)] >> (w * (d & (per - 1)))) & ((1u << w) - 1u);
     }
 }
 

@@ -144,7 +144,7 @@ __device__ __forceinline__ void k_section(const uint8_t* sec, int n, int* dots, 
 }
 
 // weighted sums over the groups of one value section: 8 groups (32 tokens) per instruction, lane 4g+t holds the
-// channels 16*mb + 8*s + g of groups t and t+4
+// channels (D/8)*g + 2*mb + s (rows g + 8s of row block mb) of groups t and t+4
 template <int D, int W>
 __device__ __forceinline__ void v_section(const uint8_t* sec, int ngroups, const uint32_t (*wts)[4], int (&acc)[D / 16][4], int g, int t) {
     constexpr int NRV = D / 8, GB = D * W / 2;
@@ -245,7 +245,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         qb[r] = fg < 2 ? v : 0u;
     }
 
-    float X[MB][2];             // channels 16*mb + 8*s + fg: this lane's share of the digit columns (summed over ft at the end)
+    float X[MB][2];             // rows fg and fg + 8 of row block mb: this lane's share of the digit columns (summed over ft at the end)
 #pragma unroll
     for (int mb = 0; mb < MB; ++mb) { X[mb][0] = 0.f; X[mb][1] = 0.f; }
     // what the accumulator columns of this lane stand for: lane ft = 0 holds the digits 2^16 and 2^8, ft = 1 the units
@@ -316,9 +316,9 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         const uint8_t* tK = stK ? ws.buf : poolK + offK;
         const uint8_t* tV = stV ? ws.buf + STAGE - stV : poolV + offV;
         // the first outlier entries of the tile (used after the section loops)
-        uint32_t eK[2], eV[2];
+        uint32_t eK[3], eV[3];
 #pragma unroll
-        for (int k = 0; k < 2; ++k) {
+        for (int k = 0; k < 3; ++k) {
             eK[k] = lane + 32 * k < ocK ? __ldg(ogK + ooK + lane + 32 * k) : 0u;
             eV[k] = lane + 32 * k < ocV ? __ldg(ogV + ooV + lane + 32 * k) : 0u;
         }
@@ -371,7 +371,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         // key outliers: q_ch * (x - mid) per token
 #pragma unroll 1
         for (uint32_t e = lane; e < ocK; e += 32) {
-            const uint32_t v = e < 64 ? (e < 32 ? eK[0] : eK[1]) : __ldg(ogK + ooK + e);
+            const uint32_t v = e < 96 ? (e < 32 ? eK[0] : (e < 64 ? eK[1] : eK[2])) : __ldg(ogK + ooK + e);
             const int tok = (v >> 24) & (QAQ_TILE - 1);
             const float tm = sm.qf[(v >> 16) & (D - 1)] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midK[tok]);
             outlier_add(&ws.kcorr[0][tok], &ws.kcorr[1][tok], tm);
@@ -526,7 +526,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         // value outliers: p_t * (v - mid) per channel
 #pragma unroll 1
         for (uint32_t e = lane; e < ocV; e += 32) {
-            const uint32_t v = e < 64 ? (e < 32 ? eV[0] : eV[1]) : __ldg(ogV + ooV + e);
+            const uint32_t v = e < 96 ? (e < 32 ? eV[0] : (e < 64 ? eV[1] : eV[2])) : __ldg(ogV + ooV + e);
             const int tok = (v >> 24) & (QAQ_TILE - 1), ch = (v >> 16) & (D - 1);
             const float tm = ws.p[tok] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midV[tok]);
             outlier_add(&ws.vcorr[0][ch], &ws.vcorr[1][ch], tm);
@@ -571,7 +571,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
             float v = X[mb][s2];
             v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
             v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
-            const int ch = 16 * mb + 8 * s2 + fg;
+            const int ch = (D / 8) * fg + 2 * mb + s2;     // row fg + 8*s2 of row block mb
             if (ft == 0) sm.macc[warp][ch] += v;
         }
     if (lane == 0) { sm.mm[warp] = m_run; sm.ml[warp] = l_run; sm.mlx[warp] = lx_run; }

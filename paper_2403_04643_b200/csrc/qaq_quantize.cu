@@ -9,7 +9,8 @@
 //   phase 2  warp 0: which slots have a piece of each width (ballots), section sizes of the tile,
 //            exclusive scan of the outlier counts, space taken from the (b,h) pools by atomicAdd
 //   phase 3  codes (binary32: one sub, one mul, round down), pieces written into a shared-memory
-//            image of the tile in the section layout of qaq_codec.cuh, vector stores; outlier
+//            image of the tile in the section layout of qaq_codec.cuh (values as token-major planes
+//            that the copy-out transposes into groups of four tokens), vector stores; outlier
 //            entries placed by popc ranks
 // A tile that is continued (an append behind a partly filled tile) is built anew: the codes of
 // its old tokens are read back from the pool, the image of old and new tokens replaces it.
@@ -289,15 +290,21 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
             else        { qaqc::section_bases<D, true>(om, ob);  qaqc::read_pieces<D, true>(src, om, ob, slot, Bx[x], p, cregs[x]); }
         }
     }
-    // ---- header and pieces into the shared-memory image of the tile
+    // ---- header and pieces into the shared-memory image of the tile (the values as token-major planes, which the
+    //      copy to global memory turns into groups of four tokens)
+    uint32_t vbase[5] = {0, 0, 0, 0, 0};
 #pragma unroll
     for (int x = X0; x < X1; ++x) {
         if (tid < 4) qaqc::write_header(s_img[x - X0], s_tm[x], tid);
-        if (!(valid || old)) continue;
         const qaqc::TileMasks tm = s_tm[x];
-        uint32_t base[5];
-        if (x == 0) { qaqc::section_bases<D, false>(tm, base); qaqc::write_pieces<D, false>(s_img[x - X0], tm, base, slot, Bx[x], p, cregs[x]); }
-        else        { qaqc::section_bases<D, true>(tm, base);  qaqc::write_pieces<D, true>(s_img[x - X0], tm, base, slot, Bx[x], p, cregs[x]); }
+        if (x == 0) {
+            uint32_t base[5];
+            qaqc::section_bases<D, false>(tm, base);
+            if (valid || old) qaqc::write_pieces<D, false>(s_img[x - X0], tm, base, slot, Bx[x], p, cregs[x]);
+        } else {
+            qaqc::section_bases<D, true>(tm, vbase);
+            if (valid || old) qaqc::write_planes_v<D>(s_img[x - X0], tm, vbase, slot, Bx[x], p, cregs[x]);
+        }
     }
     // ---- allocation results (the atomics were issued before the codes were computed).  A pool without room:
     //      the space is given back, nothing about the tile is published and the CTA stops; the device status
@@ -348,8 +355,12 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
         const TensorStore& ts = x ? a.v : a.k;
         uint8_t* dst = ts.codes + (size_t)bh * a.pool_bytes + s_base[x];
         const uint32_t nb = (s_tot[x] + 15u) & ~15u;     // tiles start 16-byte aligned and own a rounded amount
-        for (uint32_t o = tid * 16; o < nb; o += NT * 16)
-            *reinterpret_cast<uint4*>(dst + o) = *reinterpret_cast<const uint4*>(s_img[x - X0] + o);
+        for (uint32_t o = tid * 16; o < nb; o += NT * 16) {
+            uint4 v;
+            if (x == 0 || o < (uint32_t)qaqc::QAQ_TILE_HDR) v = *reinterpret_cast<const uint4*>(s_img[x - X0] + o);
+            else v = qaqc::group_unit_v<D>(s_img[x - X0], vbase, o);
+            *reinterpret_cast<uint4*>(dst + o) = v;
+        }
         // outliers in (token, channel) order: entries of lanes p' < p come first
         uint32_t ob = valid ? ~inl[x] : 0u;
         const uint32_t mine = (uint32_t)__popc(ob);
