@@ -143,6 +143,18 @@ qaq_status qaq_prefill_window(const qaq_config* cfg, const void* Q, const void* 
                               uint8_t* nvalid, float* qnorm2, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The scalar `qnorm2` of qaq_policy_from_hyper from a set of queries (Section 4.1, end of "Key cache
+ * quantization": the distribution of the squared norm of the queries is taken beforehand and its upper
+ * 10 % quantile stands for sum_d Q_d^2 in the key rule).  values: binary32 [n] on the device, e.g. the
+ * qnorm2 array of qaq_prefill_window or a longer history kept by the caller; NaNs are not counted.
+ * With N counted values sorted ascending the result is sorted[N-1-floor(upper_frac*N)], i.e. at most
+ * upper_frac*N values lie above it (0 if N = 0).  out: one binary32 on the device, written
+ * asynchronously on stream.  Exact (radix select by one CTA: meant for up to a few million values).
+ * Errors: QAQ_ERR_INVALID_ARG (null pointer, n < 1, upper_frac outside [0,1)).
+ */
+qaq_status qaq_qnorm2_quantile(const float* values, long n, double upper_frac, float* out, void* stream);
+
+/*
  * S2+S3: append n_new tokens per (b,h) to the cache: outlier split (entries outside
  * [lo,hi] are kept as binary16 in a sparse side list and take code 0), uniform
  * quantization of each token at its width (Section 4.1: the range [min,max] of the

@@ -12,6 +12,8 @@ import os
 import subprocess
 from dataclasses import dataclass
 
+import math
+
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -284,6 +286,18 @@ def prefill_window(Q_u16, K_u16, scale):
     nvalid = np.minimum(n, T - np.arange(T)).astype(np.uint8)
     qf = Q.view(np.float16).astype(np.float64) * scale
     return ring, nvalid, (qf * qf).sum(axis=1)
+
+
+def qnorm2_quantile(values, upper_frac: float = 0.1) -> float:
+    """Section 4.1 (end of "Key cache quantization"): the upper quantile of the squared query norms that stands for
+    sum_d Q_d^2 in the key rule.  With the N non-NaN values sorted ascending: sorted[N-1-floor(upper_frac*N)]
+    (at most upper_frac*N values lie above it); 0 for an empty list."""
+    v = np.asarray(values, dtype=np.float32).ravel()
+    v = np.sort(v[~np.isnan(v)])
+    if v.size == 0:
+        return 0.0
+    k = min(int(math.floor(upper_frac * v.size)), v.size - 1)
+    return float(v[v.size - 1 - k])
 
 
 def decode(q_u16, qk: QuantTensor, qv: QuantTensor, scale):

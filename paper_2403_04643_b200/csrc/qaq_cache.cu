@@ -60,15 +60,21 @@ extern "C" qaq_status qaq_cache_create(const qaq_config* cfg, qaq_cache** out) {
     size_t off = 0;
     auto carve = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     size_t o_codes[2], o_bits[2], o_mnmx[2], o_toff[2], o_tnb[2], o_tooff[2], o_tocnt[2], o_outl[2], o_pe[2], o_ope[2];
+    // three regions: pools that need no initialisation; tables that start at zero; what qaq_cache_reset clears
+    // (one contiguous range, one memset)
     for (int x = 0; x < 2; ++x) {
         o_codes[x] = carve(BH * c->pool_bytes);
-        o_bits[x] = carve(BH * c->tmax_pad);
+        o_outl[x] = carve(BH * (size_t)c->ocap * 4);
+    }
+    for (int x = 0; x < 2; ++x) {
         o_mnmx[x] = carve(BH * c->tmax_pad * 4);
         o_toff[x] = carve(BH * c->ntiles * 4);
-        o_tnb[x] = carve(BH * c->ntiles * 4);
         o_tooff[x] = carve(BH * c->ntiles * 4);
+    }
+    for (int x = 0; x < 2; ++x) {
+        o_bits[x] = carve(BH * c->tmax_pad);
+        o_tnb[x] = carve(BH * c->ntiles * 4);
         o_tocnt[x] = carve(BH * c->ntiles * 4);
-        o_outl[x] = carve(BH * (size_t)c->ocap * 4);
         o_pe[x] = carve(BH * 4);
         o_ope[x] = carve(BH * 4);
     }
@@ -90,15 +96,12 @@ extern "C" qaq_status qaq_cache_create(const qaq_config* cfg, qaq_cache** out) {
         t.opool_end = (uint32_t*)(base + o_ope[x]);
     }
     c->d_status = (int*)(base + o_status);
+    c->reset_off = o_bits[0];
+    c->reset_bytes = off - o_bits[0];
     // metadata and tables start at zero; code pools need no initialisation
-    for (int x = 0; x < 2; ++x) {
-        if (cudaMemset(c->t[x].bits, 0, o_outl[x] - o_bits[x]) != cudaSuccess ||
-            cudaMemset(c->t[x].pool_end, 0, BH * 4) != cudaSuccess ||
-            cudaMemset(c->t[x].opool_end, 0, BH * 4) != cudaSuccess) {
-            (void)cudaGetLastError(); cudaFree(c->slab); free(c); return QAQ_ERR_CUDA;
-        }
+    if (cudaMemset(base + o_mnmx[0], 0, off - o_mnmx[0]) != cudaSuccess) {
+        (void)cudaGetLastError(); cudaFree(c->slab); free(c); return QAQ_ERR_CUDA;
     }
-    if (cudaMemset(c->d_status, 0, 256) != cudaSuccess) { (void)cudaGetLastError(); cudaFree(c->slab); free(c); return QAQ_ERR_CUDA; }
     c->tokens = 0;
     *out = c;
     return QAQ_OK;
@@ -116,16 +119,8 @@ extern "C" qaq_status qaq_cache_destroy(qaq_cache* c) {
 extern "C" qaq_status qaq_cache_reset(qaq_cache* c, void* stream) {
     if (!c) return QAQ_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
-    const size_t BH = (size_t)c->BH;
-    for (int x = 0; x < 2; ++x) {
-        TensorStore& t = c->t[x];
-        QAQ_CUDA_TRY(cudaMemsetAsync(t.bits, 0, BH * c->tmax_pad, s));
-        QAQ_CUDA_TRY(cudaMemsetAsync(t.tile_nbytes, 0, BH * c->ntiles * 4, s));
-        QAQ_CUDA_TRY(cudaMemsetAsync(t.tile_ocnt, 0, BH * c->ntiles * 4, s));
-        QAQ_CUDA_TRY(cudaMemsetAsync(t.pool_end, 0, BH * 4, s));
-        QAQ_CUDA_TRY(cudaMemsetAsync(t.opool_end, 0, BH * 4, s));
-    }
-    QAQ_CUDA_TRY(cudaMemsetAsync(c->d_status, 0, 4, s));
+    // widths, tile lengths, outlier counts, pool ends and the status word: one contiguous range
+    QAQ_CUDA_TRY(cudaMemsetAsync((char*)c->slab + c->reset_off, 0, c->reset_bytes, s));
     c->tokens = 0;
     return QAQ_OK;
 }

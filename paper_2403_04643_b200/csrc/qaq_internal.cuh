@@ -39,6 +39,7 @@ struct qaq_cache {
     int* d_status;      // sticky device-side status
     void* slab;         // the one allocation everything above lives in
     size_t slab_bytes;
+    size_t reset_off, reset_bytes;   // the range of the slab that qaq_cache_reset clears
     long tokens;        // host counter
     // lazily sized staging for the *_host entry points
     void* stage[8];

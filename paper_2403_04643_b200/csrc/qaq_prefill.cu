@@ -191,6 +191,66 @@ __global__ void __launch_bounds__(256) window_normalize_kernel(const PrefillArgs
     }
 }
 
+// Upper quantile of a list of binary32 values (the squared query norms): exact 4 x 8-bit radix select on
+// order-preserving keys by one CTA.  NaNs are not counted.
+constexpr int QS_THREADS = 1024;
+__device__ __forceinline__ uint32_t order_key(float f) {
+    const uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__global__ void __launch_bounds__(QS_THREADS) quantile_kernel(const float* __restrict__ v, long n, double upper_frac, float* out) {
+    __shared__ unsigned int hist[256];
+    __shared__ unsigned long long s_count;
+    __shared__ uint32_t s_prefix;
+    __shared__ unsigned long long s_rank;
+    const int tid = threadIdx.x;
+    if (tid == 0) s_count = 0;
+    __syncthreads();
+    unsigned long long mine = 0;
+    for (long i = tid; i < n; i += QS_THREADS) mine += (v[i] == v[i]) ? 1ull : 0ull;
+    atomicAdd(&s_count, mine);
+    __syncthreads();
+    const unsigned long long N = s_count;
+    if (N == 0) { if (tid == 0) *out = 0.f; return; }
+    if (tid == 0) {
+        unsigned long long k = (unsigned long long)floor(upper_frac * (double)N);
+        if (k > N - 1) k = N - 1;
+        s_rank = N - 1 - k;          // ascending rank of the answer
+        s_prefix = 0;
+    }
+    __syncthreads();
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        const uint32_t prefix = s_prefix, pmask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+        if (tid < 256) hist[tid] = 0;
+        __syncthreads();
+        for (long i = tid; i < n; i += QS_THREADS) {
+            const float f = v[i];
+            if (f == f) {
+                const uint32_t key = order_key(f);
+                if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 0xFF], 1u);
+            }
+        }
+        __syncthreads();
+        if (tid == 0) {
+            unsigned long long r = s_rank;
+            int b = 0;
+            for (; b < 255; ++b) {
+                if (r < hist[b]) break;
+                r -= hist[b];
+            }
+            s_rank = r;
+            s_prefix = prefix | ((uint32_t)b << shift);
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        const uint32_t key = s_prefix;
+        const uint32_t u = (key & 0x80000000u) ? (key & 0x7FFFFFFFu) : ~key;
+        *out = __uint_as_float(u);
+    }
+}
+
 }  // namespace
 
 extern "C" qaq_status qaq_prefill_window_workspace_bytes(const qaq_config* cfg, int n_tokens, size_t* host_out) {
@@ -225,6 +285,13 @@ extern "C" qaq_status qaq_prefill_window(const qaq_config* cfg, const void* Q, c
         default: return QAQ_ERR_UNSUPPORTED_SHAPE;
     }
     window_normalize_kernel<<<grid, 256, 0, s>>>(a);
+    QAQ_CUDA_TRY(cudaGetLastError());
+    return QAQ_OK;
+}
+
+extern "C" qaq_status qaq_qnorm2_quantile(const float* values, long n, double upper_frac, float* out, void* stream) {
+    if (!values || !out || n < 1 || !(upper_frac >= 0.0 && upper_frac < 1.0)) return QAQ_ERR_INVALID_ARG;
+    quantile_kernel<<<1, QS_THREADS, 0, (cudaStream_t)stream>>>(values, n, upper_frac, out);
     QAQ_CUDA_TRY(cudaGetLastError());
     return QAQ_OK;
 }

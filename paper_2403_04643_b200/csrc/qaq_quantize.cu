@@ -172,8 +172,21 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
         if (XSEL != 0 && !given && valid) {
             nv_tok = a.nvalid[(size_t)bh * a.n_new + tn];
             nv_tok = nv_tok < a.W ? nv_tok : a.W;
+            // every row of the window is read (the ring is allocated in full), rows the token has no score in are
+            // left out of the maximum: the loads then depend on nothing and go out together
             const float* r = a.ring + (size_t)bh * a.W * a.n_new + tn;
-            for (int i = p; i < nv_tok; i += P) shat = fmaxf(shat, r[(size_t)i * a.n_new]);
+            int i = p;
+            for (; i + 7 * P < a.W; i += 8 * P) {
+                float v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = __ldg(r + (size_t)(i + u * P) * a.n_new);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) if (i + u * P < nv_tok) shat = fmaxf(shat, v[u]);
+            }
+            for (; i < a.W; i += P) {
+                const float v = __ldg(r + (size_t)i * a.n_new);
+                if (i < nv_tok) shat = fmaxf(shat, v);
+            }
         }
 #pragma unroll
         for (int o = 1; o < P; o <<= 1) shat = fmaxf(shat, __shfl_xor_sync(0xFFFFFFFFu, shat, o));

@@ -23,6 +23,7 @@ EXPORTED = [
     "qaq_quantize_append", "qaq_decode_workspace_bytes", "qaq_decode_attention", "qaq_quantize_append_host",
     "qaq_decode_attention_host", "qaq_cache_stats", "qaq_cache_export", "qaq_decode_attention_static",
     "qaq_requantize_down", "qaq_requantize", "qaq_cache_compact", "qaq_cache_pool_use", "qaq_prefill_window_workspace_bytes", "qaq_prefill_window",
+    "qaq_qnorm2_quantile",
 ]
 
 
@@ -87,6 +88,7 @@ def lib():
         L.qaq_prefill_window_workspace_bytes.argtypes = [C.POINTER(Config), C.c_int, C.POINTER(C.c_size_t)]
         L.qaq_prefill_window.argtypes = [C.POINTER(Config), C.c_void_p, C.c_void_p, C.c_long, C.c_long, C.c_long, C.c_int,
                                          C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qaq_qnorm2_quantile.argtypes = [C.c_void_p, C.c_long, C.c_double, C.c_void_p, C.c_void_p]
         L.qaq_cache_compact.argtypes = [C.c_void_p, C.c_void_p]
         L.qaq_cache_pool_use.argtypes = [C.c_void_p, C.POINTER(C.c_long), C.POINTER(C.c_long), C.c_void_p]
         L.qaq_requantize.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_long, C.c_long, C.c_long, C.c_void_p, C.c_void_p,
@@ -220,6 +222,15 @@ def qaq_prefill_window(cfg: Config, Q, K, softmax_scale, want_qnorm2=False):
     _check(lib().qaq_prefill_window(C.byref(cfg), _ptr(Q), _ptr(K), sb, sh, st, T, float(softmax_scale), _ptr(ring),
                                     _ptr(nvalid), _ptr(qn), _ptr(ws), ws.numel(), _stream()), "qaq_prefill_window")
     return (ring, nvalid, qn) if want_qnorm2 else (ring, nvalid)
+
+
+def qaq_qnorm2_quantile(values, upper_frac=0.1, out=None):
+    """Upper quantile of squared query norms (fp32 tensor on the device, any shape); returns a 1-element device tensor."""
+    assert values.dtype == torch.float32 and values.is_contiguous()
+    if out is None:
+        out = torch.empty((1,), dtype=torch.float32, device=values.device)
+    _check(lib().qaq_qnorm2_quantile(_ptr(values), values.numel(), float(upper_frac), _ptr(out), _stream()), "qaq_qnorm2_quantile")
+    return out
 
 
 def qaq_requantize_down(cache: Cache, *, bitsK=None, bitsV=None, policy=None, ring=None, nvalid=None):

@@ -65,3 +65,40 @@ def test_window_feeds_the_width_selection_like_any_ring():
         assert np.all(np.abs(got.astype(int) - wv.astype(int)) <= 1)
         agree += int((got == wv).sum()); total += T
     assert agree >= 0.995 * total
+
+
+@pytest.mark.parametrize("n", [1, 7, 1000, 262144])
+def test_qnorm2_quantile_equals_the_oracle(n):
+    """qaq_qnorm2_quantile (Section 4.1, squared query norm quantile) against the oracle's order statistic, bit for bit:
+    ties, negative values, zeros of both signs and NaNs in the list."""
+    rng = np.random.default_rng(100 + n)
+    v = np.round(rng.chisquare(8, size=n), 2).astype(np.float32)
+    if n >= 7:
+        v[::5] = -v[::5]
+        v[3] = np.nan
+        v[4] = 0.0
+        v[5] = -0.0
+    for frac in (0.1, 0.0, 0.5):
+        got = qaq.qaq_qnorm2_quantile(torch.from_numpy(v).cuda(), frac).cpu().numpy()[0]
+        want = np.float32(oracle.qnorm2_quantile(v, frac))
+        assert got == want, (n, frac, got, want)
+
+
+def test_policy_from_the_window_queries():
+    """The chain a caller runs after a prefill: window rows and per-query squared norms (qaq_prefill_window), their upper
+    10 % quantile (qaq_qnorm2_quantile), the policy constants; against the same chain on the oracle."""
+    wl = synth.scaled(synth.CONFIGS["C2"], tokens=640, heads=4)
+    K, _ = synth.make_kv(wl)
+    BH, D, W, T = wl.bh, wl.head_dim, wl.window, wl.tokens
+    g = torch.Generator().manual_seed(11)
+    Q = torch.randn((BH, W, D), generator=g).to(torch.float16)
+    scale = 1.0 / math.sqrt(D)
+    cfg = qaq.make_config(wl.batch, wl.heads, D, T, wl.bits_min, wl.bits_max, W, wl.alpha)
+    _, _, qn = qaq.qaq_prefill_window(cfg, Q.cuda(), K.cuda(), scale, want_qnorm2=True)
+    qd = float(qaq.qaq_qnorm2_quantile(qn, 0.1).cpu()[0])
+    qf = (Q.double() * scale) ** 2
+    want = oracle.qnorm2_quantile(qf.sum(-1).numpy().astype(np.float32), 0.1)
+    assert abs(qd - want) <= 1e-5 * want                                     # binary32 sums in another order
+    pd = qaq.qaq_policy_from_hyper(0.002, 0.01, qd, T)
+    cK, cV = oracle.policy(0.002, 0.01, want, T)
+    assert abs(pd.cK - cK) <= 1e-5 * cK and pd.cV == np.float32(cV)

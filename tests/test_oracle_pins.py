@@ -519,3 +519,25 @@ def test_prefill_window_rows_are_causal_softmax_rows_newest_first():
     # feeds the window maximum like any other ring
     shat = oracle.window_max(ring.astype(np.float32), nvalid)
     assert np.allclose(shat, ring.astype(np.float32).max(axis=0))
+
+
+# ----------------------------------------------------------------------------- squared query norm quantile
+def test_qnorm2_quantile_closed_form_counts_and_nans():
+    """Section 4.1, end of "Key cache quantization": the upper 10 % quantile of the squared query norms.  Pinned by a
+    closed form (1..100: ten values lie above 90), by the counting rule on random data with ties (at most frac*N
+    values above the result, more than frac*N at or above it), by a plain Python sort, and by NaNs being left out."""
+    assert oracle.qnorm2_quantile(np.arange(1, 101, dtype=np.float32), 0.1) == 90.0
+    assert oracle.qnorm2_quantile(np.arange(1, 101, dtype=np.float32)[::-1].copy(), 0.1) == 90.0
+    assert oracle.qnorm2_quantile(np.array([3.0], dtype=np.float32), 0.1) == 3.0
+    assert oracle.qnorm2_quantile(np.array([], dtype=np.float32), 0.1) == 0.0
+    rng = np.random.default_rng(5)
+    for n, frac in ((10, 0.1), (37, 0.1), (1000, 0.1), (1000, 0.25), (513, 0.0)):
+        v = np.round(rng.chisquare(8, size=n), 1).astype(np.float32)        # rounded: many ties
+        q = oracle.qnorm2_quantile(v, frac)
+        above, at_or_above = int(np.count_nonzero(v > q)), int(np.count_nonzero(v >= q))
+        assert above <= frac * n < at_or_above
+        k = int(math.floor(frac * n))
+        assert q == sorted(float(x) for x in v)[n - 1 - k]
+    v = np.array([np.nan, 1.0, -np.nan, 5.0, 2.0, np.nan, 4.0, 3.0], dtype=np.float32)
+    assert oracle.qnorm2_quantile(v, 0.2) == 4.0                            # five values count: sorted[5-1-1]
+    assert oracle.qnorm2_quantile(np.full(4, np.nan, dtype=np.float32), 0.1) == 0.0
