@@ -257,11 +257,13 @@ qaq_status qaq_decode_attention_host(qaq_cache* c, const void* q, float softmax_
  *   - Limit: 2 * CTAs * (head_dim+3) * 4 bytes + batch*heads*8 must fit in 4 MiB, where
  *     CTAs is the launch width qaq_decode_attention would use: at most max(592,
  *     batch*heads), and batch*heads when every (b,h) holds fewer than 4 tiles of 64 tokens
- *     (e.g. 256 (b,h) x 4096 tokens x head_dim 128 needs 0.6 MiB; up to about 4000 (b,h)
- *     at head_dim 128 always fit).  Larger shapes get QAQ_ERR_WORKSPACE and nothing is
+ *     (e.g. 256 (b,h) x 4096 tokens x head_dim 128 needs 0.6 MiB; at head_dim 128 up to
+ *     3971 (b,h) fit whatever their length).  Larger shapes get QAQ_ERR_WORKSPACE and nothing is
  *     launched -- use qaq_decode_attention with your own workspace.
  *   - The first call on each device looks up the array's device address (once, with that
- *     device current).  Make that first call outside any stream capture.
+ *     device current); the CUDA runtime may also load the library's kernels at that moment,
+ *     which can take device memory of its own.  Make that first call as a warm-up, outside
+ *     any stream capture; later calls take nothing.
  *   - All calls on a device share the one array.  Calls that may overlap on the GPU
  *     (different streams, no ordering between them) race on it and give wrong results;
  *     keep them on one stream or order them yourself.  The array keeps the previous

@@ -231,3 +231,16 @@ def test_thresholds_with_nans_of_both_signs(tokens):
         b, h = divmod(bh, wl.heads)
         want = (*oracle.thresholds(Ku[b, h], wl.alpha), *oracle.thresholds(Vu[b, h], wl.alpha))
         assert np.array_equal(thr[bh], np.array(want, dtype=np.float32)), (bh, thr[bh], want)
+
+
+def test_decode_twice_gives_the_same_bits():
+    # outlier corrections are summed with integer atomics and everything else in a fixed order: a repeat of the call,
+    # and a call with the score row requested, return the same output bit for bit
+    wl = synth.scaled(synth.CONFIGS["C4"], batch=2, heads=3, tokens=1500, alpha=0.10)      # many outliers per tile
+    K, V, q, ring, nv = make_inputs(wl)
+    pol = qaq.qaq_policy_from_hyper(*HYPER["C4"], wl.tokens)
+    cfg, cache, thr, out, scores, dev = gpu_pipeline(wl, K, V, q, ring, nv, pol)
+    first = out.cpu().numpy().view(np.uint32).copy()
+    for _ in range(3):
+        again = qaq.qaq_decode_attention(cache, dev[2], 1.0 / math.sqrt(wl.head_dim))
+        assert np.array_equal(again.cpu().numpy().view(np.uint32), first)

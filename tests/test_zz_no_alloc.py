@@ -51,6 +51,9 @@ def test_static_scratch_decode_matches_workspace_decode_twice_in_a_row():
         got = out.cpu().numpy()
         assert np.all(np.isfinite(got))
         assert np.all(np.abs(got - want) <= ATOL + RTOL * np.abs(want)), np.abs(got - want).max()
+        # both entry points run the same kernels with the same split, and every sum in them is either an exact
+        # integer sum or taken in a fixed order: the results are the same bit for bit
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
     # and once more on the first cache, after the other shape has used the array
     wl, cache = caches[0]
     q = synth.make_query(wl, step=7).cuda()
@@ -58,6 +61,36 @@ def test_static_scratch_decode_matches_workspace_decode_twice_in_a_row():
     out = torch.empty((wl.bh, wl.head_dim), dtype=torch.float32, device="cuda")
     qaq.qaq_decode_attention_static(cache, q, 1.0 / math.sqrt(wl.head_dim), out)
     assert np.all(np.abs(out.cpu().numpy() - want) <= ATOL + RTOL * np.abs(want))
+
+
+def _one_tile_cache(B, H, D=128, T=64):
+    cfg = qaq.make_config(B, H, D, T, 2, 8, 1, 0.0)
+    cache = qaq.Cache(cfg)
+    K = torch.zeros((B, H, T, D), dtype=torch.float16, device="cuda")
+    thr = torch.tensor([[-1.0, 1.0, -1.0, 1.0]], device="cuda").repeat(B * H, 1).contiguous()
+    bits = torch.full((B * H, T), 2, dtype=torch.uint8, device="cuda")
+    qaq.qaq_quantize_append(cache, K, K, thr, bitsK=bits, bitsV=bits)
+    return cache
+
+
+def test_static_scratch_limit_is_exact_and_a_warm_call_takes_no_device_memory():
+    # one tile per (b,h): the partials take (b,h) x (2 x 131 + 2) floats, so 3971 (b,h) fit the 4 MiB and 3972 do not
+    D = 128
+    fits, too_large = _one_tile_cache(11, 361), _one_tile_cache(12, 331)
+    for cache, bh, ok in ((fits, 3971, True), (too_large, 3972, False)):
+        q = torch.zeros((bh, D), dtype=torch.float16, device="cuda")
+        out = torch.empty((bh, D), dtype=torch.float32, device="cuda")
+        if ok:
+            qaq.qaq_decode_attention_static(cache, q, 1.0, out)          # first call on this device: symbol look-up, module load
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
+            qaq.qaq_decode_attention_static(cache, q, 1.0, out)
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free_before
+        else:
+            with pytest.raises(qaq.QaqError) as e:
+                qaq.qaq_decode_attention_static(cache, q, 1.0, out)
+            assert e.value.code == 5
 
 
 def test_static_scratch_rejects_shapes_beyond_its_limit():
