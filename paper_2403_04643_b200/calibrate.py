@@ -31,3 +31,68 @@ def calibrate(cfg, K, V, ring, nvalid, thr, T, qnorm2, target_k=4.0, target_v=3.
         else: hi_x = mx
     sS, sX = 10.0 ** (0.5 * (lo_s + hi_s)), 10.0 ** (0.5 * (lo_x + hi_x))
     return sS, sX, qaq.qaq_policy_from_hyper(sS, sX, qnorm2, T)
+
+
+# ----------------------------------------------------------------------------- frozen values per workload
+# The calibrated numbers are kept in hyper.json beside this file, so that runs reproduce and every arm of the
+# benchmark reports the same configuration.  `python -m paper_2403_04643_b200.calibrate` (on a GPU) writes it anew.
+import json
+import os
+
+from . import synth
+
+HYPER_JSON = os.path.join(os.path.dirname(os.path.abspath(__file__)), "hyper.json")
+# name -> (workload, tokens the widths are selected on, target mean widths (K, V))
+POINTS = {
+    "C2": ("C2", 4096, (4.0, 3.0)),
+    "C3": ("C3", 4096, (4.0, 3.0)),
+    "C3_low": ("C3", 4096, (2.2, 2.2)),
+    "C4": ("C4", 8192, (4.0, 3.0)),
+    "C5": ("C5", 32768, (4.0, 3.0)),
+}
+
+
+def frozen(name):
+    """(sigmaS_max, sigmaX_max, qnorm2) of a named point, or None if hyper.json does not hold it."""
+    try:
+        with open(HYPER_JSON) as f:
+            e = json.load(f)[name]
+        return float(e["sigmaS_max"]), float(e["sigmaX_max"]), float(e["qnorm2"])
+    except (OSError, KeyError, ValueError):
+        return None
+
+
+def qnorm2_of_queries(wl, dev, layers=None, upper_frac=0.1):
+    """Upper 10 % quantile of sum_d (q_d / sqrt(D))^2 over the workload's decode queries (Section 4.1), on the device."""
+    import torch
+    qs = [synth.make_query(wl, l, device=dev) for l in range(layers or wl.layers)]
+    q = torch.stack(qs).float() / math.sqrt(wl.head_dim)
+    return float(qaq.qaq_qnorm2_quantile((q * q).sum(-1).contiguous(), upper_frac).cpu()[0])
+
+
+def _main():
+    import torch
+    dev = torch.device("cuda", 0)
+    out = {}
+    for name, (key, T, targets) in POINTS.items():
+        wl = synth.scaled(synth.CONFIGS[key], layers=synth.CONFIGS[key].layers, tokens=T, grow_to=0)
+        K, V = synth.make_kv(wl, 0, device=dev)
+        ring, nv = synth.make_score_ring(wl, 0, device=dev)
+        cfg = qaq.make_config(wl.batch, wl.heads, wl.head_dim, T, wl.bits_min, wl.bits_max, wl.window, wl.alpha)
+        thr = qaq.qaq_outlier_thresholds(cfg, K, V)
+        qn = qnorm2_of_queries(wl, dev)
+        sS, sX, pol = calibrate(cfg, K, V, ring, nv, thr, T, qn, target_k=targets[0], target_v=targets[1])
+        mk, mv = _mean_bits(cfg, pol, K, V, ring, nv, thr)
+        out[name] = {"sigmaS_max": sS, "sigmaX_max": sX, "qnorm2": qn, "target_mean_bits": list(targets),
+                     "mean_bits_layer0": [round(mk, 3), round(mv, 3)], "workload": wl.name, "tokens": T}
+        del K, V, ring, nv
+        torch.cuda.empty_cache()
+    path = os.environ.get("QAQ_HYPER_OUT", HYPER_JSON)
+    with open(path, "w") as f:
+        json.dump(out, f, indent=1)
+        f.write("\n")
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    _main()
