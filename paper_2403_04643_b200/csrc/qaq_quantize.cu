@@ -113,7 +113,13 @@ __device__ __forceinline__ uint32_t pool_take(uint32_t* pool, uint32_t amount, u
 // XSEL: -1 = keys and values in one CTA; 0 / 1 = this launch handles only the keys / only the values of a tile
 // (half the registers and shared memory per CTA, so more tiles are in flight per SM).
 template <int D, bool SELECT_ONLY, int XSEL>
-__global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 128 ? 5 : 6)) quant_kernel(const QuantArgs a) {
+#ifndef QSPLIT_CTAS
+#define QSPLIT_CTAS 6
+#endif
+#ifndef QSPLIT_MIN_CTAS
+#define QSPLIT_MIN_CTAS 4096
+#endif
+__global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 128 ? QSPLIT_CTAS : 6)) quant_kernel(const QuantArgs a) {
     constexpr int X0 = XSEL < 0 ? 0 : XSEL, X1 = XSEL < 0 ? 2 : XSEL + 1;
     constexpr int P = D / 32;            // lanes per token
     constexpr int NT = 2 * D;            // threads
@@ -422,7 +428,7 @@ qaq_status launch_x(int D, dim3 grid, const QuantArgs& a, cudaStream_t s) {
 template <bool SELECT_ONLY>
 qaq_status launch(int D, dim3 grid, const QuantArgs& a, cudaStream_t s) {
     qaq_status st;
-    if (SELECT_ONLY || grid.x * grid.y < 4096) {
+    if (SELECT_ONLY || grid.x * grid.y < QSPLIT_MIN_CTAS) {
         st = launch_x<SELECT_ONLY, -1>(D, grid, a, s);
     } else {   // large launches: keys and values of a tile in separate CTAs
         st = launch_x<SELECT_ONLY, 0>(D, grid, a, s);
