@@ -29,8 +29,7 @@ typedef enum {
     QAQ_ERR_UNSUPPORTED_SHAPE = 2, /* head_dim not in {32,64,128}, widths outside 1..8, ... */
     QAQ_ERR_CAPACITY = 3,          /* token or outlier capacity of the cache exceeded */
     QAQ_ERR_CUDA = 4,              /* a CUDA runtime call failed */
-    QAQ_ERR_WORKSPACE = 5,         /* workspace too small or misaligned */
-    QAQ_ERR_TIMEOUT = 6            /* a bounded device-side wait ran out */
+    QAQ_ERR_WORKSPACE = 5          /* workspace too small or misaligned */
 } qaq_status;
 
 const char* qaq_status_string(qaq_status s);
@@ -199,8 +198,8 @@ qaq_status qaq_requantize_down(qaq_cache* c, const uint8_t* bitsK, const uint8_t
 
 /*
  * Re-quantization in both directions (Section 4.2, "Integration in text generation process":
- * tokens whose new width is lower are quantized further; "for those otherwise, we take the
- * unquantized KV cache from CPU memory and re-quantize it to the required bits").
+ * tokens whose new width is lower are quantized further, the others are recomputed at the
+ * width they need from the unquantized copy that the caller keeps, in CPU memory in the paper).
  * K_full, V_full: the unquantized binary16 values of the cached tokens, [batch][heads][>=tokens]
  * [head_dim] with element strides as in qaq_outlier_thresholds, in any memory the GPU can read:
  * device memory, or pinned host memory that is mapped into the device's address space (then only
@@ -210,7 +209,7 @@ qaq_status qaq_requantize_down(qaq_cache* c, const uint8_t* bitsK, const uint8_t
  * they are: a raised token keeps its min, max and outliers and gets the codes an append at the
  * new width would have produced, so after the call the cache equals one filled at the new widths.
  * A closed tile that grows is moved to the end of its (b,h) pool and its old bytes stay unused
- * until qaq_cache_reset; if the pool has no room left the tile is left as it was and
+ * until qaq_cache_compact (or qaq_cache_reset); if the pool has no room left the tile is left as it was and
  * qaq_cache_stats().device_status reports QAQ_ERR_CAPACITY.
  */
 qaq_status qaq_requantize(qaq_cache* c, const void* K_full, const void* V_full, long stride_b, long stride_h,

@@ -164,8 +164,9 @@ void qaq_oracle_window_max(const float* ring, const uint8_t* nvalid, int W, long
 }
 
 // ---- O2: range of the non-outlier values of one token (Section 4.2) -----------
-// "the distribution range is significantly reduced without outliers": min and max
-// are taken over the entries that are not outliers.  No such entry: range [0,0].
+// With the outliers set aside the range of a token shrinks a lot, which is the point of
+// setting them aside: min and max are taken over the entries that are not outliers.
+// No such entry: range [0,0].
 void qaq_oracle_masked_range(const uint16_t* x, int D, float lo, float hi, float* mn, float* mx) {
     bool any = false;
     float a = 0.f, b = 0.f;
@@ -288,8 +289,8 @@ void qaq_oracle_unpack_token(const uint8_t* bytes, int D, int B, uint8_t* codes)
 // ---- S2+S3 for one (b,h) tensor: outlier split, quantize, pack ----------------
 // Outputs (canonical form): mn[T], step[T], off[T+1] (byte offsets, exclusive prefix
 // sum of D*B/8), stream (tokens concatenated), rowptr[T+1], ch[], val[] (outliers
-// in (token, channel) order, value = the original binary16 bits: "stored accurately
-// without quantization error").  Returns the number of outliers, or -1 if out_cap
+// in (token, channel) order, value = the original binary16 bits, so that an outlier
+// comes back without any quantization error).  Returns the number of outliers, or -1 if out_cap
 // or stream_cap is too small.
 long qaq_oracle_quantize(const uint16_t* x, long T, int D, float lo, float hi, const uint8_t* bits,
                          float* mn, float* step, uint32_t* off, uint8_t* stream, long stream_cap,

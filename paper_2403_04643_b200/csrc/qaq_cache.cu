@@ -14,7 +14,6 @@ extern "C" const char* qaq_status_string(qaq_status s) {
         case QAQ_ERR_CAPACITY: return "capacity exceeded";
         case QAQ_ERR_CUDA: return "CUDA error";
         case QAQ_ERR_WORKSPACE: return "workspace too small or misaligned";
-        case QAQ_ERR_TIMEOUT: return "device-side wait timed out";
     }
     return "unknown status";
 }
