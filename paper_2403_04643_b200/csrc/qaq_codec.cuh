@@ -142,6 +142,17 @@ __device__ __forceinline__ void write_header(uint8_t* img, const TileMasks& tm, 
 __device__ __forceinline__ int rank_in(const TileMasks& tm, int c, int slot) {
     return __popcll(tm.m[c] & ((1ull << slot) - 1ull));
 }
+// The ranks of one slot in the four sections, either taken from the masks when asked for or handed over packed
+// (rank in section c in byte c; a tile has at most 64 items per section).
+struct MaskRanks {
+    const TileMasks& tm;
+    int slot;
+    __device__ __forceinline__ int operator()(int c) const { return rank_in(tm, c, slot); }
+};
+struct PackedRanks {
+    uint32_t rk;
+    __device__ __forceinline__ int operator()(int c) const { return (int)((rk >> (8 * c)) & 0xFFu); }
+};
 
 template <int NW>
 __device__ __forceinline__ void store_words(uint8_t* p, const uint32_t* w) {   // p is min(16, 4*NW)-byte aligned
@@ -172,18 +183,18 @@ __device__ __forceinline__ void load_words(const uint8_t* p, uint32_t* w) {
 
 // The pieces of one thread's 32 channels (block p of the token in `slot`, codes one per byte in creg) written
 // into a tile image (shared or global memory, 16-byte aligned).
-template <int D, bool IS_V>
-__device__ __forceinline__ void write_pieces(uint8_t* img, const TileMasks& tm, const uint32_t (&base)[5], int slot, int B,
-                                             int p, const uint32_t (&creg)[8]) {
+template <int D, bool IS_V, typename Ranks>
+__device__ __forceinline__ void write_pieces(uint8_t* img, const Ranks& rk, const uint32_t (&base)[5], int B, int p,
+                                             const uint32_t (&creg)[8]) {
     if (!IS_V) {
-        if (B & 8) store_words<8>(img + base[0] + rank_in(tm, 0, slot) * D + p * 32, creg);
+        if (B & 8) store_words<8>(img + base[0] + rk(0) * D + p * 32, creg);
         if (B & 4) {
             const int sh = B & 3;
             uint32_t w[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j)
                 w[j] = ((creg[2 * j] >> sh) & 0x0F0F0F0Fu) | (((creg[2 * j + 1] >> sh) & 0x0F0F0F0Fu) << 4);
-            store_words<4>(img + base[1] + rank_in(tm, 1, slot) * (D / 2) + p * 16, w);
+            store_words<4>(img + base[1] + rk(1) * (D / 2) + p * 16, w);
         }
         if (B & 2) {
             const int sh = B & 1;
@@ -195,18 +206,18 @@ __device__ __forceinline__ void write_pieces(uint8_t* img, const TileMasks& tm, 
                 for (int m = 0; m < 4; ++m) acc |= ((creg[4 * j + m] >> sh) & 0x03030303u) << (2 * m);
                 w[j] = acc;
             }
-            store_words<2>(img + base[2] + rank_in(tm, 2, slot) * (D / 4) + p * 8, w);
+            store_words<2>(img + base[2] + rk(2) * (D / 4) + p * 8, w);
         }
         if (B & 1) {
             uint32_t acc = 0;
 #pragma unroll
             for (int m = 0; m < 8; ++m) acc |= (creg[m] & 0x01010101u) << m;
-            *reinterpret_cast<uint32_t*>(img + base[3] + rank_in(tm, 3, slot) * (D / 8) + p * 4) = acc;
+            *reinterpret_cast<uint32_t*>(img + base[3] + rk(3) * (D / 8) + p * 4) = acc;
         }
     } else {
         // values: byte lane (rank & 3) of the words of group rank >> 2; channel 32p + 4j + b is byte b of creg[j]
         if (B & 8) {
-            const int r = rank_in(tm, 0, slot);
+            const int r = rk(0);
             uint8_t* grp = img + base[0] + (r >> 2) * (D * 4) + (r & 3);
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -214,7 +225,7 @@ __device__ __forceinline__ void write_pieces(uint8_t* img, const TileMasks& tm, 
                 for (int b = 0; b < 4; ++b) grp[4 * (32 * p + 4 * j + b)] = (uint8_t)(creg[j] >> (8 * b));
         }
         if (B & 4) {
-            const int sh = B & 3, r = rank_in(tm, 1, slot);
+            const int sh = B & 3, r = rk(1);
             uint8_t* grp = img + base[1] + (r >> 2) * (D * 2) + (r & 3);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -225,7 +236,7 @@ __device__ __forceinline__ void write_pieces(uint8_t* img, const TileMasks& tm, 
             }
         }
         if (B & 2) {
-            const int sh = B & 1, r = rank_in(tm, 2, slot);
+            const int sh = B & 1, r = rk(2);
             uint8_t* grp = img + base[2] + (r >> 2) * D + (r & 3);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -235,7 +246,7 @@ __device__ __forceinline__ void write_pieces(uint8_t* img, const TileMasks& tm, 
             }
         }
         if (B & 1) {
-            const int r = rank_in(tm, 3, slot);
+            const int r = rk(3);
             uint8_t* grp = img + base[3] + (r >> 2) * (D / 2) + (r & 3);
 #pragma unroll
             for (int j = 0; j < 8; j += 2) {
@@ -245,6 +256,12 @@ __device__ __forceinline__ void write_pieces(uint8_t* img, const TileMasks& tm, 
             }
         }
     }
+}
+
+template <int D, bool IS_V>
+__device__ __forceinline__ void write_pieces(uint8_t* img, const TileMasks& tm, const uint32_t (&base)[5], int slot, int B,
+                                             int p, const uint32_t (&creg)[8]) {
+    write_pieces<D, IS_V>(img, MaskRanks{tm, slot}, base, B, p, creg);
 }
 
 // The inverse: codes of one thread's 32 channels (one per byte) put together from the token's pieces.
@@ -326,15 +343,15 @@ __device__ __forceinline__ void read_pieces(const uint8_t* img, const TileMasks&
 // lowest bits first) on its own with vector stores: the item of rank r of section c takes the quarter (r & 3) of
 // its group.  Step 2 (group_unit_v): 16 bytes of the final layout, words 4u .. 4u+3 of a group, are the 4x4 byte
 // transpose of word u of the group's four rows.
-template <int D>
-__device__ __forceinline__ void write_planes_v(uint8_t* img, const TileMasks& tm, const uint32_t (&base)[5], int slot, int B,
-                                               int p, const uint32_t (&creg)[8]) {
+template <int D, typename Ranks>
+__device__ __forceinline__ void write_planes_v(uint8_t* img, const Ranks& rk, const uint32_t (&base)[5], int B, int p,
+                                               const uint32_t (&creg)[8]) {
     if (B & 8) {
-        const int r = rank_in(tm, 0, slot);
+        const int r = rk(0);
         store_words<8>(img + base[0] + (r >> 2) * (D * 4) + (r & 3) * D + 32 * p, creg);
     }
     if (B & 4) {
-        const int sh = B & 3, r = rank_in(tm, 1, slot);
+        const int sh = B & 3, r = rk(1);
         uint32_t y[8], w[4];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -346,7 +363,7 @@ __device__ __forceinline__ void write_planes_v(uint8_t* img, const TileMasks& tm
         store_words<4>(img + base[1] + (r >> 2) * (D * 2) + (r & 3) * (D / 2) + 16 * p, w);
     }
     if (B & 2) {
-        const int sh = B & 1, r = rank_in(tm, 2, slot);
+        const int sh = B & 1, r = rk(2);
         uint32_t w[2] = {0, 0};
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -357,7 +374,7 @@ __device__ __forceinline__ void write_planes_v(uint8_t* img, const TileMasks& tm
         store_words<2>(img + base[2] + (r >> 2) * D + (r & 3) * (D / 4) + 8 * p, w);
     }
     if (B & 1) {
-        const int r = rank_in(tm, 3, slot);
+        const int r = rk(3);
         uint32_t w = 0;
 #pragma unroll
         for (int j = 0; j < 8; ++j) w |= ((((creg[j] & 0x01010101u) * 0x01020408u) >> 24) & 15u) << (4 * j);

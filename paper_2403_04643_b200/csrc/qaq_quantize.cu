@@ -139,6 +139,8 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
     __shared__ uint8_t s_bits[2][QAQ_TILE];   // widths of the tile's slots (0: empty)
     __shared__ uint32_t s_cnt[2][QAQ_TILE];   // outlier counts of the new tokens, then exclusive offsets
     __shared__ qaqc::TileMasks s_tm[2];
+    __shared__ uint32_t s_rank[2][QAQ_TILE];   // ranks of the slots in the four sections, one per byte
+    __shared__ uint32_t s_sec[2][5];           // byte offsets of the sections
     __shared__ uint32_t s_tot[2], s_base[2], s_obase[2], s_olimit[2];
     __shared__ int s_skip;
     __shared__ __align__(16) uint8_t s_img[SELECT_ONLY ? 1 : X1 - X0][SELECT_ONLY ? 16 : IMG];  // the tile as it will be stored
@@ -260,12 +262,22 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
         for (int x = X0; x < X1; ++x) {
             const uint32_t b0 = s_bits[x][lane], b1 = s_bits[x][lane + 32];
             qaqc::TileMasks tm;
+            uint32_t rk0 = 0, rk1 = 0;       // ranks of slots lane and lane + 32
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                tm.m[c] = (unsigned long long)__ballot_sync(0xFFFFFFFFu, (b0 & (8u >> c)) != 0) |
-                          ((unsigned long long)__ballot_sync(0xFFFFFFFFu, (b1 & (8u >> c)) != 0) << 32);
+            for (int c = 0; c < 4; ++c) {
+                const unsigned lo = __ballot_sync(0xFFFFFFFFu, (b0 & (8u >> c)) != 0), hi = __ballot_sync(0xFFFFFFFFu, (b1 & (8u >> c)) != 0);
+                tm.m[c] = (unsigned long long)lo | ((unsigned long long)hi << 32);
+                const unsigned below = (1u << lane) - 1u;
+                rk0 |= (uint32_t)__popc(lo & below) << (8 * c);
+                rk1 |= (uint32_t)(__popc(lo) + __popc(hi & below)) << (8 * c);
+            }
+            s_rank[x][lane] = rk0; s_rank[x][lane + 32] = rk1;
             uint32_t base[5];
             if (x == 0) qaqc::section_bases<D, false>(tm, base); else qaqc::section_bases<D, true>(tm, base);
+            if (lane == 0) {
+#pragma unroll
+                for (int c = 0; c < 5; ++c) s_sec[x][c] = base[c];
+            }
             const uint32_t c0 = s_cnt[x][lane], c1 = s_cnt[x][lane + 32];
             uint32_t ic0 = c0, ic1 = c1;
 #pragma unroll
@@ -315,14 +327,16 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
 #pragma unroll
     for (int x = X0; x < X1; ++x) {
         if (tid < 4) qaqc::write_header(s_img[x - X0], s_tm[x], tid);
-        const qaqc::TileMasks tm = s_tm[x];
+        const qaqc::PackedRanks rk{s_rank[x][slot & (QAQ_TILE - 1)]};
         if (x == 0) {
             uint32_t base[5];
-            qaqc::section_bases<D, false>(tm, base);
-            if (valid || old) qaqc::write_pieces<D, false>(s_img[x - X0], tm, base, slot, Bx[x], p, cregs[x]);
+#pragma unroll
+            for (int c = 0; c < 5; ++c) base[c] = s_sec[x][c];
+            if (valid || old) qaqc::write_pieces<D, false>(s_img[x - X0], rk, base, Bx[x], p, cregs[x]);
         } else {
-            qaqc::section_bases<D, true>(tm, vbase);
-            if (valid || old) qaqc::write_planes_v<D>(s_img[x - X0], tm, vbase, slot, Bx[x], p, cregs[x]);
+#pragma unroll
+            for (int c = 0; c < 5; ++c) vbase[c] = s_sec[x][c];
+            if (valid || old) qaqc::write_planes_v<D>(s_img[x - X0], rk, vbase, Bx[x], p, cregs[x]);
         }
     }
     // ---- allocation results (the atomics were issued before the codes were computed).  A pool without room:
