@@ -192,8 +192,8 @@ __device__ __forceinline__ void write_pieces(uint8_t* img, const Ranks& rk, cons
             const int sh = B & 3;
             uint32_t w[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                w[j] = ((creg[2 * j] >> sh) & 0x0F0F0F0Fu) | (((creg[2 * j + 1] >> sh) & 0x0F0F0F0Fu) << 4);
+            for (int j = 0; j < 4; ++j)     // the odd register goes straight to the high nibbles: one shift by 4 - sh
+                w[j] = ((creg[2 * j] >> sh) & 0x0F0F0F0Fu) | ((creg[2 * j + 1] << (4 - sh)) & 0xF0F0F0F0u);
             store_words<4>(img + base[1] + rk(1) * (D / 2) + p * 16, w);
         }
         if (B & 2) {
@@ -201,9 +201,9 @@ __device__ __forceinline__ void write_pieces(uint8_t* img, const Ranks& rk, cons
             uint32_t w[2];
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
-                uint32_t acc = 0;
+                uint32_t acc = (creg[4 * j] >> sh) & 0x03030303u;
 #pragma unroll
-                for (int m = 0; m < 4; ++m) acc |= ((creg[4 * j + m] >> sh) & 0x03030303u) << (2 * m);
+                for (int m = 1; m < 4; ++m) acc |= (creg[4 * j + m] << (2 * m - sh)) & (0x03030303u << (2 * m));
                 w[j] = acc;
             }
             store_words<2>(img + base[2] + rk(2) * (D / 4) + p * 8, w);
@@ -364,20 +364,26 @@ __device__ __forceinline__ void write_planes_v(uint8_t* img, const Ranks& rk, co
     }
     if (B & 2) {
         const int sh = B & 1, r = rk(2);
-        uint32_t w[2] = {0, 0};
+        // the four 2-bit fields of a register gathered into one byte by a multiplication: field b (bit 8b + sh) times
+        // 2^(24 - 6b - sh) lands at bit 24 + 2b, and no other product of a field and a term reaches the top byte
+        const uint32_t msk = 0x03030303u << sh, mul = 0x01041040u >> sh;
+        uint32_t t[8], w[2];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const uint32_t x = (creg[j] >> sh) & 0x03030303u;
-            const uint32_t z = x | (x >> 6);
-            w[j >> 2] |= ((z | (z >> 12)) & 0xFFu) << (8 * (j & 3));
-        }
+        for (int j = 0; j < 8; ++j) t[j] = (creg[j] & msk) * mul;
+#pragma unroll
+        for (int k = 0; k < 2; ++k)
+            w[k] = prmt(prmt(t[4 * k], t[4 * k + 1], 0x0073u), prmt(t[4 * k + 2], t[4 * k + 3], 0x0073u), 0x5410u);
         store_words<2>(img + base[2] + (r >> 2) * D + (r & 3) * (D / 4) + 8 * p, w);
     }
     if (B & 1) {
         const int r = rk(3);
-        uint32_t w = 0;
+        // the low bits of a register's four bytes gathered into a nibble by a multiplication (bit 8b times 2^(24 - 7b)
+        // lands at bit 24 + b); odd registers are placed four bits higher, so that a pair fills the top byte
+        uint32_t t[4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) w |= ((((creg[j] & 0x01010101u) * 0x01020408u) >> 24) & 15u) << (4 * j);
+        for (int k = 0; k < 4; ++k)
+            t[k] = (((creg[2 * k] & 0x01010101u) * 0x01020408u) & 0x0F000000u) | (((creg[2 * k + 1] & 0x01010101u) * 0x10204080u) & 0xF0000000u);
+        const uint32_t w = prmt(prmt(t[0], t[1], 0x0073u), prmt(t[2], t[3], 0x0073u), 0x5410u);
         *reinterpret_cast<uint32_t*>(img + base[3] + (r >> 2) * (D / 2) + (r & 3) * (D / 8) + 4 * p) = w;
     }
 }
