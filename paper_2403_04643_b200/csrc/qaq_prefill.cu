@@ -10,6 +10,8 @@
 // on the tensor cores (mma.sync m16n8k16, binary16 in, binary32 accumulate); with n <= 64 rows it is
 // bound by reading K once.  Two kernels: logits + per-chunk (max, sum of exponentials) of every
 // row; then the rows are normalised in place with the merged (max, sum).
+#include <cooperative_groups.h>
+
 #include "qaq_internal.cuh"
 
 namespace {
@@ -191,6 +193,167 @@ __global__ void __launch_bounds__(256) window_normalize_kernel(const PrefillArgs
     }
 }
 
+// ---- one pass: the CTAs of one (b,h) form a thread-block cluster.  Each keeps the logits of its 512 tokens in
+// shared memory, the per-row (max, sum) of the CTAs are exchanged through distributed shared memory, and the
+// normalised rows are written once: K is read once and the ring written once (no logits in global memory, no
+// workspace).  Used while a (b,h) fits a portable cluster (up to 8 x 512 tokens); longer sequences take the two
+// kernels above.
+constexpr int PC_WARPS = 8;
+constexpr int PC_CHUNK = 512;           // tokens per CTA: 64 per warp
+constexpr int PC_MAXCTA = 8;            // portable cluster size
+constexpr int PC_PITCH = PC_CHUNK + 8;  // row pitch of the logits tile in floats (spreads the rows of a fragment over the banks)
+
+template <int D>
+__global__ void __launch_bounds__(PC_WARPS * 32) window_cluster_kernel(const PrefillArgs a) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    constexpr int WPL = D / 8;
+    constexpr int KS = D / 16;
+    extern __shared__ __align__(16) float s_l[];            // [n][PC_PITCH] logits of this CTA's tokens
+    __shared__ float2 s_part[PC_WARPS][32];
+    __shared__ float2 s_stat[PW_MAXQ];                       // (max, sum of exponentials) of every row over this CTA's tokens
+    __shared__ float s_m[PW_MAXQ], s_inv[PW_MAXQ];
+    const int bh = blockIdx.y, chunk = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, c = lane & 3;
+    const int b_idx = bh / a.H, h_idx = bh % a.H;
+    const __half* Kb = a.K + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
+    const __half* Qb = a.Q + (size_t)bh * a.n * D;
+    const float NEG = __int_as_float(0xff800000);
+
+    if (a.qnorm2 && chunk == 0) {
+        for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
+            float s = 0.f;
+            for (int d = 0; d < D; ++d) { const float f = a.scale * __half2float(Qb[(size_t)i * D + d]); s = fmaf(f, f, s); }
+            a.qnorm2[(size_t)bh * a.n + i] = s;
+        }
+    }
+    const int t_cta = chunk * PC_CHUNK;
+    const int t_warp = t_cta + warp * (PC_CHUNK / PC_WARPS);
+
+    for (int mp = 0; mp * 32 < a.n; ++mp) {            // two 16-row tiles of queries at a time
+        uint32_t afr[2][KS][4];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+            const int r0 = mp * 32 + mt * 16 + g, r1 = r0 + 8;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                const uint32_t* q0 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r0 * D + c * (D / 4)) + 2 * ks;
+                const uint32_t* q1 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r1 * D + c * (D / 4)) + 2 * ks;
+                afr[mt][ks][0] = r0 < a.n ? q0[0] : 0u;
+                afr[mt][ks][1] = r1 < a.n ? q1[0] : 0u;
+                afr[mt][ks][2] = r0 < a.n ? q0[1] : 0u;
+                afr[mt][ks][3] = r1 < a.n ? q1[1] : 0u;
+            }
+        }
+        float rm[2][2], rs[2][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) { rm[mt][0] = rm[mt][1] = NEG; rs[mt][0] = rs[mt][1] = 0.f; }
+
+#pragma unroll 2
+        for (int step = 0; step < PC_CHUNK / PC_WARPS / 8; ++step) {
+            const int t0 = t_warp + 8 * step;
+            if (t0 >= a.T) break;
+            uint32_t bw[WPL];
+            {
+                const int t = t0 + g;
+                const uint4* src = reinterpret_cast<const uint4*>(Kb + (size_t)(t < a.T ? t : 0) * a.st + c * (D / 4));
+#pragma unroll
+                for (int i = 0; i < WPL / 4; ++i) {
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (t < a.T) v = src[i];
+                    bw[4 * i] = v.x; bw[4 * i + 1] = v.y; bw[4 * i + 2] = v.z; bw[4 * i + 3] = v.w;
+                }
+            }
+            float acc[2][4];
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) mma_16816(acc[mt], afr[mt][ks], bw[2 * ks], bw[2 * ks + 1]);
+            }
+            // acc[mt][0..1]: row g, tokens t0+2c, t0+2c+1;  acc[mt][2..3]: row g+8
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int hr = 0; hr < 2; ++hr) {
+                    const int i = mp * 32 + mt * 16 + g + 8 * hr;          // query
+                    if (i >= a.n) continue;
+                    const int last = a.T - a.n + i;                         // last token the query sees
+                    const float l0 = a.scale * acc[mt][2 * hr], l1 = a.scale * acc[mt][2 * hr + 1];
+                    *reinterpret_cast<float2*>(&s_l[(size_t)i * PC_PITCH + (t0 - t_cta) + 2 * c]) = make_float2(l0, l1);
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int t = t0 + 2 * c + e;
+                        const float l = e ? l1 : l0;
+                        if (t < a.T && t <= last) {
+                            const float mnew = fmaxf(rm[mt][hr], l);
+                            rs[mt][hr] = rs[mt][hr] * __expf(rm[mt][hr] - mnew) + __expf(l - mnew);
+                            rm[mt][hr] = mnew;
+                        }
+                    }
+                }
+        }
+        // merge the four lanes of a row, then the warps, into this CTA's (max, sum) of the row
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int hr = 0; hr < 2; ++hr) {
+                float m = rm[mt][hr], s = rs[mt][hr];
+#pragma unroll
+                for (int o = 1; o < 4; o <<= 1) {
+                    const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, o), s2 = __shfl_xor_sync(0xFFFFFFFFu, s, o);
+                    const float mn = fmaxf(m, m2);
+                    s = (m == NEG ? 0.f : s * __expf(m - mn)) + (m2 == NEG ? 0.f : s2 * __expf(m2 - mn));
+                    m = mn;
+                }
+                if (c == 0) s_part[warp][mt * 16 + g + 8 * hr] = make_float2(m, s);
+            }
+        __syncthreads();
+        for (int il = threadIdx.x; il < 32; il += blockDim.x) {
+            const int i = mp * 32 + il;
+            if (i >= a.n) continue;
+            float m = NEG, s = 0.f;
+            for (int w = 0; w < PC_WARPS; ++w) {
+                const float2 p = s_part[w][il];
+                const float mn = fmaxf(m, p.x);
+                s = (m == NEG ? 0.f : s * __expf(m - mn)) + (p.x == NEG ? 0.f : p.y * __expf(p.x - mn));
+                m = mn;
+            }
+            s_stat[i] = make_float2(m, s);
+        }
+        __syncthreads();
+    }
+    // ---- every CTA of the (b,h) has its row statistics: merge them across the cluster
+    cluster.sync();
+    const unsigned ncta = cluster.num_blocks();
+    for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
+        float m = NEG, s = 0.f;
+        for (unsigned r = 0; r < ncta; ++r) {
+            const float2 p = *cluster.map_shared_rank(&s_stat[i], r);
+            const float mn = fmaxf(m, p.x);
+            s = (m == NEG ? 0.f : s * __expf(m - mn)) + (p.x == NEG ? 0.f : p.y * __expf(p.x - mn));
+            m = mn;
+        }
+        s_m[i] = m;
+        s_inv[i] = s > 0.f ? 1.0f / s : 0.f;
+    }
+    __syncthreads();
+    // ---- normalised rows, newest first, written once; rows-per-token counts
+    const int nt = min(PC_CHUNK, a.T - t_cta);
+    for (int r = warp; r < a.n; r += PC_WARPS) {
+        const int i = a.n - 1 - r;
+        const int last = a.T - a.n + i;
+        const float M = s_m[i], inv = s_inv[i];
+        float* row = a.ring + ((size_t)bh * a.n + r) * a.T + t_cta;
+        const float* src = s_l + (size_t)i * PC_PITCH;
+        for (int k = lane; k < nt; k += 32) row[k] = (t_cta + k <= last) ? __expf(src[k] - M) * inv : 0.f;
+    }
+    for (int k = threadIdx.x; k < nt; k += blockDim.x) a.nvalid[(size_t)bh * a.T + t_cta + k] = (uint8_t)min(a.n, a.T - (t_cta + k));
+    cluster.sync();      // nobody leaves while its statistics may still be read by the others
+}
+
 // Upper quantile of a list of binary32 values (the squared query norms): exact 4 x 8-bit radix select on
 // order-preserving keys by one CTA.  NaNs are not counted.
 constexpr int QS_THREADS = 1024;
@@ -276,8 +439,36 @@ extern "C" qaq_status qaq_prefill_window(const qaq_config* cfg, const void* Q, c
     a.H = cfg->heads; a.T = n_tokens; a.n = cfg->window; a.scale = softmax_scale;
     a.ring = score_ring; a.nvalid = nvalid; a.qnorm2 = qnorm2; a.part = (float2*)ws;
     a.nchunk = (n_tokens + PW_CHUNK - 1) / PW_CHUNK;
-    const dim3 grid((unsigned)a.nchunk, (unsigned)(cfg->batch * cfg->heads));
     cudaStream_t s = (cudaStream_t)stream;
+    const int ncl = (n_tokens + PC_CHUNK - 1) / PC_CHUNK;
+    if (ncl <= PC_MAXCTA) {
+        // one pass: the CTAs of a (b,h) are one cluster
+        const size_t smem = (size_t)cfg->window * PC_PITCH * sizeof(float);
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3((unsigned)ncl, (unsigned)(cfg->batch * cfg->heads));
+        lc.blockDim = dim3(PC_WARPS * 32);
+        lc.dynamicSmemBytes = smem;
+        lc.stream = s;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = (unsigned)ncl; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        lc.attrs = at; lc.numAttrs = 1;
+        switch (cfg->head_dim) {
+            case 32:
+                QAQ_CUDA_TRY(cudaFuncSetAttribute(window_cluster_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                QAQ_CUDA_TRY(cudaLaunchKernelEx(&lc, window_cluster_kernel<32>, a)); break;
+            case 64:
+                QAQ_CUDA_TRY(cudaFuncSetAttribute(window_cluster_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                QAQ_CUDA_TRY(cudaLaunchKernelEx(&lc, window_cluster_kernel<64>, a)); break;
+            case 128:
+                QAQ_CUDA_TRY(cudaFuncSetAttribute(window_cluster_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+                QAQ_CUDA_TRY(cudaLaunchKernelEx(&lc, window_cluster_kernel<128>, a)); break;
+            default: return QAQ_ERR_UNSUPPORTED_SHAPE;
+        }
+        QAQ_CUDA_TRY(cudaGetLastError());
+        return QAQ_OK;
+    }
+    const dim3 grid((unsigned)a.nchunk, (unsigned)(cfg->batch * cfg->heads));
     switch (cfg->head_dim) {
         case 32: window_logits_kernel<32><<<grid, PW_WARPS * 32, 0, s>>>(a); break;
         case 64: window_logits_kernel<64><<<grid, PW_WARPS * 32, 0, s>>>(a); break;

@@ -14,9 +14,10 @@ from gpu_helpers import oracle_thresholds, u16
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("D,window,tokens", [(128, 32, 1000), (64, 5, 300), (32, 64, 517), (128, 40, 23)])
+@pytest.mark.parametrize("D,window,tokens", [(128, 32, 1000), (64, 5, 300), (32, 64, 517), (128, 40, 23), (128, 64, 4096), (64, 32, 4500)])
 def test_window_rows_match_the_oracle(D, window, tokens):
-    # 1000 and 517 tokens: several 256-token chunks with a ragged tail; 23 tokens: fewer tokens than window rows
+    # 1000 and 517 tokens: several chunks with a ragged tail; 23 tokens: fewer tokens than window rows; 4096 tokens: the
+    # largest sequence the one-pass kernel takes (a cluster of 8 CTAs per (b,h)), with 64 rows; 4500: the two-kernel path
     wl = synth.scaled(synth.CONFIGS["C1"], batch=2, heads=2, head_dim=D, tokens=tokens, window=window, seed=70 + D)
     K, _ = synth.make_kv(wl)
     g = torch.Generator().manual_seed(D + window)
