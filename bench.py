@@ -550,7 +550,7 @@ def extras(qaq, dev, peak, only="", sm_mhz=None):
             # the score window after a prefill (Section 4.2): rows of the last `window` queries on the fp16 keys
             Qw = torch.randn((BH, W, D), device=dev, dtype=torch.float32).to(torch.float16)
             us_w = _time_us(lambda: qaq.qaq_prefill_window(cfg, Qw, K, scale), 10)
-            moved = BH * T * (2 * D + 3 * 4 * W + 1)           # K once; ring written, then read and written again
+            moved = BH * T * (2 * D + 4 * W + 1)               # K once, the ring once (one-pass kernel up to 4096 tokens)
             res["C3_layer_prefill_window"] = {"rows": W, "us": round(us_w, 1), "bytes": int(moved),
                                               "gbs": round(moved / us_w / 1e3, 1), "frac_of_hbm": round(moved / us_w / 1e3 / peak, 3)}
         if name == "C3_layer_low_widths":
