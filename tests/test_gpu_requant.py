@@ -253,3 +253,38 @@ def test_compaction_of_a_pool_with_many_moved_tiles():
     out = qaq.qaq_decode_attention(cache, q.cuda(), 1.0 / math.sqrt(D))
     assert_attention_close(out.cpu().numpy(), _decode_ref(wl, q, qk, qv))
     assert qaq.qaq_cache_stats(cache).device_status == 0
+
+
+def test_appends_and_decode_after_a_pool_ran_full():
+    # Raising widths moves tiles to the end of their pool until it is full; appends that find no room afterwards are
+    # reported (device status QAQ_ERR_CAPACITY), publish nothing, and decode and export keep working on what the
+    # cache holds: tokens that were not stored count with zero width.
+    wl = synth.scaled(synth.CONFIGS["C2"], heads=2, tokens=640)
+    K, V, q, ring, nv = make_inputs(wl)
+    T0 = 500
+    cfg = qaq.make_config(wl.batch, wl.heads, wl.head_dim, 640, wl.bits_min, wl.bits_max, wl.window, wl.alpha)
+    Kd, Vd, qd = K.cuda(), V.cuda(), q.cuda()
+    thr = qaq.qaq_outlier_thresholds(cfg, Kd[:, :, :T0], Vd[:, :, :T0])
+    cache = qaq.Cache(cfg)
+    low = torch.full((wl.bh, T0), 2, dtype=torch.uint8, device="cuda")
+    qaq.qaq_quantize_append(cache, Kd[:, :, :T0], Vd[:, :, :T0], thr, bitsK=low, bitsV=low)
+    for b in (3, 5, 6, 7, 8):          # every step makes the closed tiles grow and move
+        up = torch.full((wl.bh, T0), b, dtype=torch.uint8, device="cuda")
+        qaq.qaq_requantize(cache, Kd[:, :, :T0], Vd[:, :, :T0], thr, bitsK=up, bitsV=up)
+    assert qaq.qaq_cache_stats(cache).device_status == 3
+    wide = torch.full((wl.bh, 1), 8, dtype=torch.uint8, device="cuda")
+    for t in range(T0, 640):
+        qaq.qaq_quantize_append(cache, Kd[:, :, t:t + 1], Vd[:, :, t:t + 1], thr, bitsK=wide, bitsV=wide)
+    assert cache.tokens == 640
+    out = qaq.qaq_decode_attention(cache, qd, 1.0 / math.sqrt(wl.head_dim))
+    torch.cuda.synchronize()
+    assert torch.isfinite(out).all()
+    use = qaq.qaq_cache_pool_use(cache)
+    assert use[0] <= use[2] and use[1] <= use[2]
+    for x in range(2):
+        ex = qaq.qaq_cache_export(cache, x)
+        bits = ex["bits"].cpu().numpy()
+        assert set(np.unique(bits)) <= {0, 2, 3, 5, 6, 7, 8}
+    qaq.qaq_cache_compact(cache)
+    out2 = qaq.qaq_decode_attention(cache, qd, 1.0 / math.sqrt(wl.head_dim))
+    assert np.array_equal(out2.cpu().numpy().view(np.uint32), out.cpu().numpy().view(np.uint32))
