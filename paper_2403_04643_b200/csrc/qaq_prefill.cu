@@ -8,8 +8,11 @@
 //
 // This is the one dense contraction on the path ([n x D] x [D x T] per (b,h)), so the logits run
 // on the tensor cores (mma.sync m16n8k16, binary16 in, binary32 accumulate); with n <= 64 rows it is
-// bound by reading K once.  Two kernels: logits + per-chunk (max, sum of exponentials) of every
-// row; then the rows are normalised in place with the merged (max, sum).
+// bound by reading K once.  Sequences of up to 4096 tokens take one kernel whose CTAs form a
+// thread-block cluster per (b,h) (logits stay in shared memory, row statistics travel through
+// distributed shared memory, the ring is written once); longer ones take two kernels: logits +
+// per-chunk (max, sum of exponentials) of every row, then the rows are normalised in place with
+// the merged (max, sum).
 #include <cooperative_groups.h>
 
 #include "qaq_internal.cuh"
