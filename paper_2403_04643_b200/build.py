@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libqaq.so")
-SOURCES = ["qaq_cache.cu", "qaq_thresholds.cu", "qaq_quantize.cu", "qaq_requant.cu", "qaq_prefill.cu", "qaq_decode.cu"]
+SOURCES = ["qaq_cache.cu", "qaq_thresholds.cu", "qaq_quantize.cu", "qaq_requant.cu", "qaq_prefill.cu", "qaq_decode.cu", "qaq_decode_multi.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--fmad=true", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

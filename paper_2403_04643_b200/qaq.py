@@ -23,7 +23,7 @@ EXPORTED = [
     "qaq_quantize_append", "qaq_decode_workspace_bytes", "qaq_decode_attention", "qaq_quantize_append_host",
     "qaq_decode_attention_host", "qaq_cache_stats", "qaq_cache_export", "qaq_decode_attention_static",
     "qaq_requantize_down", "qaq_requantize", "qaq_cache_compact", "qaq_cache_pool_use", "qaq_prefill_window_workspace_bytes", "qaq_prefill_window",
-    "qaq_qnorm2_quantile",
+    "qaq_qnorm2_quantile", "qaq_decode_multi_workspace_bytes", "qaq_decode_attention_multi",
 ]
 
 
@@ -89,6 +89,8 @@ def lib():
         L.qaq_prefill_window.argtypes = [C.POINTER(Config), C.c_void_p, C.c_void_p, C.c_long, C.c_long, C.c_long, C.c_int,
                                          C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.qaq_qnorm2_quantile.argtypes = [C.c_void_p, C.c_long, C.c_double, C.c_void_p, C.c_void_p]
+        L.qaq_decode_multi_workspace_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
+        L.qaq_decode_attention_multi.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.qaq_cache_compact.argtypes = [C.c_void_p, C.c_void_p]
         L.qaq_cache_pool_use.argtypes = [C.c_void_p, C.POINTER(C.c_long), C.POINTER(C.c_long), C.c_void_p]
         L.qaq_requantize.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_long, C.c_long, C.c_long, C.c_void_p, C.c_void_p,
@@ -280,6 +282,23 @@ def qaq_decode_attention(cache: Cache, q, softmax_scale, out=None, scores_out=No
     ws = cache.workspace()
     _check(lib().qaq_decode_attention(cache.handle, _ptr(q), float(softmax_scale), _ptr(out), _ptr(scores_out), _ptr(ws),
                                       ws.numel(), _stream()), "qaq_decode_attention")
+    return out
+
+
+def qaq_decode_attention_multi(cache: Cache, q, softmax_scale, out=None):
+    """Several queries per (b,h): q fp16 [B*H, n_q, D] on the device; returns fp32 [B*H, n_q, D]."""
+    BH, D = cache.cfg.batch * cache.cfg.heads, cache.cfg.head_dim
+    assert q.dtype == torch.float16 and q.is_contiguous() and q.dim() == 3 and q.shape[0] == BH and q.shape[2] == D
+    n_q = q.shape[1]
+    if out is None:
+        out = torch.empty((BH, n_q, D), dtype=torch.float32, device=q.device)
+    nb = C.c_size_t()
+    _check(lib().qaq_decode_multi_workspace_bytes(cache.handle, C.byref(nb)), "qaq_decode_multi_workspace_bytes")
+    if getattr(cache, "_ws_multi", None) is None or cache._ws_multi.numel() < nb.value:
+        cache._ws_multi = torch.empty(nb.value, dtype=torch.uint8, device=q.device)
+    ws = cache._ws_multi
+    _check(lib().qaq_decode_attention_multi(cache.handle, _ptr(q), n_q, float(softmax_scale), _ptr(out), _ptr(ws), ws.numel(),
+                                            _stream()), "qaq_decode_attention_multi")
     return out
 
 

@@ -244,3 +244,29 @@ def test_decode_twice_gives_the_same_bits():
     for _ in range(3):
         again = qaq.qaq_decode_attention(cache, dev[2], 1.0 / math.sqrt(wl.head_dim))
         assert np.array_equal(again.cpu().numpy().view(np.uint32), first)
+
+
+@pytest.mark.parametrize("D,n_q", [(128, 1), (128, 3), (128, 8), (64, 5), (32, 4)])
+def test_batched_multi_query_decode(D, n_q):
+    # several queries per (b,h) in one call (Section 4.2, integration: every later query reads the same packed cache):
+    # each against the oracle's attention for that query, and against the single-query entry point; 1000 tokens with
+    # a ragged tail, CTAs that straddle two (b,h), eight queries in two passes
+    wl = synth.scaled(synth.CONFIGS["C2"], heads=3, head_dim=D, tokens=1000, seed=40 + D)
+    K, V, q, ring, nv = make_inputs(wl)
+    hyper = HYPER["C2"]
+    pol = qaq.qaq_policy_from_hyper(*hyper, wl.tokens)
+    cfg, cache, thr, out, scores, dev = gpu_pipeline(wl, K, V, q, ring, nv, pol)
+    ref = oracle_batch(wl, K, V, q, ring, nv, *oracle.policy(*hyper, wl.tokens))
+    g = torch.Generator().manual_seed(7 + n_q)
+    Q = (torch.randn((wl.bh, n_q, D), generator=g) * torch.linspace(0.5, 2.0, n_q).view(1, n_q, 1)).to(torch.float16)
+    Q[:, 0] = q.reshape(wl.bh, D)
+    scale = 1.0 / math.sqrt(D)
+    got = qaq.qaq_decode_attention_multi(cache, Q.cuda(), scale).cpu().numpy()
+    Qu = Q.numpy().view(np.uint16)
+    for j in range(n_q):
+        want = np.stack([oracle.decode(Qu[bh, j], ref.K[bh], ref.V[bh], scale)[0] for bh in range(wl.bh)])
+        assert_attention_close(got[:, j], want)
+        single = qaq.qaq_decode_attention(cache, Q[:, j].contiguous().cuda(), scale).cpu().numpy()
+        assert np.all(np.abs(got[:, j] - single) <= 1e-3 + 5e-3 * np.abs(single))     # two roundings of the same sums
+    with pytest.raises(qaq.QaqError):
+        qaq.qaq_decode_attention_multi(cache, torch.zeros((wl.bh, 9, D), dtype=torch.float16, device="cuda"), scale)
