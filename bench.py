@@ -547,6 +547,17 @@ def extras(qaq, dev, peak, only="", sm_mhz=None):
         if name == "C3_layer_low_widths":      # fewer bytes, the same instructions: the issue ceiling is the one that binds
             res[name]["note"] = "fewer bytes per token, the same per-token work: the instruction-issue ceiling binds"
         if name == "C3_layer_uniform4_with_outliers":
+            # batched decode (Section 4.2, integration): n_q queries per (b,h) in one call, against n_q single calls
+            mq = {}
+            for n_q in (1, 4, 8):
+                Qm = torch.randn((BH, n_q, D), device=dev, dtype=torch.float32).to(torch.float16)
+                om = torch.empty((BH, n_q, D), dtype=torch.float32, device=dev)
+                us_m = _time_us(lambda: qaq.qaq_decode_attention_multi(cache, Qm, scale, out=om), 10)
+                mq[f"n_q={n_q}"] = {"us": round(us_m, 1), "us_per_query": round(us_m / n_q, 1),
+                                    "packed_bytes_per_s_over_hbm_peak": round(ab["decode"] * ((n_q + 3) // 4) / us_m / 1e3 / peak, 3),
+                                    "queries_x_cached_tokens_per_s": round(n_q * wl.batch * T / (us_m * 1e-6), 1)}
+            mq["single_query_call_us"] = round(us_d, 1)
+            res["C3_layer_multi_query_decode"] = mq
             # the score window after a prefill (Section 4.2): rows of the last `window` queries on the fp16 keys
             Qw = torch.randn((BH, W, D), device=dev, dtype=torch.float32).to(torch.float16)
             us_w = _time_us(lambda: qaq.qaq_prefill_window(cfg, Qw, K, scale), 10)

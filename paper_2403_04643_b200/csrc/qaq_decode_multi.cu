@@ -9,8 +9,8 @@
 //   S.V:  the three byte digits of the 22-bit weights of two queries fill six columns; two instructions on the same
 //         operand registers serve four queries.
 // One CTA (four warps) = one run of consecutive tiles of the flattened (b,h, tile) sequence, all warps on the same
-// tile: the 16-item row blocks of the key sections are dealt out to the warps, threads 0..63 own one token each
-// (logits, softmax weights and weight digits of every query), and on the value side every warp takes its share of
+// tile: the 16-item row blocks of the key sections are dealt out to the warps, every thread owns one token for two
+// of the queries (logits, softmax weights and weight digits), and on the value side every warp takes its share of
 // the 16-channel row blocks for all tokens, so that the accumulators of four queries stay few per thread.  Whole
 // tiles are staged two deep with cp.async.  Four barriers per tile; no warp waits on another CTA.
 #include "qaq_decode_common.cuh"
@@ -107,8 +107,7 @@ __device__ __forceinline__ void v_section_mq(const uint8_t* sec, int ngroups, co
 }
 
 // Barriers of a tile: [1] its bytes have landed (and the scratch of the tile before is free), [2] key dot products
-// and key-outlier sums are complete, [3] (token warps only) the largest logits of the tile are known, [4] value
-// weights are in place.
+// and key-outlier sums are complete, [3] the largest logits of the tile are known, [4] value weights are in place.
 template <int D>
 __global__ void __launch_bounds__(MQ_THREADS, MQ_CTAS_PER_SM) decode_multi_kernel(const MultiArgs a) {
     constexpr int NR = D / 16;                       // key operand registers per lane and item
@@ -119,7 +118,7 @@ __global__ void __launch_bounds__(MQ_THREADS, MQ_CTAS_PER_SM) decode_multi_kerne
     MultiSmem<D>& sm = *reinterpret_cast<MultiSmem<D>*>(smem_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int fg = lane >> 2, ft = lane & 3;
-    const bool tokthr = tid < QAQ_TILE;              // threads 0..63 own token `tid` of the tile
+    const int tok = tid & (QAQ_TILE - 1), qh = tid >> 6;   // every thread owns token `tok` of the tile for the queries 2*qh, 2*qh+1
     const int nq = a.nq;
     const float NEG = __int_as_float(0xff800000);
 
@@ -181,9 +180,10 @@ __global__ void __launch_bounds__(MQ_THREADS, MQ_CTAS_PER_SM) decode_multi_kerne
     // query of a pair, columns 3..5 those of the second
     const float sa0 = ft == 0 ? 65536.0f : (ft == 1 ? 1.0f : 0.f), sa1 = ft == 0 ? 256.0f : 0.f;
     const float sb0 = ft == 2 ? 256.0f : 0.f, sb1 = ft == 1 ? 65536.0f : (ft == 2 ? 1.0f : 0.f);
-    float m_run[MQ], l_part[MQ], lx_part[MQ], c_part[MQ], vout[MQ];
+    float m_run[MQ], vout[MQ];
+    float l_part[2] = {0.f, 0.f}, lx_part[2] = {0.f, 0.f}, c_part[2] = {0.f, 0.f};   // sums over this thread's token, its two queries
 #pragma unroll
-    for (int j = 0; j < MQ; ++j) { m_run[j] = NEG; l_part[j] = lx_part[j] = c_part[j] = 0.f; vout[j] = 0.f; }
+    for (int j = 0; j < MQ; ++j) { m_run[j] = NEG; vout[j] = 0.f; }
 
     const size_t trow = (size_t)bh * a.ntiles_max;
     const size_t mrow = (size_t)bh * a.tmax_pad;
@@ -228,10 +228,8 @@ __global__ void __launch_bounds__(MQ_THREADS, MQ_CTAS_PER_SM) decode_multi_kerne
         Pre p;
         p.mmK = p.mmV = 0; p.eK = p.eV = 0;
         if (tile < tile_hi) {
-            if (tokthr) {
-                const size_t t0 = mrow + (size_t)tile * QAQ_TILE + tid;
-                p.mmK = __ldg(a.k.mnmx + t0); p.mmV = __ldg(a.v.mnmx + t0);
-            }
+            const size_t t0 = mrow + (size_t)tile * QAQ_TILE + tok;
+            p.mmK = __ldg(a.k.mnmx + t0); p.mmV = __ldg(a.v.mnmx + t0);
             if ((uint32_t)tid < tb.oc[0]) p.eK = __ldg(ogK + tb.oo[0] + tid);
             if ((uint32_t)tid < tb.oc[1]) p.eV = __ldg(ogV + tb.oo[1] + tid);
         }
@@ -280,18 +278,18 @@ __global__ void __launch_bounds__(MQ_THREADS, MQ_CTAS_PER_SM) decode_multi_kerne
         if (!okV) { n[1][0] = n[1][1] = n[1][2] = n[1][3] = 0; }
 
         // ---- token threads: widths, ranks in the sections, steps and midpoints of their token
-        const int tg = tile * QAQ_TILE + tid;               // token index (token threads)
-        const bool val = tokthr && tg < a.T;
+        const int tg = tile * QAQ_TILE + tok;               // token index
+        const bool val = tg < a.T;
         int BK = 0, BV = 0;
         uint32_t rkK = 0, rkV = 0;                           // rank in section c in byte c
         float stepK = 0.f, stepV = 0.f, midK = 0.f, midV = 0.f;
         int topV = 0;
-        if (tokthr) {
-            const unsigned long long below = (1ull << tid) - 1ull;
+        {
+            const unsigned long long below = (1ull << tok) - 1ull;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                if ((mk[c] >> tid) & 1ull) BK |= 8 >> c;
-                if ((mv[c] >> tid) & 1ull) BV |= 8 >> c;
+                if ((mk[c] >> tok) & 1ull) BK |= 8 >> c;
+                if ((mv[c] >> tok) & 1ull) BV |= 8 >> c;
                 rkK |= (uint32_t)__popcll(mk[c] & below) << (8 * c);
                 rkV |= (uint32_t)__popcll(mv[c] & below) << (8 * c);
             }
@@ -304,13 +302,13 @@ __global__ void __launch_bounds__(MQ_THREADS, MQ_CTAS_PER_SM) decode_multi_kerne
                 stepK = qaqc::step_of(kmn, kmx, BK); stepV = qaqc::step_of(vmn, vmx, BV);
                 midK = fmaf(0.5f, stepK, kmn); midV = fmaf(0.5f, stepV, vmn);
             }
-            sm.midV[tid] = midV;
+            if (qh == 0) sm.midV[tok] = midV;
             topV = BV ? BV - (1 << (31 - __clz(BV))) : 0;   // shift of the widest value piece
             // the largest value weight of the tile is at most the largest step * 2^shift (p <= 1)
             float wb = stepV * __int_as_float((127 + topV) << 23);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) wb = fmaxf(wb, __shfl_xor_sync(0xFFFFFFFFu, wb, o));
-            if (lane == 0) sm.wloc[warp] = wb;
+            if (lane == 0 && qh == 0) sm.wloc[warp] = wb;
         }
 
         // ---- K: integer dot products of all queries, the row blocks of the four sections dealt out to the warps
@@ -340,37 +338,36 @@ __global__ void __launch_bounds__(MQ_THREADS, MQ_CTAS_PER_SM) decode_multi_kerne
         }
         __syncthreads();                                   // [2]
 
-        // ---- token threads: logits of every query, largest logits of the tile
-        float lg[MQ];
-#pragma unroll
-        for (int j = 0; j < MQ; ++j) lg[j] = NEG;
-        if (tokthr) {
-            int dot[MQ];
-#pragma unroll
-            for (int j = 0; j < MQ; ++j) dot[j] = 0;
+        // ---- logits of this thread's token for its two queries, largest logits of the tile
+        float lg[2] = {NEG, NEG};
+        {
+            int dot[2] = {0, 0};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int w = 8 >> c;
                 if ((BK & w) && okK) {
-                    const int4 dv = *reinterpret_cast<const int4*>(&sm.dotw[c][(rkK >> (8 * c)) & 0xFF][0]);
+                    const int2 dv = *reinterpret_cast<const int2*>(&sm.dotw[c][(rkK >> (8 * c)) & 0xFF][2 * qh]);
                     const int sh = BK & (w - 1);
-                    dot[0] += dv.x << sh; dot[1] += dv.y << sh; dot[2] += dv.z << sh; dot[3] += dv.w << sh;
+                    dot[0] += dv.x << sh; dot[1] += dv.y << sh;
                 }
             }
 #pragma unroll
-            for (int j = 0; j < MQ; ++j) {
-                const int kh = sm.kcorr[0][j][tid], kl = sm.kcorr[1][j][tid];
-                if (kh | kl) { sm.kcorr[0][j][tid] = 0; sm.kcorr[1][j][tid] = 0; }
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = 2 * qh + jj;
+                const int kh = sm.kcorr[0][j][tok], kl = sm.kcorr[1][j][tok];
+                if (kh | kl) { sm.kcorr[0][j][tok] = 0; sm.kcorr[1][j][tok] = 0; }
                 if (val && j < nq) {
-                    const float qk = fmaf(sm.qscale[j] * stepK, (float)dot[j], fmaf(midK, sm.qsum[j], outlier_sum(kh, kl)));
-                    lg[j] = a.scale * qk;
+                    const float qk = fmaf(sm.qscale[j] * stepK, (float)dot[jj], fmaf(midK, sm.qsum[j], outlier_sum(kh, kl)));
+                    lg[jj] = a.scale * qk;
                 }
-                float m = lg[j];
+                float m = lg[jj];
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-                if (lane == 0) sm.mloc[warp][j] = m;
+                if (lane == 0) sm.mloc[warp & 1][j] = m;
             }
-            asm volatile("bar.sync 1, 64;" ::: "memory");     // [3] the two token warps
+        }
+        __syncthreads();                                   // [3]
+        {
             // ---- value weights p * step * 2^shift as 22-bit fixed point with one scale for the tile (the bound on the
             //      largest weight does not depend on the query).  The weight of the token's lowest piece is rounded once;
             //      the other pieces use exact multiples of it, and p is replaced by what the rounded weight stands for,
@@ -381,11 +378,13 @@ __global__ void __launch_bounds__(MQ_THREADS, MQ_CTAS_PER_SM) decode_multi_kerne
             const float wunit = wok ? __int_as_float((wex - 21) << 23) : 0.f;
             const float winv = wok ? __int_as_float((254 - (wex - 21)) << 23) : 0.f;
 #pragma unroll
-            for (int j = 0; j < MQ; ++j) {
-                const float m_new = fmaxf(m_run[j], fmaxf(sm.mloc[0][j], sm.mloc[1][j]));
-                if (tid == 0) sm.mnew[j] = m_new;
-                const float alpha = m_new == NEG ? 1.0f : __expf(m_run[j] - m_new);
-                const float pe = m_new == NEG ? 0.f : __expf(lg[j] - m_new);               // 0 for slots beyond T
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = 2 * qh + jj;
+                const float mr = qh ? m_run[2 + jj] : m_run[jj];
+                const float m_new = fmaxf(mr, fmaxf(sm.mloc[0][j], sm.mloc[1][j]));
+                if (tok == 0) sm.mnew[j] = m_new;
+                const float alpha = m_new == NEG ? 1.0f : __expf(mr - m_new);
+                const float pe = m_new == NEG ? 0.f : __expf(lg[jj] - m_new);               // 0 for slots beyond T
                 uint32_t iw = (uint32_t)__float2int_rn(fminf(pe * stepV * winv, 8388608.0f));
                 iw = min(iw, 0x7F0000u >> topV);                   // the three balanced byte digits of a shifted weight stay signed bytes
                 float p = pe;
@@ -404,10 +403,10 @@ __global__ void __launch_bounds__(MQ_THREADS, MQ_CTAS_PER_SM) decode_multi_kerne
                         gp[8] = (uint8_t)wt;
                     }
                 }
-                sm.p[j][tid] = p;
-                l_part[j] = fmaf(l_part[j], alpha, p);
-                lx_part[j] = fmaf(lx_part[j], alpha, pe);
-                c_part[j] = fmaf(c_part[j], alpha, p * midV);
+                sm.p[j][tok] = p;
+                l_part[jj] = fmaf(l_part[jj], alpha, p);
+                lx_part[jj] = fmaf(lx_part[jj], alpha, pe);
+                c_part[jj] = fmaf(c_part[jj], alpha, p * midV);
             }
             if (tid == 0) sm.wunit = wunit;
         }
@@ -489,15 +488,16 @@ __global__ void __launch_bounds__(MQ_THREADS, MQ_CTAS_PER_SM) decode_multi_kerne
                     if (ft == 0 && warp < VWARPS) sm.xs[2 * pr + w][(D / 8) * fg + 2 * (mb0 + mb) + s2] = v;
                 }
 #pragma unroll
-    for (int j = 0; j < MQ; ++j) {
-        float l = l_part[j], lx = lx_part[j], cs = c_part[j];
+    for (int jj = 0; jj < 2; ++jj) {
+        float l = l_part[jj], lx = lx_part[jj], cs = c_part[jj];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             l += __shfl_xor_sync(0xFFFFFFFFu, l, o);
             lx += __shfl_xor_sync(0xFFFFFFFFu, lx, o);
             cs += __shfl_xor_sync(0xFFFFFFFFu, cs, o);
         }
-        if (lane == 0) { sm.red[warp][j] = l; sm.red2[warp][j] = lx; sm.red3[warp][j] = cs; }
+        // warps 2*qh and 2*qh+1 hold the two halves of the tokens for queries 2*qh, 2*qh+1
+        if (lane == 0) { sm.red[warp & 1][2 * qh + jj] = l; sm.red2[warp & 1][2 * qh + jj] = lx; sm.red3[warp & 1][2 * qh + jj] = cs; }
     }
     __syncthreads();
 #pragma unroll
