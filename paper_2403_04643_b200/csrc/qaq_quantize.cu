@@ -141,7 +141,9 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
     __shared__ qaqc::TileMasks s_tm[2];
     __shared__ uint32_t s_rank[2][QAQ_TILE];   // ranks of the slots in the four sections, one per byte
     __shared__ uint32_t s_sec[2][5];           // byte offsets of the sections
-    __shared__ uint32_t s_tot[2], s_base[2], s_obase[2], s_olimit[2];
+    __shared__ uint32_t s_tot[2], s_base[2], s_obase[2], s_olimit[2], s_otot[2];
+    constexpr uint32_t OUT_STAGE = 4 * D;      // outliers of a tile whose (slot, channel) are listed on chip in entry order; more go out one by one
+    __shared__ unsigned short s_work[SELECT_ONLY ? 1 : X1 - X0][SELECT_ONLY ? 1 : OUT_STAGE];
     __shared__ int s_skip;
     __shared__ __align__(16) uint8_t s_img[SELECT_ONLY ? 1 : X1 - X0][SELECT_ONLY ? 16 : IMG];  // the tile as it will be stored
 
@@ -290,7 +292,7 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
             // a continued tile stays where it is and takes only what it grows by behind its end
             const uint32_t old_nb = starts ? 0u : (x ? a.v : a.k).tile_nbytes[ti];
             amount[x][0] = base[4] - old_nb; amount[x][1] = ctot0 + ctot1;
-            if (lane == 0) { s_tm[x] = tm; s_tot[x] = base[4]; }
+            if (lane == 0) { s_tm[x] = tm; s_tot[x] = base[4]; s_otot[x] = ctot0 + ctot1; }
         }
         if (lane >= 2 * X0 && lane < 2 * X1) {
             const int x = lane >> 1, pool = lane & 1;
@@ -337,6 +339,34 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
 #pragma unroll
             for (int c = 0; c < 5; ++c) vbase[c] = s_sec[x][c];
             if (valid || old) qaqc::write_planes_v<D>(s_img[x - X0], rk, vbase, Bx[x], p, cregs[x]);
+        }
+    }
+    // ---- where the outliers of the new tokens are: (slot, channel) in (token, channel) order - entries of lanes
+    //      p' < p of a token come first - listed in shared memory; their place needs only the scan of the counts.
+    //      The values are fetched and the entries written afterwards by all threads, one entry each.
+    uint32_t before[2] = {0, 0};
+#pragma unroll
+    for (int x = X0; x < X1; ++x) {
+        uint32_t ob = valid ? ~inl[x] : 0u;
+        const uint32_t mine = (uint32_t)__popc(ob);
+#pragma unroll
+        for (int d = 1; d < P; ++d) {
+            const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, mine, d);
+            if (p >= d) before[x] += o;
+        }
+        if (ob) {
+            const uint32_t all = ob;
+            const uint32_t lp0 = s_cnt[x][slot & (QAQ_TILE - 1)] + before[x];
+            while (ob) {
+                const int bit = __ffs(ob) - 1;
+                ob &= ob - 1;
+                const int k = bit & 15, hi = bit >> 4;
+                const int c = 2 * k + hi;                                   // channel inside the lane's 32
+                // entries of lower channels: pairs k' < k, plus channel 2k when this is 2k+1
+                const uint32_t lower = (((1u << k) - 1u) * 0x00010001u) | (hi ? (1u << k) : 0u);
+                const uint32_t lp = lp0 + (uint32_t)__popc(all & lower);
+                if (lp < OUT_STAGE) s_work[x - X0][lp] = (unsigned short)(((slot & (QAQ_TILE - 1)) << 8) | (32 * p + c));
+            }
         }
     }
     // ---- allocation results (the atomics were issued before the codes were computed).  A pool without room:
@@ -394,30 +424,34 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
             else v = qaqc::group_unit_v<D>(s_img[x - X0], vbase, o);
             *reinterpret_cast<uint4*>(dst + o) = v;
         }
-        // outliers in (token, channel) order: entries of lanes p' < p come first
-        uint32_t ob = valid ? ~inl[x] : 0u;
-        const uint32_t mine = (uint32_t)__popc(ob);
-        uint32_t before = 0;
-#pragma unroll
-        for (int d = 1; d < P; ++d) {
-            const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, mine, d);
-            if (p >= d) before += o;
-        }
-        if (ob) {
-            const uint32_t all = ob;
-            const uint32_t pos0 = s_obase[x] + s_cnt[x][slot & (QAQ_TILE - 1)] + before;
-            const __half* row = (x ? a.V : a.K) + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh + (size_t)tn * a.st + 32 * p;
-            while (ob) {
-                const int bit = __ffs(ob) - 1;
-                ob &= ob - 1;
-                const int k = bit & 15, hi = bit >> 4;
-                const int c = 2 * k + hi;                                   // channel inside the lane's 32
-                // entries of lower channels: pairs k' < k, plus channel 2k when this is 2k+1
-                const uint32_t lower = (((1u << k) - 1u) * 0x00010001u) | (hi ? (1u << k) : 0u);
-                const uint32_t pos = pos0 + (uint32_t)__popc(all & lower);
+        // outlier entries: one listed outlier per thread (value read again from the input: the registers hold -inf in
+        // its place), stores next to each other; a tile with more outliers than are listed writes the rest one by one
+        {
+            const uint32_t ntot = s_otot[x], nst = ntot < OUT_STAGE ? ntot : OUT_STAGE;
+            const __half* X = (x ? a.V : a.K) + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
+            for (uint32_t i = tid; i < nst; i += NT) {
+                const uint32_t w = s_work[x - X0][i], sl = w >> 8, ch = w & 0xFFu;
+                const uint32_t pos = s_obase[x] + i;
                 if (pos < s_olimit[x])
-                    ts.outl[(size_t)bh * a.ocap + pos] = (uint32_t)__half_as_ushort(row[c]) | ((uint32_t)(32 * p + c) << 16) |
-                                                          ((uint32_t)(slot & (QAQ_TILE - 1)) << 24);
+                    ts.outl[(size_t)bh * a.ocap + pos] = (uint32_t)__half_as_ushort(X[(size_t)(tile * QAQ_TILE + (int)sl - a.t_old) * a.st + ch]) |
+                                                          (ch << 16) | (sl << 24);
+            }
+            if (ntot > OUT_STAGE) {
+                uint32_t ob = valid ? ~inl[x] : 0u;
+                const uint32_t all = ob;
+                const uint32_t lp0 = s_cnt[x][slot & (QAQ_TILE - 1)] + before[x];
+                const __half* row = X + (size_t)tn * a.st + 32 * p;
+                while (ob) {
+                    const int bit = __ffs(ob) - 1;
+                    ob &= ob - 1;
+                    const int k = bit & 15, hi = bit >> 4;
+                    const int c = 2 * k + hi;
+                    const uint32_t lower = (((1u << k) - 1u) * 0x00010001u) | (hi ? (1u << k) : 0u);
+                    const uint32_t lp = lp0 + (uint32_t)__popc(all & lower);
+                    if (lp >= OUT_STAGE && s_obase[x] + lp < s_olimit[x])
+                        ts.outl[(size_t)bh * a.ocap + s_obase[x] + lp] = (uint32_t)__half_as_ushort(row[c]) | ((uint32_t)(32 * p + c) << 16) |
+                                                                           ((uint32_t)(slot & (QAQ_TILE - 1)) << 24);
+                }
             }
         }
         if (valid && p == 0) {
