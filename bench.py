@@ -610,9 +610,71 @@ def extras(qaq, dev, peak, only="", sm_mhz=None):
             res["C3_layer_requantize_up"] = up
         del cache, K, V, ring
         torch.cuda.empty_cache()
+    if not only or "C2_generation_loop".startswith(only):
+        res["C2_generation_loop"] = generation_loop_c2(qaq, dev)
     if not only or "C5_stream_all_steps".startswith(only):
         res["C5_stream_all_steps"] = stream_c5(qaq, dev)
     return res
+
+
+def generation_loop_c2(qaq, dev, steps=256):
+    """The per-step loop of Section 4.2 ("Integration in text generation process") on one 7B-shaped layer at batch 1:
+    append the new token, decode with the normalised score row written out, put that row into the window (the
+    caller's ring: plain tensor copies), then lower the widths of all cached tokens to what the rules give with the
+    new window (qaq_requantize_down)."""
+    from paper_2403_04643_b200.calibrate import frozen
+    wl = synth.CONFIGS["C2"]
+    T0, D, BH, W = wl.tokens, wl.head_dim, wl.bh, wl.window
+    T1 = T0 + steps
+    wlx = synth.scaled(wl, tokens=T1)
+    K, V = synth.make_kv(wlx, 0, device=dev)
+    q = synth.make_query(wlx, 0, device=dev)
+    ring0, nv0 = synth.make_score_ring(wl, 0, device=dev)
+    ring = torch.zeros((wl.batch, wl.heads, W, T1), dtype=torch.float32, device=dev)
+    nvalid = torch.zeros((wl.batch, wl.heads, T1), dtype=torch.uint8, device=dev)
+    ring[:, :, :, :T0] = ring0; nvalid[:, :, :T0] = nv0
+    # room for tiles that move: a value tile whose widths are lowered can need more padding of its groups than before
+    cfg = qaq.make_config(wl.batch, wl.heads, D, 2 * T1, wl.bits_min, wl.bits_max, W, wl.alpha)
+    thr = qaq.qaq_outlier_thresholds(cfg, K[:, :, :T0], V[:, :, :T0])
+    hy = frozen("C2")
+    cache = qaq.Cache(cfg)
+    qaq.qaq_quantize_append(cache, K[:, :, :T0], V[:, :, :T0], thr, policy=qaq.qaq_policy_from_hyper(*hy, T0), ring=ring0, nvalid=nv0)
+    st0 = qaq.qaq_cache_stats(cache)
+    outb = torch.empty((BH, D), dtype=torch.float32, device=dev)
+    r1 = torch.zeros((wl.batch, wl.heads, W, 1), dtype=torch.float32, device=dev)
+    n1 = torch.zeros((wl.batch, wl.heads, 1), dtype=torch.uint8, device=dev)
+    scale = 1.0 / math.sqrt(D)
+
+    def one(t):
+        pol = qaq.qaq_policy_from_hyper(*hy, t + 1)
+        qaq.qaq_quantize_append(cache, K[:, :, t:t + 1], V[:, :, t:t + 1], thr, policy=pol, ring=r1, nvalid=n1)
+        qaq.qaq_decode_attention(cache, q, scale, out=outb, scores_out=scores_view(t + 1))
+        ring[:, :, t % W, :t + 1] = scores_view(t + 1).view(wl.batch, wl.heads, t + 1)
+        nvalid[:, :, :t + 1] = torch.clamp(nvalid[:, :, :t + 1] + 1, max=W)
+        qaq.qaq_requantize_down(cache, policy=pol, ring=ring, nvalid=nvalid)
+        if (t - T0) % 64 == 63:
+            qaq.qaq_cache_compact(cache)      # closes the gaps moved tiles leave in the pools
+
+    sbuf = torch.empty((BH * T1,), dtype=torch.float32, device=dev)
+
+    def scores_view(n):
+        return sbuf[:BH * n].view(BH, n)
+
+    for t in range(T0, T0 + 8):
+        one(t)
+    torch.cuda.synchronize()
+    a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+    a.record()
+    for t in range(T0 + 8, T1):
+        one(t)
+    b.record(); torch.cuda.synchronize()
+    st1 = qaq.qaq_cache_stats(cache)
+    n = T1 - T0 - 8
+    mb = lambda st, x: round(st.code_bytes[x] * 8 / (BH * st.tokens * D), 2)
+    return {"steps": n, "us_per_step": round(a.elapsed_time(b) * 1e3 / n, 1), "tokens_at_end": int(st1.tokens),
+            "mean_bits_after_prefill": [mb(st0, 0), mb(st0, 1)], "mean_bits_at_end": [mb(st1, 0), mb(st1, 1)],
+            "cr_paper_at_end": round(st1.cr_paper, 3), "device_status": int(st1.device_status),
+            "note": "append 1 + decode with score row + window update (tensor copies) + qaq_requantize_down over the whole cache, per step"}
 
 
 def stream_c5(qaq, dev):
