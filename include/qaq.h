@@ -189,6 +189,12 @@ qaq_status qaq_quantize_append(qaq_cache* c, const void* K_new, const void* V_ne
  * [batch*heads][window][n_cols]; nvalid: u8 [batch*heads][n_cols]; n_cols >= cached tokens.
  * Tiles are rewritten in place: the bytes read by qaq_decode_attention and the counters of
  * qaq_cache_stats shrink; pool space inside closed tiles is not handed back to later appends.
+ * One exception: the values of a tile are stored in groups of four tokens per piece width, and a
+ * tile whose lowered widths need more group padding than before can come out a few bytes larger;
+ * it is then placed anew at the end of its pool like a raised tile (see qaq_requantize).  A caller
+ * that lowers widths every step gives the cache some room beyond the tokens it will hold and calls
+ * qaq_cache_compact now and then; without room the tile stays as it was and the device status
+ * reports QAQ_ERR_CAPACITY.
  * Device pointers; asynchronous on stream.  Errors: QAQ_ERR_INVALID_ARG (missing arrays,
  * n_cols too small), QAQ_ERR_UNSUPPORTED_SHAPE, QAQ_ERR_CUDA; an empty cache is a no-op.
  */
