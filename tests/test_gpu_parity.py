@@ -270,3 +270,21 @@ def test_batched_multi_query_decode(D, n_q):
         assert np.all(np.abs(got[:, j] - single) <= 1e-3 + 5e-3 * np.abs(single))     # two roundings of the same sums
     with pytest.raises(qaq.QaqError):
         qaq.qaq_decode_attention_multi(cache, torch.zeros((wl.bh, 9, D), dtype=torch.float16, device="cuda"), scale)
+
+
+@pytest.mark.parametrize("tokens,alpha", [(1, 0.01), (65, 0.01), (640, 0.10)])
+def test_batched_decode_edge_cases(tokens, alpha):
+    # a single token, one token past a tile, and tiles with more outliers than one pass over the threads handles
+    wl = synth.scaled(synth.CONFIGS["C4"], batch=1, heads=2, tokens=tokens, alpha=alpha)
+    K, V, q, ring, nv = make_inputs(wl)
+    pol = qaq.qaq_policy_from_hyper(*HYPER["C4"], tokens)
+    cfg, cache, thr, out, scores, dev = gpu_pipeline(wl, K, V, q, ring, nv, pol)
+    ref = oracle_batch(wl, K, V, q, ring, nv, *oracle.policy(*HYPER["C4"], tokens))
+    D, scale = wl.head_dim, 1.0 / math.sqrt(wl.head_dim)
+    g = torch.Generator().manual_seed(3)
+    Q = torch.randn((wl.bh, 2, D), generator=g).to(torch.float16)
+    got = qaq.qaq_decode_attention_multi(cache, Q.cuda(), scale).cpu().numpy()
+    Qu = Q.numpy().view(np.uint16)
+    for j in range(2):
+        want = np.stack([oracle.decode(Qu[bh, j], ref.K[bh], ref.V[bh], scale)[0] for bh in range(wl.bh)])
+        assert_attention_close(got[:, j], want)
