@@ -251,7 +251,8 @@ qaq_status qaq_decode_attention_host(qaq_cache* c, const void* q, float softmax_
  * Decode attention for several queries per (b,h) in one call (Section 4.2, "Integration in text generation
  * process"; the packed cache is what every query reads).  Per query the result is what qaq_decode_attention
  * returns for it, within the same tolerance; up to four queries share one pass over the packed cache (a tile is
- * staged and taken apart once, the queries are columns of the tensor-core operand), so n_q = 5..8 takes two passes.
+ * staged and taken apart once, the queries are columns of the tensor-core operand), so n_q = 5..8 takes two passes;
+ * a pass left with one or two queries runs the single-query kernel on each of them (it is cheaper there).
  * q: binary16 [batch*heads][n_q][head_dim]; out: binary32 [batch*heads][n_q][head_dim]; 1 <= n_q <= 8;
  * ws: qaq_decode_multi_workspace_bytes bytes, 16-byte aligned.  Device pointers, asynchronous on stream.
  * Errors: QAQ_ERR_INVALID_ARG (null pointer, empty cache, n_q outside 1..8), QAQ_ERR_WORKSPACE.

@@ -52,6 +52,7 @@ struct DecArgs {
     int tmax_pad, ntiles_max;
     int T;
     const __half* q;
+    long q_stride, out_stride;   // elements between the rows of consecutive (b,h) in q and in out
     float scale;
     float* part;       // [ncta][2][D+3]: accumulators, running max, sum of the weights used, exact sum
     float* ml;         // [BH][2]   merged (max, sum) for score normalisation
@@ -156,7 +157,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
     // ---- q: float copy, fixed-point byte digits per lane
     float qmax = 0.f, qs = 0.f;
     for (int d = tid; d < D; d += DEC_THREADS) {
-        const float f = __half2float(a.q[(size_t)bh * D + d]);
+        const float f = __half2float(a.q[(size_t)bh * a.q_stride + d]);
         sm.qf[d] = f;
         qmax = fmaxf(qmax, fabsf(f));
         qs += f;
@@ -569,7 +570,7 @@ __global__ void merge_kernel(const DecArgs a) {
         LX = fmaf(w, p[D + 2], LX);
         x = fmaf(w, p[d], x);
     }
-    a.out[(size_t)bh * D + d] = L > 0.f ? x / L : 0.f;
+    a.out[(size_t)bh * a.out_stride + d] = L > 0.f ? x / L : 0.f;
     if (d == 0) { a.ml[2 * bh] = M; a.ml[2 * bh + 1] = LX; }
 }
 
@@ -639,7 +640,7 @@ extern "C" qaq_status qaq_decode_attention(const qaq_cache* c, const void* q, fl
     DecArgs a;
     a.k = c->t[0]; a.v = c->t[1]; a.pool_bytes = c->pool_bytes; a.ocap = c->ocap;
     a.tmax_pad = c->tmax_pad; a.ntiles_max = c->ntiles; a.T = (int)c->tokens;
-    a.q = (const __half*)q; a.scale = softmax_scale;
+    a.q = (const __half*)q; a.scale = softmax_scale; a.q_stride = c->cfg.head_dim; a.out_stride = c->cfg.head_dim;
     const int ntiles = (a.T + QAQ_TILE - 1) / QAQ_TILE;
     const DecPlan plan = plan_decode(BH, ntiles);
     a.BH = BH; a.run = plan.run; a.ncta = plan.ncta;
@@ -647,6 +648,29 @@ extern "C" qaq_status qaq_decode_attention(const qaq_cache* c, const void* q, fl
     a.ml = a.part + (size_t)2 * plan.ncta * (D + 3);
     a.out = out; a.scores = scores_out;
     cudaStream_t s = (cudaStream_t)stream;
+    switch (D) {
+        case 32: return run_decode<32>(a, BH, s);
+        case 64: return run_decode<64>(a, BH, s);
+        case 128: return run_decode<128>(a, BH, s);
+    }
+    return QAQ_ERR_UNSUPPORTED_SHAPE;
+}
+
+// One query per (b,h) taken from / written to rows that lie q_stride / out_stride elements apart (used by the
+// batched entry point for the queries that do not fill a pass of their own); ws as for qaq_decode_attention.
+qaq_status qaq_decode_strided(const qaq_cache* c, const void* q, long q_stride, float softmax_scale, float* out, long out_stride,
+                              void* ws, cudaStream_t s) {
+    const int D = c->cfg.head_dim, BH = c->BH;
+    DecArgs a;
+    a.k = c->t[0]; a.v = c->t[1]; a.pool_bytes = c->pool_bytes; a.ocap = c->ocap;
+    a.tmax_pad = c->tmax_pad; a.ntiles_max = c->ntiles; a.T = (int)c->tokens;
+    a.q = (const __half*)q; a.scale = softmax_scale; a.q_stride = q_stride; a.out_stride = out_stride;
+    const int ntiles = (a.T + QAQ_TILE - 1) / QAQ_TILE;
+    const DecPlan plan = plan_decode(BH, ntiles);
+    a.BH = BH; a.run = plan.run; a.ncta = plan.ncta;
+    a.part = (float*)ws;
+    a.ml = a.part + (size_t)2 * plan.ncta * (D + 3);
+    a.out = out; a.scores = nullptr;
     switch (D) {
         case 32: return run_decode<32>(a, BH, s);
         case 64: return run_decode<64>(a, BH, s);
@@ -702,7 +726,7 @@ extern "C" qaq_status qaq_decode_attention_static(const qaq_cache* c, const void
     DecArgs a;
     a.k = c->t[0]; a.v = c->t[1]; a.pool_bytes = c->pool_bytes; a.ocap = c->ocap;
     a.tmax_pad = c->tmax_pad; a.ntiles_max = c->ntiles; a.T = T;
-    a.q = (const __half*)q; a.scale = softmax_scale;
+    a.q = (const __half*)q; a.scale = softmax_scale; a.q_stride = c->cfg.head_dim; a.out_stride = c->cfg.head_dim;
     a.BH = BH; a.run = plan.run; a.ncta = plan.ncta;
     // Every partial that the merge reads and every (max,sum) pair is written before it is read,
     // so nothing in the scratch has to be cleared between calls.

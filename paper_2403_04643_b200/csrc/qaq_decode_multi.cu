@@ -564,7 +564,8 @@ qaq_status run_multi(const MultiArgs& a, cudaStream_t s) {
 
 extern "C" qaq_status qaq_decode_multi_workspace_bytes(const qaq_cache* c, size_t* host_out) {
     if (!c || !host_out) return QAQ_ERR_INVALID_ARG;
-    // plan_multi never uses more CTAs than max(MQ_SLOTS, BH), whatever the token count; the passes of a call reuse the space
+    // plan_multi never uses more CTAs than max(MQ_SLOTS, BH), whatever the token count; the passes of a call reuse the
+    // space, and the partials of the single-query kernel (at most 2 * max(592, BH) * (head_dim + 3) + 2 * BH floats) fit it too
     const int ncta_max = c->BH > MQ_SLOTS ? c->BH : MQ_SLOTS;
     *host_out = (size_t)2 * ncta_max * MQ * (c->cfg.head_dim + 3) * sizeof(float);
     return QAQ_OK;
@@ -591,6 +592,16 @@ extern "C" qaq_status qaq_decode_attention_multi(const qaq_cache* c, const void*
     for (int q0 = 0; q0 < n_q; q0 += MQ) {          // four queries per pass over the cache
         a.q0 = q0; a.nq = n_q - q0 < MQ ? n_q - q0 : MQ;
         qaq_status st;
+        if (a.nq <= 2) {
+            // one or two queries do not pay for a pass of this kernel (it is laid out for four): the single-query
+            // kernel takes them one by one (its partials fit the same workspace)
+            for (int j = 0; j < a.nq; ++j) {
+                st = qaq_decode_strided(c, (const __half*)q + (size_t)(q0 + j) * D, (long)n_q * D, softmax_scale,
+                                        out + (size_t)(q0 + j) * D, (long)n_q * D, ws, s);
+                if (st != QAQ_OK) return st;
+            }
+            continue;
+        }
         switch (D) {
             case 32: st = run_multi<32>(a, s); break;
             case 64: st = run_multi<64>(a, s); break;

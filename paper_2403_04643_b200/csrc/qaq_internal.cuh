@@ -64,3 +64,6 @@ qaq_status qaq_launch_select(const qaq_config* cfg, const qaq_policy* pol, const
 qaq_status qaq_launch_append(qaq_cache* c, const void* K, const void* V, long sb, long sh, long st, int n_new,
                              const uint8_t* bitsK, const uint8_t* bitsV, const qaq_policy* pol, const float* ring,
                              const uint8_t* nvalid, const float* thr, cudaStream_t s);
+// single-query decode on strided query / output rows (qaq_decode.cu); ws: qaq_decode_workspace_bytes bytes
+qaq_status qaq_decode_strided(const qaq_cache* c, const void* q, long q_stride, float softmax_scale, float* out, long out_stride,
+                              void* ws, cudaStream_t s);

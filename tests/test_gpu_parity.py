@@ -246,7 +246,7 @@ def test_decode_twice_gives_the_same_bits():
         assert np.array_equal(again.cpu().numpy().view(np.uint32), first)
 
 
-@pytest.mark.parametrize("D,n_q", [(128, 1), (128, 3), (128, 8), (64, 5), (32, 4)])
+@pytest.mark.parametrize("D,n_q", [(128, 1), (128, 3), (128, 8), (64, 5), (32, 4), (64, 6), (32, 2)])
 def test_batched_multi_query_decode(D, n_q):
     # several queries per (b,h) in one call (Section 4.2, integration: every later query reads the same packed cache):
     # each against the oracle's attention for that query, and against the single-query entry point; 1000 tokens with
