@@ -39,7 +39,7 @@ import hashlib
 COUNTERS_JSON = os.path.join(ROOT, "profiles", "counters_C3.json")
 CSRC = os.path.join(ROOT, "paper_2403_04643_b200", "csrc")
 ISSUE_SLOTS_PER_CLOCK = 148 * 4
-KERNEL_KEYS = {"quant_keys": "quant_kernel<128, 0, 0>", "quant_values": "quant_kernel<128, 0, 1>", "decode": "decode_kernel<128>",
+KERNEL_KEYS = {"quant_keys": "quant_kernel<128, 0, 0>", "quant_values": "quant_kernel<128, 0, 1>", "decode": "decode_kernel<128, 0>",
                "thr_scan": "thr_scan_kernel"}
 
 

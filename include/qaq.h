@@ -262,6 +262,35 @@ qaq_status qaq_decode_attention_multi(const qaq_cache* c, const void* q, int n_q
                                       void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The generation step with the token count kept in device memory (Section 4.2, "Integration in text generation
+ * process": every step appends the new token's K and V rows to the quantized cache and attends over the whole of it).
+ * The calls above take the token count from the host-side handle, so each step needs the host to issue launches that
+ * depend on it.  Between qaq_stream_begin and qaq_stream_end the count lives in the cache's device memory instead:
+ * qaq_stream_append reads it, stores one token per (b,h) behind it and advances it; qaq_stream_decode attends over as
+ * many tokens as it says.  Neither touches host state, and their launch shapes do not depend on the count, so one
+ * append + decode pair can be captured in a CUDA graph once and replayed for every step (the buffers behind the
+ * pointers must then stay where they are; their contents are read at replay time).  While the count is on the device
+ * the host-side count is stale: call no other function on the cache until qaq_stream_end has brought it back.
+ *
+ * qaq_stream_begin: writes the host count to the device (asynchronous on stream).
+ * qaq_stream_append: k_new / v_new binary16, one row of head_dim per (b,h), element strides between batches and heads
+ *   given; the other arguments as for qaq_quantize_append with n_new = 1 (score_col: [batch*heads][window][1],
+ *   nvalid: [batch*heads][1]; or given widths bitK / bitV [batch*heads][1]).  A cache that is full keeps its count
+ *   and sets the device status to QAQ_ERR_CAPACITY (read by qaq_cache_stats).
+ * qaq_stream_decode: as qaq_decode_attention; rows of scores_out lie scores_stride >= max_tokens elements apart.
+ *   A count of zero yields zeros.
+ * qaq_stream_end: copies the count back and waits for the stream (the one call of the four that synchronises).
+ * Errors: QAQ_ERR_INVALID_ARG, QAQ_ERR_WORKSPACE, QAQ_ERR_UNSUPPORTED_SHAPE, QAQ_ERR_CUDA as above.
+ */
+qaq_status qaq_stream_begin(qaq_cache* c, void* stream);
+qaq_status qaq_stream_append(qaq_cache* c, const void* k_new, const void* v_new, long stride_b, long stride_h,
+                             const uint8_t* bitK, const uint8_t* bitV, const qaq_policy* policy,
+                             const float* score_col, const uint8_t* nvalid, const float* thr, void* stream);
+qaq_status qaq_stream_decode(const qaq_cache* c, const void* q, float softmax_scale, float* out, float* scores_out,
+                             long scores_stride, void* ws, size_t ws_bytes, void* stream);
+qaq_status qaq_stream_end(qaq_cache* c, void* stream);
+
+/*
  * Decode attention without a caller-supplied workspace and without any allocation.
  * (No counterpart in the paper: this exists for the sake of the callers, not the method.)
  *

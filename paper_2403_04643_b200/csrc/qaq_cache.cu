@@ -124,6 +124,30 @@ extern "C" qaq_status qaq_cache_reset(qaq_cache* c, void* stream) {
     return QAQ_OK;
 }
 
+namespace {
+__global__ void set_count_kernel(int* count, unsigned* ticket, int value) { *count = value; *ticket = 0u; }
+}  // namespace
+
+// The token count moves to device memory (qaq_stream_begin) and back (qaq_stream_end); between the two the
+// qaq_stream_* calls read and advance it there, and the host counter is stale.
+extern "C" qaq_status qaq_stream_begin(qaq_cache* c, void* stream) {
+    if (!c) return QAQ_ERR_INVALID_ARG;
+    set_count_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(qaq_d_count(c), qaq_d_ticket(c), (int)c->tokens);
+    QAQ_CUDA_TRY(cudaGetLastError());
+    return QAQ_OK;
+}
+
+extern "C" qaq_status qaq_stream_end(qaq_cache* c, void* stream) {
+    if (!c) return QAQ_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    int count = -1;
+    QAQ_CUDA_TRY(cudaMemcpyAsync(&count, qaq_d_count(c), sizeof(int), cudaMemcpyDeviceToHost, s));
+    QAQ_CUDA_TRY(cudaStreamSynchronize(s));
+    if (count < 0 || count > c->cfg.max_tokens) return QAQ_ERR_INVALID_ARG;
+    c->tokens = count;
+    return QAQ_OK;
+}
+
 int g_qaq_last_cuda_error = 0;
 
 extern "C" const char* qaq_last_cuda_error(void) { return cudaGetErrorName((cudaError_t)g_qaq_last_cuda_error); }

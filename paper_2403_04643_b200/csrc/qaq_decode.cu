@@ -51,6 +51,7 @@ struct DecArgs {
     uint32_t ocap;
     int tmax_pad, ntiles_max;
     int T;
+    const int* d_count;          // counted kernels only: the token count in device memory (T, run and ncta are then derived from it)
     const __half* q;
     long q_stride, out_stride;   // elements between the rows of consecutive (b,h) in q and in out
     float scale;
@@ -58,8 +59,26 @@ struct DecArgs {
     float* ml;         // [BH][2]   merged (max, sum) for score normalisation
     int BH, run, ncta; // (b,h) count; tiles per CTA of the flattened (b,h, tile) sequence; CTAs
     float* out;        // [BH][D]
-    float* scores;     // [BH][T] or null
+    float* scores;     // [BH][scores_stride] or null
+    long scores_stride;
 };
+
+// The flattened sequence of BH * ntiles tiles is cut into runs of `run` consecutive tiles, one CTA
+// each: enough CTAs to fill every SM (148 SMs, 4 resident CTAs each) evenly, at least one tile per
+// warp where there are that many, and never more than one (b,h) boundary inside a run.
+constexpr int DEC_SLOTS = 148 * DEC_CTAS_PER_SM;
+struct DecPlan { int run, ncta; };
+__host__ __device__ inline DecPlan plan_decode(int BH, int ntiles) {
+    const long long total = (long long)BH * ntiles;
+    long long run = (total + DEC_SLOTS - 1) / DEC_SLOTS;
+    const int floor_run = ntiles < DEC_WARPS ? ntiles : DEC_WARPS;
+    if (run < floor_run) run = floor_run;
+    if (run > ntiles) run = ntiles;
+    DecPlan p;
+    p.run = (int)run;
+    p.ncta = (int)((total + run - 1) / run);
+    return p;
+}
 
 // per-warp scratch for the tile a warp is working on
 template <int D>
@@ -129,7 +148,9 @@ __device__ __forceinline__ void v_section(const uint8_t* sec, int ngroups, const
 // own: own running max / sum / accumulators, own staging buffer, no CTA barrier in the loop; the
 // warps are merged once at the end.  Lane l looks after tokens l and l + 32 of the tile (logit, softmax
 // weight, fixed-point value weight); in the section loops lane 4g+t is lane (g, t) of the tensor-core fragments.
-template <int D>
+// COUNTED: the token count is read from device memory and the split derived from it here (the grid is then the
+// largest one any count needs; CTAs beyond the split find no tiles and leave).
+template <int D, bool COUNTED>
 __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(const DecArgs a) {
     constexpr int NR = D / 16;       // key operand registers per lane and item
     constexpr int MB = D / 16;       // 16-channel row blocks of the value side
@@ -141,6 +162,9 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
     const int fg = lane >> 2, ft = lane & 3;
     const unsigned lt = (1u << lane) - 1u;
     WarpScratch<D>& ws = sm.ws[warp];
+    const int T = COUNTED ? *a.d_count : a.T;
+    if (COUNTED && T < 1) return;
+    const int run = COUNTED ? plan_decode(a.BH, (T + QAQ_TILE - 1) / QAQ_TILE).run : a.run;
 
 #pragma unroll 1
     for (int seg = 0; seg < 2; ++seg) {
@@ -148,8 +172,8 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
     // index is read afresh for each segment so that none of this stays in registers over the tile loop.
     int cta;
     asm volatile("mov.u32 %0, %%ctaid.x;" : "=r"(cta));
-    const int ntiles = (a.T + QAQ_TILE - 1) / QAQ_TILE;
-    const int flat_lo = cta * a.run, flat_hi = min(a.BH * ntiles, flat_lo + a.run);
+    const int ntiles = (T + QAQ_TILE - 1) / QAQ_TILE;
+    const int flat_lo = cta * run, flat_hi = min(a.BH * ntiles, flat_lo + run);
     const int bh = flat_lo / ntiles + seg;
     const int tile_lo = max(flat_lo, bh * ntiles) - bh * ntiles, tile_hi = min(flat_hi, (bh + 1) * ntiles) - bh * ntiles;
     if (tile_lo >= tile_hi) continue;   // the same for every thread of the CTA
@@ -261,7 +285,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         const uint32_t ooV = __shfl_sync(0xFFFFFFFFu, cur.tb, 6), ocV = __shfl_sync(0xFFFFFFFFu, cur.tb, 7);
         const bool has_next = tile + DEC_WARPS < tile_hi;
         const int t0 = tile * QAQ_TILE + lane;              // this lane's tokens: t0 and t0 + 32
-        const bool val0 = t0 < a.T, val1 = t0 + HALF < a.T;
+        const bool val0 = t0 < T, val1 = t0 + HALF < T;
         const uint8_t* tK = stK ? ws.buf : poolK + offK;
         const uint8_t* tV = stV ? ws.buf + STAGE - stV : poolV + offV;
         // the first outlier entries of the tile (used after the section loops)
@@ -351,7 +375,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
             if (j ? val1 : val0) {
                 const float qk = fmaf(qscale * stepK[j], (float)dot, fmaf(ws.midK[tk], qsum, outlier_sum(kh, kl)));
                 lg[j] = a.scale * qk;
-                if (a.scores) a.scores[(size_t)bh * a.T + t0 + HALF * j] = lg[j];
+                if (a.scores) a.scores[(size_t)bh * a.scores_stride + t0 + HALF * j] = lg[j];
             }
         }
         float m = fmaxf(lg[0], lg[1]);
@@ -550,14 +574,17 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
 }
 
 // log-sum-exp merge of the partials -> X, and (max, sum) for the score row
-template <int D>
+template <int D, bool COUNTED>
 __global__ void merge_kernel(const DecArgs a) {
     const int bh = blockIdx.x, d = threadIdx.x;
+    const int T = COUNTED ? *a.d_count : a.T;
+    if (COUNTED && T < 1) { a.out[(size_t)bh * a.out_stride + d] = 0.f; return; }
+    const int ntiles = (T + QAQ_TILE - 1) / QAQ_TILE;
+    const int run = COUNTED ? plan_decode(a.BH, ntiles).run : a.run;
     // the CTAs of decode_kernel whose runs meet this (b,h); a CTA's first segment has slot 0
-    const int ntiles = (a.T + QAQ_TILE - 1) / QAQ_TILE;
-    const int c_lo = (bh * ntiles) / a.run, c_hi = ((bh + 1) * ntiles - 1) / a.run;
+    const int c_lo = (bh * ntiles) / run, c_hi = ((bh + 1) * ntiles - 1) / run;
     // only the first of them can have begun in the (b,h) before
-    auto slot = [&](int c) { return a.part + (size_t)(2 * c + (c * a.run < bh * ntiles ? 1 : 0)) * (D + 3); };
+    auto slot = [&](int c) { return a.part + (size_t)(2 * c + (c * run < bh * ntiles ? 1 : 0)) * (D + 3); };
     float M = __int_as_float(0xff800000);
     for (int c = c_lo; c <= c_hi; ++c) M = fmaxf(M, slot(c)[D]);
     float L = 0.f, LX = 0.f, x = 0.f;
@@ -574,46 +601,31 @@ __global__ void merge_kernel(const DecArgs a) {
     if (d == 0) { a.ml[2 * bh] = M; a.ml[2 * bh + 1] = LX; }
 }
 
-__global__ void scores_kernel(float* scores, const float* ml, int T) {
+__global__ void scores_kernel(float* scores, long stride, const float* ml, int T, const int* d_count) {
     const int bh = blockIdx.y;
+    if (d_count) T = *d_count;
     const float M = ml[2 * bh], L = ml[2 * bh + 1];
     const float inv = L > 0.f ? 1.0f / L : 0.f;
     for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < T; t += gridDim.x * blockDim.x) {
-        float* s = scores + (size_t)bh * T + t;
+        float* s = scores + (size_t)bh * stride + t;
         *s = __expf(*s - M) * inv;
     }
 }
 
-// The flattened sequence of BH * ntiles tiles is cut into runs of `run` consecutive tiles, one CTA
-// each: enough CTAs to fill every SM (148 SMs, 4 resident CTAs each) evenly, at least one tile per
-// warp where there are that many, and never more than one (b,h) boundary inside a run.
-constexpr int DEC_SLOTS = 148 * DEC_CTAS_PER_SM;
-struct DecPlan { int run, ncta; };
-DecPlan plan_decode(int BH, int ntiles) {
-    const long long total = (long long)BH * ntiles;
-    long long run = (total + DEC_SLOTS - 1) / DEC_SLOTS;
-    const int floor_run = ntiles < DEC_WARPS ? ntiles : DEC_WARPS;
-    if (run < floor_run) run = floor_run;
-    if (run > ntiles) run = ntiles;
-    DecPlan p;
-    p.run = (int)run;
-    p.ncta = (int)((total + run - 1) / run);
-    return p;
-}
 // floats of workspace for the partials (two slots per CTA) and the merged (max, sum) pairs
 size_t decode_ws_floats(int BH, int ncta, int D) { return (size_t)2 * ncta * (D + 3) + (size_t)BH * 2; }
 
-template <int D>
+template <int D, bool COUNTED = false>
 qaq_status run_decode(const DecArgs& a, int BH, cudaStream_t s) {
     const size_t smem = sizeof(DecSmem<D>);
     if (smem > 48 * 1024)
-        QAQ_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    decode_kernel<D><<<a.ncta, DEC_THREADS, smem, s>>>(a);
-    merge_kernel<D><<<BH, D, 0, s>>>(a);
+        QAQ_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D, COUNTED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    decode_kernel<D, COUNTED><<<a.ncta, DEC_THREADS, smem, s>>>(a);
+    merge_kernel<D, COUNTED><<<BH, D, 0, s>>>(a);
     if (a.scores) {
-        int gx = (a.T + 1023) / 1024;
+        int gx = (a.T + 1023) / 1024;     // counted: a.T holds the capacity
         if (gx > 64) gx = 64;
-        scores_kernel<<<dim3(gx, BH), 256, 0, s>>>(a.scores, a.ml, a.T);
+        scores_kernel<<<dim3(gx, BH), 256, 0, s>>>(a.scores, a.scores_stride, a.ml, a.T, COUNTED ? a.d_count : nullptr);
     }
     QAQ_CUDA_TRY(cudaGetLastError());
     return QAQ_OK;
@@ -646,7 +658,7 @@ extern "C" qaq_status qaq_decode_attention(const qaq_cache* c, const void* q, fl
     a.BH = BH; a.run = plan.run; a.ncta = plan.ncta;
     a.part = (float*)ws;
     a.ml = a.part + (size_t)2 * plan.ncta * (D + 3);
-    a.out = out; a.scores = scores_out;
+    a.out = out; a.scores = scores_out; a.scores_stride = a.T; a.d_count = nullptr;
     cudaStream_t s = (cudaStream_t)stream;
     switch (D) {
         case 32: return run_decode<32>(a, BH, s);
@@ -670,7 +682,7 @@ qaq_status qaq_decode_strided(const qaq_cache* c, const void* q, long q_stride, 
     a.BH = BH; a.run = plan.run; a.ncta = plan.ncta;
     a.part = (float*)ws;
     a.ml = a.part + (size_t)2 * plan.ncta * (D + 3);
-    a.out = out; a.scores = nullptr;
+    a.out = out; a.scores = nullptr; a.scores_stride = 0; a.d_count = nullptr;
     switch (D) {
         case 32: return run_decode<32>(a, BH, s);
         case 64: return run_decode<64>(a, BH, s);
@@ -732,12 +744,41 @@ extern "C" qaq_status qaq_decode_attention_static(const qaq_cache* c, const void
     // so nothing in the scratch has to be cleared between calls.
     a.part = (float*)scratch;
     a.ml = a.part + (size_t)2 * plan.ncta * (D + 3);
-    a.out = out; a.scores = nullptr;
+    a.out = out; a.scores = nullptr; a.scores_stride = 0; a.d_count = nullptr;
     cudaStream_t s = (cudaStream_t)stream;
     switch (D) {
         case 32: return run_decode<32>(a, BH, s);
         case 64: return run_decode<64>(a, BH, s);
         case 128: return run_decode<128>(a, BH, s);
+    }
+    return QAQ_ERR_UNSUPPORTED_SHAPE;
+}
+
+// Decode attention over as many tokens as the device-side count says (qaq_stream_begin / qaq_stream_append): the
+// split over CTAs is derived from the count inside the kernels, the grid is the largest any count needs, and nothing
+// on the host is read or changed, so the call can be captured in a CUDA graph and replayed while the cache grows.
+extern "C" qaq_status qaq_stream_decode(const qaq_cache* c, const void* q, float softmax_scale, float* out,
+                                        float* scores_out, long scores_stride, void* ws, size_t ws_bytes, void* stream) {
+    if (!c || !q || !out || !ws) return QAQ_ERR_INVALID_ARG;
+    if (scores_out && scores_stride < c->cfg.max_tokens) return QAQ_ERR_INVALID_ARG;
+    size_t need = 0;
+    qaq_decode_workspace_bytes(c, &need);
+    if (ws_bytes < need || ((uintptr_t)ws & 15)) return QAQ_ERR_WORKSPACE;
+    const int D = c->cfg.head_dim, BH = c->BH;
+    DecArgs a;
+    a.k = c->t[0]; a.v = c->t[1]; a.pool_bytes = c->pool_bytes; a.ocap = c->ocap;
+    a.tmax_pad = c->tmax_pad; a.ntiles_max = c->ntiles; a.T = (int)c->cfg.max_tokens;
+    a.d_count = qaq_d_count(c);
+    a.q = (const __half*)q; a.scale = softmax_scale; a.q_stride = D; a.out_stride = D;
+    a.BH = BH; a.run = 0; a.ncta = BH > DEC_SLOTS ? BH : DEC_SLOTS;
+    a.part = (float*)ws;
+    a.ml = a.part + (size_t)2 * a.ncta * (D + 3);
+    a.out = out; a.scores = scores_out; a.scores_stride = scores_stride;
+    cudaStream_t s = (cudaStream_t)stream;
+    switch (D) {
+        case 32: return run_decode<32, true>(a, BH, s);
+        case 64: return run_decode<64, true>(a, BH, s);
+        case 128: return run_decode<128, true>(a, BH, s);
     }
     return QAQ_ERR_UNSUPPORTED_SHAPE;
 }

@@ -36,7 +36,7 @@ struct qaq_cache {
     size_t pool_bytes;  // per (b,h)
     uint32_t ocap;      // outlier entries per (b,h)
     TensorStore t[2];
-    int* d_status;      // sticky device-side status
+    int* d_status;      // sticky device-side status; the two words behind it: see qaq_d_count / qaq_d_ticket
     void* slab;         // the one allocation everything above lives in
     size_t slab_bytes;
     size_t reset_off, reset_bytes;   // the range of the slab that qaq_cache_reset clears
@@ -54,6 +54,11 @@ extern int g_qaq_last_cuda_error;
         cudaError_t _e = (expr);                            \
         if (_e != cudaSuccess) { g_qaq_last_cuda_error = (int)_e; (void)cudaGetLastError(); return QAQ_ERR_CUDA; } \
     } while (0)
+
+// the token count in device memory that the qaq_stream_* calls work with (valid between qaq_stream_begin and
+// qaq_stream_end), and the arrival counter of the kernel that advances it (zero between launches)
+static inline int* qaq_d_count(const qaq_cache* c) { return c->d_status + 1; }
+static inline unsigned* qaq_d_ticket(const qaq_cache* c) { return (unsigned*)(c->d_status + 2); }
 
 static inline bool qaq_dim_ok(int D) { return D == 32 || D == 64 || D == 128; }
 

@@ -41,6 +41,9 @@ struct QuantArgs {
     uint32_t ocap;
     int tmax_pad, ntiles;
     int* status;
+    int* d_count;          // null, or the token count kept in device memory: read instead of t_old / first_tile and
+    unsigned* d_ticket;    //   advanced by the last CTA of the launch to finish (small appends only)
+    int max_tokens;
     uint8_t* out_bitsK;    // selection only
     uint8_t* out_bitsV;
 };
@@ -124,17 +127,39 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
     constexpr int P = D / 32;            // lanes per token
     constexpr int NT = 2 * D;            // threads
     constexpr int IMG = qaqc::v_tile_bytes_max(D);
+    constexpr bool COUNTED = XSEL < 0 && !SELECT_ONLY;   // the launches that may take the token count from device memory
     const int bh = blockIdx.y;
-    const int tile = a.first_tile + blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slot = tid / P, p = tid % P;
+    int t_old = a.t_old, first_tile = a.first_tile;
+    if (COUNTED && a.d_count) {
+        t_old = *a.d_count;                // the same value in every thread of the launch: it is written only by tick()
+        first_tile = t_old / QAQ_TILE;
+        if (t_old + a.tok_hi > a.max_tokens) {             // no room: nothing is stored, the count stays
+            if (tid == 0) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
+            return;
+        }
+    }
+    const int tile = first_tile + blockIdx.x;
+    // counted launches: the last CTA to get here moves the count on.  Every thread of every CTA has used the count it
+    // read by then (the barrier), and nothing else of the launch reads it afterwards.
+    auto tick = [&]() {
+        if (COUNTED && a.d_count) {
+            __syncthreads();
+            if (tid == 0) {
+                __threadfence();
+                const unsigned n = gridDim.x * gridDim.y;
+                if (atomicInc(a.d_ticket, n - 1) == n - 1) *a.d_count = t_old + a.tok_hi;
+            }
+        }
+    };
 
-    const int abs_lo = max(tile * QAQ_TILE, a.t_old + a.tok_lo);
-    const int abs_hi = min((tile + 1) * QAQ_TILE, a.t_old + a.tok_hi);
+    const int abs_lo = max(tile * QAQ_TILE, t_old + a.tok_lo);
+    const int abs_hi = min((tile + 1) * QAQ_TILE, t_old + a.tok_hi);
     const int s_lo = abs_lo - tile * QAQ_TILE, s_hi = abs_hi - tile * QAQ_TILE;
     const bool valid = slot >= s_lo && slot < s_hi;       // a new token
     const bool old = !SELECT_ONLY && slot < s_lo;         // a token the tile already holds
-    const int tn = tile * QAQ_TILE + slot - a.t_old;      // index among the new tokens
+    const int tn = tile * QAQ_TILE + slot - t_old;        // index among the new tokens
 
     __shared__ uint8_t s_bits[2][QAQ_TILE];   // widths of the tile's slots (0: empty)
     __shared__ uint32_t s_cnt[2][QAQ_TILE];   // outlier counts of the new tokens, then exclusive offsets
@@ -410,7 +435,7 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
         }
     }
     __syncthreads();   // [C] image complete, pool positions known, every old byte of the tile has been read
-    if (s_skip) return;
+    if (s_skip) { tick(); return; }
 
     // ---- the image goes out with vector stores; outlier list; per-token metadata
 #pragma unroll
@@ -433,7 +458,7 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
                 const uint32_t w = s_work[x - X0][i], sl = w >> 8, ch = w & 0xFFu;
                 const uint32_t pos = s_obase[x] + i;
                 if (pos < s_olimit[x])
-                    ts.outl[(size_t)bh * a.ocap + pos] = (uint32_t)__half_as_ushort(X[(size_t)(tile * QAQ_TILE + (int)sl - a.t_old) * a.st + ch]) |
+                    ts.outl[(size_t)bh * a.ocap + pos] = (uint32_t)__half_as_ushort(X[(size_t)(tile * QAQ_TILE + (int)sl - t_old) * a.st + ch]) |
                                                           (ch << 16) | (sl << 24);
             }
             if (ntot > OUT_STAGE) {
@@ -459,6 +484,7 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
             ts.mnmx[mt] = (uint32_t)__half_as_ushort(__float2half_rn(mnf[x])) | ((uint32_t)__half_as_ushort(__float2half_rn(mxf[x])) << 16);
         }
     }
+    tick();
 }
 
 
@@ -573,4 +599,30 @@ extern "C" qaq_status qaq_quantize_append(qaq_cache* c, const void* K_new, const
     if (n_new == 0) return QAQ_OK;
     return qaq_launch_append(c, K_new, V_new, stride_b, stride_h, stride_t, n_new, bitsK, bitsV, policy, score_ring,
                              nvalid, thr, (cudaStream_t)stream);
+}
+
+// One new token per (b,h) with the token count taken from (and advanced in) device memory: the open tile (or a new one)
+// of every (b,h) is rebuilt by one CTA, as in the head / tail launch of qaq_launch_append.  Nothing on the host changes,
+// so the call can be captured in a CUDA graph and replayed.
+extern "C" qaq_status qaq_stream_append(qaq_cache* c, const void* k_new, const void* v_new, long stride_b, long stride_h,
+                                        const uint8_t* bitK, const uint8_t* bitV, const qaq_policy* policy,
+                                        const float* score_col, const uint8_t* nvalid, const float* thr, void* stream) {
+    if (!c || !thr) return QAQ_ERR_INVALID_ARG;
+    if ((bitK == nullptr) != (bitV == nullptr)) return QAQ_ERR_INVALID_ARG;
+    if (!bitK && (!policy || !score_col || !nvalid)) return QAQ_ERR_INVALID_ARG;
+    const int D = c->cfg.head_dim;
+    qaq_status st = check_dense(k_new, v_new, stride_b, stride_h, D, D);
+    if (st != QAQ_OK) return st;
+    QuantArgs a{};
+    a.K = (const __half*)k_new; a.V = (const __half*)v_new; a.sb = stride_b; a.sh = stride_h; a.st = D;
+    a.H = c->cfg.heads; a.n_new = 1; a.tok_lo = 0; a.tok_hi = 1;
+    a.bitsK = bitK; a.bitsV = bitV; a.ring = score_col; a.nvalid = nvalid; a.W = c->cfg.window; a.thr = thr;
+    a.cK = policy ? policy->cK : 0.f; a.cV = policy ? policy->cV : 0.f; a.bmin = c->cfg.bits_min; a.bmax = c->cfg.bits_max;
+    a.k = c->t[0]; a.v = c->t[1]; a.pool_bytes = c->pool_bytes; a.ocap = c->ocap;
+    a.tmax_pad = c->tmax_pad; a.ntiles = c->ntiles; a.status = c->d_status;
+    a.d_count = qaq_d_count(c); a.d_ticket = qaq_d_ticket(c); a.max_tokens = (int)c->cfg.max_tokens;
+    st = launch_x<false, -1>(D, dim3(1, c->BH), a, (cudaStream_t)stream);
+    if (st != QAQ_OK) return st;
+    QAQ_CUDA_TRY(cudaGetLastError());
+    return QAQ_OK;
 }

@@ -24,6 +24,7 @@ EXPORTED = [
     "qaq_decode_attention_host", "qaq_cache_stats", "qaq_cache_export", "qaq_decode_attention_static",
     "qaq_requantize_down", "qaq_requantize", "qaq_cache_compact", "qaq_cache_pool_use", "qaq_prefill_window_workspace_bytes", "qaq_prefill_window",
     "qaq_qnorm2_quantile", "qaq_decode_multi_workspace_bytes", "qaq_decode_attention_multi",
+    "qaq_stream_begin", "qaq_stream_append", "qaq_stream_decode", "qaq_stream_end",
 ]
 
 
@@ -91,6 +92,12 @@ def lib():
         L.qaq_qnorm2_quantile.argtypes = [C.c_void_p, C.c_long, C.c_double, C.c_void_p, C.c_void_p]
         L.qaq_decode_multi_workspace_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
         L.qaq_decode_attention_multi.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qaq_stream_begin.argtypes = [C.c_void_p, C.c_void_p]
+        L.qaq_stream_end.argtypes = [C.c_void_p, C.c_void_p]
+        L.qaq_stream_append.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_long, C.c_long, C.c_void_p, C.c_void_p,
+                                        C.POINTER(Policy), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.qaq_stream_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_long, C.c_void_p,
+                                        C.c_size_t, C.c_void_p]
         L.qaq_cache_compact.argtypes = [C.c_void_p, C.c_void_p]
         L.qaq_cache_pool_use.argtypes = [C.c_void_p, C.POINTER(C.c_long), C.POINTER(C.c_long), C.c_void_p]
         L.qaq_requantize.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_long, C.c_long, C.c_long, C.c_void_p, C.c_void_p,
@@ -299,6 +306,44 @@ def qaq_decode_attention_multi(cache: Cache, q, softmax_scale, out=None):
     ws = cache._ws_multi
     _check(lib().qaq_decode_attention_multi(cache.handle, _ptr(q), n_q, float(softmax_scale), _ptr(out), _ptr(ws), ws.numel(),
                                             _stream()), "qaq_decode_attention_multi")
+    return out
+
+
+def qaq_stream_begin(cache: Cache):
+    """The token count moves to device memory: from here to qaq_stream_end only the qaq_stream_* calls may be used."""
+    _check(lib().qaq_stream_begin(cache.handle, _stream()), "qaq_stream_begin")
+
+
+def qaq_stream_end(cache: Cache):
+    """Brings the token count back to the host (synchronises the current stream); returns it."""
+    _check(lib().qaq_stream_end(cache.handle, _stream()), "qaq_stream_end")
+    return cache.tokens
+
+
+def qaq_stream_append(cache: Cache, k_new, v_new, thr, *, bitK=None, bitV=None, policy=None, score_col=None, nvalid=None):
+    """One token per (b,h) behind the device-side count: k_new / v_new fp16 [B,H,1,D] (or [B,H,D])."""
+    if k_new.dim() == 3:
+        k_new, v_new = k_new.unsqueeze(2), v_new.unsqueeze(2)
+    assert k_new.shape[2] == 1
+    sb, sh, _ = _strides(k_new)
+    assert _strides(v_new)[:2] == (sb, sh)
+    pol = C.byref(policy) if policy is not None else None
+    _check(lib().qaq_stream_append(cache.handle, _ptr(k_new), _ptr(v_new), sb, sh, _ptr(bitK), _ptr(bitV), pol,
+                                   _ptr(score_col), _ptr(nvalid), _ptr(thr), _stream()), "qaq_stream_append")
+
+
+def qaq_stream_decode(cache: Cache, q, softmax_scale, out, scores_out=None):
+    """Decode attention over as many tokens as the device-side count says; scores_out fp32 [B*H, >= max_tokens]."""
+    BH, D = cache.cfg.batch * cache.cfg.heads, cache.cfg.head_dim
+    assert q.dtype == torch.float16 and q.is_contiguous() and q.numel() == BH * D
+    assert out.dtype == torch.float32 and out.is_contiguous() and out.numel() == BH * D
+    stride = 0
+    if scores_out is not None:
+        assert scores_out.dtype == torch.float32 and scores_out.is_contiguous() and scores_out.shape[0] == BH
+        stride = scores_out.shape[1]
+    ws = cache.workspace()
+    _check(lib().qaq_stream_decode(cache.handle, _ptr(q), float(softmax_scale), _ptr(out), _ptr(scores_out), stride, _ptr(ws),
+                                   ws.numel(), _stream()), "qaq_stream_decode")
     return out
 
 
