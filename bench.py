@@ -536,12 +536,37 @@ def extras(qaq, dev, peak, only="", sm_mhz=None):
             stream()
         b.record(); torch.cuda.synchronize()
         us_s = a.elapsed_time(b) * 1e3 / reps
+        # the same step with the token count in device memory, captured once in a CUDA graph and replayed
+        qaq.qaq_stream_begin(cache)
+
+        def stream_counted():
+            if uniform is None:
+                qaq.qaq_stream_append(cache, k1, v1, thr, policy=pol, score_col=r1, nvalid=n1)
+            else:
+                qaq.qaq_stream_append(cache, k1, v1, thr, bitK=b1, bitV=b1)
+            qaq.qaq_stream_decode(cache, q, scale, outb)
+        stream_counted()                      # loads the kernels before the capture
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            stream_counted()
+        reps_g = min(24, cfg.max_tokens - t_now - reps - 1)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps_g - 3):
+            graph.replay()
+        b.record(); torch.cuda.synchronize()
+        us_g = a.elapsed_time(b) * 1e3 / (reps_g - 3)
+        assert qaq.qaq_stream_end(cache) == t_now + reps + 1 + reps_g
+        del graph
         res[name] = {"tokens": T, "bh": BH, "quantize_us": round(us_q, 1), "quantize_gbs": round(ab["quantize"] / us_q / 1e3, 1),
                      "quantize_frac_of_hbm": round(ab["quantize"] / us_q / 1e3 / peak, 3),
                      "decode_us": round(us_d, 1), "decode_gbs": round(ab["decode"] / us_d / 1e3, 1),
                      "decode_frac_of_hbm": round(ab["decode"] / us_d / 1e3 / peak, 3),
                      "cached_tokens_per_s": round(wl.batch * T / (us_d * 1e-6), 1),
-                     "append1_plus_decode_us": round(us_s, 1),
+                     "append1_plus_decode_us": round(us_s, 1), "append1_plus_decode_graph_replay_us": round(us_g, 1),
                      "mean_bits": [round(st.code_bytes[0] * 8 / (BH * T * D), 2), round(st.code_bytes[1] * 8 / (BH * T * D), 2)],
                      "cr_paper": round(st.cr_paper, 3)}
         if name == "C3_layer_low_widths":      # fewer bytes, the same instructions: the issue ceiling is the one that binds
@@ -708,10 +733,43 @@ def stream_c5(qaq, dev):
     b.record(); torch.cuda.synchronize()
     sec = a.elapsed_time(b) * 1e-3
     st = qaq.qaq_cache_stats(cache)
-    return {"steps": T1 - T0, "seconds": round(sec, 2), "us_per_step": round(sec / (T1 - T0) * 1e6, 1),
-            "generated_tokens_per_s": round(wl.batch * (T1 - T0) / sec, 1), "final_tokens": int(st.tokens),
-            "device_status": int(st.device_status), "clocks": sampler.stop(),
-            "note": "host-launched steps (one append launch, decode + merge per step); values of appended tokens stay at 8 bits"}
+    res = {"steps": T1 - T0, "seconds": round(sec, 2), "us_per_step": round(sec / (T1 - T0) * 1e6, 1),
+           "generated_tokens_per_s": round(wl.batch * (T1 - T0) / sec, 1), "final_tokens": int(st.tokens),
+           "device_status": int(st.device_status),
+           "note": "host-launched steps (one append launch, decode + merge per step); values of appended tokens stay at 8 bits"}
+    # the same run with the token count in device memory: one captured append + decode pair replayed 98304 times, the
+    # new token's rows copied into the captured buffers before every replay
+    cache.reset()
+    qaq.qaq_quantize_append(cache, K[:, :, :T0], V[:, :, :T0], thr, policy=pol, ring=ring, nvalid=nv)
+    k1 = torch.empty((wl.batch, wl.heads, 1, D), dtype=torch.float16, device=dev)
+    v1 = torch.empty_like(k1)
+    warm = qaq.Cache(qaq.make_config(wl.batch, wl.heads, D, 64, wl.bits_min, wl.bits_max, W, wl.alpha))
+    k1.zero_(); v1.zero_()
+    qaq.qaq_stream_begin(warm)                 # one eager step on a scratch cache loads the kernels before the capture
+    qaq.qaq_stream_append(warm, k1, v1, thr, policy=pol, score_col=r1, nvalid=n1)
+    qaq.qaq_stream_decode(warm, q, scale, outb)
+    qaq.qaq_stream_end(warm)
+    warm.close()
+    cache.workspace()
+    qaq.qaq_stream_begin(cache)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        qaq.qaq_stream_append(cache, k1, v1, thr, policy=pol, score_col=r1, nvalid=n1)
+        qaq.qaq_stream_decode(cache, q, scale, outb)
+    a.record()
+    for t in range(T0, T1):
+        k1.copy_(K[:, :, t:t + 1]); v1.copy_(V[:, :, t:t + 1])
+        graph.replay()
+    b.record(); torch.cuda.synchronize()
+    sec_g = a.elapsed_time(b) * 1e-3
+    final = qaq.qaq_stream_end(cache)
+    st = qaq.qaq_cache_stats(cache)
+    res["graph_replay"] = {"seconds": round(sec_g, 2), "us_per_step": round(sec_g / (T1 - T0) * 1e6, 1),
+                           "generated_tokens_per_s": round(wl.batch * (T1 - T0) / sec_g, 1), "final_tokens": int(final),
+                           "device_status": int(st.device_status)}
+    res["clocks"] = sampler.stop()
+    return res
 
 
 def cpu_baseline(wl, hyper, budget_s=15.0):
