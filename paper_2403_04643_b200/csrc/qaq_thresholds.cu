@@ -19,13 +19,14 @@ namespace {
 
 constexpr int SAMPLE_TOKENS = 64;
 constexpr int SCAN_TOKENS = 256;     // tokens per CTA of the scan
-constexpr int CHUNK_PIECES = 4 * 256; // 16-byte pieces looked at between two barriers (four per thread)
+constexpr int WARP_FLAGS = 192;      // 16-byte pieces a warp of the scan can set aside before it has to look at them
 constexpr int CTA_LIST = 4096;       // candidates per tail a scan CTA can hold
 constexpr int SELECT_KEYS = 16384;   // candidates of one tail the select kernel keeps in shared memory
 
 __device__ __forceinline__ uint32_t key_of(unsigned short h) { return (h & 0x8000u) ? (uint32_t)(~h & 0xFFFFu) : (uint32_t)(h | 0x8000u); }
 __device__ __forceinline__ unsigned short half_of_key(uint32_t k) { return (k & 0x8000u) ? (unsigned short)(k & 0x7FFFu) : (unsigned short)(~k & 0xFFFFu); }
 __device__ __forceinline__ bool is_nan_bits(unsigned short h) { return (h & 0x7FFFu) > 0x7C00u; }
+__device__ __forceinline__ __half2 h2_of(uint32_t x) { return *reinterpret_cast<__half2*>(&x); }
 __device__ __forceinline__ float float_of_key(uint32_t k) { return __half2float(__ushort_as_half(half_of_key(k))); }
 
 struct Problem {          // per (b,h,tensor), in the workspace
@@ -296,85 +297,116 @@ __global__ void __launch_bounds__(256) thr_sample_kernel(const ThrArgs a) {
     }
 }
 
-// ---- 2. the one pass over the data: compaction of the tail candidates
+// ---- 2. the one pass over the data: compaction of the tail candidates.
+// Almost all entries are inside [lo, hi], so the pass is a cheap filter first: a 16-byte piece whose smallest entry is
+// at least lo and whose largest is at most hi (NaN-propagating min / max, so a NaN fails both) is dropped; the others
+// (about one in ten at alpha = 1 %) are set aside in a buffer of the warp's own, and when enough of them have come
+// together the warp looks at them entry by entry with all lanes busy.  Nothing in the loop needs the other warps:
+// no CTA barrier, one shared-memory reservation per warp, tail and batch of set-aside pieces.
 __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
     const int bhx = blockIdx.y, bh = bhx >> 1, x = bhx & 1;
     Problem* pr = a.prob + bhx;
     if (pr->done) return;
     __shared__ unsigned short s_list[2][CTA_LIST];
-    __shared__ uint4 s_flag[CHUNK_PIECES];                    // 16-byte pieces with something outside [lo, hi]
-    __shared__ uint32_t s_n[2], s_base[2], s_nan, s_nflag;
+    __shared__ uint4 s_flag[8][WARP_FLAGS];                   // per warp: pieces with something outside [lo, hi]
+    __shared__ uint32_t s_n[2], s_base[2], s_nan;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned lt = (1u << lane) - 1u;
     if (threadIdx.x < 2) s_n[threadIdx.x] = 0;
     if (threadIdx.x == 2) s_nan = 0;
-    if (threadIdx.x == 3) s_nflag = 0;
     __syncthreads();
     const float flo = float_of_key(pr->klo), fhi = float_of_key(pr->khi);
     const __half2 lo2 = __float2half2_rn(flo), hi2 = __float2half2_rn(fhi);   // exact: both are binary16 values
     const int b_idx = bh / a.H, h_idx = bh % a.H;
-    const __half* X = a.X[x] + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
-    const int t0 = blockIdx.x * SCAN_TOKENS, t1 = min(a.T, t0 + SCAN_TOKENS);
-    const int tok_shift = 31 - __clz(a.D / 8);                   // 16-byte pieces per token is a power of two
-    const int n = (t1 - t0) << tok_shift;
-    for (int i0 = 0; i0 < n; i0 += 4 * 256) {
+    const int t0 = blockIdx.x * SCAN_TOKENS, ntok = min(a.T, t0 + SCAN_TOKENS) - t0;
+    const int tok_shift = 31 - __clz(a.D / 8);                   // 16-byte pieces per token is a power of two (4, 8, 16)
+    // thread tid looks at piece (tid mod pieces per token) of tokens tid >> tok_shift, + 256 >> tok_shift, ...
+    int tok = (int)threadIdx.x >> tok_shift;
+    const int tok_step = 256 >> tok_shift;
+    const __half* ptr = (x ? a.X[1] : a.X[0]) + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh + (size_t)(t0 + tok) * a.st +
+                        (((int)threadIdx.x & ((1 << tok_shift) - 1)) << 3);
+    const size_t ptr_step = (size_t)tok_step * a.st;
+    uint4* wflag = s_flag[warp];
+    uint32_t nflag = 0;      // pieces set aside by this warp (the same in all its lanes)
+    uint32_t nnan = 0;
+
+    for (int c0 = 0; c0 < ntok; c0 += 4 * tok_step) {
         // four independent 16-byte loads per thread before any of them is looked at
         uint4 raw[4];
+        bool in_range[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int i = i0 + u * 256 + threadIdx.x;
+            in_range[u] = tok + u * tok_step < ntok;
             raw[u] = make_uint4(0, 0, 0, 0);
-            if (i < n) raw[u] = *reinterpret_cast<const uint4*>(X + (size_t)(t0 + (i >> tok_shift)) * a.st + ((i & ((1 << tok_shift) - 1)) << 3));
+            if (in_range[u]) raw[u] = *reinterpret_cast<const uint4*>(ptr + u * ptr_step);
         }
+        tok += 4 * tok_step;
+        ptr += 4 * ptr_step;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            // cheap filter: almost all entries are inside [lo, hi]; a 16-byte piece holding anything
-            // else is set aside and looked at entry by entry afterwards, with all lanes busy
-            const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
-            // all-ones iff every entry of the piece is inside [lo, hi] (a NaN compares false)
-            uint32_t all_in = 0xFFFFFFFFu;
+            const __half2 v0 = h2_of(raw[u].x), v1 = h2_of(raw[u].y), v2 = h2_of(raw[u].z), v3 = h2_of(raw[u].w);
+            const __half2 mn = __hmin2_nan(__hmin2_nan(v0, v1), __hmin2_nan(v2, v3));
+            const __half2 mx = __hmax2_nan(__hmax2_nan(v0, v1), __hmax2_nan(v2, v3));
+            const bool flag = in_range[u] && !(__hbge2(mn, lo2) && __hble2(mx, hi2));
+            const unsigned bal = __ballot_sync(0xFFFFFFFFu, flag);
+            if (flag) wflag[nflag + __popc(bal & lt)] = raw[u];
+            nflag += (uint32_t)__popc(bal);
+        }
+        __syncwarp();
+        // the next round may set aside 128 more; the last round empties the buffer
+        if (!(nflag > (uint32_t)(WARP_FLAGS - 128) || c0 + 4 * tok_step >= ntok)) continue;
+        // the warp's set-aside pieces entry by entry: per lane the entries below lo, above hi and NaN; one reservation
+        // per tail for the whole batch, then every lane writes its keys
+        for (uint32_t i0 = 0; i0 < nflag; i0 += 32) {
+            const bool have = i0 + lane < nflag;
+            const uint4 r = have ? wflag[i0 + lane] : make_uint4(0, 0, 0, 0);
+            const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+            uint32_t below = 0, above = 0, nans = 0;              // bit j / 16 + j: low / high half of word j
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const __half2 v = *reinterpret_cast<const __half2*>(&w[j]);
-                all_in &= __hge2_mask(v, lo2) & __hle2_mask(v, hi2);
+                const __half2 v = h2_of(w[j]);
+                const uint32_t ge = __hge2_mask(v, lo2), le = __hle2_mask(v, hi2);   // a NaN compares false twice
+                below |= (~ge & le & 0x00010001u) << j;
+                above |= (ge & ~le & 0x00010001u) << j;
+                nans |= (~(ge | le) & 0x00010001u) << j;
             }
-            const bool inside = all_in == 0xFFFFFFFFu;
-            // one shared-memory reservation per warp for its flagged pieces
-            const bool flag = !inside && i0 + u * 256 + (int)threadIdx.x < n;
-            const unsigned bal = __ballot_sync(0xFFFFFFFFu, flag);
-            if (bal) {
-                const int lane = threadIdx.x & 31;
-                uint32_t base = 0;
-                if (lane == 0) base = atomicAdd(&s_nflag, (uint32_t)__popc(bal));
-                base = __shfl_sync(0xFFFFFFFFu, base, 0);
-                if (flag) s_flag[base + __popc(bal & ((1u << lane) - 1u))] = raw[u];
-            }
-        }
-    __syncthreads();
-    for (uint32_t i = threadIdx.x; i < s_nflag; i += blockDim.x) {
-        const uint4 r = s_flag[i];
-        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
-        // bit j / 16 + j: low / high half of word j is not inside [lo, hi] (a candidate or a NaN)
-        uint32_t out = 0;
+            if (!have) { below = 0; above = 0; nans = 0; }
+            nnan += (uint32_t)__popc(nans);
+            const uint32_t pk = (uint32_t)__popc(below) | ((uint32_t)__popc(above) << 16);   // at most 8 each
+            uint32_t inc = pk;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const __half2 v = *reinterpret_cast<const __half2*>(&w[j]);
-            out |= (~(__hge2_mask(v, lo2) & __hle2_mask(v, hi2)) & 0x00010001u) << j;
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                if (lane >= d) inc += t;
+            }
+            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);
+            uint32_t b0 = 0, b1 = 0;
+            if (lane == 0) {
+                if (tot & 0xFFFFu) b0 = atomicAdd(&s_n[0], tot & 0xFFFFu);
+                if (tot >> 16) b1 = atomicAdd(&s_n[1], tot >> 16);
+            }
+            uint32_t pos[2] = {__shfl_sync(0xFFFFFFFFu, b0, 0) + ((inc - pk) & 0xFFFFu), __shfl_sync(0xFFFFFFFFu, b1, 0) + ((inc - pk) >> 16)};
+#pragma unroll
+            for (int side = 0; side < 2; ++side) {
+                uint32_t m = side ? above : below;
+                while (m) {
+                    const int bit = __ffs(m) - 1;
+                    m &= m - 1;
+                    const int j = bit & 3;
+                    const uint32_t wj = (j & 2) ? ((j & 1) ? w[3] : w[2]) : ((j & 1) ? w[1] : w[0]);
+                    const unsigned short h = (unsigned short)((bit >> 4) ? (wj >> 16) : (wj & 0xFFFFu));
+                    if (pos[side] < (uint32_t)CTA_LIST) s_list[side][pos[side]] = (unsigned short)key_of(h);
+                    ++pos[side];
+                }
+            }
         }
-        while (out) {
-            const int bit = __ffs(out) - 1;
-            out &= out - 1;
-            const int j = bit & 3;
-            const uint32_t wj = (j & 2) ? ((j & 1) ? w[3] : w[2]) : ((j & 1) ? w[1] : w[0]);
-            const unsigned short h = (unsigned short)((bit >> 4) ? (wj >> 16) : (wj & 0xFFFF));
-            if (is_nan_bits(h)) { atomicAdd(&s_nan, 1u); continue; }
-            const int side = __half2float(__ushort_as_half(h)) < flo ? 0 : 1;   // outside [lo, hi]: below lo or above hi
-            const uint32_t pos = atomicAdd(&s_n[side], 1u);
-            if (pos < CTA_LIST) s_list[side][pos] = (unsigned short)key_of(h);
-        }
+        nflag = 0;
+        __syncwarp();     // the buffer is free again
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) nnan += __shfl_xor_sync(0xFFFFFFFFu, nnan, o);
+    if (lane == 0 && nnan) atomicAdd(&s_nan, nnan);
     __syncthreads();
-    if (threadIdx.x == 0) s_nflag = 0;   // the next chunk starts an empty list of flagged pieces
-    __syncthreads();
-    }   // chunks
     if (threadIdx.x < 2) s_base[threadIdx.x] = s_n[threadIdx.x] ? atomicAdd(&pr->cnt[threadIdx.x], s_n[threadIdx.x]) : 0u;
     if (threadIdx.x == 2 && s_nan) atomicAdd(&pr->nan, s_nan);
     __syncthreads();
