@@ -18,8 +18,11 @@
 namespace {
 
 constexpr int SAMPLE_TOKENS = 64;
-constexpr int SCAN_TOKENS = 256;     // tokens per CTA of the scan
-constexpr int WARP_FLAGS = 192;      // 16-byte pieces a warp of the scan can set aside before it has to look at them
+#ifndef QWARP_FLAGS
+#define QWARP_FLAGS 192
+#endif
+constexpr int SCAN_TOKENS_MAX = 512; // tokens per CTA of the scan (fewer where alpha is large: see scan_tokens_for)
+constexpr int WARP_FLAGS = QWARP_FLAGS;      // 16-byte pieces a warp of the scan can set aside before it has to look at them
 constexpr int CTA_LIST = 4096;       // candidates per tail a scan CTA can hold
 constexpr int SELECT_KEYS = 16384;   // candidates of one tail the select kernel keeps in shared memory
 
@@ -34,7 +37,8 @@ struct Problem {          // per (b,h,tensor), in the workspace
     uint32_t cnt[2];      // candidates found (may exceed the capacity: then the list is incomplete)
     uint32_t nan;         // NaN entries seen by the scan
     uint32_t done;        // solved by the sample kernel
-    uint32_t pad[2];
+    uint32_t overflow;    // bit `tail`: a scan CTA found more candidates than it can hold, the list has holes
+    uint32_t pad;
 };
 
 struct ThrArgs {
@@ -45,6 +49,7 @@ struct ThrArgs {
     Problem* prob;        // [BH*2]
     unsigned short* list; // [BH*2][2][cap]
     uint32_t cap;
+    int scan_tokens;      // tokens per CTA of the scan
     float* thr;           // [BH][4]
 };
 
@@ -268,7 +273,7 @@ __global__ void __launch_bounds__(256) thr_sample_kernel(const ThrArgs a) {
     const bool whole = (ns == a.T);
     if (Mv == 0) {
         if (threadIdx.x == 0) {
-            pr->klo = 0; pr->khi = 0xFFFF; pr->cnt[0] = pr->cnt[1] = 0; pr->nan = 0; pr->done = whole ? 1u : 0u;
+            pr->klo = 0; pr->khi = 0xFFFF; pr->cnt[0] = pr->cnt[1] = 0; pr->nan = 0; pr->overflow = 0; pr->done = whole ? 1u : 0u;
             if (whole) { a.thr[(size_t)bh * 4 + 2 * x] = 0.f; a.thr[(size_t)bh * 4 + 2 * x + 1] = 0.f; }
         }
         return;
@@ -289,7 +294,7 @@ __global__ void __launch_bounds__(256) thr_sample_kernel(const ThrArgs a) {
     uint32_t klo, khi;
     cta_select_keys(s_keys, (uint32_t)M, r_lo + n_neg_nan, r_hi + n_neg_nan, hist, s_tmp, klo, khi);
     if (threadIdx.x == 0) {
-        pr->klo = klo; pr->khi = khi; pr->cnt[0] = pr->cnt[1] = 0; pr->nan = 0; pr->done = whole ? 1u : 0u;
+        pr->klo = klo; pr->khi = khi; pr->cnt[0] = pr->cnt[1] = 0; pr->nan = 0; pr->overflow = 0; pr->done = whole ? 1u : 0u;
         if (whole) {
             a.thr[(size_t)bh * 4 + 2 * x] = float_of_key(klo);
             a.thr[(size_t)bh * 4 + 2 * x + 1] = float_of_key(khi);
@@ -318,7 +323,7 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
     const float flo = float_of_key(pr->klo), fhi = float_of_key(pr->khi);
     const __half2 lo2 = __float2half2_rn(flo), hi2 = __float2half2_rn(fhi);   // exact: both are binary16 values
     const int b_idx = bh / a.H, h_idx = bh % a.H;
-    const int t0 = blockIdx.x * SCAN_TOKENS, ntok = min(a.T, t0 + SCAN_TOKENS) - t0;
+    const int t0 = blockIdx.x * a.scan_tokens, ntok = min(a.T, t0 + a.scan_tokens) - t0;
     const int tok_shift = 31 - __clz(a.D / 8);                   // 16-byte pieces per token is a power of two (4, 8, 16)
     // thread tid looks at piece (tid mod pieces per token) of tokens tid >> tok_shift, + 256 >> tok_shift, ...
     int tok = (int)threadIdx.x >> tok_shift;
@@ -413,9 +418,8 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
 #pragma unroll
     for (int side = 0; side < 2; ++side) {
         const uint32_t cnt = s_n[side];
-        // a CTA list that overflowed makes the global count exceed what was stored: the select
-        // kernel sees cnt > cap or a hole and falls back; mark it by a huge count
-        if (cnt > CTA_LIST) { if (threadIdx.x == 0) atomicAdd(&pr->cnt[side], 0x40000000u); continue; }
+        // a CTA list that overflowed leaves a hole in the global list: the select kernel falls back for that tail
+        if (cnt > CTA_LIST) { if (threadIdx.x == 0) atomicOr(&pr->overflow, 1u << side); continue; }
         unsigned short* dst = a.list + ((size_t)bhx * 2 + side) * a.cap;
         for (uint32_t i = threadIdx.x; i < cnt; i += blockDim.x) {
             const uint32_t pos = s_base[side] + i;
@@ -438,7 +442,7 @@ __global__ void __launch_bounds__(256) thr_select_kernel(const ThrArgs a) {
     if (N > 0) {
         const unsigned long long k = rank_k(a.alpha, N);
         const uint32_t c = pr->cnt[side];
-        if (c > k && c <= a.cap) {
+        if (c > k && c <= a.cap && !((pr->overflow >> side) & 1u)) {
             // rank k from below in the low list, rank k from above in the high list
             const uint32_t want = side == 0 ? (uint32_t)k : (uint32_t)(c - 1 - k);
             const unsigned short* l = a.list + ((size_t)bhx * 2 + side) * a.cap;   // 16-byte aligned
@@ -467,6 +471,15 @@ __global__ void __launch_bounds__(256) thr_select_kernel(const ThrArgs a) {
         }
     }
     if (threadIdx.x == 0) a.thr[(size_t)bh * 4 + 2 * x + side] = res;
+}
+
+// Tokens per CTA of the scan: as many as keep the expected number of candidates per tail (1.25 times the tail mass
+// plus the bracket's slack) well inside the CTA's list; a CTA that overflows sends its problem to the exact fallback.
+int scan_tokens_for(double alpha, int D) {
+    const double per_token = (0.625 * alpha + 0.004) * D;
+    int tokens = SCAN_TOKENS_MAX;
+    while (tokens > 64 && per_token * tokens > 0.6 * CTA_LIST) tokens /= 2;
+    return tokens;
 }
 
 uint32_t list_capacity(const qaq_config* cfg, int n_tokens) {
@@ -514,9 +527,11 @@ extern "C" qaq_status qaq_outlier_thresholds(const qaq_config* cfg, const void* 
     if (a.cap < 64) return QAQ_ERR_WORKSPACE;
     a.list = (unsigned short*)((char*)ws + head);
     a.thr = thr;
+    a.scan_tokens = SCAN_TOKENS_MAX;
     thr_sample_kernel<<<BH * 2, 256, 0, s>>>(a);
     if (n_tokens > SAMPLE_TOKENS) {
-        dim3 grid((n_tokens + SCAN_TOKENS - 1) / SCAN_TOKENS, BH * 2);
+        a.scan_tokens = scan_tokens_for(cfg->outlier_frac, cfg->head_dim);
+        dim3 grid((n_tokens + a.scan_tokens - 1) / a.scan_tokens, BH * 2);
         thr_scan_kernel<<<grid, 256, 0, s>>>(a);
         thr_select_kernel<<<BH * 4, 256, 0, s>>>(a);
     }

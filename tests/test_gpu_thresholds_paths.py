@@ -59,3 +59,13 @@ def test_constant_tensor_and_single_distinct_tail_value():
     K[:] = 1.5                       # every entry equal: both thresholds are that value, no outliers
     V[:, :, :, ::2] = -2.0           # half of the entries tie at the lower tail
     check(K, V, wl, wl.alpha)
+
+
+@pytest.mark.parametrize("alpha", [0.3, 0.5, 1.0])
+def test_tails_so_heavy_that_every_scan_block_overflows(alpha):
+    # a third of the entries (or more) beyond the bracket per tail: every block of the scan finds more candidates
+    # than it can hold, while the global list would have room for the count - the holes must send the problem to the
+    # exact select over its data
+    wl = synth.scaled(synth.CONFIGS["C2"], heads=2, tokens=2048)
+    K, V = synth.make_kv(wl, 0)
+    check(K, V, wl, alpha)
