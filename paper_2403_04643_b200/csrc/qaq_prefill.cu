@@ -201,18 +201,21 @@ __global__ void __launch_bounds__(256) window_normalize_kernel(const PrefillArgs
 // normalised rows are written once: K is read once and the ring written once (no logits in global memory, no
 // workspace).  Used while a (b,h) fits a portable cluster (up to 8 x 512 tokens); longer sequences take the two
 // kernels above.
-constexpr int PC_WARPS = 8;
-constexpr int PC_CHUNK = 512;           // tokens per CTA: 64 per warp
+constexpr int PC_WARPS = 16;            // 32 tokens per warp
+constexpr int PC_MINCTA = 2;            // two CTAs per SM (64 registers per thread)
+constexpr int PC_CHUNK = 512;           // tokens per CTA
 constexpr int PC_MAXCTA = 8;            // portable cluster size
 constexpr int PC_PITCH = PC_CHUNK + 8;  // row pitch of the logits tile in floats (spreads the rows of a fragment over the banks)
 
 template <int D>
-__global__ void __launch_bounds__(PC_WARPS * 32) window_cluster_kernel(const PrefillArgs a) {
+__global__ void __launch_bounds__(PC_WARPS * 32, PC_MINCTA) window_cluster_kernel(const PrefillArgs a) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     constexpr int WPL = D / 8;
     constexpr int KS = D / 16;
-    extern __shared__ __align__(16) float s_l[];            // [n][PC_PITCH] logits of this CTA's tokens
+    extern __shared__ __align__(16) float s_l[];            // [n][PC_PITCH] logits of this CTA's tokens, then the queries
+    // the queries as A-operand fragments, one uint4 per (16-row tile, k step, lane): every warp reads the same ones
+    uint4* s_q = reinterpret_cast<uint4*>(s_l + (size_t)a.n * PC_PITCH);
     __shared__ float2 s_part[PC_WARPS][32];
     __shared__ float2 s_stat[PW_MAXQ];                       // (max, sum of exponentials) of every row over this CTA's tokens
     __shared__ float s_m[PW_MAXQ], s_inv[PW_MAXQ];
@@ -234,21 +237,22 @@ __global__ void __launch_bounds__(PC_WARPS * 32) window_cluster_kernel(const Pre
     const int t_cta = chunk * PC_CHUNK;
     const int t_warp = t_cta + warp * (PC_CHUNK / PC_WARPS);
 
+    const int ntile = 2 * ((a.n + 31) / 32);
+    for (int idx = threadIdx.x; idx < ntile * KS * 32; idx += blockDim.x) {
+        const int ln = idx & 31, ks = (idx >> 5) % KS, tile = idx / (32 * KS);
+        const int r0 = tile * 16 + (ln >> 2), r1 = r0 + 8, cc = ln & 3;
+        const uint32_t* q0 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r0 * D + cc * (D / 4)) + 2 * ks;
+        const uint32_t* q1 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r1 * D + cc * (D / 4)) + 2 * ks;
+        uint4 f;
+        f.x = r0 < a.n ? q0[0] : 0u;
+        f.y = r1 < a.n ? q1[0] : 0u;
+        f.z = r0 < a.n ? q0[1] : 0u;
+        f.w = r1 < a.n ? q1[1] : 0u;
+        s_q[idx] = f;
+    }
+    __syncthreads();
+
     for (int mp = 0; mp * 32 < a.n; ++mp) {            // two 16-row tiles of queries at a time
-        uint32_t afr[2][KS][4];
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-            const int r0 = mp * 32 + mt * 16 + g, r1 = r0 + 8;
-#pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                const uint32_t* q0 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r0 * D + c * (D / 4)) + 2 * ks;
-                const uint32_t* q1 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r1 * D + c * (D / 4)) + 2 * ks;
-                afr[mt][ks][0] = r0 < a.n ? q0[0] : 0u;
-                afr[mt][ks][1] = r1 < a.n ? q1[0] : 0u;
-                afr[mt][ks][2] = r0 < a.n ? q0[1] : 0u;
-                afr[mt][ks][3] = r1 < a.n ? q1[1] : 0u;
-            }
-        }
         float rm[2][2], rs[2][2];
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) { rm[mt][0] = rm[mt][1] = NEG; rs[mt][0] = rs[mt][1] = 0.f; }
@@ -274,7 +278,11 @@ __global__ void __launch_bounds__(PC_WARPS * 32) window_cluster_kernel(const Pre
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
 #pragma unroll
-                for (int ks = 0; ks < KS; ++ks) mma_16816(acc[mt], afr[mt][ks], bw[2 * ks], bw[2 * ks + 1]);
+                for (int ks = 0; ks < KS; ++ks) {
+                    const uint4 f = s_q[((2 * mp + mt) * KS + ks) * 32 + lane];
+                    const uint32_t fr[4] = {f.x, f.y, f.z, f.w};
+                    mma_16816(acc[mt], fr, bw[2 * ks], bw[2 * ks + 1]);
+                }
             }
             // acc[mt][0..1]: row g, tokens t0+2c, t0+2c+1;  acc[mt][2..3]: row g+8
 #pragma unroll
@@ -345,13 +353,26 @@ __global__ void __launch_bounds__(PC_WARPS * 32) window_cluster_kernel(const Pre
     __syncthreads();
     // ---- normalised rows, newest first, written once; rows-per-token counts
     const int nt = min(PC_CHUNK, a.T - t_cta);
+    const bool vec_ok = (a.T & 3) == 0 && ((uintptr_t)a.ring & 15) == 0;      // rows start 16-byte aligned, no ragged end
     for (int r = warp; r < a.n; r += PC_WARPS) {
         const int i = a.n - 1 - r;
         const int last = a.T - a.n + i;
         const float M = s_m[i], inv = s_inv[i];
         float* row = a.ring + ((size_t)bh * a.n + r) * a.T + t_cta;
         const float* src = s_l + (size_t)i * PC_PITCH;
-        for (int k = lane; k < nt; k += 32) row[k] = (t_cta + k <= last) ? __expf(src[k] - M) * inv : 0.f;
+        if (vec_ok) {     // four tokens per lane and store
+            for (int k = 4 * lane; k < nt; k += 128) {
+                const float4 l = *reinterpret_cast<const float4*>(src + k);
+                float4 o;
+                o.x = (t_cta + k <= last) ? __expf(l.x - M) * inv : 0.f;
+                o.y = (t_cta + k + 1 <= last) ? __expf(l.y - M) * inv : 0.f;
+                o.z = (t_cta + k + 2 <= last) ? __expf(l.z - M) * inv : 0.f;
+                o.w = (t_cta + k + 3 <= last) ? __expf(l.w - M) * inv : 0.f;
+                *reinterpret_cast<float4*>(row + k) = o;
+            }
+        } else {
+            for (int k = lane; k < nt; k += 32) row[k] = (t_cta + k <= last) ? __expf(src[k] - M) * inv : 0.f;
+        }
     }
     for (int k = threadIdx.x; k < nt; k += blockDim.x) a.nvalid[(size_t)bh * a.T + t_cta + k] = (uint8_t)min(a.n, a.T - (t_cta + k));
     cluster.sync();      // nobody leaves while its statistics may still be read by the others
@@ -446,7 +467,8 @@ extern "C" qaq_status qaq_prefill_window(const qaq_config* cfg, const void* Q, c
     const int ncl = (n_tokens + PC_CHUNK - 1) / PC_CHUNK;
     if (ncl <= PC_MAXCTA) {
         // one pass: the CTAs of a (b,h) are one cluster
-        const size_t smem = (size_t)cfg->window * PC_PITCH * sizeof(float);
+        const size_t smem = (size_t)cfg->window * PC_PITCH * sizeof(float) +
+                            (size_t)(2 * ((cfg->window + 31) / 32)) * (cfg->head_dim / 16) * 32 * sizeof(uint4);   // logits, query fragments
         cudaLaunchConfig_t lc = {};
         lc.gridDim = dim3((unsigned)ncl, (unsigned)(cfg->batch * cfg->heads));
         lc.blockDim = dim3(PC_WARPS * 32);
