@@ -216,9 +216,11 @@ __global__ void __launch_bounds__(PC_WARPS * 32, PC_MINCTA) window_cluster_kerne
     extern __shared__ __align__(16) float s_l[];            // [n][PC_PITCH] logits of this CTA's tokens, then the queries
     // the queries as A-operand fragments, one uint4 per (16-row tile, k step, lane): every warp reads the same ones
     uint4* s_q = reinterpret_cast<uint4*>(s_l + (size_t)a.n * PC_PITCH);
-    __shared__ float2 s_part[PC_WARPS][32];
-    __shared__ float2 s_stat[PW_MAXQ];                       // (max, sum of exponentials) of every row over this CTA's tokens
-    __shared__ float s_m[PW_MAXQ], s_inv[PW_MAXQ];
+    __shared__ float s_part[PC_WARPS][32];                   // per warp: maximum of every row of the current 32 over its tokens
+    __shared__ float s_mcta[PW_MAXQ];                        // maximum of every row over this CTA's tokens
+    __shared__ float2 s_all[PC_MAXCTA][PW_MAXQ];             // (max, sum of exponentials) of every row over the tokens of every CTA
+                                                             // of the cluster: each CTA writes its entries into all the copies
+    __shared__ float s_inv[PW_MAXQ];
     const int bh = blockIdx.y, chunk = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, c = lane & 3;
@@ -236,13 +238,24 @@ __global__ void __launch_bounds__(PC_WARPS * 32, PC_MINCTA) window_cluster_kerne
     }
     const int t_cta = chunk * PC_CHUNK;
     const int t_warp = t_cta + warp * (PC_CHUNK / PC_WARPS);
+    // this warp's keys are on their way to L2 while the queries are laid out
+    constexpr int LPT = D >= 64 ? D / 64 : 1;                                    // 128-byte lines per token
+    for (int ln = lane; ln < (PC_CHUNK / PC_WARPS) * LPT; ln += 32) {
+        const int t = t_warp + ln / LPT;
+        if (t < a.T) asm volatile("prefetch.global.L2 [%0];" ::"l"(Kb + (size_t)t * a.st + (ln % LPT) * 64));
+    }
+    // first half of a cluster barrier: by the time the row statistics are exchanged every CTA of the cluster is known
+    // to be running (its shared memory may be written)
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 
     const int ntile = 2 * ((a.n + 31) / 32);
     for (int idx = threadIdx.x; idx < ntile * KS * 32; idx += blockDim.x) {
         const int ln = idx & 31, ks = (idx >> 5) % KS, tile = idx / (32 * KS);
         const int r0 = tile * 16 + (ln >> 2), r1 = r0 + 8, cc = ln & 3;
-        const uint32_t* q0 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r0 * D + cc * (D / 4)) + 2 * ks;
-        const uint32_t* q1 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r1 * D + cc * (D / 4)) + 2 * ks;
+        // k step ks of lane (., cc): words 2 (ks mod 2), + 1 of the 16-byte piece 4 (ks / 2) + cc of the row
+        const int w0 = 4 * (4 * (ks >> 1) + cc) + 2 * (ks & 1);
+        const uint32_t* q0 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r0 * D) + w0;
+        const uint32_t* q1 = reinterpret_cast<const uint32_t*>(Qb + (size_t)r1 * D) + w0;
         uint4 f;
         f.x = r0 < a.n ? q0[0] : 0u;
         f.y = r1 < a.n ? q1[0] : 0u;
@@ -253,129 +266,135 @@ __global__ void __launch_bounds__(PC_WARPS * 32, PC_MINCTA) window_cluster_kerne
     __syncthreads();
 
     for (int mp = 0; mp * 32 < a.n; ++mp) {            // two 16-row tiles of queries at a time
-        float rm[2][2], rs[2][2];
+        float rm[2][2];                 // running maximum of rows g, g + 8 of the two tiles over the tokens this lane sees
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt) { rm[mt][0] = rm[mt][1] = NEG; rs[mt][0] = rs[mt][1] = 0.f; }
+        for (int mt = 0; mt < 2; ++mt) rm[mt][0] = rm[mt][1] = NEG;
 
-#pragma unroll 2
-        for (int step = 0; step < PC_CHUNK / PC_WARPS / 8; ++step) {
+#pragma unroll 1
+        for (int step = 0; step < PC_CHUNK / PC_WARPS / 8; step += 2) {    // two groups of 8 tokens per set of query fragments
             const int t0 = t_warp + 8 * step;
             if (t0 >= a.T) break;
-            uint32_t bw[WPL];
-            {
-                const int t = t0 + g;
-                const uint4* src = reinterpret_cast<const uint4*>(Kb + (size_t)(t < a.T ? t : 0) * a.st + c * (D / 4));
+            // lane (g, c) holds, of token t0 + g (and t0 + 8 + g), the 16-byte pieces c, c + 4, ...: the four lanes of a
+            // token read 64 consecutive bytes at a time, and the words of piece 4i + c are the B operands of k steps
+            // 2i and 2i + 1 (the queries are laid out to match)
+            uint32_t bw[2][WPL];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int t = t0 + 8 * h + g;
+                const uint4* src = reinterpret_cast<const uint4*>(Kb + (size_t)(t < a.T ? t : 0) * a.st) + c;
 #pragma unroll
                 for (int i = 0; i < WPL / 4; ++i) {
                     uint4 v = make_uint4(0, 0, 0, 0);
-                    if (t < a.T) v = src[i];
-                    bw[4 * i] = v.x; bw[4 * i + 1] = v.y; bw[4 * i + 2] = v.z; bw[4 * i + 3] = v.w;
+                    if (t < a.T) v = src[4 * i];
+                    bw[h][4 * i] = v.x; bw[h][4 * i + 1] = v.y; bw[h][4 * i + 2] = v.z; bw[h][4 * i + 3] = v.w;
                 }
             }
-            float acc[2][4];
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt) {
+                float acc[2][4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
+                for (int i = 0; i < 4; ++i) { acc[0][i] = 0.f; acc[1][i] = 0.f; }
 #pragma unroll
                 for (int ks = 0; ks < KS; ++ks) {
                     const uint4 f = s_q[((2 * mp + mt) * KS + ks) * 32 + lane];
                     const uint32_t fr[4] = {f.x, f.y, f.z, f.w};
-                    mma_16816(acc[mt], fr, bw[2 * ks], bw[2 * ks + 1]);
+                    mma_16816(acc[0], fr, bw[0][2 * ks], bw[0][2 * ks + 1]);
+                    mma_16816(acc[1], fr, bw[1][2 * ks], bw[1][2 * ks + 1]);
                 }
-            }
-            // acc[mt][0..1]: row g, tokens t0+2c, t0+2c+1;  acc[mt][2..3]: row g+8
-#pragma unroll
-            for (int mt = 0; mt < 2; ++mt)
+                // acc[h][0..1]: row g, tokens t0+8h+2c, +1;  acc[h][2..3]: row g+8
 #pragma unroll
                 for (int hr = 0; hr < 2; ++hr) {
                     const int i = mp * 32 + mt * 16 + g + 8 * hr;          // query
                     if (i >= a.n) continue;
                     const int last = a.T - a.n + i;                         // last token the query sees
-                    const float l0 = a.scale * acc[mt][2 * hr], l1 = a.scale * acc[mt][2 * hr + 1];
-                    *reinterpret_cast<float2*>(&s_l[(size_t)i * PC_PITCH + (t0 - t_cta) + 2 * c]) = make_float2(l0, l1);
 #pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int t = t0 + 2 * c + e;
-                        const float l = e ? l1 : l0;
-                        if (t < a.T && t <= last) {
-                            const float mnew = fmaxf(rm[mt][hr], l);
-                            rs[mt][hr] = rs[mt][hr] * __expf(rm[mt][hr] - mnew) + __expf(l - mnew);
-                            rm[mt][hr] = mnew;
-                        }
+                    for (int h = 0; h < 2; ++h) {
+                        const int t = t0 + 8 * h + 2 * c;
+                        const float l0 = a.scale * acc[h][2 * hr], l1 = a.scale * acc[h][2 * hr + 1];
+                        *reinterpret_cast<float2*>(&s_l[(size_t)i * PC_PITCH + (t - t_cta)]) = make_float2(l0, l1);
+                        if (t <= last) rm[mt][hr] = fmaxf(rm[mt][hr], l0);       // last < T: one bound does for both
+                        if (t + 1 <= last) rm[mt][hr] = fmaxf(rm[mt][hr], l1);
                     }
                 }
+            }
         }
-        // merge the four lanes of a row, then the warps, into this CTA's (max, sum) of the row
+        // merge the four lanes of a row, then the warps, into this CTA's maximum of the row
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
             for (int hr = 0; hr < 2; ++hr) {
-                float m = rm[mt][hr], s = rs[mt][hr];
-#pragma unroll
-                for (int o = 1; o < 4; o <<= 1) {
-                    const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, o), s2 = __shfl_xor_sync(0xFFFFFFFFu, s, o);
-                    const float mn = fmaxf(m, m2);
-                    s = (m == NEG ? 0.f : s * __expf(m - mn)) + (m2 == NEG ? 0.f : s2 * __expf(m2 - mn));
-                    m = mn;
-                }
-                if (c == 0) s_part[warp][mt * 16 + g + 8 * hr] = make_float2(m, s);
+                float m = rm[mt][hr];
+                m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+                m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+                if (c == 0) s_part[warp][mt * 16 + g + 8 * hr] = m;
             }
         __syncthreads();
-        for (int il = threadIdx.x; il < 32; il += blockDim.x) {
-            const int i = mp * 32 + il;
-            if (i >= a.n) continue;
-            float m = NEG, s = 0.f;
-            for (int w = 0; w < PC_WARPS; ++w) {
-                const float2 p = s_part[w][il];
-                const float mn = fmaxf(m, p.x);
-                s = (m == NEG ? 0.f : s * __expf(m - mn)) + (p.x == NEG ? 0.f : p.y * __expf(p.x - mn));
-                m = mn;
-            }
-            s_stat[i] = make_float2(m, s);
+        if (threadIdx.x < 32 && mp * 32 + (int)threadIdx.x < a.n) {
+            float m = NEG;
+#pragma unroll
+            for (int w = 0; w < PC_WARPS; ++w) m = fmaxf(m, s_part[w][threadIdx.x]);
+            s_mcta[mp * 32 + threadIdx.x] = m;
         }
         __syncthreads();
     }
-    // ---- every CTA of the (b,h) has its row statistics: merge them across the cluster
+    // ---- the logits become exponentials relative to the CTA's row maximum, in place (one exponential per entry in
+    //      all; entries a query cannot see become 0), and every row gets its sum over this CTA's tokens
+    const int nt = min(PC_CHUNK, a.T - t_cta);
+    const unsigned ncta = cluster.num_blocks(), rank = cluster.block_rank();
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");       // second half of the barrier begun at the start
+    for (int i = warp; i < a.n; i += PC_WARPS) {
+        const int last = a.T - a.n + i;
+        const float m = s_mcta[i];
+        float* rowl = s_l + (size_t)i * PC_PITCH;
+        float sum = 0.f;
+        for (int k = 4 * lane; k < nt; k += 128) {       // the pitch covers the four of a ragged end; what is there is not used
+            const float4 l = *reinterpret_cast<const float4*>(rowl + k);
+            float4 e;
+            e.x = (t_cta + k <= last) ? __expf(l.x - m) : 0.f;
+            e.y = (t_cta + k + 1 <= last) ? __expf(l.y - m) : 0.f;
+            e.z = (t_cta + k + 2 <= last) ? __expf(l.z - m) : 0.f;
+            e.w = (t_cta + k + 3 <= last) ? __expf(l.w - m) : 0.f;
+            *reinterpret_cast<float4*>(rowl + k) = e;
+            sum += (e.x + e.y) + (e.z + e.w);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+        if (lane < (int)ncta) *cluster.map_shared_rank(&s_all[rank][i], lane) = make_float2(m, sum);
+    }
+    // ---- every CTA of the (b,h) has the row statistics of all of them (the remote stores are complete at the cluster
+    //      barrier, and nothing is read from or written to another CTA afterwards): merge them
     cluster.sync();
-    const unsigned ncta = cluster.num_blocks();
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
         float m = NEG, s = 0.f;
         for (unsigned r = 0; r < ncta; ++r) {
-            const float2 p = *cluster.map_shared_rank(&s_stat[i], r);
+            const float2 p = s_all[r][i];
             const float mn = fmaxf(m, p.x);
             s = (m == NEG ? 0.f : s * __expf(m - mn)) + (p.x == NEG ? 0.f : p.y * __expf(p.x - mn));
             m = mn;
         }
-        s_m[i] = m;
-        s_inv[i] = s > 0.f ? 1.0f / s : 0.f;
+        // what this CTA's exponentials are multiplied by: exp(own maximum - maximum of the row) / sum of the row
+        const float own = s_mcta[i];
+        s_inv[i] = (s > 0.f && own != NEG) ? __expf(own - m) / s : 0.f;
     }
     __syncthreads();
     // ---- normalised rows, newest first, written once; rows-per-token counts
-    const int nt = min(PC_CHUNK, a.T - t_cta);
     const bool vec_ok = (a.T & 3) == 0 && ((uintptr_t)a.ring & 15) == 0;      // rows start 16-byte aligned, no ragged end
     for (int r = warp; r < a.n; r += PC_WARPS) {
         const int i = a.n - 1 - r;
-        const int last = a.T - a.n + i;
-        const float M = s_m[i], inv = s_inv[i];
+        const float f = s_inv[i];
         float* row = a.ring + ((size_t)bh * a.n + r) * a.T + t_cta;
         const float* src = s_l + (size_t)i * PC_PITCH;
         if (vec_ok) {     // four tokens per lane and store
             for (int k = 4 * lane; k < nt; k += 128) {
-                const float4 l = *reinterpret_cast<const float4*>(src + k);
-                float4 o;
-                o.x = (t_cta + k <= last) ? __expf(l.x - M) * inv : 0.f;
-                o.y = (t_cta + k + 1 <= last) ? __expf(l.y - M) * inv : 0.f;
-                o.z = (t_cta + k + 2 <= last) ? __expf(l.z - M) * inv : 0.f;
-                o.w = (t_cta + k + 3 <= last) ? __expf(l.w - M) * inv : 0.f;
+                float4 o = *reinterpret_cast<const float4*>(src + k);
+                o.x *= f; o.y *= f; o.z *= f; o.w *= f;
                 *reinterpret_cast<float4*>(row + k) = o;
             }
         } else {
-            for (int k = lane; k < nt; k += 32) row[k] = (t_cta + k <= last) ? __expf(src[k] - M) * inv : 0.f;
+            for (int k = lane; k < nt; k += 32) row[k] = src[k] * f;
         }
     }
     for (int k = threadIdx.x; k < nt; k += blockDim.x) a.nvalid[(size_t)bh * a.T + t_cta + k] = (uint8_t)min(a.n, a.T - (t_cta + k));
-    cluster.sync();      // nobody leaves while its statistics may still be read by the others
 }
 
 // Upper quantile of a list of binary32 values (the squared query norms): exact 4 x 8-bit radix select on
