@@ -369,19 +369,19 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
     // ---- where the outliers of the new tokens are: (slot, channel) in (token, channel) order - entries of lanes
     //      p' < p of a token come first - listed in shared memory; their place needs only the scan of the counts.
     //      The values are fetched and the entries written afterwards by all threads, one entry each.
-    uint32_t before[2] = {0, 0};
 #pragma unroll
     for (int x = X0; x < X1; ++x) {
         uint32_t ob = valid ? ~inl[x] : 0u;
         const uint32_t mine = (uint32_t)__popc(ob);
+        uint32_t before = 0;
 #pragma unroll
         for (int d = 1; d < P; ++d) {
             const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, mine, d);
-            if (p >= d) before[x] += o;
+            if (p >= d) before += o;
         }
         if (ob) {
             const uint32_t all = ob;
-            const uint32_t lp0 = s_cnt[x][slot & (QAQ_TILE - 1)] + before[x];
+            const uint32_t lp0 = s_cnt[x][slot & (QAQ_TILE - 1)] + before;
             while (ob) {
                 const int bit = __ffs(ob) - 1;
                 ob &= ob - 1;
@@ -443,6 +443,16 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
         const TensorStore& ts = x ? a.v : a.k;
         uint8_t* dst = ts.codes + (size_t)bh * a.pool_bytes + s_base[x];
         const uint32_t nb = (s_tot[x] + 15u) & ~15u;     // tiles start 16-byte aligned and own a rounded amount
+        // the value of the first listed outlier of this thread is on its way (read again from the input: the
+        // registers hold -inf in its place) while the image goes out
+        const uint32_t ntot = s_otot[x], nst = ntot < OUT_STAGE ? ntot : OUT_STAGE;
+        const __half* X = (x ? a.V : a.K) + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
+        uint32_t w_first = 0;
+        unsigned short v_first = 0;
+        if ((uint32_t)tid < nst) {
+            w_first = s_work[x - X0][tid];
+            v_first = __half_as_ushort(X[(size_t)(tile * QAQ_TILE + (int)(w_first >> 8) - t_old) * a.st + (w_first & 0xFFu)]);
+        }
         for (uint32_t o = tid * 16; o < nb; o += NT * 16) {
             uint4 v;
             if (x == 0 || o < (uint32_t)qaqc::QAQ_TILE_HDR) v = *reinterpret_cast<const uint4*>(s_img[x - X0] + o);
@@ -452,9 +462,11 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
         // outlier entries: one listed outlier per thread (value read again from the input: the registers hold -inf in
         // its place), stores next to each other; a tile with more outliers than are listed writes the rest one by one
         {
-            const uint32_t ntot = s_otot[x], nst = ntot < OUT_STAGE ? ntot : OUT_STAGE;
-            const __half* X = (x ? a.V : a.K) + (size_t)b_idx * a.sb + (size_t)h_idx * a.sh;
-            for (uint32_t i = tid; i < nst; i += NT) {
+            if ((uint32_t)tid < nst) {
+                const uint32_t pos = s_obase[x] + tid;
+                if (pos < s_olimit[x]) ts.outl[(size_t)bh * a.ocap + pos] = (uint32_t)v_first | ((w_first & 0xFFu) << 16) | ((w_first >> 8) << 24);
+            }
+            for (uint32_t i = tid + NT; i < nst; i += NT) {
                 const uint32_t w = s_work[x - X0][i], sl = w >> 8, ch = w & 0xFFu;
                 const uint32_t pos = s_obase[x] + i;
                 if (pos < s_olimit[x])
@@ -462,10 +474,26 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
                                                           (ch << 16) | (sl << 24);
             }
             if (ntot > OUT_STAGE) {
-                uint32_t ob = valid ? ~inl[x] : 0u;
+                // rare.  Nothing of the listing pass is kept in registers for this: the lane reads its 32 channels
+                // again and repeats the outlier test (same bounds, same bit order as analyze32)
+                const __half2 lo2 = __half2half2(__float2half_ru(thr[2 * x])), hi2 = __half2half2(__float2half_rd(thr[2 * x + 1]));
+                const __half* row = X + (size_t)(valid ? tn : 0) * a.st + 32 * p;
+                uint32_t ob = 0;
+                if (valid) {
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        const __half2 v = as_h2(reinterpret_cast<const uint32_t*>(row)[k]);
+                        ob |= (~(__hge2_mask(v, lo2) & __hle2_mask(v, hi2)) & 0x00010001u) << k;
+                    }
+                }
+                const uint32_t mine = (uint32_t)__popc(ob);
+                uint32_t lp0 = s_cnt[x][slot & (QAQ_TILE - 1)];
+#pragma unroll
+                for (int d = 1; d < P; ++d) {
+                    const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, mine, d);
+                    if (p >= d) lp0 += o;
+                }
                 const uint32_t all = ob;
-                const uint32_t lp0 = s_cnt[x][slot & (QAQ_TILE - 1)] + before[x];
-                const __half* row = X + (size_t)tn * a.st + 32 * p;
                 while (ob) {
                     const int bit = __ffs(ob) - 1;
                     ob &= ob - 1;
