@@ -359,11 +359,15 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
         }
         __syncwarp();
         // the next round may set aside 128 more; the last round empties the buffer
-        if (!(nflag > (uint32_t)(WARP_FLAGS - 128) || c0 + 4 * tok_step >= ntok)) continue;
+        const bool last_round = c0 + 4 * tok_step >= ntok;
+        if (!(nflag > (uint32_t)(WARP_FLAGS - 128) || last_round)) continue;
+        // whole batches of 32 only (every lane busy); what is left over stays in the buffer for the next time,
+        // except in the last round
+        const uint32_t ntake = last_round ? nflag : (nflag & ~31u);
         // the warp's set-aside pieces entry by entry: per lane the entries below lo, above hi and NaN; one reservation
         // per tail for the whole batch, then every lane writes its keys
-        for (uint32_t i0 = 0; i0 < nflag; i0 += 32) {
-            const bool have = i0 + lane < nflag;
+        for (uint32_t i0 = 0; i0 < ntake; i0 += 32) {
+            const bool have = i0 + lane < ntake;
             const uint4 r = have ? wflag[i0 + lane] : make_uint4(0, 0, 0, 0);
             const uint32_t w[4] = {r.x, r.y, r.z, r.w};
             uint32_t below = 0, above = 0, nans = 0;              // bit j / 16 + j: low / high half of word j
@@ -405,8 +409,13 @@ __global__ void __launch_bounds__(256) thr_scan_kernel(const ThrArgs a) {
                 }
             }
         }
-        nflag = 0;
-        __syncwarp();     // the buffer is free again
+        const uint32_t left = nflag - ntake;           // fewer than 32
+        uint4 keep = make_uint4(0, 0, 0, 0);
+        if ((uint32_t)lane < left) keep = wflag[ntake + lane];
+        __syncwarp();
+        if ((uint32_t)lane < left) wflag[lane] = keep;
+        nflag = left;
+        __syncwarp();     // the rest of the buffer is free again
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) nnan += __shfl_xor_sync(0xFFFFFFFFu, nnan, o);
