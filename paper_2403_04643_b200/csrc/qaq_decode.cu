@@ -80,13 +80,18 @@ __host__ __device__ inline DecPlan plan_decode(int BH, int ntiles) {
     return p;
 }
 
+constexpr int OL_STAGED = 96;     // outlier entries per tile and tensor that come through shared memory; more are read in place
+
 // per-warp scratch for the tile a warp is working on
 template <int D>
 struct WarpScratch {
     static constexpr int STAGE = 72 * D;      // bytes of the staging buffer (9 KB at head_dim 128: four CTAs per SM)
     alignas(16) uint8_t buf[STAGE];           // keys of a tile from the front, values from the back
-    int dotw[4][QAQ_TILE];                    // integer q . piece per section and rank
-    alignas(16) uint32_t wts[4][QAQ_TILE / 4][4];  // per section and value group: the three byte digits of the four weights
+    union alignas(16) {                       // the key phase is over (logits taken) before the value weights are written
+        int dotw[4][QAQ_TILE];                // integer q . piece per section and rank
+        uint32_t wts[4][QAQ_TILE / 4][4];     // per section and value group: the three byte digits of the four weights
+    };
+    uint32_t olist[2][OL_STAGED];             // the first outlier entries of the tile's keys / values (copied in with the packed words)
     float midK[QAQ_TILE];       // min + step/2
     float midV[QAQ_TILE];
     float p[QAQ_TILE];          // attention weights of the tile's tokens at the current scale of the running sums
@@ -265,6 +270,15 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
 #pragma unroll 1
         for (uint32_t o = lane * 16; o < nb; o += 32 * 16) cp_async<16>(dst + o, src + o);
     };
+    // the first entries of a tile's outlier list, 4 bytes each, into the warp's scratch (part of the copy group open then)
+    auto stage_list = [&](uint32_t* dst, const uint32_t* src, uint32_t cnt) {
+#pragma unroll
+        for (int k = 0; k < OL_STAGED / 32; ++k)
+            if (lane + 32 * k < cnt) {
+                const unsigned sa = (unsigned)__cvta_generic_to_shared(dst + lane + 32 * k);
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(sa), "l"(src + lane + 32 * k));
+            }
+    };
     int tile = tile_lo + warp;
     Meta cur = fetch_meta(tile);
     Meta nxt = fetch_meta(tile + DEC_WARPS);
@@ -273,8 +287,10 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
     if (tile < tile_hi) {
         const uint32_t nbK = (__shfl_sync(0xFFFFFFFFu, cur.tb, 1) + 15u) & ~15u, nbV = (__shfl_sync(0xFFFFFFFFu, cur.tb, 5) + 15u) & ~15u;
         if (nbK <= STAGE) { stK = nbK; stage(ws.buf, poolK + __shfl_sync(0xFFFFFFFFu, cur.tb, 0), nbK); }
+        stage_list(ws.olist[0], ogK + __shfl_sync(0xFFFFFFFFu, cur.tb, 2), __shfl_sync(0xFFFFFFFFu, cur.tb, 3));
         cp_async_commit();
         if (stK + nbV <= STAGE) { stV = nbV; stage(ws.buf + STAGE - nbV, poolV + __shfl_sync(0xFFFFFFFFu, cur.tb, 4), nbV); }
+        stage_list(ws.olist[1], ogV + __shfl_sync(0xFFFFFFFFu, cur.tb, 6), __shfl_sync(0xFFFFFFFFu, cur.tb, 7));
         cp_async_commit();
     }
 
@@ -288,13 +304,6 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         const bool val0 = t0 < T, val1 = t0 + HALF < T;
         const uint8_t* tK = stK ? ws.buf : poolK + offK;
         const uint8_t* tV = stV ? ws.buf + STAGE - stV : poolV + offV;
-        // the first outlier entries of the tile (used after the section loops)
-        uint32_t eK[3], eV[3];
-#pragma unroll
-        for (int k = 0; k < 3; ++k) {
-            eK[k] = lane + 32 * k < ocK ? __ldg(ogK + ooK + lane + 32 * k) : 0u;
-            eV[k] = lane + 32 * k < ocV ? __ldg(ogV + ooV + lane + 32 * k) : 0u;
-        }
         cp_async_wait<1>();     // this tile's keys have landed (its values may still be in flight)
         __syncwarp();
 
@@ -344,7 +353,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         // key outliers: q_ch * (x - mid) per token
 #pragma unroll 1
         for (uint32_t e = lane; e < ocK; e += 32) {
-            const uint32_t v = e < 96 ? (e < 32 ? eK[0] : (e < 64 ? eK[1] : eK[2])) : __ldg(ogK + ooK + e);
+            const uint32_t v = e < (uint32_t)OL_STAGED ? ws.olist[0][e] : __ldg(ogK + ooK + e);
             const int tok = (v >> 24) & (QAQ_TILE - 1);
             const float tm = sm.qf[(v >> 16) & (D - 1)] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midK[tok]);
             outlier_add(&ws.kcorr[0][tok], &ws.kcorr[1][tok], tm);
@@ -355,6 +364,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         if (has_next) {
             const uint32_t nb = (__shfl_sync(0xFFFFFFFFu, nxt.tb, 1) + 15u) & ~15u;
             if (nb + stV <= STAGE) { stKn = nb; stage(ws.buf, poolK + __shfl_sync(0xFFFFFFFFu, nxt.tb, 0), nb); }
+            stage_list(ws.olist[0], ogK + __shfl_sync(0xFFFFFFFFu, nxt.tb, 2), __shfl_sync(0xFFFFFFFFu, nxt.tb, 3));
         }
         cp_async_commit();
 
@@ -499,7 +509,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         // value outliers: p_t * (v - mid) per channel
 #pragma unroll 1
         for (uint32_t e = lane; e < ocV; e += 32) {
-            const uint32_t v = e < 96 ? (e < 32 ? eV[0] : (e < 64 ? eV[1] : eV[2])) : __ldg(ogV + ooV + e);
+            const uint32_t v = e < (uint32_t)OL_STAGED ? ws.olist[1][e] : __ldg(ogV + ooV + e);
             const int tok = (v >> 24) & (QAQ_TILE - 1), ch = (v >> 16) & (D - 1);
             const float tm = ws.p[tok] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midV[tok]);
             outlier_add(&ws.vcorr[0][ch], &ws.vcorr[1][ch], tm);
@@ -521,6 +531,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         if (has_next) {
             const uint32_t nb = (__shfl_sync(0xFFFFFFFFu, nxt.tb, 5) + 15u) & ~15u;
             if (nb + stKn <= STAGE) { stVn = nb; stage(ws.buf + STAGE - nb, poolV + __shfl_sync(0xFFFFFFFFu, nxt.tb, 4), nb); }
+            stage_list(ws.olist[1], ogV + __shfl_sync(0xFFFFFFFFu, nxt.tb, 6), __shfl_sync(0xFFFFFFFFu, nxt.tb, 7));
         }
         cp_async_commit();
         stK = stKn; stV = stVn;
