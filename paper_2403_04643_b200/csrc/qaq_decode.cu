@@ -271,13 +271,19 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         for (uint32_t o = lane * 16; o < nb; o += 32 * 16) cp_async<16>(dst + o, src + o);
     };
     // the first entries of a tile's outlier list, 4 bytes each, into the warp's scratch (part of the copy group open then)
+    // (lists of whole tiles start on 16-byte boundaries: four entries per copy, reading up to three entries past the
+    // list, which the capacity's read-ahead margin covers; a list that grew with an open tile may start anywhere)
     auto stage_list = [&](uint32_t* dst, const uint32_t* src, uint32_t cnt) {
+        if (((uintptr_t)src & 15) == 0) {
+            if (lane < OL_STAGED / 4 && 4u * lane < cnt) cp_async<16>(dst + 4 * lane, src + 4 * lane);
+        } else {
 #pragma unroll
-        for (int k = 0; k < OL_STAGED / 32; ++k)
-            if (lane + 32 * k < cnt) {
-                const unsigned sa = (unsigned)__cvta_generic_to_shared(dst + lane + 32 * k);
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(sa), "l"(src + lane + 32 * k));
-            }
+            for (int k = 0; k < OL_STAGED / 32; ++k)
+                if (lane + 32 * k < cnt) {
+                    const unsigned sa = (unsigned)__cvta_generic_to_shared(dst + lane + 32 * k);
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(sa), "l"(src + lane + 32 * k));
+                }
+        }
     };
     int tile = tile_lo + warp;
     Meta cur = fetch_meta(tile);
