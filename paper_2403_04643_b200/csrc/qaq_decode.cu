@@ -244,31 +244,41 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
     // ---- tile metadata in registers: table words in lanes 0..7 (offset and length of the bytes, first entry and
     //      length of the outlier list; keys in lanes 0..3, values in 4..7), min/max of tokens lane, lane+32.
     //      Table entries that point outside the pool or the list are not followed (length 0).
+    //      The loads are only issued here; nothing looks at what they return before settle() does, a tile later.
     struct Meta { uint32_t tb, mm[4]; };
     auto fetch_meta = [&](int tile) {
         Meta m;
         m.tb = 0; m.mm[0] = m.mm[1] = m.mm[2] = m.mm[3] = 0;
         if (tile < tile_hi) {
-            uint32_t first = 0, len = 0;
             if (lane < 8) {
                 const TensorStore& ts = (lane >= 4) ? a.v : a.k;
-                const size_t ti = trow + tile;
-                if (lane & 2) { first = ts.tile_ooff[ti]; len = ts.tile_ocnt[ti]; if ((size_t)first + len > a.ocap) len = 0; }
-                else {
-                    first = ts.tile_off[ti]; len = ts.tile_nbytes[ti];
-                    if ((first & 15u) || len < (uint32_t)qaqc::QAQ_TILE_HDR || (size_t)first + ((len + 15u) & ~15u) > a.pool_bytes) len = 0;
-                }
-                m.tb = (lane & 1) ? len : first;
+                const uint32_t* tab = (lane & 2) ? ((lane & 1) ? ts.tile_ocnt : ts.tile_ooff) : ((lane & 1) ? ts.tile_nbytes : ts.tile_off);
+                m.tb = tab[trow + tile];
             }
             const size_t t0 = mrow + (size_t)tile * QAQ_TILE + lane;
             m.mm[0] = a.k.mnmx[t0]; m.mm[1] = a.k.mnmx[t0 + 32]; m.mm[2] = a.v.mnmx[t0]; m.mm[3] = a.v.mnmx[t0 + 32];
         }
         return m;
     };
+    // the table words of a tile as they are used: a length becomes 0 where offset and length point outside the pool
+    // or the list (lanes 2k, 2k+1 hold an offset and its length)
+    auto settle = [&](uint32_t tb) -> uint32_t {
+        const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, tb, 1);
+        const uint32_t first = (lane & 1) ? other : tb, len = (lane & 1) ? tb : other;
+        const bool bad = (lane & 2) ? ((size_t)first + len > a.ocap)
+                                    : ((first & 15u) || len < (uint32_t)qaqc::QAQ_TILE_HDR || (size_t)first + ((len + 15u) & ~15u) > a.pool_bytes);
+        return lane < 8 ? ((lane & 1) ? (bad ? 0u : len) : first) : 0u;
+    };
     // copies nb bytes (a multiple of 16) of a tile to the staging buffer
     auto stage = [&](uint8_t* dst, const uint8_t* src, uint32_t nb) {
+        unsigned sa = (unsigned)__cvta_generic_to_shared(dst) + lane * 16;
+        const uint8_t* g = src + lane * 16;
 #pragma unroll 1
-        for (uint32_t o = lane * 16; o < nb; o += 32 * 16) cp_async<16>(dst + o, src + o);
+        for (uint32_t o = lane * 16; o < nb; o += 4 * 512, sa += 4 * 512, g += 4 * 512) {      // four copies per round
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (o + 512u * u < nb) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(sa + 512u * u), "l"(g + 512 * u));
+        }
     };
     // the first entries of a tile's outlier list, 4 bytes each, into the warp's scratch (part of the copy group open then)
     // (lists of whole tiles start on 16-byte boundaries: four entries per copy, reading up to three entries past the
@@ -288,6 +298,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
     int tile = tile_lo + warp;
     Meta cur = fetch_meta(tile);
     Meta nxt = fetch_meta(tile + DEC_WARPS);
+    cur.tb = settle(cur.tb);
     // what is staged: bytes (rounded up to 16) of the current keys / values in the buffer, 0 = read in place
     uint32_t stK = 0, stV = 0;
     if (tile < tile_hi) {
@@ -367,6 +378,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         __syncwarp();
         // ---- the front of the buffer is free: start the copy of the next tile's keys (beside this tile's values)
         uint32_t stKn = 0;
+        nxt.tb = settle(nxt.tb);       // fetched a tile ago
         if (has_next) {
             const uint32_t nb = (__shfl_sync(0xFFFFFFFFu, nxt.tb, 1) + 15u) & ~15u;
             if (nb + stV <= STAGE) { stKn = nb; stage(ws.buf, poolK + __shfl_sync(0xFFFFFFFFu, nxt.tb, 0), nb); }
