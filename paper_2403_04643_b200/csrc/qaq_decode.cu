@@ -368,13 +368,16 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
         k_section<D, 2>(tK + kb[2], n[0][2], ws.dotw[2], qb, fg, ft);
         k_section<D, 1>(tK + kb[3], n[0][3], ws.dotw[3], qb, fg, ft);
         // key outliers: q_ch * (x - mid) per token
-#pragma unroll 1
-        for (uint32_t e = lane; e < ocK; e += 32) {
-            const uint32_t v = e < (uint32_t)OL_STAGED ? ws.olist[0][e] : __ldg(ogK + ooK + e);
+        auto k_outlier = [&](uint32_t v) {
             const int tok = (v >> 24) & (QAQ_TILE - 1);
             const float tm = sm.qf[(v >> 16) & (D - 1)] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midK[tok]);
             outlier_add(&ws.kcorr[0][tok], &ws.kcorr[1][tok], tm);
-        }
+        };
+#pragma unroll
+        for (int k = 0; k < OL_STAGED / 32; ++k)         // the staged entries: independent chains, side by side
+            if (lane + 32u * k < ocK) k_outlier(ws.olist[0][lane + 32 * k]);
+#pragma unroll 1
+        for (uint32_t e = lane + OL_STAGED; e < ocK; e += 32) k_outlier(__ldg(ogK + ooK + e));
         __syncwarp();
         // ---- the front of the buffer is free: start the copy of the next tile's keys (beside this tile's values)
         uint32_t stKn = 0;
@@ -525,13 +528,16 @@ __global__ void __launch_bounds__(DEC_THREADS, DEC_CTAS_PER_SM) decode_kernel(co
             }
         }
         // value outliers: p_t * (v - mid) per channel
-#pragma unroll 1
-        for (uint32_t e = lane; e < ocV; e += 32) {
-            const uint32_t v = e < (uint32_t)OL_STAGED ? ws.olist[1][e] : __ldg(ogV + ooV + e);
+        auto v_outlier = [&](uint32_t v) {
             const int tok = (v >> 24) & (QAQ_TILE - 1), ch = (v >> 16) & (D - 1);
             const float tm = ws.p[tok] * (__half2float(__ushort_as_half((unsigned short)(v & 0xFFFF))) - ws.midV[tok]);
             outlier_add(&ws.vcorr[0][ch], &ws.vcorr[1][ch], tm);
-        }
+        };
+#pragma unroll
+        for (int k = 0; k < OL_STAGED / 32; ++k)
+            if (lane + 32u * k < ocV) v_outlier(ws.olist[1][lane + 32 * k]);
+#pragma unroll 1
+        for (uint32_t e = lane + OL_STAGED; e < ocV; e += 32) v_outlier(__ldg(ogV + ooV + e));
         __syncwarp();
         if (ocV) {
 #pragma unroll
