@@ -279,12 +279,13 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
     if (SELECT_ONLY) return;
     __syncthreads();   // [A] widths and outlier counts visible
 
-    // ---- warp 0: section masks of the tile, scan of the outlier counts; lanes 0..3 each take space from one
-    //      pool (four atomics in flight)
+    // ---- warp 0: section masks of the tile, ranks and section offsets, space for the bytes; warp 1: scan of the
+    //      outlier counts, space for the entries (the two halves do not depend on each other; the atomics - lane 2x of
+    //      warp 0 and lane 2x + 1 of warp 1 for tensor x - stay in flight while every warp computes its codes)
     const bool starts = (s_lo == 0), closes = (s_hi == QAQ_TILE), whole = starts && closes;
     uint32_t my_base = 0, my_amount = 0, my_taken = 0;
     if (warp == 0) {
-        uint32_t amount[2][2];   // [tensor][0: bytes, 1: outliers]
+        uint32_t amount[2];
 #pragma unroll
         for (int x = X0; x < X1; ++x) {
             const uint32_t b0 = s_bits[x][lane], b1 = s_bits[x][lane + 32];
@@ -305,6 +306,20 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
 #pragma unroll
                 for (int c = 0; c < 5; ++c) s_sec[x][c] = base[c];
             }
+            // a continued tile stays where it is and takes only what it grows by behind its end
+            const uint32_t old_nb = starts ? 0u : (x ? a.v : a.k).tile_nbytes[ti];
+            amount[x] = base[4] - old_nb;
+            if (lane == 0) { s_tm[x] = tm; s_tot[x] = base[4]; }
+        }
+        if (!(lane & 1) && lane >= 2 * X0 && lane < 2 * X1) {
+            const int x = lane >> 1;
+            my_amount = x ? amount[1] : amount[0];
+            my_base = pool_take(&(x ? a.v : a.k).pool_end[bh], my_amount, 15u, whole, closes, my_taken);
+        }
+    } else if (warp == 1) {
+        uint32_t amount[2];
+#pragma unroll
+        for (int x = X0; x < X1; ++x) {
             const uint32_t c0 = s_cnt[x][lane], c1 = s_cnt[x][lane + 32];
             uint32_t ic0 = c0, ic1 = c1;
 #pragma unroll
@@ -314,16 +329,13 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
             }
             const uint32_t ctot0 = __shfl_sync(0xFFFFFFFFu, ic0, 31), ctot1 = __shfl_sync(0xFFFFFFFFu, ic1, 31);
             s_cnt[x][lane] = ic0 - c0; s_cnt[x][lane + 32] = ctot0 + ic1 - c1;
-            // a continued tile stays where it is and takes only what it grows by behind its end
-            const uint32_t old_nb = starts ? 0u : (x ? a.v : a.k).tile_nbytes[ti];
-            amount[x][0] = base[4] - old_nb; amount[x][1] = ctot0 + ctot1;
-            if (lane == 0) { s_tm[x] = tm; s_tot[x] = base[4]; s_otot[x] = ctot0 + ctot1; }
+            amount[x] = ctot0 + ctot1;
+            if (lane == 0) s_otot[x] = ctot0 + ctot1;
         }
-        if (lane >= 2 * X0 && lane < 2 * X1) {
-            const int x = lane >> 1, pool = lane & 1;
-            const TensorStore& ts = x ? a.v : a.k;
-            my_amount = x ? amount[1][pool] : amount[0][pool];
-            my_base = pool_take(pool ? &ts.opool_end[bh] : &ts.pool_end[bh], my_amount, pool ? 3u : 15u, whole, closes, my_taken);
+        if ((lane & 1) && lane >= 2 * X0 && lane < 2 * X1) {
+            const int x = lane >> 1;
+            my_amount = x ? amount[1] : amount[0];
+            my_base = pool_take(&(x ? a.v : a.k).opool_end[bh], my_amount, 3u, whole, closes, my_taken);
         }
     }
 
@@ -397,44 +409,51 @@ __global__ void __launch_bounds__(2 * D, XSEL < 0 ? (D == 128 ? 3 : 4) : (D == 1
     // ---- allocation results (the atomics were issued before the codes were computed).  A pool without room:
     //      the space is given back, nothing about the tile is published and the CTA stops; the device status
     //      reports the lost tokens.
-    if (warp == 0) {
+    if (warp == 0) {          // the byte pools
         bool fail = false;
-        if (lane >= 2 * X0 && lane < 2 * X1) {
-            const int x = lane >> 1, pool = lane & 1;
-            const TensorStore& ts = x ? a.v : a.k;
-            if (pool == 0) {
-                const uint32_t off = starts ? my_base : ts.tile_off[ti];
-                fail = (size_t)my_base + my_taken + 16 > a.pool_bytes || (size_t)off + s_tot[x] + 16 > a.pool_bytes;
-                s_base[x] = off;
-            } else {
-                const uint32_t room = my_base + 8 < a.ocap ? a.ocap - 8 - my_base : 0;  // 8 entries of read-ahead margin
-                const uint32_t stored = my_amount < room ? my_amount : room;
-                if (stored < my_amount) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
-                s_obase[x] = my_base;
-                s_olimit[x] = my_base + stored;
-            }
+        const bool mine = !(lane & 1) && lane >= 2 * X0 && lane < 2 * X1;
+        const int x = lane >> 1;
+        const TensorStore& ts = x ? a.v : a.k;
+        if (mine) {
+            const uint32_t off = starts ? my_base : ts.tile_off[ti];
+            fail = (size_t)my_base + my_taken + 16 > a.pool_bytes || (size_t)off + s_tot[x] + 16 > a.pool_bytes;
+            s_base[x] = off;
         }
         const bool any_fail = __any_sync(0xFFFFFFFFu, fail);
-        if (lane >= 2 * X0 && lane < 2 * X1) {
-            const int x = lane >> 1, pool = lane & 1;
-            const TensorStore& ts = x ? a.v : a.k;
+        if (mine) {
             if (any_fail) {
-                if (my_taken) atomicSub(pool ? &ts.opool_end[bh] : &ts.pool_end[bh], my_taken);
-            } else if (pool == 0) {
+                if (my_taken) atomicSub(&ts.pool_end[bh], my_taken);
+            } else {
                 if (starts) ts.tile_off[ti] = my_base;
                 ts.tile_nbytes[ti] = s_tot[x];
-            } else {
-                const uint32_t stored = s_olimit[x] - s_obase[x];
-                if (starts) { ts.tile_ooff[ti] = my_base; ts.tile_ocnt[ti] = stored; }
-                else ts.tile_ocnt[ti] += stored;
             }
         }
         if (lane == 0) {
             s_skip = any_fail ? 1 : 0;
             if (any_fail) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
         }
+    } else if (warp == 1) {   // the outlier lists: what fits is known now, the table is written once the byte pools have answered
+        if ((lane & 1) && lane >= 2 * X0 && lane < 2 * X1) {
+            const int x = lane >> 1;
+            const uint32_t room = my_base + 8 < a.ocap ? a.ocap - 8 - my_base : 0;  // 8 entries of read-ahead margin
+            const uint32_t stored = my_amount < room ? my_amount : room;
+            if (stored < my_amount) atomicMax(a.status, (int)QAQ_ERR_CAPACITY);
+            s_obase[x] = my_base;
+            s_olimit[x] = my_base + stored;
+        }
     }
     __syncthreads();   // [C] image complete, pool positions known, every old byte of the tile has been read
+    if (warp == 1 && (lane & 1) && lane >= 2 * X0 && lane < 2 * X1) {
+        const int x = lane >> 1;
+        const TensorStore& ts = x ? a.v : a.k;
+        if (s_skip) {
+            if (my_taken) atomicSub(&ts.opool_end[bh], my_taken);
+        } else {
+            const uint32_t stored = s_olimit[x] - s_obase[x];
+            if (starts) { ts.tile_ooff[ti] = my_base; ts.tile_ocnt[ti] = stored; }
+            else ts.tile_ocnt[ti] += stored;
+        }
+    }
     if (s_skip) { tick(); return; }
 
     // ---- the image goes out with vector stores; outlier list; per-token metadata
