@@ -227,7 +227,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--extras", default="", help="run only the extra points whose name starts with this")
-    ap.add_argument("--streams", type=int, default=2, help="streams the independent layers of a step are spread over")
+    ap.add_argument("--streams", type=int, default=3, help="streams the independent layers of a step are spread over")
     ap.add_argument("--no-graph", action="store_true", help="launch the timed steps on the stream instead of replaying a CUDA graph")
     ap.add_argument("--write-counters", default="", help="parse an ncu --csv log and write profiles/counters_C3.json (no GPU needed)")
     args = ap.parse_args()
